@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Benchmark of the libsdllm hot path: cached-KV tokens/s per layer (refresh + sparse attention).
+
+A "step" is one decoding block of the workload's attention stack: for every layer one refresh
+(dense block attention + saliency + pooling, top-k, K/V compaction) followed by the block's
+cache-reuse steps (sparse block attention over [K_c ; K_n]), issued in model order (step-major,
+layer-minor), so consecutive calls touch different layers' K/V and caches. The dense step 0 of each
+block (cache_state 0) is not part of this path and is not timed. "Cached-KV tokens" of a call are the
+key/value positions it consumes: L for a refresh, n + b for a reuse step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2_llada] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0). `--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2508_02558_b200 import workloads as W
+
+METRIC = "cached_kv_tokens_per_s_per_layer"
+UNIT = "tokens/s"
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the sparse-attention kernel pair on this workload,
+# from the ncu capture summarised under profiles/ (None until a capture exists for the workload).
+NCU_TRAFFIC_BYTES = {"c2_llada": None}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_llada", choices=["c2_llada", "c3_dream"])
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (0 = the workload's)")
+    ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------ workload
+def tokens_per_step(cfg: W.WorkloadConfig, n_layers: int, n_keep: int) -> int:
+    reuse_steps = cfg.steps_per_block - 2
+    return n_layers * (cfg.seq_len + reuse_steps * (n_keep + cfg.block_len))
+
+
+def algorithmic_bytes(cfg: W.WorkloadConfig, n_keep: int):
+    """Bytes each call must move (K and V once, Q and O once, scores / indices), per layer."""
+    e = 2 if cfg.dtype == "bf16" else 4
+    L, b, Hq, Hkv, D = cfg.seq_len, cfg.block_len, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    refresh = 2 * L * Hkv * D * e + 2 * b * Hq * D * e + 4 * (L - b) * Hkv
+    topk = 4 * (L - b) * Hkv + 4 * n_keep * Hkv
+    compact = 2 * (2 * n_keep * Hkv * D * e) + 4 * n_keep * Hkv
+    sparse = 2 * (n_keep + b) * Hkv * D * e + 2 * b * Hq * D * e
+    return {"refresh": refresh, "topk": topk, "compact": compact, "sparse": sparse}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush(); self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        os.unlink(self.file.name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------ CPU oracle arm
+def oracle_block_sample(cfg: W.WorkloadConfig, seed: int):
+    """One layer x one decoding block through the CPU oracle: 1 refresh + the block's reuse steps. Returns (tokens, seconds)."""
+    import oracle
+    s = W.make_sequence(cfg, seed=seed, layer=0, block=0)
+    q, k, v = s.refresh_inputs(1)
+    steps = [s.sparse_inputs(i) for i in range(2, cfg.steps_per_block)]
+    t0 = time.perf_counter()
+    r = oracle.refresh(q, k, v, s.block_off, cfg.retention, cfg.pool_window)
+    k_c, v_c = oracle.gather_rows(k, r.kept_idx), oracle.gather_rows(v, r.kept_idx)
+    for q2, kn, vn in steps:
+        oracle.sparse_block_attention(q2, k_c, v_c, kn, vn)
+    dt = time.perf_counter() - t0
+    return cfg.seq_len + len(steps) * (r.n_keep + cfg.block_len), dt
+
+
+def omp_threads() -> int:
+    env = os.environ.get("OMP_NUM_THREADS")
+    return int(env) if env else len(os.sched_getaffinity(0))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = W.CONFIGS[args.workload]
+    import oracle
+    oracle.build()
+    for i in range(args.warmup):
+        oracle_block_sample(cfg, seed=1000 + i) if i == 0 else None      # one warm pass is enough for a CPU loop
+    tok, sec = 0, 0.0
+    for i in range(args.steps):
+        t, s = oracle_block_sample(cfg, seed=i)
+        tok += t; sec += s
+    value = tok / sec
+    sample = "per step: 1 layer x 1 block (1 refresh + %d reuse steps) of %s" % (cfg.steps_per_block - 2, cfg.name)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": omp_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ------------------------------------------------------------------------------------------------ CUDA arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2508_02558_b200 import binding as B
+    from paper_2508_02558_b200.session import LayerCache
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: libsdllm has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()
+
+    cfg = W.CONFIGS[args.workload]
+    n_layers = args.layers or cfg.n_layers
+    Hq, Hkv, D, L, b = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.seq_len, cfg.block_len
+    reuse_steps = cfg.steps_per_block - 2
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    bdt = B.BF16 if cfg.dtype == "bf16" else B.F32
+
+    def to_dev(x):
+        if cfg.dtype == "bf16":
+            return torch.from_numpy(W.f32_to_bf16_bits(x).reshape(x.shape).view(np.int16)).view(torch.bfloat16).to(dev)
+        return torch.from_numpy(x).to(dev)
+
+    # ---- inputs: base tensors from the seeded host generator (one (layer, block=0) each); per-step drift on the device
+    caches, Ks, Vs, Qr = [], [], [], []
+    gen = torch.Generator(device=dev); gen.manual_seed(1234 + rank)
+    for l in range(n_layers):
+        s = W.make_sequence(cfg, seed=rank, layer=l, block=0)
+        q, k, v = s.refresh_inputs(1)
+        Ks.append(to_dev(k)[None]); Vs.append(to_dev(v)[None]); Qr.append(to_dev(q)[None])
+        caches.append(LayerCache(batch=1, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, seq_len_max=L, block_len=b, dtype=bdt,
+                                 retention=cfg.retention, pool_window=cfg.pool_window, device=str(dev),
+                                 share_scratch_with=caches[0] if caches else None))
+    o = cfg.prompt_len
+    n_keep = B.keep_count(caches[0].desc, L, o)[0]
+    block_off = torch.tensor([o], dtype=torch.int32, device=dev)
+    drift = cfg.drift_std / np.sqrt(D)
+    # fresh block rows for every (reuse step, layer): Q_b', K_n, V_n = base + drift, rounded to the compute dtype
+    Qs = torch.empty((reuse_steps, n_layers, 1, Hq, b, D), dtype=tdt, device=dev)
+    Kn = torch.empty((reuse_steps, n_layers, 1, Hkv, b, D), dtype=tdt, device=dev)
+    Vn = torch.empty_like(Kn)
+    for l in range(n_layers):
+        for t in range(reuse_steps):
+            Qs[t, l] = (Qr[l].float() + drift * torch.randn(Qr[l].shape, device=dev, generator=gen)).to(tdt)
+            Kn[t, l] = (Ks[l][:, :, o:o + b].float() + drift * torch.randn((1, Hkv, b, D), device=dev, generator=gen)).to(tdt)
+            Vn[t, l] = (Vs[l][:, :, o:o + b].float() + drift * torch.randn((1, Hkv, b, D), device=dev, generator=gen)).to(tdt)
+    out_r = torch.empty((n_layers, 1, Hq, b, D), dtype=tdt, device=dev)
+    out_s = torch.empty((reuse_steps, n_layers, 1, Hq, b, D), dtype=tdt, device=dev)
+
+    stream = torch.cuda.Stream(device=dev)
+
+    def one_step():
+        """One decoding block: refresh every layer, then every reuse step over every layer (model order)."""
+        for l in range(n_layers):
+            caches[l].refresh(Qr[l], Ks[l], Vs[l], None, block_off, out=out_r[l], stream=stream)
+        for t in range(reuse_steps):
+            for l in range(n_layers):
+                caches[l].sparse_step(Qs[t, l], Kn[t, l], Vn[t, l], out_s[t, l], stream=stream)
+
+    def sparse_only():
+        for t in range(reuse_steps):
+            for l in range(n_layers):
+                caches[l].sparse_step(Qs[t, l], Kn[t, l], Vn[t, l], out_s[t, l], stream=stream)
+
+    def refresh_only():
+        for l in range(n_layers):
+            caches[l].refresh(Qr[l], Ks[l], Vs[l], None, block_off, out=out_r[l], stream=stream)
+
+    def make_runner(fn):
+        if args.no_graph:
+            return fn
+        with torch.cuda.stream(stream):
+            fn()                                    # first eager call sets kernel attributes outside the capture
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            fn()
+        return graph.replay
+
+    def timed(runner, iters, warm):
+        with torch.cuda.stream(stream):
+            for _ in range(warm):
+                runner()
+            stream.synchronize()
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(iters):
+                runner()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
+        return e0.elapsed_time(e1) / 1e3
+
+    launches_per_step = n_layers * (4 + 2 * reuse_steps)
+    step_runner = make_runner(one_step)
+    sampler = ClockSampler(local) if rank == 0 else None
+    sec = timed(step_runner, args.steps, max(args.warmup, 3))
+    clocks = sampler.stop() if sampler else None
+    if world > 1:
+        t = torch.tensor([sec], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        sec = float(t.item())
+    tok = tokens_per_step(cfg, n_layers, n_keep)
+    value = world * tok * args.steps / sec
+
+    # ---- roofline of the dominant call (sparse block attention: 30 of the 31 calls per layer per block)
+    ab = algorithmic_bytes(cfg, n_keep)
+    sp_runner = make_runner(sparse_only)
+    sp_sec = timed(sp_runner, max(3, args.steps // 2), 3) / max(3, args.steps // 2) / (n_layers * reuse_steps)
+    rf_runner = make_runner(refresh_only)
+    rf_sec = timed(rf_runner, max(3, args.steps // 2), 3) / max(3, args.steps // 2) / n_layers
+    peak, peak_kind = peaks()
+    achieved = ab["sparse"] / sp_sec / 1e9
+    roofline = {"bound": "hbm", "kernel": "sdllm_sparse_block_attn (split-K partial + merge)", "achieved": achieved,
+                "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                "frac_of_8TBps": achieved / 8000.0, "algorithmic_bytes_per_launch": ab["sparse"], "us_per_launch": sp_sec * 1e6,
+                "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+                "refresh_chain": {"us_per_layer": rf_sec * 1e6, "algorithmic_bytes": ab["refresh"] + ab["topk"] + ab["compact"],
+                                  "achieved": (ab["refresh"] + ab["topk"] + ab["compact"]) / rf_sec / 1e9,
+                                  "frac": (ab["refresh"] + ab["topk"] + ab["compact"]) / rf_sec / 1e9 / peak}}
+
+    # ---- end to end: inputs start in pinned host memory, results are read back, every step
+    e2e = None
+    if not args.no_e2e:
+        hK = [x.cpu().pin_memory() for x in Ks]; hV = [x.cpu().pin_memory() for x in Vs]; hQ = [x.cpu().pin_memory() for x in Qr]
+        hQs, hKn, hVn = Qs.cpu().pin_memory(), Kn.cpu().pin_memory(), Vn.cpu().pin_memory()
+        h_out_r, h_out_s = out_r.cpu().pin_memory(), out_s.cpu().pin_memory()
+        dK, dV, dQ = torch.empty_like(Ks[0]), torch.empty_like(Vs[0]), torch.empty_like(Qr[0])
+        dQs, dKn, dVn = torch.empty_like(Qs[0, 0]), torch.empty_like(Kn[0, 0]), torch.empty_like(Vn[0, 0])
+
+        def e2e_step():
+            with torch.cuda.stream(stream):
+                for l in range(n_layers):
+                    dQ.copy_(hQ[l], non_blocking=True); dK.copy_(hK[l], non_blocking=True); dV.copy_(hV[l], non_blocking=True)
+                    caches[l].refresh(dQ, dK, dV, None, block_off, out=out_r[l], stream=stream)
+                    h_out_r[l].copy_(out_r[l], non_blocking=True)
+                for t in range(reuse_steps):
+                    for l in range(n_layers):
+                        dQs.copy_(hQs[t, l], non_blocking=True); dKn.copy_(hKn[t, l], non_blocking=True); dVn.copy_(hVn[t, l], non_blocking=True)
+                        caches[l].sparse_step(dQs, dKn, dVn, out_s[t, l], stream=stream)
+                        h_out_s[t, l].copy_(out_s[t, l], non_blocking=True)
+        e2e_iters = max(2, min(args.steps, 5))
+        e2e_sec = timed(e2e_step, e2e_iters, 1)
+        if world > 1:
+            t = torch.tensor([e2e_sec], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_sec = float(t.item())
+        esz = Ks[0].element_size()
+        h2d = n_layers * ((2 * Hkv * L * D + Hq * b * D) * esz + reuse_steps * (2 * Hkv * b * D + Hq * b * D) * esz)
+        d2h = n_layers * (1 + reuse_steps) * Hq * b * D * esz
+        e2e = {"value": world * tok * e2e_iters / e2e_sec, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": 1e3 * e2e_sec / e2e_iters}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        oracle_block_sample(cfg, seed=99)            # warm the caches and the OpenMP pool
+        ctok, csec = oracle_block_sample(cfg, seed=0)
+        cpu_baseline = {"value": ctok / csec, "unit": UNIT, "cores": omp_threads(), "kind": "oracle", "seconds": csec,
+                        "sample": "1 layer x 1 block (1 refresh + %d reuse steps) of %s, fp64" % (reuse_steps, cfg.name)}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": cfg.name, "layers": n_layers, "seq_len": L, "block_len": b, "n_q_heads": Hq, "n_kv_heads": Hkv,
+                       "head_dim": D, "retention": cfg.retention, "pool_window": cfg.pool_window, "n_keep": n_keep,
+                       "step": "1 decoding block: %d layers x (1 refresh chain + %d reuse steps)" % (n_layers, reuse_steps),
+                       "l2": "no flush: one step streams %.0f MB of K/V and caches across layers, larger than L2" % (
+                           n_layers * (ab["refresh"] + reuse_steps * 0 + 2 * n_keep * Hkv * D * 2) / 1e6),
+                       "launch": "eager" if args.no_graph else "cuda_graph_replay", "parallelism": "replicas" if world > 1 else "1gpu"},
+            "block_steps_per_s": world * n_layers * (1 + reuse_steps) * args.steps / sec,
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks,
+            "gpu_launches": launches_per_step * args.steps,
+        }))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,150 @@
+/*
+ * libsdllm — cache refresh and sparse block attention for diffusion LLMs (Sparse-dLLM), C ABI.
+ *
+ * One layer, one decoding block. At the refresh step of a block (cache_state 1 of the paper's
+ * Algorithm 2) the block's b query rows attend over the whole bidirectional K/V, a saliency score
+ * per key is reduced over the block queries and pooled along the key axis, a per-KV-head top-k at
+ * the retention ratio r picks the prefix/suffix entries to keep, and the kept K/V rows are gathered
+ * into a compacted cache (Algorithm 1). Every later step of the block (cache_state 2, Algorithm 3)
+ * attends over Concat(K_c, K_n): the compacted cache followed by the block's fresh K/V.
+ *
+ * Conventions for every call
+ *   - All data pointers are DEVICE pointers unless a parameter says "host". The library never
+ *     allocates, frees or keeps a pointer; buffers and workspace belong to the caller.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *     No call synchronises with the host.
+ *   - Layout: the last axis (head_dim, D) is contiguous. The other axes (batch, head, position) are
+ *     addressed through the *_stride arrays of sdllm_desc, given in ELEMENTS. Every base pointer and
+ *     every stride*element_size must be a multiple of 16 bytes.
+ *   - Query head h reads KV head h / G, G = n_q_heads / n_kv_heads.
+ *   - Arguments are validated on the host before anything is launched: a bad argument returns a
+ *     status and launches nothing. Kernels never trap or assert.
+ *   - Positions >= seq_len[i] of sequence i are padding and are ignored.
+ */
+#ifndef SDLLM_H_
+#define SDLLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SDLLM_VERSION 100
+
+typedef enum {
+  SDLLM_OK = 0,
+  SDLLM_ERR_INVALID_ARG = 1, /* null/misaligned pointer, inconsistent shape, even pool window, r outside [0,1] ... */
+  SDLLM_ERR_UNSUPPORTED = 2, /* shape or mode outside what the kernels cover, or not an sm_100 device */
+  SDLLM_ERR_WORKSPACE = 3,   /* workspace NULL or smaller than sdllm_workspace_bytes() */
+  SDLLM_ERR_CUDA = 4,        /* a CUDA runtime call or launch failed */
+  SDLLM_ERR_TIMEOUT = 5      /* reserved: a bounded device-side wait gave up */
+} sdllm_status;
+
+typedef enum { SDLLM_F32 = 0, SDLLM_BF16 = 1 } sdllm_dtype;
+
+/* Saliency of a candidate key (Algorithm 1, "Calculate attention scores").
+ * LOGIT_MEAN: a_c = scale * <Mean(Q_b), k_c>, the pre-softmax score of the paper's equation and pseudocode.
+ * PROB_MEAN : a_c = mean over the block queries of softmax(scale * Q_b K^T)[., c], normalised over all keys. */
+typedef enum { SDLLM_SCORE_LOGIT_MEAN = 0, SDLLM_SCORE_PROB_MEAN = 1 } sdllm_score_kind;
+
+/* Key-axis pooling (Algorithm 1, MaxPool1D with kernel_size = s, padding = s/2, stride 1). AVG is the
+ * paper's AvgPool ablation: padding counts as zero and the divisor is always s. */
+typedef enum { SDLLM_POOL_MAX = 0, SDLLM_POOL_AVG = 1 } sdllm_pool_kind;
+
+/* How many entries are kept and from where.
+ * JOINT_FLOOR     : Algorithm 1 as printed. One top-n over Concat(prefix, suffix), n = floor((L-b)*r);
+ *                   the pooling window runs across the prefix/suffix seam.
+ * PER_REGION_CEIL : ceil(r*o) from the prefix and ceil(r*(L-o-b)) from the suffix, pooled per region.
+ * PREFIX_ONLY     : Algorithm 5 (prefix-sparse). floor(o*r) from the prefix, the whole suffix is kept. */
+typedef enum { SDLLM_SELECT_JOINT_FLOOR = 0, SDLLM_SELECT_PER_REGION_CEIL = 1, SDLLM_SELECT_PREFIX_ONLY = 2 } sdllm_select_mode;
+
+typedef enum {
+  SDLLM_OP_REFRESH_SCORES = 0,
+  SDLLM_OP_SELECT_TOPK = 1,
+  SDLLM_OP_COMPACT_KV = 2,
+  SDLLM_OP_SPARSE_BLOCK_ATTN = 3
+} sdllm_op;
+
+/* Problem description, filled by the caller. Plain data; set struct_size = sizeof(sdllm_desc). */
+typedef struct sdllm_desc {
+  uint32_t struct_size;
+  int32_t batch;        /* B: independent sequences */
+  int32_t n_q_heads;    /* Hq */
+  int32_t n_kv_heads;   /* Hkv, divides Hq */
+  int32_t head_dim;     /* D: 64 or 128 */
+  int32_t seq_len_max;  /* padded length of the position axis of k, v and pooled_scores (>= every seq_len[i]) */
+  int32_t block_len;    /* b: rows of the current decoding block; b * G <= 256 */
+  int32_t dtype;        /* sdllm_dtype of q, k, v, out, k_c, v_c */
+  float softmax_scale;  /* 0 selects 1/sqrt(D) */
+  int32_t pool_window;  /* s: odd, >= 1 */
+  int32_t pool;         /* sdllm_pool_kind */
+  int32_t score;        /* sdllm_score_kind */
+  int32_t select;       /* sdllm_select_mode */
+  int32_t n_keep_max;   /* rows per (sequence, KV head) of kept_idx, k_c and v_c; kept counts are clamped to it */
+  double retention;     /* r in [0, 1] */
+  /* strides in elements for the (batch, head, position) axes */
+  int64_t q_stride[3];   /* q_blk  [B, Hq,  b,          D] */
+  int64_t kv_stride[3];  /* k, v   [B, Hkv, seq_len_max, D] */
+  int64_t o_stride[3];   /* out    [B, Hq,  b,          D] */
+  int64_t c_stride[3];   /* k_c,v_c[B, Hkv, n_keep_max, D] */
+  int64_t blk_stride[3]; /* k_blk,v_blk [B, Hkv, b,     D] */
+} sdllm_desc;
+
+/* Library version (SDLLM_VERSION of the build). */
+int sdllm_version(void);
+
+/* Static, human-readable name of a status code. */
+const char* sdllm_status_string(sdllm_status status);
+
+/* Bytes of device workspace a call of `op` needs for this description (host-only, no GPU needed).
+ * Returns 0 for an invalid description or when the op needs none. The workspace needs 256-byte alignment
+ * and no initialisation; its contents after a call are unspecified. */
+size_t sdllm_workspace_bytes(const sdllm_desc* desc, int op);
+
+/* Host-only. Number of cache entries kept for a sequence of length seq_len whose block starts at block_off:
+ * n = floor(|I| * r) of Algorithm 1 (or the other policies of sdllm_select_mode), products taken in double.
+ * n_total is always written; n_prefix / n_suffix receive the per-region quotas, or -1 when the split is data
+ * dependent (JOINT_FLOOR). Not clamped to n_keep_max. Any output pointer may be NULL. */
+sdllm_status sdllm_keep_count(const sdllm_desc* desc, int32_t seq_len, int32_t block_off, int32_t* n_total,
+                              int32_t* n_prefix, int32_t* n_suffix);
+
+/* Host-only. Cache state of step i within a block for delay step x (Algorithm 2 is x = 1; Algorithm 4 general):
+ * 0 = dense step (cache unused), 1 = refresh (run Algorithm 1), 2 = reuse the compacted cache. */
+int32_t sdllm_cache_state(int32_t step_in_block, int32_t delay);
+
+/* Refresh step, part 1 (cache_state 1; Algorithm 1 up to the importance scores).
+ *   out[i, h, :, :]  = softmax(scale * Q_b K^T) V for the block rows over ALL seq_len[i] keys (prefix+block+suffix)
+ *   lse[i, h, :]     = log-sum-exp of the scaled logits per row            [B, Hq, b] fp32, nullable
+ *   pooled_scores    = importance I after saliency + key-axis pooling      [B, Hkv, seq_len_max] fp32, nullable;
+ *                      indexed by ABSOLUTE position; block positions and padding hold -inf.
+ * `out` may be NULL (scores only). seq_len NULL means every sequence has seq_len_max keys. block_off[i] = o.
+ * The probability matrix is never written to memory. */
+sdllm_status sdllm_refresh_scores(const sdllm_desc* desc, const void* q_blk, const void* k, const void* v,
+                                  const int32_t* seq_len, const int32_t* block_off, void* out, float* lse,
+                                  float* pooled_scores, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Refresh step, part 2 (Algorithm 1, "n <- floor(|I| r)", "TopKIndices"). Per (sequence, KV head): the n
+ * candidates with the largest pooled score; equal scores go to the lower position; written as ascending
+ * absolute positions into kept_idx [B, Hkv, n_keep_max] int32, entries past the count are -1.
+ * kept_cnt [B] int32 receives min(n, n_keep_max) (the same for every head of a sequence). */
+sdllm_status sdllm_select_topk(const sdllm_desc* desc, const float* pooled_scores, const int32_t* seq_len,
+                               const int32_t* block_off, int32_t* kept_idx, int32_t* kept_cnt, void* workspace,
+                               size_t workspace_bytes, void* cuda_stream);
+
+/* Refresh step, part 3 (Algorithm 1, "Select" and the cache store): k_c[i, g, j, :] = k[i, g, kept_idx[i, g, j], :],
+ * same for v, bit-exact. Rows j >= kept_cnt[i] are zero-filled. */
+sdllm_status sdllm_compact_kv(const sdllm_desc* desc, const void* k, const void* v, const int32_t* kept_idx,
+                              const int32_t* kept_cnt, void* k_c, void* v_c, void* cuda_stream);
+
+/* Reuse step (cache_state 2, Algorithm 3): out = softmax(scale * Q_b' [K_c ; K_n]^T) [V_c ; V_n] over the first
+ * kept_cnt[i] rows of the compacted cache followed by the block's b fresh rows k_blk, v_blk. */
+sdllm_status sdllm_sparse_block_attn(const sdllm_desc* desc, const void* q_blk, const void* k_c, const void* v_c,
+                                     const int32_t* kept_cnt, const void* k_blk, const void* v_blk, void* out,
+                                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDLLM_H_ */

@@ -1,0 +1,246 @@
+// C ABI of libsdllm: argument validation, workspace layout and kernel dispatch. Host code only.
+#include <math.h>
+#include <stdlib.h>
+
+#include "common.cuh"
+
+using namespace sdllm;
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int elem_size(int dtype) { return dtype == SDLLM_BF16 ? 2 : 4; }
+
+bool strides_ok(const int64_t* s, int es) {
+  for (int i = 0; i < 3; ++i)
+    if (s[i] < 0 || (s[i] * es) % 16 != 0) return false;
+  return true;
+}
+
+// Shape and policy checks shared by every entry point.
+sdllm_status check_desc(const sdllm_desc* d) {
+  if (d == nullptr || d->struct_size != sizeof(sdllm_desc)) return SDLLM_ERR_INVALID_ARG;
+  if (d->batch < 1 || d->n_q_heads < 1 || d->n_kv_heads < 1 || d->block_len < 1 || d->seq_len_max < 1) return SDLLM_ERR_INVALID_ARG;
+  if (d->n_q_heads % d->n_kv_heads != 0) return SDLLM_ERR_INVALID_ARG;
+  if (d->dtype != SDLLM_F32 && d->dtype != SDLLM_BF16) return SDLLM_ERR_INVALID_ARG;
+  if (d->pool_window < 1 || d->pool_window % 2 == 0) return SDLLM_ERR_INVALID_ARG;
+  if (d->pool != SDLLM_POOL_MAX && d->pool != SDLLM_POOL_AVG) return SDLLM_ERR_INVALID_ARG;
+  if (d->score != SDLLM_SCORE_LOGIT_MEAN && d->score != SDLLM_SCORE_PROB_MEAN) return SDLLM_ERR_INVALID_ARG;
+  if (d->select < SDLLM_SELECT_JOINT_FLOOR || d->select > SDLLM_SELECT_PREFIX_ONLY) return SDLLM_ERR_INVALID_ARG;
+  if (!(d->retention >= 0.0 && d->retention <= 1.0)) return SDLLM_ERR_INVALID_ARG;
+  if (!(d->softmax_scale >= 0.f) || isinf(d->softmax_scale)) return SDLLM_ERR_INVALID_ARG;
+  if (d->n_keep_max < 0 || d->block_len > d->seq_len_max) return SDLLM_ERR_INVALID_ARG;
+  const int es = elem_size(d->dtype);
+  if (!strides_ok(d->q_stride, es) || !strides_ok(d->kv_stride, es) || !strides_ok(d->o_stride, es) ||
+      !strides_ok(d->c_stride, es) || !strides_ok(d->blk_stride, es))
+    return SDLLM_ERR_INVALID_ARG;
+  if (d->head_dim != 64 && d->head_dim != 128) return SDLLM_ERR_UNSUPPORTED;
+  if ((int64_t)d->block_len * (d->n_q_heads / d->n_kv_heads) > kMaxRows) return SDLLM_ERR_UNSUPPORTED;
+  if (d->batch > 65535 || d->n_kv_heads > 65535) return SDLLM_ERR_UNSUPPORTED;
+  if (d->score == SDLLM_SCORE_PROB_MEAN) return SDLLM_ERR_UNSUPPORTED;
+  return SDLLM_OK;
+}
+
+// The kernels are built for sm_100a only.
+sdllm_status check_device() {
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SDLLM_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return SDLLM_ERR_CUDA;
+  return major == 10 ? SDLLM_OK : SDLLM_ERR_UNSUPPORTED;
+}
+
+float scale_of(const sdllm_desc* d) { return d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / sqrtf((float)d->head_dim); }
+
+struct WsLayout {
+  size_t part_o, part_ml, raw, total;
+};
+
+WsLayout attn_ws(const sdllm_desc* d, const AttnPlan& pl, bool scores) {
+  WsLayout w{};
+  const int G = d->n_q_heads / d->n_kv_heads, M = G * d->block_len;
+  size_t off = 0;
+  w.part_o = off;
+  if (pl.splits > 1) off += align_up((size_t)d->batch * d->n_kv_heads * pl.splits * M * d->head_dim * 4, 256);
+  w.part_ml = off;
+  if (pl.splits > 1) off += align_up((size_t)d->batch * d->n_kv_heads * pl.splits * M * 2 * 4, 256);
+  w.raw = off;
+  if (scores) off += align_up((size_t)d->batch * d->n_kv_heads * d->seq_len_max * 4, 256);
+  w.total = off;
+  return w;
+}
+
+AttnPlan plan_for(const sdllm_desc* d, int op) {
+  const int G = d->n_q_heads / d->n_kv_heads;
+  const int n_keys = op == SDLLM_OP_REFRESH_SCORES ? d->seq_len_max : d->n_keep_max + d->block_len;
+  AttnPlan pl = plan_attention(d->dtype, d->head_dim, G * d->block_len, d->batch, d->n_kv_heads, n_keys,
+                               op == SDLLM_OP_REFRESH_SCORES);
+  if (const char* e = getenv("SDLLM_SPLITS")) {   // tuning aid: force the number of key splits
+    const int s = atoi(e);
+    const int n_tiles = (n_keys + pl.key_tile - 1) / pl.key_tile;
+    if (s >= 1) pl.splits = s > kMaxSplits ? kMaxSplits : (s > n_tiles ? n_tiles : s);
+  }
+  return pl;
+}
+
+void fill_common(AttnParams& p, const sdllm_desc* d, const AttnPlan& pl) {
+  p.B = d->batch; p.Hq = d->n_q_heads; p.Hkv = d->n_kv_heads; p.G = p.Hq / p.Hkv; p.b = d->block_len; p.M = p.G * p.b;
+  p.splits = pl.splits;
+  p.scale = scale_of(d);
+  p.scale_log2 = p.scale * kLog2e;
+  for (int i = 0; i < 3; ++i) { p.q_stride[i] = d->q_stride[i]; p.o_stride[i] = d->o_stride[i]; }
+}
+
+}  // namespace
+
+extern "C" {
+
+int sdllm_version(void) { return SDLLM_VERSION; }
+
+const char* sdllm_status_string(sdllm_status s) {
+  switch (s) {
+    case SDLLM_OK: return "ok";
+    case SDLLM_ERR_INVALID_ARG: return "invalid argument";
+    case SDLLM_ERR_UNSUPPORTED: return "unsupported shape, mode or device";
+    case SDLLM_ERR_WORKSPACE: return "workspace missing or too small";
+    case SDLLM_ERR_CUDA: return "CUDA error";
+    case SDLLM_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+size_t sdllm_workspace_bytes(const sdllm_desc* d, int op) {
+  if (check_desc(d) != SDLLM_OK) return 0;
+  if (op == SDLLM_OP_REFRESH_SCORES) return attn_ws(d, plan_for(d, op), true).total;
+  if (op == SDLLM_OP_SPARSE_BLOCK_ATTN) return attn_ws(d, plan_for(d, op), false).total;
+  return 0;
+}
+
+sdllm_status sdllm_keep_count(const sdllm_desc* d, int32_t seq_len, int32_t block_off, int32_t* n_total, int32_t* n_prefix,
+                              int32_t* n_suffix) {
+  const sdllm_status st = check_desc(d);
+  if (st != SDLLM_OK) return st;
+  if (seq_len < d->block_len || block_off < 0 || block_off + d->block_len > seq_len) return SDLLM_ERR_INVALID_ARG;
+  int np, ns;
+  const int nt = keep_count_total(block_off, seq_len - block_off - d->block_len, d->retention, d->select, &np, &ns);
+  if (n_total) *n_total = nt;
+  if (n_prefix) *n_prefix = np;
+  if (n_suffix) *n_suffix = ns;
+  return SDLLM_OK;
+}
+
+int32_t sdllm_cache_state(int32_t i, int32_t delay) { return i > delay ? 2 : (i == delay ? 1 : 0); }
+
+sdllm_status sdllm_refresh_scores(const sdllm_desc* d, const void* q_blk, const void* k, const void* v, const int32_t* seq_len,
+                                  const int32_t* block_off, void* out, float* lse, float* pooled_scores, void* ws, size_t ws_bytes,
+                                  void* cuda_stream) {
+  sdllm_status st = check_desc(d);
+  if (st != SDLLM_OK) return st;
+  if (!q_blk || !k || !v || !block_off || (!out && !pooled_scores)) return SDLLM_ERR_INVALID_ARG;
+  if (!aligned16(q_blk) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(pooled_scores) || !aligned16(lse))
+    return SDLLM_ERR_INVALID_ARG;
+  if (lse && !out) return SDLLM_ERR_INVALID_ARG;
+  const AttnPlan pl = plan_for(d, SDLLM_OP_REFRESH_SCORES);
+  const WsLayout w = attn_ws(d, pl, true);
+  if (w.total > 0 && (ws == nullptr || ws_bytes < w.total || (reinterpret_cast<uintptr_t>(ws) & 255u))) return SDLLM_ERR_WORKSPACE;
+  if ((st = check_device()) != SDLLM_OK) return st;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  char* wsb = reinterpret_cast<char*>(ws);
+
+  AttnParams p{};
+  fill_common(p, d, pl);
+  p.q = q_blk; p.k1 = k; p.v1 = v; p.k2 = nullptr; p.v2 = nullptr;
+  p.n1_per_seq = seq_len; p.block_off = block_off;
+  p.out = out; p.lse = lse;
+  p.part_o = reinterpret_cast<float*>(wsb + w.part_o);
+  p.part_ml = reinterpret_cast<float*>(wsb + w.part_ml);
+  p.raw_scores = pooled_scores ? reinterpret_cast<float*>(wsb + w.raw) : nullptr;
+  p.n1_max = d->seq_len_max; p.n2 = 0;
+  p.want_scores = pooled_scores != nullptr;
+  for (int i = 0; i < 3; ++i) { p.k1_stride[i] = d->kv_stride[i]; p.k2_stride[i] = 0; }
+  if (launch_attn_partial(p, pl, d->dtype, d->head_dim, stream) != cudaSuccess) return SDLLM_ERR_CUDA;
+
+  MergeParams m{};
+  m.part_o = (out && pl.splits > 1) ? p.part_o : nullptr;
+  m.part_ml = p.part_ml; m.out = out; m.lse = lse;
+  m.B = p.B; m.Hq = p.Hq; m.Hkv = p.Hkv; m.G = p.G; m.b = p.b; m.M = p.M; m.D = d->head_dim; m.splits = pl.splits; m.dtype = d->dtype;
+  for (int i = 0; i < 3; ++i) m.o_stride[i] = d->o_stride[i];
+  m.raw_scores = p.raw_scores; m.pooled = pooled_scores; m.seq_len = seq_len; m.block_off = block_off;
+  m.Lmax = d->seq_len_max; m.window = d->pool_window; m.pool_kind = d->pool;
+  m.per_region = d->select != SDLLM_SELECT_JOINT_FLOOR;
+  if (launch_merge_pool(m, stream) != cudaSuccess) return SDLLM_ERR_CUDA;
+  return SDLLM_OK;
+}
+
+sdllm_status sdllm_select_topk(const sdllm_desc* d, const float* pooled_scores, const int32_t* seq_len, const int32_t* block_off,
+                               int32_t* kept_idx, int32_t* kept_cnt, void* ws, size_t ws_bytes, void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  sdllm_status st = check_desc(d);
+  if (st != SDLLM_OK) return st;
+  if (!pooled_scores || !block_off || !kept_idx || !kept_cnt) return SDLLM_ERR_INVALID_ARG;
+  if (!aligned16(pooled_scores) || !aligned16(kept_idx)) return SDLLM_ERR_INVALID_ARG;
+  if ((st = check_device()) != SDLLM_OK) return st;
+  SelectParams p{};
+  p.pooled = pooled_scores; p.seq_len = seq_len; p.block_off = block_off; p.kept_idx = kept_idx; p.kept_cnt = kept_cnt;
+  p.B = d->batch; p.Hkv = d->n_kv_heads; p.Lmax = d->seq_len_max; p.b = d->block_len; p.n_keep_max = d->n_keep_max;
+  p.mode = d->select; p.retention = d->retention;
+  const int cand = d->seq_len_max - d->block_len;
+  p.smem_keys = cand <= 45056 ? cand : 0;
+  if (launch_select_topk(p, reinterpret_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return SDLLM_ERR_CUDA;
+  return SDLLM_OK;
+}
+
+sdllm_status sdllm_compact_kv(const sdllm_desc* d, const void* k, const void* v, const int32_t* kept_idx, const int32_t* kept_cnt,
+                              void* k_c, void* v_c, void* cuda_stream) {
+  sdllm_status st = check_desc(d);
+  if (st != SDLLM_OK) return st;
+  if (!k || !v || !kept_idx || !kept_cnt || !k_c || !v_c) return SDLLM_ERR_INVALID_ARG;
+  if (!aligned16(k) || !aligned16(v) || !aligned16(k_c) || !aligned16(v_c)) return SDLLM_ERR_INVALID_ARG;
+  if ((st = check_device()) != SDLLM_OK) return st;
+  const int es = elem_size(d->dtype);
+  CompactParams p{};
+  p.k = k; p.v = v; p.kept_idx = kept_idx; p.kept_cnt = kept_cnt; p.k_c = k_c; p.v_c = v_c;
+  p.B = d->batch; p.Hkv = d->n_kv_heads; p.n_keep_max = d->n_keep_max; p.row_bytes = d->head_dim * es; p.Lmax = d->seq_len_max;
+  for (int i = 0; i < 3; ++i) { p.kv_stride_bytes[i] = d->kv_stride[i] * es; p.c_stride_bytes[i] = d->c_stride[i] * es; }
+  if (launch_compact(p, reinterpret_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return SDLLM_ERR_CUDA;
+  return SDLLM_OK;
+}
+
+sdllm_status sdllm_sparse_block_attn(const sdllm_desc* d, const void* q_blk, const void* k_c, const void* v_c, const int32_t* kept_cnt,
+                                     const void* k_blk, const void* v_blk, void* out, void* ws, size_t ws_bytes, void* cuda_stream) {
+  sdllm_status st = check_desc(d);
+  if (st != SDLLM_OK) return st;
+  if (!q_blk || !k_blk || !v_blk || !out || !kept_cnt) return SDLLM_ERR_INVALID_ARG;
+  if (d->n_keep_max > 0 && (!k_c || !v_c)) return SDLLM_ERR_INVALID_ARG;
+  if (!aligned16(q_blk) || !aligned16(k_c) || !aligned16(v_c) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out))
+    return SDLLM_ERR_INVALID_ARG;
+  const AttnPlan pl = plan_for(d, SDLLM_OP_SPARSE_BLOCK_ATTN);
+  const WsLayout w = attn_ws(d, pl, false);
+  if (w.total > 0 && (ws == nullptr || ws_bytes < w.total || (reinterpret_cast<uintptr_t>(ws) & 255u))) return SDLLM_ERR_WORKSPACE;
+  if ((st = check_device()) != SDLLM_OK) return st;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  char* wsb = reinterpret_cast<char*>(ws);
+
+  AttnParams p{};
+  fill_common(p, d, pl);
+  p.q = q_blk; p.k1 = k_c ? k_c : k_blk; p.v1 = v_c ? v_c : v_blk; p.k2 = k_blk; p.v2 = v_blk;
+  p.n1_per_seq = kept_cnt; p.block_off = nullptr;
+  p.out = out; p.lse = nullptr;
+  p.part_o = reinterpret_cast<float*>(wsb + w.part_o);
+  p.part_ml = reinterpret_cast<float*>(wsb + w.part_ml);
+  p.raw_scores = nullptr;
+  p.n1_max = d->n_keep_max; p.n2 = d->block_len;
+  p.want_scores = 0;
+  for (int i = 0; i < 3; ++i) { p.k1_stride[i] = d->c_stride[i]; p.k2_stride[i] = d->blk_stride[i]; }
+  if (launch_attn_partial(p, pl, d->dtype, d->head_dim, stream) != cudaSuccess) return SDLLM_ERR_CUDA;
+  if (pl.splits > 1) {
+    MergeParams m{};
+    m.part_o = p.part_o; m.part_ml = p.part_ml; m.out = out; m.lse = nullptr;
+    m.B = p.B; m.Hq = p.Hq; m.Hkv = p.Hkv; m.G = p.G; m.b = p.b; m.M = p.M; m.D = d->head_dim; m.splits = pl.splits; m.dtype = d->dtype;
+    for (int i = 0; i < 3; ++i) m.o_stride[i] = d->o_stride[i];
+    if (launch_merge_pool(m, stream) != cudaSuccess) return SDLLM_ERR_CUDA;
+  }
+  return SDLLM_OK;
+}
+
+}  // extern "C"

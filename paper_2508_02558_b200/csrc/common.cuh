@@ -1,0 +1,103 @@
+// Shared declarations of the libsdllm CUDA sources (sm_100a only).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sdllm.h"
+
+namespace sdllm {
+
+constexpr int kNumSMs = 148;          // B200
+constexpr int kMaxRows = 256;         // b * G rows of one KV head handled by one CTA
+constexpr int kMaxSplits = 64;        // key-axis splits per (sequence, KV head)
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// How one attention launch is cut into CTAs; a pure function of the description so that the workspace
+// query and the launch always agree.
+struct AttnPlan {
+  int key_tile;     // keys per pipeline stage
+  int m_warps;      // warps along the query rows (16 rows each, bf16) / row chunks (32 rows each, fp32)
+  int c_warps;      // warps along the keys of a tile (bf16 only)
+  int stages;       // shared-memory pipeline depth
+  int splits;       // CTAs along the key axis per (sequence, KV head)
+  int threads;
+  size_t smem_bytes;
+};
+
+// Key sources of one attention launch. The virtual key axis is [src1 rows 0..n1) ++ [src2 rows 0..n2).
+// refresh: src1 = full K/V with n1 = seq_len[i], n2 = 0.  reuse: src1 = compacted cache with n1 = kept_cnt[i],
+// src2 = the block's fresh rows with n2 = b.
+struct AttnParams {
+  const void* q;
+  const void* k1; const void* v1;
+  const void* k2; const void* v2;
+  const int32_t* n1_per_seq;   // nullable -> n1_max
+  const int32_t* block_off;    // refresh only
+  void* out;                   // nullable
+  float* lse;                  // nullable
+  float* part_o;               // [B][Hkv][splits][M][D]
+  float* part_ml;              // [B][Hkv][splits][M][2]  (running max in log2 units, running sum)
+  float* raw_scores;           // [B][Hkv][n1_max] or null
+  int B, Hq, Hkv, G, b, M;     // M = G * b rows per KV head
+  int n1_max, n2;
+  int splits;
+  int want_scores;             // compute mean-query logit scores for src1 keys
+  float scale;                 // softmax scale
+  float scale_log2;            // scale * log2(e)
+  int64_t q_stride[3], k1_stride[3], k2_stride[3], o_stride[3];
+};
+
+struct MergeParams {
+  const float* part_o; const float* part_ml;
+  void* out; float* lse;
+  int B, Hq, Hkv, G, b, M, D, splits, dtype;
+  int64_t o_stride[3];
+  int merge_blocks;            // blocks [0, merge_blocks) merge; the rest pool
+  // pooling of raw scores -> pooled scores
+  const float* raw_scores; float* pooled;
+  const int32_t* seq_len; const int32_t* block_off;
+  int Lmax, window, pool_kind, per_region;
+};
+
+struct SelectParams {
+  const float* pooled; const int32_t* seq_len; const int32_t* block_off;
+  int32_t* kept_idx; int32_t* kept_cnt;
+  int B, Hkv, Lmax, b, n_keep_max, mode;
+  double retention;
+  int smem_keys;               // candidates cached in shared memory (0 = read global every pass)
+};
+
+struct CompactParams {
+  const void* k; const void* v; const int32_t* kept_idx; const int32_t* kept_cnt;
+  void* k_c; void* v_c;
+  int B, Hkv, n_keep_max, row_bytes, Lmax;
+  int64_t kv_stride_bytes[3], c_stride_bytes[3];
+};
+
+AttnPlan plan_attention(int dtype, int D, int M, int B, int Hkv, int n_keys_max, bool want_scores);
+
+cudaError_t launch_attn_partial(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st);
+cudaError_t launch_merge_pool(const MergeParams& p, cudaStream_t st);
+cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st);
+cudaError_t launch_compact(const CompactParams& p, cudaStream_t st);
+
+__host__ __device__ inline int keep_count_total(int pre, int suf, double r, int mode, int* n_pre, int* n_suf) {
+  // Algorithm 1: n = floor(|I| * r) in double; the other policies are described in sdllm.h.
+  auto clampll = [](long long x, int hi) { return (int)(x < 0 ? 0 : (x > hi ? hi : x)); };
+  if (mode == SDLLM_SELECT_JOINT_FLOOR) {
+    *n_pre = -1; *n_suf = -1;
+    return clampll((long long)floor((double)(pre + suf) * r), pre + suf);
+  }
+  if (mode == SDLLM_SELECT_PER_REGION_CEIL) {
+    *n_pre = clampll((long long)ceil((double)pre * r), pre);
+    *n_suf = clampll((long long)ceil((double)suf * r), suf);
+    return *n_pre + *n_suf;
+  }
+  *n_pre = clampll((long long)floor((double)pre * r), pre);
+  *n_suf = suf;
+  return *n_pre + *n_suf;
+}
+
+}  // namespace sdllm
