@@ -99,8 +99,9 @@ int sdllm_version(void);
 const char* sdllm_status_string(sdllm_status status);
 
 /* Bytes of device workspace a call of `op` needs for this description (host-only, no GPU needed).
- * Returns 0 for an invalid description or when the op needs none. The workspace needs 256-byte alignment
- * and no initialisation; its contents after a call are unspecified. */
+ * Returns 0 for an invalid description or when the op needs none. The workspace needs 256-byte alignment; its
+ * first 4 bytes are a status word the caller zeroes once (see sdllm_read_status), the rest needs no initialisation
+ * and is unspecified after a call. One workspace may serve any number of calls that run one after another. */
 size_t sdllm_workspace_bytes(const sdllm_desc* desc, int op);
 
 /* Host-only. Number of cache entries kept for a sequence of length seq_len whose block starts at block_off:
@@ -113,6 +114,13 @@ sdllm_status sdllm_keep_count(const sdllm_desc* desc, int32_t seq_len, int32_t b
 /* Host-only. Cache state of step i within a block for delay step x (Algorithm 2 is x = 1; Algorithm 4 general):
  * 0 = dense step (cache unused), 1 = refresh (run Algorithm 1), 2 = reuse the compacted cache. */
 int32_t sdllm_cache_state(int32_t step_in_block, int32_t delay);
+
+/* Reads the device status word kept in the first 4 bytes of an attention workspace. The kernels bound every wait
+ * on a shared-memory barrier; if one ever expires they record a non-zero code there and run to the end instead of
+ * hanging (the outputs of that call are then invalid). The caller zeroes those 4 bytes once after allocating the
+ * workspace. This call copies the word to the host and SYNCHRONISES the stream (the only call that does).
+ * Returns SDLLM_OK when the word is zero, SDLLM_ERR_TIMEOUT otherwise; *device_status receives the raw code. */
+sdllm_status sdllm_read_status(const void* workspace, void* cuda_stream, int32_t* device_status);
 
 /* Refresh step, part 1 (cache_state 1; Algorithm 1 up to the importance scores).
  *   out[i, h, :, :]  = softmax(scale * Q_b K^T) V for the block rows over ALL seq_len[i] keys (prefix+block+suffix)

@@ -21,6 +21,7 @@ SELECT_JOINT_FLOOR, SELECT_PER_REGION_CEIL, SELECT_PREFIX_ONLY = 0, 1, 2
 OP_REFRESH_SCORES, OP_SELECT_TOPK, OP_COMPACT_KV, OP_SPARSE_BLOCK_ATTN = range(4)
 
 EXPORTS = ("sdllm_version", "sdllm_status_string", "sdllm_workspace_bytes", "sdllm_keep_count", "sdllm_cache_state",
+           "sdllm_read_status",
            "sdllm_refresh_scores", "sdllm_select_topk", "sdllm_compact_kv", "sdllm_sparse_block_attn")
 
 
@@ -64,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.sdllm_keep_count.argtypes = [dp, ctypes.c_int32, ctypes.c_int32] + [ctypes.POINTER(ctypes.c_int32)] * 3
         L.sdllm_cache_state.restype = ctypes.c_int32
         L.sdllm_cache_state.argtypes = [ctypes.c_int32, ctypes.c_int32]
+        L.sdllm_read_status.restype = ctypes.c_int
+        L.sdllm_read_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
         L.sdllm_refresh_scores.restype = ctypes.c_int
         L.sdllm_refresh_scores.argtypes = [dp, vp, vp, vp, i32p, i32p, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.sdllm_select_topk.restype = ctypes.c_int
@@ -154,6 +157,15 @@ def keep_count(desc: Desc, seq_len: int, block_off: int):
 
 def cache_state(step_in_block: int, delay: int = 1) -> int:
     return int(lib().sdllm_cache_state(int(step_in_block), int(delay)))
+
+
+def read_status(workspace, stream=None) -> int:
+    """Device status word of a workspace (0 = no bounded wait ever expired). Synchronises the stream."""
+    v = ctypes.c_int32(0)
+    st = lib().sdllm_read_status(_ptr(workspace), _stream(stream), ctypes.byref(v))
+    if st not in (OK, ERR_TIMEOUT):
+        raise SdllmError(st, "sdllm_read_status")
+    return v.value
 
 
 def refresh_scores(desc: Desc, q_blk, k, v, seq_len, block_off, out, lse, pooled_scores, workspace, stream=None):

@@ -1,5 +1,6 @@
 // C ABI of libsdllm: argument validation, workspace layout and kernel dispatch. Host code only.
 #include <math.h>
+#include <stdio.h>
 #include <stdlib.h>
 
 #include "common.cuh"
@@ -50,16 +51,27 @@ sdllm_status check_device() {
   return major == 10 ? SDLLM_OK : SDLLM_ERR_UNSUPPORTED;
 }
 
+// SDLLM_DEBUG=1 prints the CUDA error behind an SDLLM_ERR_CUDA to stderr.
+bool cuda_failed(cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return false;
+  const char* dbg = getenv("SDLLM_DEBUG");
+  if (dbg && dbg[0] == '1') fprintf(stderr, "libsdllm: %s: %s\n", what, cudaGetErrorString(e));
+  (void)cudaGetLastError();
+  return true;
+}
+
 float scale_of(const sdllm_desc* d) { return d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / sqrtf((float)d->head_dim); }
 
 struct WsLayout {
-  size_t part_o, part_ml, raw, total;
+  size_t status, part_o, part_ml, raw, total;
 };
 
 WsLayout attn_ws(const sdllm_desc* d, const AttnPlan& pl, bool scores) {
   WsLayout w{};
   const int G = d->n_q_heads / d->n_kv_heads, M = G * d->block_len;
   size_t off = 0;
+  w.status = off;
+  off += 256;                          // device status word (sdllm_read_status)
   w.part_o = off;
   if (pl.splits > 1) off += align_up((size_t)d->batch * d->n_kv_heads * pl.splits * M * d->head_dim * 4, 256);
   w.part_ml = off;
@@ -72,20 +84,15 @@ WsLayout attn_ws(const sdllm_desc* d, const AttnPlan& pl, bool scores) {
 
 AttnPlan plan_for(const sdllm_desc* d, int op) {
   const int G = d->n_q_heads / d->n_kv_heads;
-  const int n_keys = op == SDLLM_OP_REFRESH_SCORES ? d->seq_len_max : d->n_keep_max + d->block_len;
-  AttnPlan pl = plan_attention(d->dtype, d->head_dim, G * d->block_len, d->batch, d->n_kv_heads, n_keys,
-                               op == SDLLM_OP_REFRESH_SCORES);
-  if (const char* e = getenv("SDLLM_SPLITS")) {   // tuning aid: force the number of key splits
-    const int s = atoi(e);
-    const int n_tiles = (n_keys + pl.key_tile - 1) / pl.key_tile;
-    if (s >= 1) pl.splits = s > kMaxSplits ? kMaxSplits : (s > n_tiles ? n_tiles : s);
-  }
-  return pl;
+  const bool refresh = op == SDLLM_OP_REFRESH_SCORES;
+  return plan_attention(d->dtype, d->head_dim, G * d->block_len, d->batch, d->n_kv_heads,
+                        refresh ? d->seq_len_max : d->n_keep_max, refresh ? 0 : d->block_len);
 }
 
 void fill_common(AttnParams& p, const sdllm_desc* d, const AttnPlan& pl) {
   p.B = d->batch; p.Hq = d->n_q_heads; p.Hkv = d->n_kv_heads; p.G = p.Hq / p.Hkv; p.b = d->block_len; p.M = p.G * p.b;
   p.splits = pl.splits;
+  p.splits_total = pl.splits * pl.cluster;
   p.scale = scale_of(d);
   p.scale_log2 = p.scale * kLog2e;
   for (int i = 0; i < 3; ++i) { p.q_stride[i] = d->q_stride[i]; p.o_stride[i] = d->o_stride[i]; }
@@ -131,6 +138,16 @@ sdllm_status sdllm_keep_count(const sdllm_desc* d, int32_t seq_len, int32_t bloc
 
 int32_t sdllm_cache_state(int32_t i, int32_t delay) { return i > delay ? 2 : (i == delay ? 1 : 0); }
 
+sdllm_status sdllm_read_status(const void* workspace, void* cuda_stream, int32_t* device_status) {
+  if (!workspace || !device_status) return SDLLM_ERR_INVALID_ARG;
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  int32_t v = 0;
+  if (cudaMemcpyAsync(&v, workspace, sizeof(v), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return SDLLM_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return SDLLM_ERR_CUDA;
+  *device_status = v;
+  return v == 0 ? SDLLM_OK : SDLLM_ERR_TIMEOUT;
+}
+
 sdllm_status sdllm_refresh_scores(const sdllm_desc* d, const void* q_blk, const void* k, const void* v, const int32_t* seq_len,
                                   const int32_t* block_off, void* out, float* lse, float* pooled_scores, void* ws, size_t ws_bytes,
                                   void* cuda_stream) {
@@ -152,13 +169,14 @@ sdllm_status sdllm_refresh_scores(const sdllm_desc* d, const void* q_blk, const 
   p.q = q_blk; p.k1 = k; p.v1 = v; p.k2 = nullptr; p.v2 = nullptr;
   p.n1_per_seq = seq_len; p.block_off = block_off;
   p.out = out; p.lse = lse;
+  p.status = reinterpret_cast<int32_t*>(wsb + w.status);
   p.part_o = reinterpret_cast<float*>(wsb + w.part_o);
   p.part_ml = reinterpret_cast<float*>(wsb + w.part_ml);
   p.raw_scores = pooled_scores ? reinterpret_cast<float*>(wsb + w.raw) : nullptr;
   p.n1_max = d->seq_len_max; p.n2 = 0;
   p.want_scores = pooled_scores != nullptr;
   for (int i = 0; i < 3; ++i) { p.k1_stride[i] = d->kv_stride[i]; p.k2_stride[i] = 0; }
-  if (launch_attn_partial(p, pl, d->dtype, d->head_dim, stream) != cudaSuccess) return SDLLM_ERR_CUDA;
+  if (cuda_failed(launch_attn_partial(p, pl, d->dtype, d->head_dim, stream), "attention launch")) return SDLLM_ERR_CUDA;
 
   MergeParams m{};
   m.part_o = (out && pl.splits > 1) ? p.part_o : nullptr;
@@ -168,7 +186,7 @@ sdllm_status sdllm_refresh_scores(const sdllm_desc* d, const void* q_blk, const 
   m.raw_scores = p.raw_scores; m.pooled = pooled_scores; m.seq_len = seq_len; m.block_off = block_off;
   m.Lmax = d->seq_len_max; m.window = d->pool_window; m.pool_kind = d->pool;
   m.per_region = d->select != SDLLM_SELECT_JOINT_FLOOR;
-  if (launch_merge_pool(m, stream) != cudaSuccess) return SDLLM_ERR_CUDA;
+  if (cuda_failed(launch_merge_pool(m, stream), "merge/pool launch")) return SDLLM_ERR_CUDA;
   return SDLLM_OK;
 }
 
@@ -186,7 +204,7 @@ sdllm_status sdllm_select_topk(const sdllm_desc* d, const float* pooled_scores, 
   p.mode = d->select; p.retention = d->retention;
   const int cand = d->seq_len_max - d->block_len;
   p.smem_keys = cand <= 45056 ? cand : 0;
-  if (launch_select_topk(p, reinterpret_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return SDLLM_ERR_CUDA;
+  if (cuda_failed(launch_select_topk(p, reinterpret_cast<cudaStream_t>(cuda_stream)), "select launch")) return SDLLM_ERR_CUDA;
   return SDLLM_OK;
 }
 
@@ -202,7 +220,7 @@ sdllm_status sdllm_compact_kv(const sdllm_desc* d, const void* k, const void* v,
   p.k = k; p.v = v; p.kept_idx = kept_idx; p.kept_cnt = kept_cnt; p.k_c = k_c; p.v_c = v_c;
   p.B = d->batch; p.Hkv = d->n_kv_heads; p.n_keep_max = d->n_keep_max; p.row_bytes = d->head_dim * es; p.Lmax = d->seq_len_max;
   for (int i = 0; i < 3; ++i) { p.kv_stride_bytes[i] = d->kv_stride[i] * es; p.c_stride_bytes[i] = d->c_stride[i] * es; }
-  if (launch_compact(p, reinterpret_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return SDLLM_ERR_CUDA;
+  if (cuda_failed(launch_compact(p, reinterpret_cast<cudaStream_t>(cuda_stream)), "compact launch")) return SDLLM_ERR_CUDA;
   return SDLLM_OK;
 }
 
@@ -226,19 +244,20 @@ sdllm_status sdllm_sparse_block_attn(const sdllm_desc* d, const void* q_blk, con
   p.q = q_blk; p.k1 = k_c ? k_c : k_blk; p.v1 = v_c ? v_c : v_blk; p.k2 = k_blk; p.v2 = v_blk;
   p.n1_per_seq = kept_cnt; p.block_off = nullptr;
   p.out = out; p.lse = nullptr;
+  p.status = reinterpret_cast<int32_t*>(wsb + w.status);
   p.part_o = reinterpret_cast<float*>(wsb + w.part_o);
   p.part_ml = reinterpret_cast<float*>(wsb + w.part_ml);
   p.raw_scores = nullptr;
   p.n1_max = d->n_keep_max; p.n2 = d->block_len;
   p.want_scores = 0;
   for (int i = 0; i < 3; ++i) { p.k1_stride[i] = d->c_stride[i]; p.k2_stride[i] = d->blk_stride[i]; }
-  if (launch_attn_partial(p, pl, d->dtype, d->head_dim, stream) != cudaSuccess) return SDLLM_ERR_CUDA;
+  if (cuda_failed(launch_attn_partial(p, pl, d->dtype, d->head_dim, stream), "attention launch")) return SDLLM_ERR_CUDA;
   if (pl.splits > 1) {
     MergeParams m{};
     m.part_o = p.part_o; m.part_ml = p.part_ml; m.out = out; m.lse = nullptr;
     m.B = p.B; m.Hq = p.Hq; m.Hkv = p.Hkv; m.G = p.G; m.b = p.b; m.M = p.M; m.D = d->head_dim; m.splits = pl.splits; m.dtype = d->dtype;
     for (int i = 0; i < 3; ++i) m.o_stride[i] = d->o_stride[i];
-    if (launch_merge_pool(m, stream) != cudaSuccess) return SDLLM_ERR_CUDA;
+    if (cuda_failed(launch_merge_pool(m, stream), "merge/pool launch")) return SDLLM_ERR_CUDA;
   }
   return SDLLM_OK;
 }

@@ -20,9 +20,12 @@ struct AttnPlan {
   int key_tile;     // keys per pipeline stage
   int m_warps;      // warps along the query rows (16 rows each, bf16) / row chunks (32 rows each, fp32)
   int c_warps;      // warps along the keys of a tile (bf16 only)
+  int warp_keys;    // keys per warp per tile (bf16 TMA kernel: 16, 32 or 64)
   int stages;       // shared-memory pipeline depth
-  int splits;       // CTAs along the key axis per (sequence, KV head)
+  int cluster;      // CTAs of one (sequence, KV head) that merge through distributed shared memory
+  int splits;       // partials per (sequence, KV head) left in the workspace (1 = final output written directly)
   int threads;
+  bool tma;         // bf16 TMA kernel (else the cp.async kernels)
   size_t smem_bytes;
 };
 
@@ -42,7 +45,9 @@ struct AttnParams {
   float* raw_scores;           // [B][Hkv][n1_max] or null
   int B, Hq, Hkv, G, b, M;     // M = G * b rows per KV head
   int n1_max, n2;
-  int splits;
+  int splits;                  // partials per (sequence, KV head) in the workspace
+  int splits_total;            // CTAs along the key axis per (sequence, KV head) = splits * cluster size
+  int32_t* status;             // device status word: set non-zero when a bounded wait gave up
   int want_scores;             // compute mean-query logit scores for src1 keys
   float scale;                 // softmax scale
   float scale_log2;            // scale * log2(e)
@@ -76,7 +81,7 @@ struct CompactParams {
   int64_t kv_stride_bytes[3], c_stride_bytes[3];
 };
 
-AttnPlan plan_attention(int dtype, int D, int M, int B, int Hkv, int n_keys_max, bool want_scores);
+AttnPlan plan_attention(int dtype, int D, int M, int B, int Hkv, int n1_max, int n2);
 
 cudaError_t launch_attn_partial(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st);
 cudaError_t launch_merge_pool(const MergeParams& p, cudaStream_t st);

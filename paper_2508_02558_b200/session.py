@@ -49,7 +49,7 @@ class LayerCache:
         else:
             self.pooled = torch.empty((batch, n_kv_heads, seq_len_max), dtype=torch.float32, device=dev)
             ws = max(B.workspace_bytes(self.desc, op) for op in range(4))
-            self.workspace = torch.empty((max(ws, 256),), dtype=torch.uint8, device=dev)
+            self.workspace = torch.zeros((max(ws, 256),), dtype=torch.uint8, device=dev)   # status word starts at 0
 
     # cache_state 1: dense block attention + Algorithm 1
     def refresh(self, q_blk, k, v, seq_len, block_off, out=None, lse=None, stream=None):

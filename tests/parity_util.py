@@ -74,6 +74,7 @@ def gpu_refresh(q, k, v, seq_len: Sequence[int], block_off: Sequence[int], dtype
     cache.k_c.fill_(float("nan")); cache.v_c.fill_(float("nan"))
     cache.refresh(qd, kd, vd, sl, bo, out=out, lse=lse)
     torch.cuda.synchronize()
+    assert B.read_status(cache.workspace) == 0, "a bounded device-side wait expired"
     return GpuRefresh(cache, to_host_f32(out), lse.cpu().numpy(), cache.pooled.cpu().numpy(),
                       cache.kept_idx.cpu().numpy(), cache.kept_cnt.cpu().numpy(), kd, vd)
 
@@ -150,6 +151,7 @@ def gpu_sparse_step(g: GpuRefresh, q2, kn, vn, dtype: str) -> np.ndarray:
     out = torch.full(q2.shape, float("nan"), dtype=g.cache.tdtype, device=DEV)
     g.cache.sparse_step(qd, knd, vnd, out)
     torch.cuda.synchronize()
+    assert B.read_status(g.cache.workspace) == 0, "a bounded device-side wait expired"
     return to_host_f32(out)
 
 

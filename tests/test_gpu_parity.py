@@ -108,6 +108,16 @@ def test_pool_windows(window):
     assert stats["set_mismatch"] == 0
 
 
+@pytest.mark.parametrize("env", [{"SDLLM_NO_TMA": "1"}, {"SDLLM_CLUSTER": "1", "SDLLM_SPLITS": "3"}, {"SDLLM_PDL": "0"},
+                                 {"SDLLM_SPLITS": "7"}, {"SDLLM_SPLITS": "1"}])
+def test_alternative_launch_plans_agree_with_oracle(env, monkeypatch):
+    """The cp.async kernel, the global-workspace merge (no cluster), and other split counts give the same answers."""
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    _run_sequence_case(_small("alt_mha", "bf16", 4, 4, 128, 403, 130, salient_frac=0.02), seed=12, block=1)
+    _run_sequence_case(_small("alt_gqa", "bf16", 8, 2, 128, 300, 64, retention=0.3, salient_frac=0.02), seed=13, block=0)
+
+
 def test_ragged_batch():
     import parity_util as U
     cfg = _small("rag", "bf16", 4, 4, 128, 64, 64, salient_frac=0.02)
