@@ -76,7 +76,7 @@ def attention(q, k, v, scale: Optional[float] = None, return_probs: bool = False
 
 
 def scores_logit_mean(q, k, block_off: int, scale: Optional[float] = None, matrix_form: bool = False) -> np.ndarray:
-    """Mean-query logit saliency over the candidates (Algorithm 1 lines 4-6). Returns [Hkv, L-b]."""
+    """Mean-query logit saliency over the candidates (Algorithm 1, steps "Mean(Q_b)" and "MatMul(qbar, K_f^T)"). Returns [Hkv, L-b]."""
     q, k = _f64(q), _f64(k)
     Hq, b, D = q.shape
     Hkv, L, _ = k.shape
@@ -97,7 +97,7 @@ def scores_prob_mean(probs, n_kv_heads: int, block_off: int) -> np.ndarray:
 
 
 def pool(a, window: int, kind: int = POOL_MAX, seam: int = -1) -> np.ndarray:
-    """Key-axis pooling with stride 1 and padding window//2 (Algorithm 1 line 7). a [Hkv, C]."""
+    """Key-axis pooling with stride 1 and padding window//2 (Algorithm 1, step "MaxPool1D"). a [Hkv, C]."""
     a = _f64(a)
     out = np.empty_like(a)
     _check(lib().orc_pool(_dp(a), a.shape[0], a.shape[1], int(window), int(kind), int(seam), _dp(out)), "pool")
@@ -106,7 +106,7 @@ def pool(a, window: int, kind: int = POOL_MAX, seam: int = -1) -> np.ndarray:
 
 def keep_count(seq_len: int, block_len: int, block_off: int, retention: float,
                mode: int = SELECT_JOINT_FLOOR) -> Tuple[int, int, int]:
-    """(n_total, n_prefix, n_suffix); quotas are -1 in joint mode (Algorithm 1 line 8)."""
+    """(n_total, n_prefix, n_suffix); quotas are -1 in joint mode (Algorithm 1, step "n <- floor(|I| r)")."""
     n = [ctypes.c_int(0) for _ in range(3)]
     _check(lib().orc_keep_count(int(seq_len), int(block_len), int(block_off), ctypes.c_double(retention), int(mode),
                                 *[ctypes.byref(x) for x in n]), "keep_count")

@@ -32,7 +32,7 @@ const double kNegInf = -std::numeric_limits<double>::infinity();
 extern "C" {
 
 // Softmax attention of the block queries over nk keys (Section 3.3 / Appendix A.2: the refresh step
-// still performs bidirectional attention; Algorithm 3 lines for cache_state 2 attend over Concat(K_c, K_n)).
+// still performs bidirectional attention; Algorithm 3 at cache_state 2 attends over Concat(K_c, K_n)).
 //   S_ij = scale * <q_i, k_j>,  P = row-softmax(S),  out_i = sum_j P_ij v_j,  lse_i = log sum_j exp(S_ij)
 // out [Hq][b][D]; lse [Hq][b] (nullable); probs [Hq][b][nk] (nullable).
 int orc_attention(const double* q, const double* k, const double* v, int Hq, int Hkv, int b, int nk, int D,
@@ -69,11 +69,11 @@ int orc_attention(const double* q, const double* k, const double* v, int Hq, int
   return 0;
 }
 
-// Candidate position map of Algorithm 1 lines 1-3: K_f = Concat(K[:o], K[o+b:]); candidate c sits at
+// Candidate position map of Algorithm 1 ("extract the candidates"): K_f = Concat(K[:o], K[o+b:]); candidate c sits at
 // absolute position c (prefix) or c + b (suffix).
 int orc_candidate_pos(int c, int o, int b) { return c < o ? c : c + b; }
 
-// Saliency of Algorithm 1 lines 4-6 with the 1/sqrt(d_k) of the body's attention-score equation:
+// Saliency of Algorithm 1 ("Mean(Q_b)", "MatMul(qbar, K_f^T)") with the 1/sqrt(d_k) of the body's attention-score equation:
 //   qbar_g = Mean over the b*G block queries of KV head g;   a[g][c] = scale * <qbar_g, K_f[g][c]>
 // k is the full-sequence K [Hkv][L][D]; a is [Hkv][L-b].
 int orc_scores_logit_mean(const double* q, const double* k, int Hq, int Hkv, int b, int L, int D, int o,
@@ -137,7 +137,7 @@ int orc_scores_prob_mean(const double* probs, int Hq, int Hkv, int b, int L, int
   return 0;
 }
 
-// Algorithm 1 line 7: I = Pool1D(A, kernel_size = s, padding = s/2), stride 1, odd s, so |I| = |A|.
+// Algorithm 1, pooling step: I = Pool1D(A, kernel_size = s, padding = s/2), stride 1, odd s, so |I| = |A|.
 // kind 0: max pooling, padding acts as -inf. kind 1: average pooling, padding counts as zeros and the
 // divisor is always s (the default behaviour of a framework AvgPool1d).
 // seam < 0: one window axis over all C candidates (the literal Concat reading: the last prefix key and the
@@ -161,7 +161,7 @@ int orc_pool(const double* a, int Hkv, int C, int s, int kind, int seam, double*
   return 0;
 }
 
-// Algorithm 1 line 8 (n = floor(|I| * r)) and the two other counting policies.
+// Algorithm 1, count step (n = floor(|I| * r)) and the two other counting policies.
 //   mode 0 joint     : n_total = floor((L-b) * r); quotas are data dependent (-1).
 //   mode 1 per region: ceil(r * o) from the prefix, ceil(r * (L-o-b)) from the suffix.
 //   mode 2 prefix only (Algorithm 5): floor(o * r) from the prefix, the whole suffix.
@@ -187,7 +187,7 @@ int orc_keep_count(int L, int b, int o, double r, int mode, int* n_total, int* n
   return 0;
 }
 
-// Algorithm 1 line 9: TopKIndices(I, n) on one head's scores x[0..C). Ties go to the lowest index; the
+// Algorithm 1, selection step: TopKIndices(I, n) on one head's scores x[0..C). Ties go to the lowest index; the
 // result is returned in ascending index order. Done as a full stable sort by descending score.
 int orc_select_topk(const double* x, int C, int n, int32_t* idx_out) {
   if (n < 0 || n > C) return 1;
@@ -200,7 +200,7 @@ int orc_select_topk(const double* x, int C, int n, int32_t* idx_out) {
   return 0;
 }
 
-// Algorithm 1 lines 10-12: K_c = Select(K, idx) for one tensor; src [Hkv][L][D], idx [Hkv][n] absolute
+// Algorithm 1, Select and cache store: K_c = Select(K, idx) for one tensor; src [Hkv][L][D], idx [Hkv][n] absolute
 // positions, dst [Hkv][n][D]. Element size is given in bytes so the copy is bit-exact for any dtype.
 int orc_gather_rows(const void* src, const int32_t* idx, int Hkv, int L, int n, size_t row_bytes, void* dst) {
   for (int g = 0; g < Hkv; ++g)

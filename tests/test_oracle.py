@@ -72,7 +72,7 @@ def test_attention_invariants():
         np.testing.assert_allclose(out0[h], np.broadcast_to(v[h // 2].mean(0), (b, D)), atol=1e-13)
 
 
-# ------------------------------------------------------------------ saliency score (Algorithm 1 lines 4-6)
+# ------------------------------------------------------------------ saliency score (Algorithm 1, mean query and score)
 def test_scores_linearity_two_evaluation_orders():
     Hq, Hkv, b, L, D, o = 6, 2, 4, 29, 16, 10
     q, k = _rand((Hq, b, D), 11), _rand((Hkv, L, D), 12)
@@ -129,7 +129,7 @@ def test_scores_prob_mean_mass():
     np.testing.assert_allclose(oracle.scores_prob_mean(pu, Hkv, o), 1.0 / L, atol=1e-15)
 
 
-# ------------------------------------------------------------------ pooling (Algorithm 1 line 7)
+# ------------------------------------------------------------------ pooling (Algorithm 1, MaxPool1D)
 @pytest.mark.parametrize("s", [1, 3, 5, 7, 9])
 def test_pool_matches_library(s):
     a = _rand((3, 41), 20 + s)
@@ -163,7 +163,7 @@ def test_pool_invariants():
         oracle.pool(a, 4)
 
 
-# ------------------------------------------------------------------ counts (Algorithm 1 line 8; k = (L-b) x r)
+# ------------------------------------------------------------------ counts (Algorithm 1, n = floor(|I| r); Section 3.3.1, k = (L-b) x r)
 def test_keep_counts_golden():
     rows = [l.split("#")[0].split() for l in open(os.path.join(GOLD, "keep_counts.txt")) if l.split("#")[0].strip()]
     assert len(rows) >= 8
@@ -184,7 +184,7 @@ def test_keep_count_edges():
         oracle.keep_count(256, 32, 10, 1.5)
 
 
-# ------------------------------------------------------------------ selection (Algorithm 1 line 9)
+# ------------------------------------------------------------------ selection (Algorithm 1, TopKIndices)
 def test_select_matches_library_stable_sort_and_tie_rule():
     rng = np.random.default_rng(40)
     for C, n in [(1, 0), (1, 1), (7, 3), (64, 64), (257, 100), (1000, 1)]:
@@ -219,7 +219,7 @@ def test_select_monotone_in_retention():
         prev = cur
 
 
-# ------------------------------------------------------------------ gather (Algorithm 1 lines 10-12)
+# ------------------------------------------------------------------ gather (Algorithm 1, Select)
 def test_gather_is_fancy_indexing_bit_exact():
     rng = np.random.default_rng(50)
     src32 = rng.standard_normal((3, 37, 8)).astype(np.float32)
