@@ -551,6 +551,8 @@ cudaError_t launch_inst(const TmaMaps& tm, const AttnParams& p, const AttnPlan& 
   if (pl.smem_bytes > configured) {
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
     if (e != cudaSuccess) return e;
+    // ask for the largest shared-memory carve-out so that two CTAs of the small-row shapes fit on one SM
+    (void)cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     configured = pl.smem_bytes;
   }
   cudaLaunchConfig_t cfg{};
@@ -623,7 +625,7 @@ AttnPlan plan_attention(int dtype, int D, int M, int B, int Hkv, int n1_max, int
   if (total > tiles) total = tiles;
   if (total < 1) total = 1;
   if (total > 8 * kMaxSplits) total = 8 * kMaxSplits;
-  int max_cluster = 8;
+  int max_cluster = 1;   // merging through the workspace measured faster than cluster launches on every shape tried
   if (const char* e = getenv("SDLLM_CLUSTER")) { if (atoi(e) >= 1 && atoi(e) <= 8) max_cluster = atoi(e); }
   const int outer = (int)((total + max_cluster - 1) / max_cluster);
   pl.cluster = (int)((total + outer - 1) / outer);
