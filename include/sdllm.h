@@ -99,9 +99,10 @@ int sdllm_version(void);
 const char* sdllm_status_string(sdllm_status status);
 
 /* Bytes of device workspace a call of `op` needs for this description (host-only, no GPU needed).
- * Returns 0 for an invalid description or when the op needs none. The workspace needs 256-byte alignment; its
- * first 4 bytes are a status word the caller zeroes once (see sdllm_read_status), the rest needs no initialisation
- * and is unspecified after a call. One workspace may serve any number of calls that run one after another. */
+ * Returns 0 for an invalid description or when the op needs none. The workspace needs 256-byte alignment and the
+ * caller zeroes ALL of it once after allocating it: its first 4 bytes are a status word (see sdllm_read_status) and
+ * it holds completion counters that every call leaves at zero again; the rest is unspecified after a call. One
+ * workspace may serve any number of calls that run one after another on the GPU, never two that overlap. */
 size_t sdllm_workspace_bytes(const sdllm_desc* desc, int op);
 
 /* Host-only. Number of cache entries kept for a sequence of length seq_len whose block starts at block_off:

@@ -63,7 +63,7 @@ bool cuda_failed(cudaError_t e, const char* what) {
 float scale_of(const sdllm_desc* d) { return d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / sqrtf((float)d->head_dim); }
 
 struct WsLayout {
-  size_t status, part_o, part_ml, raw, total;
+  size_t status, counters, part_o, part_ml, raw, total;
 };
 
 WsLayout attn_ws(const sdllm_desc* d, const AttnPlan& pl, bool scores) {
@@ -71,11 +71,14 @@ WsLayout attn_ws(const sdllm_desc* d, const AttnPlan& pl, bool scores) {
   const int G = d->n_q_heads / d->n_kv_heads, M = G * d->block_len;
   size_t off = 0;
   w.status = off;
+  (void)M;
   off += 256;                          // device status word (sdllm_read_status)
+  w.counters = off;                    // completion counters: zero between calls
+  off += align_up(pl.n_counters * 4, 256);
   w.part_o = off;
-  if (pl.splits > 1) off += align_up((size_t)d->batch * d->n_kv_heads * pl.splits * M * d->head_dim * 4, 256);
+  off += align_up((size_t)d->batch * d->n_kv_heads * pl.part_rows * d->head_dim * 4, 256);
   w.part_ml = off;
-  if (pl.splits > 1) off += align_up((size_t)d->batch * d->n_kv_heads * pl.splits * M * 2 * 4, 256);
+  off += align_up((size_t)d->batch * d->n_kv_heads * pl.part_rows * 2 * 4, 256);
   w.raw = off;
   if (scores) off += align_up((size_t)d->batch * d->n_kv_heads * d->seq_len_max * 4, 256);
   w.total = off;
@@ -85,7 +88,7 @@ WsLayout attn_ws(const sdllm_desc* d, const AttnPlan& pl, bool scores) {
 AttnPlan plan_for(const sdllm_desc* d, int op) {
   const int G = d->n_q_heads / d->n_kv_heads;
   const bool refresh = op == SDLLM_OP_REFRESH_SCORES;
-  return plan_attention(d->dtype, d->head_dim, G * d->block_len, d->batch, d->n_kv_heads,
+  return plan_attention(d->dtype, d->head_dim, G * d->block_len, d->block_len, d->batch, d->n_kv_heads,
                         refresh ? d->seq_len_max : d->n_keep_max, refresh ? 0 : d->block_len);
 }
 
@@ -175,8 +178,12 @@ sdllm_status sdllm_refresh_scores(const sdllm_desc* d, const void* q_blk, const 
   p.raw_scores = pooled_scores ? reinterpret_cast<float*>(wsb + w.raw) : nullptr;
   p.n1_max = d->seq_len_max; p.n2 = 0;
   p.want_scores = pooled_scores != nullptr;
+  p.counters = reinterpret_cast<int32_t*>(wsb + w.counters);
+  p.pooled = pooled_scores; p.window = d->pool_window; p.pool_kind = d->pool;
+  p.per_region = d->select != SDLLM_SELECT_JOINT_FLOOR;
   for (int i = 0; i < 3; ++i) { p.k1_stride[i] = d->kv_stride[i]; p.k2_stride[i] = 0; }
   if (cuda_failed(launch_attn_partial(p, pl, d->dtype, d->head_dim, stream), "attention launch")) return SDLLM_ERR_CUDA;
+  if (pl.fused_tail) return SDLLM_OK;
 
   MergeParams m{};
   m.part_o = (out && pl.splits > 1) ? p.part_o : nullptr;
@@ -250,9 +257,11 @@ sdllm_status sdllm_sparse_block_attn(const sdllm_desc* d, const void* q_blk, con
   p.raw_scores = nullptr;
   p.n1_max = d->n_keep_max; p.n2 = d->block_len;
   p.want_scores = 0;
+  p.counters = reinterpret_cast<int32_t*>(wsb + w.counters);
+  p.pooled = nullptr;
   for (int i = 0; i < 3; ++i) { p.k1_stride[i] = d->c_stride[i]; p.k2_stride[i] = d->blk_stride[i]; }
   if (cuda_failed(launch_attn_partial(p, pl, d->dtype, d->head_dim, stream), "attention launch")) return SDLLM_ERR_CUDA;
-  if (pl.splits > 1) {
+  if (pl.splits > 1 && !pl.fused_tail) {
     MergeParams m{};
     m.part_o = p.part_o; m.part_ml = p.part_ml; m.out = out; m.lse = nullptr;
     m.B = p.B; m.Hq = p.Hq; m.Hkv = p.Hkv; m.G = p.G; m.b = p.b; m.M = p.M; m.D = d->head_dim; m.splits = pl.splits; m.dtype = d->dtype;

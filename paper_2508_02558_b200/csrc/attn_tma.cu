@@ -26,6 +26,9 @@ using namespace dev;
 size_t attn_legacy_smem_bytes(int dtype, int D, const AttnPlan& plan);
 AttnPlan plan_attention_legacy(int dtype, int D, int M, int B, int Hkv, int n_keys_max);
 cudaError_t launch_attn_legacy(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st);
+bool umma_supported(int dtype, int D, int M, int b);
+AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, int n2);
+cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cudaStream_t st);
 
 namespace {
 
@@ -595,15 +598,28 @@ cudaError_t launch_tma_d(const TmaMaps& tm, const AttnParams& p, const AttnPlan&
 
 }  // namespace
 
-AttnPlan plan_attention(int dtype, int D, int M, int B, int Hkv, int n1_max, int n2) {
+// Partial rows the mma.sync kernels leave per (sequence, KV head).
+static void finish_plan(AttnPlan& pl, int M) {
+  pl.part_rows = pl.splits > 1 ? (size_t)pl.splits * M : 0;
+  pl.n_counters = 0; pl.fused_tail = false;
+  pl.rep = 1; pl.row_tiles = 1; pl.parts = pl.splits; pl.rows_rep = M; pl.key_tile2 = pl.key_tile;
+}
+
+AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_max, int n2) {
+  // SDLLM_KERNEL = cpasync | tma | umma picks a kernel family for bf16 (tuning and test aid); default: tcgen05 where it applies
+  const char* kern = getenv("SDLLM_KERNEL");
   const char* no_tma = getenv("SDLLM_NO_TMA");
-  if (dtype != SDLLM_BF16 || (no_tma && no_tma[0] == '1') || encode_fn() == nullptr) {
+  const bool want_cpasync = (no_tma && no_tma[0] == '1') || (kern && kern[0] == 'c');
+  const bool want_tma = kern && kern[0] == 't';
+  if (dtype != SDLLM_BF16 || want_cpasync || encode_fn() == nullptr) {
     AttnPlan pl = plan_attention_legacy(dtype, D, M, B, Hkv, n1_max + n2);
-    pl.tma = false; pl.cluster = 1; pl.warp_keys = 32;
+    pl.tma = false; pl.cluster = 1; pl.warp_keys = 32; pl.kind = 0;
+    finish_plan(pl, M);
     return pl;
   }
+  if (!want_tma && umma_supported(dtype, D, M, b)) return plan_attention_umma(D, M, b, B, Hkv, n1_max, n2);
   AttnPlan pl{};
-  pl.tma = true;
+  pl.tma = true; pl.kind = 1;
   pl.m_warps = (M + 15) / 16;
   if (pl.m_warps <= 2) { pl.c_warps = 8 / pl.m_warps; pl.warp_keys = 16; }        // 8 warps, 64- or 128-key tiles
   else if (pl.m_warps <= 4) { pl.c_warps = 2; pl.warp_keys = 32; }                // 6-8 warps, 64-key tiles
@@ -631,10 +647,12 @@ AttnPlan plan_attention(int dtype, int D, int M, int B, int Hkv, int n1_max, int
   pl.cluster = (int)((total + outer - 1) / outer);
   pl.splits = outer;
   pl.smem_bytes = tma_smem_bytes(D, pl);
+  finish_plan(pl, M);
   return pl;
 }
 
 cudaError_t launch_attn_partial(const AttnParams& p_in, const AttnPlan& plan, int dtype, int D, cudaStream_t st) {
+  if (plan.kind == 2) return launch_attn_umma(p_in, plan, D, st);
   if (!plan.tma) return launch_attn_legacy(p_in, plan, dtype, D, st);
   AttnParams p = p_in;
   TmaMaps tm;

@@ -359,3 +359,416 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
       }
     }
   } else if (warp < 6) {
+    // ======================================= softmax warps =======================================
+    if (do_attn) {
+      const int q4 = warp & 3;                         // TMEM lane quadrant this warp may access
+      const int row = q4 * 32 + lane;
+      const int rep = row / rows_rep;                  // warp-uniform
+      const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16);
+      const int chunk_keys = KT / R;                   // key slice of a tile owned by this replica
+#pragma unroll
+      for (int d = 0; d < D; ++d) o_reg[d] = 0.f;
+      float alpha_prev = 1.f;
+      int it = 0;
+      bool ok = true;
+      auto accumulate = [&](int j, float alpha) -> bool {
+        const int ob = j & 1;
+        if (!wait_bar_warp(BAR(O_FULL + ob), (j >> 1) & 1, abort_flag, p.status, 8)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(lane_addr + 256u + (uint32_t)ob * 128u + c * 32, v);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o_reg[c * 32 + i] = fmaf(o_reg[c * 32 + i], alpha, __uint_as_float(v[i]));
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(O_FREE + ob));
+        return true;
+      };
+      for (int t = t_begin; t < t_end && ok; ++t) {
+        const Tile x = tile_of(t, tiles1, KT, KT2, n1, n2);
+        if (x.nv == 0) continue;
+        const int s = it % NS, sb = it & 1;
+        // columns of this tile owned by this replica
+        const int c_lo = min(rep * chunk_keys, x.nv), c_hi = min((rep + 1) * chunk_keys, x.nv);
+        if (!wait_bar_warp(BAR(S_FULL + sb), (it >> 1) & 1, abort_flag, p.status, 9)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t s_addr = lane_addr + (uint32_t)sb * 128u;
+        // ---- pass 1: row maximum over the owned, valid columns ----
+        float mx = -INFINITY;
+        for (int c0 = 0; c0 < x.n_mma; c0 += 32) {
+          if (c0 >= c_hi || c0 + 32 <= c_lo) continue;
+          uint32_t v[32];
+          tmem_ld32(s_addr + c0, v);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (c0 + i >= c_lo && c0 + i < c_hi) mx = fmaxf(mx, __uint_as_float(v[i]));
+        }
+        const float m_new = fmaxf(m_run, mx * p.scale_log2);
+        const float mu = (m_new == -INFINITY) ? 0.f : m_new;
+        const float alpha = fast_exp2(m_run - mu);
+        m_run = m_new;
+        // ---- pass 2: P = exp2(S * scale_log2 - mu) as bf16 over the S columns; zero outside the owned slice ----
+        float psum = 0.f;
+        for (int c0 = 0; c0 < x.n_mma; c0 += 32) {
+          uint32_t pk[16];
+          if (c0 >= c_hi || c0 + 32 <= c_lo) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+          } else {
+            uint32_t v[32];
+            tmem_ld32(s_addr + c0, v);
+            tc_wait_ld();
+            float e[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const bool in = c0 + i >= c_lo && c0 + i < c_hi;
+              e[i] = in ? fast_exp2(fmaf(__uint_as_float(v[i]), p.scale_log2, -mu)) : 0.f;
+              psum += e[i];
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(e[2 * i], e[2 * i + 1]);
+          }
+          tmem_st16(s_addr + (c0 >> 1), pk);
+        }
+        l_run = fmaf(l_run, alpha, psum);
+        // ---- V rows past the source's count may hold anything: zero them so that 0 * V stays 0 ----
+        if (x.nv < x.n_mma) {
+          if (!wait_bar_warp(BAR(FULL_V + s), (it / NS) & 1, abort_flag, p.status, 10)) { ok = false; break; }
+          unsigned char* vs = stage0 + (size_t)s * stage_bytes + kv_bytes;
+          const int nz = (x.n_mma - x.nv) * H * 8;     // 16-byte chunks to clear
+          for (int i = (warp - 2) * 32 + lane; i < nz; i += 128) {
+            const int rr = x.nv + i / (H * 8), c = i % (H * 8);
+            *reinterpret_cast<uint4*>(vs + (c >> 3) * half_bytes + rr * 128 + (((c & 7) ^ (rr & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+          }
+          fence_proxy_async();
+        }
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(P_FULL + sb));
+        if (it > 0 && !accumulate(it - 1, alpha_prev)) { ok = false; break; }
+        alpha_prev = alpha;
+        ++it;
+      }
+      if (ok && it > 0) ok = accumulate(it - 1, alpha_prev);
+    }
+  } else {
+    // ======================================= saliency warps (refresh) =======================================
+    if (do_scores) {
+      // qbar <- Mean(Q_b) over the b*G rows of the KV head, fp32, fixed order
+      for (int d = tid - 192; d < D; d += 64) {
+        float acc = 0.f;
+        for (int hg = 0; hg < p.G; ++hg) {
+          const __nv_bfloat16* qh = reinterpret_cast<const __nv_bfloat16*>(p.q) + (int64_t)bi * p.q_stride[0] +
+                                    (int64_t)(g * p.G + hg) * p.q_stride[1];
+          for (int i = 0; i < p.b; ++i) acc += __bfloat162float(qh[(int64_t)i * p.q_stride[2] + d]);
+        }
+        qbar_s[d] = acc / (float)p.M;
+      }
+      asm volatile("bar.sync 1, 64;\n" ::: "memory");
+      const int l8 = lane & 7;
+      int it = 0;
+      for (int t = t_begin; t < t_end; ++t) {
+        const Tile x = tile_of(t, tiles1, KT, KT2, n1, n2);
+        if (x.nv == 0) continue;
+        const int s = it % NS;
+        if (!wait_bar_warp(BAR(FULL_K + s), (it / NS) & 1, abort_flag, p.status, 11)) break;
+        if (x.src1) {
+          const unsigned char* kst = stage0 + (size_t)s * stage_bytes;
+          for (int k0 = (warp - 6) * 4; k0 < x.nv; k0 += 8) {      // warp-uniform trip count: the shuffles need all lanes
+            const int kk = k0 + (lane >> 3);                       // < KT always; rows past nv are computed and dropped
+            float acc = 0.f;
+#pragma unroll
+            for (int h = 0; h < H; ++h) {
+              const uint4 raw = *reinterpret_cast<const uint4*>(kst + h * half_bytes + kk * 128 + ((l8 ^ (kk & 7)) << 4));
+              const float4 qa = *reinterpret_cast<const float4*>(qbar_s + h * 64 + l8 * 8);
+              const float4 qb = *reinterpret_cast<const float4*>(qbar_s + h * 64 + l8 * 8 + 4);
+              const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+              float2 f;
+              f = __bfloat1622float2(h2[0]); acc = fmaf(qa.x, f.x, acc); acc = fmaf(qa.y, f.y, acc);
+              f = __bfloat1622float2(h2[1]); acc = fmaf(qa.z, f.x, acc); acc = fmaf(qa.w, f.y, acc);
+              f = __bfloat1622float2(h2[2]); acc = fmaf(qb.x, f.x, acc); acc = fmaf(qb.y, f.y, acc);
+              f = __bfloat1622float2(h2[3]); acc = fmaf(qb.z, f.x, acc); acc = fmaf(qb.w, f.y, acc);
+            }
+            acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+            acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+            acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+            if (l8 == 0 && kk < x.nv) p.raw_scores[(int64_t)(bi * p.Hkv + g) * p.n1_max + x.row0 + kk] = acc * p.scale;
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(EMPTY_K + s));
+        ++it;
+      }
+    }
+  }
+
+  // ======================================= epilogue =======================================
+  const int64_t unit = (int64_t)(bi * p.Hkv + g) * up.row_tiles + rt;      // (sequence, KV head, row tile)
+  if (do_attn && warp >= 2 && warp < 6) {
+    const int row = (warp & 3) * 32 + lane;
+    const int rep = row / rows_rep, m_local = row - rep * rows_rep;
+    if (m_local < M_rt && !*abort_flag) {
+      const int m = rt * 128 + m_local;                // row within the KV head: m = head_in_group * b + i
+      const int hg = m / p.b, i = m - hg * p.b;
+      if (up.parts == 1) {
+        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
+                           (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2];
+#pragma unroll
+        for (int d = 0; d < D; d += 8) {
+          uint4 w;
+          w.x = pack_bf16(o_reg[d] * inv, o_reg[d + 1] * inv);
+          w.y = pack_bf16(o_reg[d + 2] * inv, o_reg[d + 3] * inv);
+          w.z = pack_bf16(o_reg[d + 4] * inv, o_reg[d + 5] * inv);
+          w.w = pack_bf16(o_reg[d + 6] * inv, o_reg[d + 7] * inv);
+          *reinterpret_cast<uint4*>(o + d) = w;
+        }
+        if (p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (m_run + log2f(l_run)) * kLn2;
+      } else {
+        const int64_t prow = (unit * up.parts + split * R + rep) * rows_rep + m_local;
+        float* o = p.part_o + prow * D;
+#pragma unroll
+        for (int d = 0; d < D; d += 4)
+          *reinterpret_cast<float4*>(o + d) = make_float4(o_reg[d], o_reg[d + 1], o_reg[d + 2], o_reg[d + 3]);
+        reinterpret_cast<float2*>(p.part_ml)[prow] = make_float2(m_run, l_run);
+      }
+    }
+  }
+
+  // ---- the last CTA of the unit merges the partials and pools the saliency; nobody waits for anybody ----
+  const bool need_counter = p.splits > 1;
+  const bool have_tail = (do_attn && up.parts > 1) || (do_scores && p.pooled != nullptr);
+  if (have_tail) {
+    __threadfence();
+    tc_fence_before();
+    __syncthreads();
+    if (need_counter) {
+      if (tid == 0) {
+        const int old = atomicAdd(p.counters + unit, 1);
+        *last_flag = (old == p.splits - 1) ? 1 : 0;
+      }
+      __syncthreads();
+    }
+    const bool last = need_counter ? (*last_flag != 0) : true;
+    if (last && !*abort_flag) {
+      __threadfence();
+      if (do_attn && up.parts > 1) {
+        constexpr int D4 = D / 4;
+        const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + unit * up.parts * rows_rep;
+        const float* po = p.part_o + unit * up.parts * rows_rep * D;
+        for (int m_local = warp; m_local < M_rt; m_local += UM_THREADS / 32) {
+          float mstar = -INFINITY;
+          for (int pi = lane; pi < up.parts; pi += 32) {
+            const float2 x = __ldcg(ml + (int64_t)pi * rows_rep + m_local);
+            if (x.y > 0.f) mstar = fmaxf(mstar, x.x);
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, o));
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          float l = 0.f;
+          for (int pi = 0; pi < up.parts; ++pi) {
+            const float2 x = __ldcg(ml + (int64_t)pi * rows_rep + m_local);
+            if (!(x.y > 0.f)) continue;
+            const float w = exp2f(x.x - mstar);
+            l = fmaf(x.y, w, l);
+            if (lane < D4) {
+              const float4 o = __ldcg(reinterpret_cast<const float4*>(po + ((int64_t)pi * rows_rep + m_local) * D) + lane);
+              acc.x = fmaf(o.x, w, acc.x); acc.y = fmaf(o.y, w, acc.y); acc.z = fmaf(o.z, w, acc.z); acc.w = fmaf(o.w, w, acc.w);
+            }
+          }
+          const float inv = l > 0.f ? 1.f / l : 0.f;
+          const int m = rt * 128 + m_local;
+          const int hg = m / p.b, i = m - hg * p.b;
+          if (lane < D4) {
+            __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
+                               (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + lane * 4;
+            uint2 w2;
+            w2.x = pack_bf16(acc.x * inv, acc.y * inv);
+            w2.y = pack_bf16(acc.z * inv, acc.w * inv);
+            *reinterpret_cast<uint2*>(o) = w2;
+          }
+          if (lane == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
+        }
+      }
+      if (do_scores && p.pooled != nullptr) {
+        // Algorithm 1, MaxPool1D(A, kernel_size = s, padding = s/2) over the candidate axis Concat(prefix, suffix);
+        // block positions and padding get -inf
+        const int L = n1, b = p.b;
+        int o = p.block_off[bi];
+        o = min(max(o, 0), max(L - b, 0));
+        const int C = max(L - b, 0), w = (p.window - 1) / 2;
+        const float* a = p.raw_scores + (int64_t)(bi * p.Hkv + g) * p.n1_max;
+        float* dst = p.pooled + (int64_t)(bi * p.Hkv + g) * p.n1_max;
+        for (int pos = tid; pos < p.n1_max; pos += UM_THREADS) {
+          float outv = -INFINITY;
+          if (pos < L && (pos < o || pos >= o + b)) {
+            const int c = pos < o ? pos : pos - b;
+            int lo = 0, hi = C;
+            if (p.per_region) { if (c < o) hi = o; else lo = o; }
+            float mx = -INFINITY, sum = 0.f;
+            for (int t = c - w; t <= c + w; ++t) {
+              if (t < lo || t >= hi) continue;
+              const float x = __ldcg(a + (t < o ? t : t + b));
+              mx = fmaxf(mx, x);
+              sum += x;
+            }
+            outv = p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
+          }
+          dst[pos] = outv;
+        }
+      }
+      if (need_counter && tid == 0) p.counters[unit] = 0;     // ready for the next call
+    }
+  }
+
+  // ---- free the tensor memory ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
+}
+
+// 4-D bf16 tensor (D, rows, heads, batch) with element strides for the three outer axes; box = (64, box_rows, box_heads, 1),
+// 128-byte swizzle, out-of-range rows read as zero.
+bool make_map(CUtensorMap* m, const void* base, int D, int rows, int heads, int batch, const int64_t* stride_bhr, int box_rows,
+              int box_heads) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc || rows < 1) return false;
+  const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)rows, (cuuint64_t)heads, (cuuint64_t)batch};
+  auto st = [&](int64_t s) { return (cuuint64_t)(s > 0 ? s * 2 : (int64_t)D * 2); };   // unused strides stay legal
+  const cuuint64_t strides[3] = {st(stride_bhr[2]), st(stride_bhr[1]), st(stride_bhr[0])};
+  const cuuint32_t box[4] = {64u, (cuuint32_t)box_rows, (cuuint32_t)box_heads, 1u};
+  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+size_t umma_smem_bytes(int D, int KT) {
+  const size_t H = D / 64;
+  const size_t need = 1024 /*alignment slack*/ + 1024 /*barriers, qbar*/ + H * 128 * 128 + (size_t)UM_STAGES * 2 * H * KT * 128;
+  // every CTA allocates all 512 TMEM columns, so two CTAs must never share an SM: ask for more than half its shared memory
+  return need > 120 * 1024 ? need : 120 * 1024;
+}
+
+template <int D>
+cudaError_t launch_umma_d(const UmmaMaps& tm, const UmmaParams& up, const AttnPlan& pl, cudaStream_t st) {
+  auto kern = attn_umma_bf16_kernel<D>;
+  static size_t configured = 0;
+  if (pl.smem_bytes > configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
+    if (e != cudaSuccess) return e;
+    (void)cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    configured = pl.smem_bytes;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(pl.splits, up.a.Hkv * up.row_tiles, up.a.B);
+  cfg.blockDim = dim3(UM_THREADS);
+  cfg.dynamicSmemBytes = pl.smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  int na = 0;
+  const char* e = getenv("SDLLM_PDL");       // SDLLM_PDL=0 turns programmatic dependent launch off (tuning and test aid)
+  if (!(e && e[0] == '0')) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = attr; cfg.numAttrs = na;
+  return cudaLaunchKernelEx(&cfg, kern, tm, up);
+}
+
+}  // namespace
+
+// Whether the tcgen05 kernel covers a shape: bf16, D in {64, 128}, block length a multiple of 16 that either keeps all
+// b*G rows inside one 128-row tile or divides 128.
+bool umma_supported(int dtype, int D, int M, int b) {
+  if (dtype != SDLLM_BF16 || (D != 64 && D != 128) || encode_fn() == nullptr) return false;
+  if (b % 16 != 0 || b > 128) return false;
+  return M <= 128 || 128 % b == 0;
+}
+
+AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, int n2) {
+  AttnPlan pl{};
+  pl.kind = 2; pl.tma = true; pl.cluster = 1; pl.fused_tail = true;
+  pl.threads = UM_THREADS; pl.stages = UM_STAGES;
+  const int G = M / b;
+  pl.row_tiles = M <= 128 ? 1 : (G + 128 / b - 1) / (128 / b);
+  pl.rep = M <= 32 ? 4 : (M <= 64 ? 2 : 1);
+  const long long units = (long long)B * Hkv * pl.row_tiles;
+  long long want = kNumSMs / units;
+  if (want < 1) want = 1;
+  if (const char* e = getenv("SDLLM_SPLITS")) { if (atoi(e) >= 1) want = atoi(e); }   // tuning aid
+  const int kt2 = n2 > 0 ? (n2 < 128 ? n2 : 128) : 0;
+  pl.key_tile = 128;
+  if (pl.rep <= 2 && (n1_max + 127) / 128 + (n2 > 0 ? 1 : 0) < want) pl.key_tile = 64;
+  if (const char* e = getenv("SDLLM_KEY_TILE")) {   // tuning aid
+    if (atoi(e) == 64 && pl.rep <= 2) pl.key_tile = 64;
+    if (atoi(e) == 128) pl.key_tile = 128;
+  }
+  pl.key_tile2 = kt2 > 0 ? (kt2 < pl.key_tile ? kt2 : pl.key_tile) : pl.key_tile;
+  const int tiles = (n1_max + pl.key_tile - 1) / pl.key_tile + (n2 > 0 ? (n2 + pl.key_tile2 - 1) / pl.key_tile2 : 0);
+  if (want > tiles) want = tiles;
+  if (want > kMaxSplits) want = kMaxSplits;
+  if (want < 1) want = 1;
+  pl.splits = (int)want;
+  pl.parts = pl.splits * pl.rep;
+  pl.rows_rep = 128 / pl.rep;
+  pl.part_rows = pl.parts > 1 ? (size_t)pl.row_tiles * pl.parts * pl.rows_rep : 0;
+  pl.n_counters = (size_t)B * Hkv * pl.row_tiles;
+  pl.smem_bytes = umma_smem_bytes(D, pl.key_tile);
+  return pl;
+}
+
+cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cudaStream_t st) {
+  UmmaMaps tm;
+  UmmaParams up{};
+  up.a = p;
+  up.a.splits = pl.splits;
+  up.KT = pl.key_tile; up.KT2 = pl.key_tile2; up.R = pl.rep; up.row_tiles = pl.row_tiles;
+  up.heads_rt = pl.row_tiles == 1 ? p.G : 128 / p.b;
+  up.parts = pl.parts;
+  memset(&tm, 0, sizeof(tm));
+  bool ok = true;
+  if (p.out != nullptr) ok = make_map(&tm.q, p.q, D, p.b, p.Hq, p.B, p.q_stride, p.b, up.heads_rt);
+  if (p.n1_max > 0) {
+    ok = ok && make_map(&tm.k1, p.k1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, pl.key_tile, 1);
+    ok = ok && make_map(&tm.v1, p.v1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, pl.key_tile, 1);
+  }
+  if (p.n2 > 0) {
+    ok = ok && make_map(&tm.k2, p.k2, D, p.n2, p.Hkv, p.B, p.k2_stride, pl.key_tile2, 1);
+    ok = ok && make_map(&tm.v2, p.v2, D, p.n2, p.Hkv, p.B, p.k2_stride, pl.key_tile2, 1);
+    if (p.n1_max <= 0) { tm.k1 = tm.k2; tm.v1 = tm.v2; }
+  } else {
+    tm.k2 = tm.k1; tm.v2 = tm.v1;
+  }
+  if (!ok) return cudaErrorInvalidValue;
+  return D == 128 ? launch_umma_d<128>(tm, up, pl, st) : launch_umma_d<64>(tm, up, pl, st);
+}
+
+}  // namespace sdllm

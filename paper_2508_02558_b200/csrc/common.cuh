@@ -27,6 +27,15 @@ struct AttnPlan {
   int threads;
   bool tma;         // bf16 TMA kernel (else the cp.async kernels)
   size_t smem_bytes;
+  int kind;         // 0: cp.async kernels, 1: TMA + mma.sync kernel, 2: TMA + tcgen05 kernel
+  int key_tile2;    // tcgen05 kernel: keys per tile of source 2
+  int rep;          // tcgen05 kernel: replicas of the query rows along the 128 accumulator rows
+  int row_tiles;    // tcgen05 kernel: 128-row tiles of the b*G rows
+  int parts;        // partials per (sequence, KV head, row tile) = splits * rep
+  int rows_rep;     // rows of one partial
+  bool fused_tail;  // the attention kernel merges the partials and pools the scores itself
+  size_t part_rows; // partial rows per (sequence, KV head) in the workspace (0: none)
+  size_t n_counters;// completion counters in the workspace
 };
 
 // Key sources of one attention launch. The virtual key axis is [src1 rows 0..n1) ++ [src2 rows 0..n2).
@@ -48,6 +57,9 @@ struct AttnParams {
   int splits;                  // partials per (sequence, KV head) in the workspace
   int splits_total;            // CTAs along the key axis per (sequence, KV head) = splits * cluster size
   int32_t* status;             // device status word: set non-zero when a bounded wait gave up
+  int32_t* counters;           // completion counters (tcgen05 kernel), zero between calls
+  float* pooled;               // refresh with a fused tail: pooled scores [B][Hkv][n1_max], else null
+  int window, pool_kind, per_region;
   int want_scores;             // compute mean-query logit scores for src1 keys
   float scale;                 // softmax scale
   float scale_log2;            // scale * log2(e)
@@ -81,7 +93,7 @@ struct CompactParams {
   int64_t kv_stride_bytes[3], c_stride_bytes[3];
 };
 
-AttnPlan plan_attention(int dtype, int D, int M, int B, int Hkv, int n1_max, int n2);
+AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_max, int n2);
 
 cudaError_t launch_attn_partial(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st);
 cudaError_t launch_merge_pool(const MergeParams& p, cudaStream_t st);
