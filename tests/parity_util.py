@@ -81,13 +81,13 @@ def gpu_refresh(q, k, v, seq_len: Sequence[int], block_off: Sequence[int], dtype
 
 def check_refresh_against_oracle(g: GpuRefresh, q, k, v, seq_len, block_off, dtype, retention, window, *,
                                  heads: Optional[List[int]] = None, select=oracle.SELECT_JOINT_FLOOR,
-                                 pool_kind=oracle.POOL_MAX, score_rtol: float = 1e-4):
+                                 pool_kind=oracle.POOL_MAX, score_rtol: float = 1e-4, seqs: Optional[List[int]] = None):
     """Element-by-element comparison of one refresh (all sequences; optionally a subset of KV heads)."""
     Bn, Hq, b, D = q.shape
     Hkv = k.shape[1]
     G = Hq // Hkv
     stats = {"band_keys": 0, "set_mismatch": 0}
-    for i in range(Bn):
+    for i in (range(Bn) if seqs is None else seqs):
         L, o = int(seq_len[i]), int(block_off[i])
         hs = list(range(Hkv)) if heads is None else heads
         qh = np.concatenate([q[i, h * G:(h + 1) * G] for h in hs])
@@ -155,16 +155,17 @@ def gpu_sparse_step(g: GpuRefresh, q2, kn, vn, dtype: str) -> np.ndarray:
     return to_host_f32(out)
 
 
-def check_sparse_against_oracle(g: GpuRefresh, out_gpu, q2, kn, vn, dtype, heads: Optional[List[int]] = None):
+def check_sparse_against_oracle(g: GpuRefresh, out_gpu, q2, kn, vn, dtype, heads: Optional[List[int]] = None,
+                                seqs: Optional[List[int]] = None):
     """Oracle attention over [K_c ; K_n], with K_c read back from the device (it is bit-exact K[kept_idx])."""
     Bn, Hq, b, D = q2.shape
     Hkv = kn.shape[1]
     G = Hq // Hkv
-    kc, vc = to_host_f32(g.cache.k_c), to_host_f32(g.cache.v_c)
-    for i in range(Bn):
+    for i in (range(Bn) if seqs is None else seqs):
         cnt = int(g.kept_cnt[i])
         hs = list(range(Hkv)) if heads is None else heads
         qh = np.concatenate([q2[i, h * G:(h + 1) * G] for h in hs])
-        ref, _ = oracle.sparse_block_attention(qh, kc[i, hs, :cnt], vc[i, hs, :cnt], kn[i, hs], vn[i, hs])
+        kc, vc = to_host_f32(g.cache.k_c[i, hs, :cnt]), to_host_f32(g.cache.v_c[i, hs, :cnt])
+        ref, _ = oracle.sparse_block_attention(qh, kc, vc, kn[i, hs], vn[i, hs])
         for j, h in enumerate(hs):
             assert_close(out_gpu[i, h * G:(h + 1) * G], ref[j * G:(j + 1) * G], dtype, f"sparse out seq {i} head {h}")
