@@ -14,9 +14,11 @@
 //               "A <- MatMul(qbar, K_f^T)") from the K tile in shared memory, fp32
 // When b*G <= 64 the query rows are replicated R = 2 or 4 times along the 128 accumulator rows and every replica
 // takes its own slice of each key tile, so all four softmax warps work; the replicas are merged like key splits.
-// Key splits (and replicas) leave (max, sum, O) partials in the workspace; the last CTA of a (sequence, KV head,
-// row tile) to finish - found with one atomic counter, nobody waits - merges them, writes the output and, at the
-// refresh step, pools the head's saliency along the key axis (Algorithm 1, MaxPool1D).
+// The replicas are merged inside the CTA through shared memory. Key splits leave (max, sum, O) partials in the
+// workspace. While the tail is small, the last CTA of a (sequence, KV head, row tile) to finish - found with one
+// atomic counter, nobody waits - merges them, writes the output and, at the refresh step, pools the head's saliency
+// along the key axis (Algorithm 1, MaxPool1D); for large partial volumes or long sequences a second small launch
+// does the same work spread over the whole GPU.
 //
 // Every wait on an mbarrier is bounded. On expiry the thread sets an abort flag that all other waits poll, records a
 // code in the status word and the CTA runs to its end (freeing its TMEM); the outputs of that call are then invalid.
@@ -45,7 +47,7 @@ struct UmmaParams {
   int R;             // replicas of the query rows along the 128 accumulator rows (1, 2, 4)
   int row_tiles;     // 128-row tiles of the b*G rows
   int heads_rt;      // query heads per row tile
-  int parts;         // partials per (sequence, KV head, row tile) = splits * R
+  int fused_tail;    // 1: the last CTA of a unit merges and pools; 0: umma_tail_kernel does
 };
 
 // ---------------------------------------------------------------------------------------------------------
@@ -181,6 +183,102 @@ __device__ __forceinline__ void drain_bar(uint32_t bar, uint32_t parity) {
   while (!mbar_try_wait(bar, parity)) {
     if (clock64() - t0 > kWaitCycles) return;
   }
+}
+
+// Importance of one absolute position: Algorithm 1, MaxPool1D(A, kernel_size = s, padding = s/2) over the candidate
+// axis Concat(prefix, suffix) (AvgPool for the ablation); block positions and padding get -inf. `a` holds the raw
+// saliency by absolute position.
+__device__ __forceinline__ float pool_at(const AttnParams& p, const float* a, int L, int o_in, int pos) {
+  const int b = p.b;
+  const int o = min(max(o_in, 0), max(L - b, 0));
+  if (pos >= L || (pos >= o && pos < o + b)) return -INFINITY;
+  const int C = max(L - b, 0), w = (p.window - 1) / 2;
+  const int c = pos < o ? pos : pos - b;
+  int lo = 0, hi = C;
+  if (p.per_region) { if (c < o) hi = o; else lo = o; }
+  float mx = -INFINITY, sum = 0.f;
+  for (int t = c - w; t <= c + w; ++t) {
+    if (t < lo || t >= hi) continue;
+    const float x = a[t < o ? t : t + b];
+    mx = fmaxf(mx, x);
+    sum += x;
+  }
+  return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
+}
+
+// Merge of the key-split partials of one (row, float4 column) slot of a unit and the final store. Loads of four
+// partials are issued together so that their latencies overlap.
+template <int D>
+__device__ __forceinline__ void merge_slot(const AttnParams& p, int64_t unit, int bi, int g, int rt, int m_local, int d4) {
+  const int P = p.splits;
+  const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + unit * P * 128 + m_local;
+  const float4* po = reinterpret_cast<const float4*>(p.part_o + (unit * P * 128 + m_local) * D) + d4;
+  float mstar = -INFINITY;
+  for (int pi = 0; pi < P; ++pi) {
+    const float2 x = __ldcg(ml + (int64_t)pi * 128);
+    if (x.y > 0.f) mstar = fmaxf(mstar, x.x);
+  }
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float l = 0.f;
+  for (int p0 = 0; p0 < P; p0 += 4) {
+    float2 x[4];
+    float4 o[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int pi = min(p0 + u, P - 1);
+      x[u] = __ldcg(ml + (int64_t)pi * 128);
+      o[u] = __ldcg(po + (int64_t)pi * 128 * (D / 4));
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (p0 + u >= P || !(x[u].y > 0.f)) continue;
+      const float w = fast_exp2(x[u].x - mstar);
+      l = fmaf(x[u].y, w, l);
+      acc.x = fmaf(o[u].x, w, acc.x); acc.y = fmaf(o[u].y, w, acc.y); acc.z = fmaf(o[u].z, w, acc.z); acc.w = fmaf(o[u].w, w, acc.w);
+    }
+  }
+  const float inv = l > 0.f ? 1.f / l : 0.f;
+  const int m = rt * 128 + m_local;
+  const int hg = m / p.b, i = m - hg * p.b;
+  __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
+                       (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
+  uint2 w2;
+  w2.x = pack_bf16(acc.x * inv, acc.y * inv);
+  w2.y = pack_bf16(acc.z * inv, acc.w * inv);
+  *reinterpret_cast<uint2*>(out) = w2;
+  if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
+}
+
+// Deferred tail (large partial volumes or long sequences): one launch that merges the key splits, one thread per
+// (row, float4 column), and pools the saliency, one thread per position.
+template <int D>
+__global__ void __launch_bounds__(256) umma_tail_kernel(const UmmaParams up, const int merge_blocks) {
+  const AttnParams& p = up.a;
+  grid_dependency_wait();
+  grid_launch_dependents();
+  if ((int)blockIdx.x < merge_blocks) {
+    constexpr int D4 = D / 4;
+    const int64_t slot = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    const int d4 = (int)(slot % D4);
+    const int64_t r = slot / D4;
+    const int m_local = (int)(r % 128);
+    const int64_t unit = r / 128;
+    if (unit >= (int64_t)p.B * p.Hkv * up.row_tiles) return;
+    const int rt = (int)(unit % up.row_tiles);
+    const int64_t bg = unit / up.row_tiles;
+    const int g = (int)(bg % p.Hkv), bi = (int)(bg / p.Hkv);
+    if (m_local >= min(p.M - rt * 128, 128)) return;
+    merge_slot<D>(p, unit, bi, g, rt, m_local, d4);
+    return;
+  }
+  const int64_t idx = (int64_t)(blockIdx.x - merge_blocks) * 256 + threadIdx.x;
+  if (idx >= (int64_t)p.B * p.Hkv * p.n1_max) return;
+  const int pos = (int)(idx % p.n1_max);
+  const int64_t bh = idx / p.n1_max;
+  const int bi = (int)(bh / p.Hkv);
+  int L = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
+  L = min(max(L, 0), p.n1_max);
+  p.pooled[idx] = pool_at(p, p.raw_scores + bh * p.n1_max, L, p.block_off[bi], pos);
 }
 
 template <int D>
@@ -509,121 +607,90 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   }
 
   // ======================================= epilogue =======================================
+  // The ring is idle now (every load was consumed and the last tcgen05.commit the softmax warps waited for covers all
+  // MMAs), so it doubles as scratch: o_s [128][D] fp32 with the float4 index XOR-swizzled by the row, then ml_s [128].
   const int64_t unit = (int64_t)(bi * p.Hkv + g) * up.row_tiles + rt;      // (sequence, KV head, row tile)
-  if (do_attn && warp >= 2 && warp < 6) {
+  float* o_s = reinterpret_cast<float*>(stage0);
+  float2* ml_s = reinterpret_cast<float2*>(stage0 + 128 * D * 4);
+  if (do_attn && warp >= 2 && warp < 6 && !*abort_flag) {
+    constexpr int D4 = D / 4;
     const int row = (warp & 3) * 32 + lane;
-    const int rep = row / rows_rep, m_local = row - rep * rows_rep;
-    if (m_local < M_rt && !*abort_flag) {
+    ml_s[row] = make_float2(m_run, l_run);
+#pragma unroll
+    for (int j = 0; j < D4; ++j)
+      *reinterpret_cast<float4*>(o_s + row * D + ((j ^ (row & (D4 - 1))) << 2)) =
+          make_float4(o_reg[4 * j], o_reg[4 * j + 1], o_reg[4 * j + 2], o_reg[4 * j + 3]);
+    asm volatile("bar.sync 2, 128;\n" ::: "memory");
+    // merge the R replicas of every row; consecutive threads take consecutive float4 of a row (coalesced stores)
+    const int st = (warp - 2) * 32 + lane;
+    for (int slot = st; slot < M_rt * D4; slot += 128) {
+      const int m_local = slot / D4, d4 = slot - m_local * D4;
+      float mstar = -INFINITY;
+      for (int rep = 0; rep < R; ++rep) {
+        const float2 x = ml_s[rep * rows_rep + m_local];
+        if (x.y > 0.f) mstar = fmaxf(mstar, x.x);
+      }
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      float l = 0.f;
+      for (int rep = 0; rep < R; ++rep) {
+        const int rr = rep * rows_rep + m_local;
+        const float2 x = ml_s[rr];
+        if (!(x.y > 0.f)) continue;
+        const float w = fast_exp2(x.x - mstar);
+        l = fmaf(x.y, w, l);
+        const float4 o = *reinterpret_cast<const float4*>(o_s + rr * D + ((d4 ^ (rr & (D4 - 1))) << 2));
+        acc.x = fmaf(o.x, w, acc.x); acc.y = fmaf(o.y, w, acc.y); acc.z = fmaf(o.z, w, acc.z); acc.w = fmaf(o.w, w, acc.w);
+      }
       const int m = rt * 128 + m_local;                // row within the KV head: m = head_in_group * b + i
       const int hg = m / p.b, i = m - hg * p.b;
-      if (up.parts == 1) {
-        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+      if (p.splits == 1) {
+        const float inv = l > 0.f ? 1.f / l : 0.f;
         __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
-                           (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2];
-#pragma unroll
-        for (int d = 0; d < D; d += 8) {
-          uint4 w;
-          w.x = pack_bf16(o_reg[d] * inv, o_reg[d + 1] * inv);
-          w.y = pack_bf16(o_reg[d + 2] * inv, o_reg[d + 3] * inv);
-          w.z = pack_bf16(o_reg[d + 4] * inv, o_reg[d + 5] * inv);
-          w.w = pack_bf16(o_reg[d + 6] * inv, o_reg[d + 7] * inv);
-          *reinterpret_cast<uint4*>(o + d) = w;
-        }
-        if (p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (m_run + log2f(l_run)) * kLn2;
+                           (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
+        uint2 w2;
+        w2.x = pack_bf16(acc.x * inv, acc.y * inv);
+        w2.y = pack_bf16(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2*>(o) = w2;
+        if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
       } else {
-        const int64_t prow = (unit * up.parts + split * R + rep) * rows_rep + m_local;
-        float* o = p.part_o + prow * D;
-#pragma unroll
-        for (int d = 0; d < D; d += 4)
-          *reinterpret_cast<float4*>(o + d) = make_float4(o_reg[d], o_reg[d + 1], o_reg[d + 2], o_reg[d + 3]);
-        reinterpret_cast<float2*>(p.part_ml)[prow] = make_float2(m_run, l_run);
+        const int64_t prow = (unit * p.splits + split) * 128 + m_local;
+        *reinterpret_cast<float4*>(p.part_o + prow * D + d4 * 4) = acc;
+        if (d4 == 0) reinterpret_cast<float2*>(p.part_ml)[prow] = make_float2(mstar, l);
       }
     }
   }
 
-  // ---- the last CTA of the unit merges the partials and pools the saliency; nobody waits for anybody ----
-  const bool need_counter = p.splits > 1;
-  const bool have_tail = (do_attn && up.parts > 1) || (do_scores && p.pooled != nullptr);
-  if (have_tail) {
+  // ---- fused tail: the last CTA of the unit merges the key splits and pools the saliency; nobody waits ----
+  const bool tail_merge = do_attn && p.splits > 1;
+  const bool tail_pool = do_scores && p.pooled != nullptr;
+  if (up.fused_tail && (tail_merge || tail_pool)) {
     __threadfence();
-    tc_fence_before();
     __syncthreads();
-    if (need_counter) {
+    bool last = true;
+    if (p.splits > 1) {
       if (tid == 0) {
         const int old = atomicAdd(p.counters + unit, 1);
         *last_flag = (old == p.splits - 1) ? 1 : 0;
       }
       __syncthreads();
+      last = *last_flag != 0;
     }
-    const bool last = need_counter ? (*last_flag != 0) : true;
     if (last && !*abort_flag) {
       __threadfence();
-      if (do_attn && up.parts > 1) {
-        constexpr int D4 = D / 4;
-        const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + unit * up.parts * rows_rep;
-        const float* po = p.part_o + unit * up.parts * rows_rep * D;
-        for (int m_local = warp; m_local < M_rt; m_local += UM_THREADS / 32) {
-          float mstar = -INFINITY;
-          for (int pi = lane; pi < up.parts; pi += 32) {
-            const float2 x = __ldcg(ml + (int64_t)pi * rows_rep + m_local);
-            if (x.y > 0.f) mstar = fmaxf(mstar, x.x);
-          }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, o));
-          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-          float l = 0.f;
-          for (int pi = 0; pi < up.parts; ++pi) {
-            const float2 x = __ldcg(ml + (int64_t)pi * rows_rep + m_local);
-            if (!(x.y > 0.f)) continue;
-            const float w = exp2f(x.x - mstar);
-            l = fmaf(x.y, w, l);
-            if (lane < D4) {
-              const float4 o = __ldcg(reinterpret_cast<const float4*>(po + ((int64_t)pi * rows_rep + m_local) * D) + lane);
-              acc.x = fmaf(o.x, w, acc.x); acc.y = fmaf(o.y, w, acc.y); acc.z = fmaf(o.z, w, acc.z); acc.w = fmaf(o.w, w, acc.w);
-            }
-          }
-          const float inv = l > 0.f ? 1.f / l : 0.f;
-          const int m = rt * 128 + m_local;
-          const int hg = m / p.b, i = m - hg * p.b;
-          if (lane < D4) {
-            __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
-                               (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + lane * 4;
-            uint2 w2;
-            w2.x = pack_bf16(acc.x * inv, acc.y * inv);
-            w2.y = pack_bf16(acc.z * inv, acc.w * inv);
-            *reinterpret_cast<uint2*>(o) = w2;
-          }
-          if (lane == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
-        }
-      }
-      if (do_scores && p.pooled != nullptr) {
-        // Algorithm 1, MaxPool1D(A, kernel_size = s, padding = s/2) over the candidate axis Concat(prefix, suffix);
-        // block positions and padding get -inf
-        const int L = n1, b = p.b;
-        int o = p.block_off[bi];
-        o = min(max(o, 0), max(L - b, 0));
-        const int C = max(L - b, 0), w = (p.window - 1) / 2;
+      if (tail_merge)
+        for (int slot = tid; slot < M_rt * (D / 4); slot += UM_THREADS)
+          merge_slot<D>(p, unit, bi, g, rt, slot / (D / 4), slot % (D / 4));
+      if (tail_pool) {
+        // stage the head's raw saliency in shared memory (the ring is free), then pool from there
+        float* a_s = reinterpret_cast<float*>(stage0);
         const float* a = p.raw_scores + (int64_t)(bi * p.Hkv + g) * p.n1_max;
-        float* dst = p.pooled + (int64_t)(bi * p.Hkv + g) * p.n1_max;
-        for (int pos = tid; pos < p.n1_max; pos += UM_THREADS) {
-          float outv = -INFINITY;
-          if (pos < L && (pos < o || pos >= o + b)) {
-            const int c = pos < o ? pos : pos - b;
-            int lo = 0, hi = C;
-            if (p.per_region) { if (c < o) hi = o; else lo = o; }
-            float mx = -INFINITY, sum = 0.f;
-            for (int t = c - w; t <= c + w; ++t) {
-              if (t < lo || t >= hi) continue;
-              const float x = __ldcg(a + (t < o ? t : t + b));
-              mx = fmaxf(mx, x);
-              sum += x;
-            }
-            outv = p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
-          }
-          dst[pos] = outv;
-        }
+        __syncthreads();
+        for (int i = tid; i < n1; i += UM_THREADS) a_s[i] = __ldcg(a + i);
+        __syncthreads();
+        for (int pos = tid; pos < p.n1_max; pos += UM_THREADS)
+          p.pooled[(int64_t)(bi * p.Hkv + g) * p.n1_max + pos] = pool_at(p, a_s, n1, p.block_off[bi], pos);
       }
-      if (need_counter && tid == 0) p.counters[unit] = 0;     // ready for the next call
+      if (p.splits > 1 && tid == 0) p.counters[unit] = 0;      // ready for the next call
     }
   }
 
@@ -737,9 +804,9 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
   if (want > kMaxSplits) want = kMaxSplits;
   if (want < 1) want = 1;
   pl.splits = (int)want;
-  pl.parts = pl.splits * pl.rep;
+  pl.parts = pl.splits;                 // replicas are merged inside the CTA
   pl.rows_rep = 128 / pl.rep;
-  pl.part_rows = pl.parts > 1 ? (size_t)pl.row_tiles * pl.parts * pl.rows_rep : 0;
+  pl.part_rows = pl.splits > 1 ? (size_t)pl.row_tiles * pl.splits * 128 : 0;
   pl.n_counters = (size_t)B * Hkv * pl.row_tiles;
   pl.smem_bytes = umma_smem_bytes(D, pl.key_tile);
   return pl;
@@ -752,7 +819,12 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
   up.a.splits = pl.splits;
   up.KT = pl.key_tile; up.KT2 = pl.key_tile2; up.R = pl.rep; up.row_tiles = pl.row_tiles;
   up.heads_rt = pl.row_tiles == 1 ? p.G : 128 / p.b;
-  up.parts = pl.parts;
+  // The last CTA of a unit does the tail itself while that is a small job; otherwise a second launch spreads it
+  // over the whole GPU.
+  const size_t merge_bytes = pl.splits > 1 ? (size_t)pl.splits * (p.M < 128 ? p.M : 128) * D * 4 : 0;
+  const bool pool = p.want_scores && p.pooled != nullptr;
+  up.fused_tail = (merge_bytes <= 256 * 1024 && (!pool || p.n1_max <= 8192)) ? 1 : 0;
+  if (const char* e = getenv("SDLLM_FUSED_TAIL")) up.fused_tail = e[0] == '1' && (!pool || p.n1_max <= 8192);   // tuning aid
   memset(&tm, 0, sizeof(tm));
   bool ok = true;
   if (p.out != nullptr) ok = make_map(&tm.q, p.q, D, p.b, p.Hq, p.B, p.q_stride, p.b, up.heads_rt);
@@ -768,7 +840,28 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
     tm.k2 = tm.k1; tm.v2 = tm.v1;
   }
   if (!ok) return cudaErrorInvalidValue;
-  return D == 128 ? launch_umma_d<128>(tm, up, pl, st) : launch_umma_d<64>(tm, up, pl, st);
+  cudaError_t err = D == 128 ? launch_umma_d<128>(tm, up, pl, st) : launch_umma_d<64>(tm, up, pl, st);
+  if (err != cudaSuccess || up.fused_tail) return err;
+  const bool merge = p.out != nullptr && pl.splits > 1;
+  if (!merge && !pool) return cudaSuccess;
+  const long long merge_threads = merge ? (long long)p.B * p.Hkv * pl.row_tiles * 128 * (D / 4) : 0;
+  const long long pool_threads = pool ? (long long)p.B * p.Hkv * p.n1_max : 0;
+  const int merge_blocks = (int)((merge_threads + 255) / 256);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)(merge_blocks + (pool_threads + 255) / 256));
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  int na = 0;
+  const char* e = getenv("SDLLM_PDL");
+  if (!(e && e[0] == '0')) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = attr; cfg.numAttrs = na;
+  return D == 128 ? cudaLaunchKernelEx(&cfg, umma_tail_kernel<128>, up, merge_blocks)
+                  : cudaLaunchKernelEx(&cfg, umma_tail_kernel<64>, up, merge_blocks);
 }
 
 }  // namespace sdllm
