@@ -603,6 +603,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         if (lane == 0) mbar_arrive(BAR(EMPTY_K + s));
         ++it;
       }
+      // the softmax warps reuse the ring as scratch once they are done: tell them the K tiles are no longer read
+      if (do_attn) asm volatile("bar.sync 3, 192;\n" ::: "memory");
     }
   }
 
@@ -612,6 +614,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   const int64_t unit = (int64_t)(bi * p.Hkv + g) * up.row_tiles + rt;      // (sequence, KV head, row tile)
   float* o_s = reinterpret_cast<float*>(stage0);
   float2* ml_s = reinterpret_cast<float2*>(stage0 + 128 * D * 4);
+  if (do_attn && do_scores && warp >= 2 && warp < 6)
+    asm volatile("bar.sync 3, 192;\n" ::: "memory");                   // the saliency warps have left the ring
   if (do_attn && warp >= 2 && warp < 6 && !*abort_flag) {
     constexpr int D4 = D / 4;
     const int row = (warp & 3) * 32 + lane;
