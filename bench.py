@@ -220,6 +220,7 @@ def run_ours(args):
     out_s = torch.empty((reuse_steps, n_layers, 1, Hq, b, D), dtype=tdt, device=dev)
 
     stream = torch.cuda.Stream(device=dev)
+    torch.cuda.synchronize(dev)                     # the inputs above were produced on the default stream
 
     def one_step():
         """One decoding block: refresh every layer, then every reuse step over every layer (model order)."""

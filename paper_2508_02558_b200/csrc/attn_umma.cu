@@ -8,8 +8,9 @@
 //   warp 0      TMA producer: K and V tiles (128-byte swizzle) into a shared-memory ring, one mbarrier pair per slot
 //   warp 1      one thread issues tcgen05.mma: S = Q K^T (A, B from shared memory) into TMEM, then
 //               O_tile = P V with P read from TMEM (A) and V from shared memory (B, MN-major)
-//   warps 2-5   softmax: each thread owns one of the 128 accumulator rows (TMEM lane), reads S with tcgen05.ld,
-//               keeps the running max / sum, writes P (bf16) over S in TMEM, and accumulates O in registers
+//   warps 2-5   softmax: each thread owns one of the 128 accumulator rows (TMEM lane), reads its S row with
+//               tcgen05.ld, keeps the running max / sum and writes P (bf16) over S in TMEM; O accumulates in TMEM
+//               across the tiles and is rescaled in place only when a row's maximum grows by more than 2^8
 //   warps 6-7   refresh only: mean-query saliency of every streamed key (Algorithm 1, "qbar <- Mean(Q_b)",
 //               "A <- MatMul(qbar, K_f^T)") from the K tile in shared memory, fp32
 // When b*G <= 64 the query rows are replicated R = 2 or 4 times along the 128 accumulator rows and every replica
@@ -285,6 +286,7 @@ template <int D>
 __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __grid_constant__ UmmaMaps tm, const UmmaParams up) {
   constexpr int H = D / 64;            // 128-byte column halves of a row
   constexpr int NS = UM_STAGES;
+  constexpr uint32_t O_COL = 256;      // TMEM columns: S/P buffers at 0 and 128, the O accumulator at 256
   const AttnParams& p = up.a;
   extern __shared__ unsigned char smem_raw[];
 
@@ -302,6 +304,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   const int M_rt = min(p.M - rt * 128, 128);          // valid query rows of this row tile (<= rows_rep when R > 1)
   const bool do_attn = p.out != nullptr;
   const bool do_scores = p.want_scores && rt == 0;
+  const int n2 = p.n2;
 
   // ---- shared memory carve-up (1024-byte aligned for the 128-byte swizzle) ----
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -309,7 +312,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   const uint32_t bars = smem_u32(smem);
   auto BAR = [&](int i) { return bars + 8u * (uint32_t)i; };
   const int Q_FULL = 0, FULL_K = 1, FULL_V = 1 + NS, EMPTY_K = 1 + 2 * NS, EMPTY_V = 1 + 3 * NS;
-  const int S_FULL = 1 + 4 * NS, P_FULL = S_FULL + 2, O_FULL = S_FULL + 4, O_FREE = S_FULL + 6, DRAIN = S_FULL + 8;
+  const int S_FULL = 1 + 4 * NS, P_FULL = S_FULL + 2, PV_DONE = S_FULL + 4, DRAIN = S_FULL + 5;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 260);
   int* last_flag = reinterpret_cast<int*>(smem + 264);
@@ -319,6 +322,48 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   const int half_bytes = KT * 128;                     // one 64-column half of a K or V tile
   const int kv_bytes = H * half_bytes;                 // a whole K (or V) tile
   const int stage_bytes = 2 * kv_bytes;
+  // Q rows that no TMA box covers must not hold non-finite garbage; only shapes with b*G below the replica's rows need it
+  const bool zero_q = do_attn && p.b * up.heads_rt < rows_rep;
+  if (tid == 0) {                        // the descriptors live in the kernel parameters: fetch them while the CTA sets up
+    prefetch_tmap(&tm.k1); prefetch_tmap(&tm.v1);
+    if (n2 > 0) { prefetch_tmap(&tm.k2); prefetch_tmap(&tm.v2); }
+    if (do_attn) prefetch_tmap(&tm.q);
+  }
+
+  // The producer lane sets the barriers up and, unless the Q tile has to be cleared first, starts the first loads
+  // before the rest of the CTA is ready: the loads need nothing but the barriers.
+  int prod_it = 0, prod_t = t_begin, prod_n1 = 0;
+  bool prod_ok = true;
+  auto produce = [&](int limit) {     // issue loads for up to `limit` further tiles (producer lane only)
+    while (prod_t < t_end && limit > 0 && prod_ok) {
+      const Tile x = tile_of(prod_t, tiles1, KT, KT2, prod_n1, n2);
+      ++prod_t;
+      if (x.nv == 0) continue;
+      const int it = prod_it, s = it % NS;
+      const uint32_t ph = ((it / NS) - 1) & 1;
+      const uint32_t kdst = smem_u32(stage0 + (size_t)s * stage_bytes), vdst = kdst + kv_bytes;
+      const CUtensorMap* mk = x.src1 ? &tm.k1 : &tm.k2;
+      const CUtensorMap* mv = x.src1 ? &tm.v1 : &tm.v2;
+      const uint32_t tile_tx = (uint32_t)(H * (x.src1 ? KT : KT2) * 128);
+      if (it >= NS && !wait_bar(BAR(EMPTY_K + s), ph, abort_flag, p.status, 1)) { prod_ok = false; break; }
+      mbar_expect_tx(BAR(FULL_K + s), tile_tx);
+      for (int h = 0; h < H; ++h) tma_load_4d(kdst + h * half_bytes, mk, BAR(FULL_K + s), h * 64, x.row0, g, bi);
+      if (it == 0 && do_attn) {        // the Q tile right after the first K tile: S_0 needs both
+        mbar_expect_tx(BAR(Q_FULL), (uint32_t)(R * H * p.b * up.heads_rt * 128));
+        for (int rep = 0; rep < R; ++rep)
+          for (int h = 0; h < H; ++h)
+            tma_load_4d(smem_u32(q_s + h * 128 * 128 + rep * rows_rep * 128), &tm.q, BAR(Q_FULL), h * 64, 0,
+                        g * p.G + rt * up.heads_rt, bi);
+      }
+      if (do_attn) {
+        if (it >= NS && !wait_bar(BAR(EMPTY_V + s), ph, abort_flag, p.status, 2)) { prod_ok = false; break; }
+        mbar_expect_tx(BAR(FULL_V + s), tile_tx);
+        for (int h = 0; h < H; ++h) tma_load_4d(vdst + h * half_bytes, mv, BAR(FULL_V + s), h * 64, x.row0, g, bi);
+      }
+      ++prod_it;
+      --limit;
+    }
+  };
 
   if (tid == 0) {
     mbar_init(BAR(Q_FULL), 1);
@@ -331,18 +376,22 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     for (int i = 0; i < 2; ++i) {
       mbar_init(BAR(S_FULL + i), 1);
       mbar_init(BAR(P_FULL + i), 4);
-      mbar_init(BAR(O_FULL + i), 1);
-      mbar_init(BAR(O_FREE + i), 4);
     }
+    mbar_init(BAR(PV_DONE), 1);
     mbar_init(BAR(DRAIN), 1);
     *abort_flag = 0;
     *last_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    if (!zero_q && (do_attn || do_scores)) {
+      grid_dependency_wait();          // the loads below read what earlier kernels in the stream wrote
+      prod_n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
+      prod_n1 = min(max(prod_n1, 0), p.n1_max);
+      produce(NS);                     // the first NS slots are free: no waiting here
+    }
   }
-  // Q rows that no TMA box covers must not hold non-finite garbage: clear the tile first
-  if (do_attn)
+  if (zero_q)
     for (int i = tid; i < H * 128 * 128 / 16; i += UM_THREADS) reinterpret_cast<uint4*>(q_s)[i] = make_uint4(0u, 0u, 0u, 0u);
-  if (warp == 0) {
+  if (warp == 1) {                     // the MMA warp owns the tensor memory
     tmem_alloc(smem_u32(tmem_slot), 512);
     tmem_relinquish();
   }
@@ -357,74 +406,43 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
 
   int n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
   n1 = min(max(n1, 0), p.n1_max);
-  const int n2 = p.n2;
 
-  // per-thread softmax state (softmax warps only)
+  // softmax state of this thread's accumulator row (softmax warps only)
   float o_reg[D];
   float m_run = -INFINITY, l_run = 0.f;
 
   if (warp == 0) {
     // ======================================= TMA producer =======================================
-    if (lane == 0) {
-      prefetch_tmap(&tm.k1); prefetch_tmap(&tm.v1);
-      if (n2 > 0) { prefetch_tmap(&tm.k2); prefetch_tmap(&tm.v2); }
-      if (do_attn) {
-        prefetch_tmap(&tm.q);
-        mbar_expect_tx(BAR(Q_FULL), (uint32_t)(R * H * p.b * up.heads_rt * 128));
-        for (int rep = 0; rep < R; ++rep)
-          for (int h = 0; h < H; ++h)
-            tma_load_4d(smem_u32(q_s + h * 128 * 128 + rep * rows_rep * 128), &tm.q, BAR(Q_FULL), h * 64, 0,
-                        g * p.G + rt * up.heads_rt, bi);
-      }
-      int it = 0;
-      bool ok = true;
-      for (int t = t_begin; t < t_end && ok && (do_attn || do_scores); ++t) {
-        const Tile x = tile_of(t, tiles1, KT, KT2, n1, n2);
-        if (x.nv == 0) continue;
-        const int s = it % NS;
-        const uint32_t ph = ((it / NS) - 1) & 1;
-        const uint32_t kdst = smem_u32(stage0 + (size_t)s * stage_bytes), vdst = kdst + kv_bytes;
-        const CUtensorMap* mk = x.src1 ? &tm.k1 : &tm.k2;
-        const CUtensorMap* mv = x.src1 ? &tm.v1 : &tm.v2;
-        const int box_rows = x.src1 ? KT : KT2;
-        const uint32_t tile_tx = (uint32_t)(H * box_rows * 128);
-        if (it >= NS && !wait_bar(BAR(EMPTY_K + s), ph, abort_flag, p.status, 1)) { ok = false; break; }
-        mbar_expect_tx(BAR(FULL_K + s), tile_tx);
-        for (int h = 0; h < H; ++h) tma_load_4d(kdst + h * half_bytes, mk, BAR(FULL_K + s), h * 64, x.row0, g, bi);
-        if (do_attn) {
-          if (it >= NS && !wait_bar(BAR(EMPTY_V + s), ph, abort_flag, p.status, 2)) { ok = false; break; }
-          mbar_expect_tx(BAR(FULL_V + s), tile_tx);
-          for (int h = 0; h < H; ++h) tma_load_4d(vdst + h * half_bytes, mv, BAR(FULL_V + s), h * 64, x.row0, g, bi);
-        }
-        ++it;
-      }
+    if (lane == 0 && (do_attn || do_scores)) {
+      prod_n1 = n1;
+      produce(1 << 30);
       if (*abort_flag) {
         // let the copies that were issued land before the CTA retires
-        for (int j = max(it - NS, 0); j < it; ++j) {
+        for (int j = max(prod_it - NS, 0); j < prod_it; ++j) {
           drain_bar(BAR(FULL_K + j % NS), (j / NS) & 1);
           if (do_attn) drain_bar(BAR(FULL_V + j % NS), (j / NS) & 1);
         }
+        if (do_attn && prod_it > 0) drain_bar(BAR(Q_FULL), 0);
       }
     }
   } else if (warp == 1) {
     // ======================================= MMA issuer =======================================
     if (lane == 0 && do_attn) {
       const uint32_t idesc_pv = instr_desc(D, true);
-      bool ok = wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 3);
+      bool ok = true, have_q = false;
       int it = 0;
       Tile prev{}; int prev_it = -1;
       auto issue_pv = [&](const Tile& x, int j) -> bool {
         const int s = j % NS, pb = j & 1;
         if (!wait_bar(BAR(P_FULL + pb), (j >> 1) & 1, abort_flag, p.status, 4)) return false;
         if (!wait_bar(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 5)) return false;
-        if (j >= 2 && !wait_bar(BAR(O_FREE + pb), ((j >> 1) - 1) & 1, abort_flag, p.status, 6)) return false;
         tc_fence_after();
         const uint32_t vsm = smem_u32(stage0 + (size_t)s * stage_bytes) + kv_bytes;
-        const uint32_t d_t = tmem_base + 256u + (uint32_t)pb * 128u;
         const uint32_t a_t = tmem_base + (uint32_t)pb * 128u;
         for (int ks = 0; ks < x.n_mma / 16; ++ks)
-          mma_ts(d_t, a_t + ks * 8, smem_desc(vsm + ks * 2048, (uint32_t)half_bytes, 1024u), idesc_pv, ks > 0 ? 1u : 0u);
-        tc_commit(BAR(O_FULL + pb));
+          mma_ts(tmem_base + O_COL, a_t + ks * 8, smem_desc(vsm + ks * 2048, (uint32_t)half_bytes, 1024u), idesc_pv,
+                 (j > 0 || ks > 0) ? 1u : 0u);
+        tc_commit(BAR(PV_DONE));       // phase j of this barrier completes when O holds tiles 0..j
         tc_commit(BAR(EMPTY_V + s));
         return true;
       };
@@ -433,6 +451,10 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         if (x.nv == 0) continue;
         const int s = it % NS, sb = it & 1;
         if (!wait_bar(BAR(FULL_K + s), (it / NS) & 1, abort_flag, p.status, 7)) { ok = false; break; }
+        if (!have_q) {
+          if (!wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 3)) { ok = false; break; }
+          have_q = true;
+        }
         tc_fence_after();
         const uint32_t ksm = smem_u32(stage0 + (size_t)s * stage_bytes);
         const uint32_t qsm = smem_u32(q_s);
@@ -464,28 +486,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
       const int rep = row / rows_rep;                  // warp-uniform
       const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16);
       const int chunk_keys = KT / R;                   // key slice of a tile owned by this replica
-#pragma unroll
-      for (int d = 0; d < D; ++d) o_reg[d] = 0.f;
-      float alpha_prev = 1.f;
       int it = 0;
       bool ok = true;
-      auto accumulate = [&](int j, float alpha) -> bool {
-        const int ob = j & 1;
-        if (!wait_bar_warp(BAR(O_FULL + ob), (j >> 1) & 1, abort_flag, p.status, 8)) return false;
-        tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t v[32];
-          tmem_ld32(lane_addr + 256u + (uint32_t)ob * 128u + c * 32, v);
-          tc_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o_reg[c * 32 + i] = fmaf(o_reg[c * 32 + i], alpha, __uint_as_float(v[i]));
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(O_FREE + ob));
-        return true;
-      };
       for (int t = t_begin; t < t_end && ok; ++t) {
         const Tile x = tile_of(t, tiles1, KT, KT2, n1, n2);
         if (x.nv == 0) continue;
@@ -495,45 +497,72 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         if (!wait_bar_warp(BAR(S_FULL + sb), (it >> 1) & 1, abort_flag, p.status, 9)) { ok = false; break; }
         tc_fence_after();
         const uint32_t s_addr = lane_addr + (uint32_t)sb * 128u;
-        // ---- pass 1: row maximum over the owned, valid columns ----
-        float mx = -INFINITY;
-        for (int c0 = 0; c0 < x.n_mma; c0 += 32) {
-          if (c0 >= c_hi || c0 + 32 <= c_lo) continue;
-          uint32_t v[32];
-          tmem_ld32(s_addr + c0, v);
-          tc_wait_ld();
+        // ---- the owned part of the S row, all loads in flight together ----
+        uint32_t sv[4][32];
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (c0 + i >= c_lo && c0 + i < c_hi) mx = fmaxf(mx, __uint_as_float(v[i]));
-        }
+        for (int c = 0; c < 4; ++c)
+          if (c * 32 < c_hi && c * 32 + 32 > c_lo) tmem_ld32(s_addr + c * 32, sv[c]);
+        tc_wait_ld();
+        float mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (c * 32 < c_hi && c * 32 + 32 > c_lo) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (c * 32 + i >= c_lo && c * 32 + i < c_hi) mx = fmaxf(mx, __uint_as_float(sv[c][i]));
+          }
+        // ---- running maximum: O (in TMEM) and l are rescaled only when the maximum grows by more than 2^8, so P stays
+        //      below 2^8 and the accumulator is touched on very few tiles ----
         const float m_new = fmaxf(m_run, mx * p.scale_log2);
-        const float mu = (m_new == -INFINITY) ? 0.f : m_new;
-        const float alpha = fast_exp2(m_run - mu);
-        m_run = m_new;
-        // ---- pass 2: P = exp2(S * scale_log2 - mu) as bf16 over the S columns; zero outside the owned slice ----
+        const bool grow = m_new > m_run + 8.f;          // also true on the first finite maximum
+        float alpha = 1.f;
+        if (grow) {
+          alpha = fast_exp2(m_run - m_new);             // 0 when m_run is -inf
+          m_run = m_new;
+          l_run *= alpha;
+        }
+        if (it > 0 && __any_sync(0xffffffffu, grow)) {
+          // every PV issued so far must have landed before the rows are rewritten; PV of this tile waits for our arrive
+          if (!wait_bar_warp(BAR(PV_DONE), (it - 1) & 1, abort_flag, p.status, 8)) { ok = false; break; }
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t ov[32];
+            tmem_ld32(lane_addr + O_COL + c * 32, ov);
+            tc_wait_ld();
+            uint32_t lo[16], hi[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              lo[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+              hi[i] = __float_as_uint(__uint_as_float(ov[16 + i]) * alpha);
+            }
+            tmem_st16(lane_addr + O_COL + c * 32, lo);
+            tmem_st16(lane_addr + O_COL + c * 32 + 16, hi);
+          }
+        }
+        const float mu = (m_run == -INFINITY) ? 0.f : m_run;
+        // ---- P = exp2(S * scale_log2 - mu) as bf16 over the S columns; zero outside the owned slice ----
         float psum = 0.f;
-        for (int c0 = 0; c0 < x.n_mma; c0 += 32) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (c * 32 >= x.n_mma) continue;
           uint32_t pk[16];
-          if (c0 >= c_hi || c0 + 32 <= c_lo) {
+          if (c * 32 < c_hi && c * 32 + 32 > c_lo) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const int j0 = c * 32 + 2 * i;
+              const float e0 = (j0 >= c_lo && j0 < c_hi) ? fast_exp2(fmaf(__uint_as_float(sv[c][2 * i]), p.scale_log2, -mu)) : 0.f;
+              const float e1 = (j0 + 1 >= c_lo && j0 + 1 < c_hi) ? fast_exp2(fmaf(__uint_as_float(sv[c][2 * i + 1]), p.scale_log2, -mu)) : 0.f;
+              psum += e0 + e1;
+              pk[i] = pack_bf16(e0, e1);
+            }
+          } else {
 #pragma unroll
             for (int i = 0; i < 16; ++i) pk[i] = 0u;
-          } else {
-            uint32_t v[32];
-            tmem_ld32(s_addr + c0, v);
-            tc_wait_ld();
-            float e[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const bool in = c0 + i >= c_lo && c0 + i < c_hi;
-              e[i] = in ? fast_exp2(fmaf(__uint_as_float(v[i]), p.scale_log2, -mu)) : 0.f;
-              psum += e[i];
-            }
-#pragma unroll
-            for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(e[2 * i], e[2 * i + 1]);
           }
-          tmem_st16(s_addr + (c0 >> 1), pk);
+          tmem_st16(s_addr + c * 16, pk);
         }
-        l_run = fmaf(l_run, alpha, psum);
+        l_run += psum;
         // ---- V rows past the source's count may hold anything: zero them so that 0 * V stays 0 ----
         if (x.nv < x.n_mma) {
           if (!wait_bar_warp(BAR(FULL_V + s), (it / NS) & 1, abort_flag, p.status, 10)) { ok = false; break; }
@@ -549,11 +578,22 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(BAR(P_FULL + sb));
-        if (it > 0 && !accumulate(it - 1, alpha_prev)) { ok = false; break; }
-        alpha_prev = alpha;
         ++it;
       }
-      if (ok && it > 0) ok = accumulate(it - 1, alpha_prev);
+      // ---- the finished accumulator row: TMEM -> registers ----
+#pragma unroll
+      for (int d = 0; d < D; ++d) o_reg[d] = 0.f;
+      if (ok && it > 0 && wait_bar_warp(BAR(PV_DONE), (it - 1) & 1, abort_flag, p.status, 6)) {
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t ov[32];
+          tmem_ld32(lane_addr + O_COL + c * 32, ov);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o_reg[c * 32 + i] = __uint_as_float(ov[i]);
+        }
+      }
     }
   } else {
     // ======================================= saliency warps (refresh) =======================================
@@ -569,7 +609,12 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         qbar_s[d] = acc / (float)p.M;
       }
       asm volatile("bar.sync 1, 64;\n" ::: "memory");
-      const int l8 = lane & 7;
+      float qb[D];                                       // the whole mean query in registers
+#pragma unroll
+      for (int d = 0; d < D; d += 4) {
+        const float4 v4 = *reinterpret_cast<const float4*>(qbar_s + d);
+        qb[d] = v4.x; qb[d + 1] = v4.y; qb[d + 2] = v4.z; qb[d + 3] = v4.w;
+      }
       int it = 0;
       for (int t = t_begin; t < t_end; ++t) {
         const Tile x = tile_of(t, tiles1, KT, KT2, n1, n2);
@@ -577,26 +622,23 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         const int s = it % NS;
         if (!wait_bar_warp(BAR(FULL_K + s), (it / NS) & 1, abort_flag, p.status, 11)) break;
         if (x.src1) {
+          // one key per lane: a_j = scale * <qbar, k_j>; the 128-byte swizzle keeps 32 consecutive rows conflict-free
           const unsigned char* kst = stage0 + (size_t)s * stage_bytes;
-          for (int k0 = (warp - 6) * 4; k0 < x.nv; k0 += 8) {      // warp-uniform trip count: the shuffles need all lanes
-            const int kk = k0 + (lane >> 3);                       // < KT always; rows past nv are computed and dropped
-            float acc = 0.f;
+          for (int kk = (warp - 6) * 32 + lane; kk < x.nv; kk += 64) {
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-            for (int h = 0; h < H; ++h) {
-              const uint4 raw = *reinterpret_cast<const uint4*>(kst + h * half_bytes + kk * 128 + ((l8 ^ (kk & 7)) << 4));
-              const float4 qa = *reinterpret_cast<const float4*>(qbar_s + h * 64 + l8 * 8);
-              const float4 qb = *reinterpret_cast<const float4*>(qbar_s + h * 64 + l8 * 8 + 4);
-              const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
-              float2 f;
-              f = __bfloat1622float2(h2[0]); acc = fmaf(qa.x, f.x, acc); acc = fmaf(qa.y, f.y, acc);
-              f = __bfloat1622float2(h2[1]); acc = fmaf(qa.z, f.x, acc); acc = fmaf(qa.w, f.y, acc);
-              f = __bfloat1622float2(h2[2]); acc = fmaf(qb.x, f.x, acc); acc = fmaf(qb.y, f.y, acc);
-              f = __bfloat1622float2(h2[3]); acc = fmaf(qb.z, f.x, acc); acc = fmaf(qb.w, f.y, acc);
+            for (int c = 0; c < H * 8; ++c) {
+              const uint4 raw = *reinterpret_cast<const uint4*>(kst + (c >> 3) * half_bytes + kk * 128 + (((c & 7) ^ (kk & 7)) << 4));
+              a0 = fmaf(qb[c * 8 + 0], __uint_as_float(raw.x << 16), a0);
+              a1 = fmaf(qb[c * 8 + 1], __uint_as_float(raw.x & 0xffff0000u), a1);
+              a2 = fmaf(qb[c * 8 + 2], __uint_as_float(raw.y << 16), a2);
+              a3 = fmaf(qb[c * 8 + 3], __uint_as_float(raw.y & 0xffff0000u), a3);
+              a0 = fmaf(qb[c * 8 + 4], __uint_as_float(raw.z << 16), a0);
+              a1 = fmaf(qb[c * 8 + 5], __uint_as_float(raw.z & 0xffff0000u), a1);
+              a2 = fmaf(qb[c * 8 + 6], __uint_as_float(raw.w << 16), a2);
+              a3 = fmaf(qb[c * 8 + 7], __uint_as_float(raw.w & 0xffff0000u), a3);
             }
-            acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-            acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-            acc += __shfl_xor_sync(0xffffffffu, acc, 4);
-            if (l8 == 0 && kk < x.nv) p.raw_scores[(int64_t)(bi * p.Hkv + g) * p.n1_max + x.row0 + kk] = acc * p.scale;
+            p.raw_scores[(int64_t)(bi * p.Hkv + g) * p.n1_max + x.row0 + kk] = ((a0 + a1) + (a2 + a3)) * p.scale;
           }
         }
         __syncwarp();
@@ -604,62 +646,101 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         ++it;
       }
       // the softmax warps reuse the ring as scratch once they are done: tell them the K tiles are no longer read
-      if (do_attn) asm volatile("bar.sync 3, 192;\n" ::: "memory");
+      if (do_attn && R > 1) asm volatile("bar.sync 3, 192;\n" ::: "memory");
     }
   }
 
   // ======================================= epilogue =======================================
-  // The ring is idle now (every load was consumed and the last tcgen05.commit the softmax warps waited for covers all
-  // MMAs), so it doubles as scratch: o_s [128][D] fp32 with the float4 index XOR-swizzled by the row, then ml_s [128].
   const int64_t unit = (int64_t)(bi * p.Hkv + g) * up.row_tiles + rt;      // (sequence, KV head, row tile)
-  float* o_s = reinterpret_cast<float*>(stage0);
-  float2* ml_s = reinterpret_cast<float2*>(stage0 + 128 * D * 4);
-  if (do_attn && do_scores && warp >= 2 && warp < 6)
-    asm volatile("bar.sync 3, 192;\n" ::: "memory");                   // the saliency warps have left the ring
-  if (do_attn && warp >= 2 && warp < 6 && !*abort_flag) {
+  if (do_attn && warp >= 2 && warp < 6) {
     constexpr int D4 = D / 4;
     const int row = (warp & 3) * 32 + lane;
-    ml_s[row] = make_float2(m_run, l_run);
+    const int rep = row / rows_rep, m_local = row - rep * rows_rep;
+    if (R == 1) {
+      // one accumulator row per query row: straight from registers
+      if (m_local < M_rt && !*abort_flag) {
+        const int m = rt * 128 + m_local;              // row within the KV head: m = head_in_group * b + i
+        const int hg = m / p.b, i = m - hg * p.b;
+        if (p.splits == 1) {
+          const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+          __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
+                             (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2];
 #pragma unroll
-    for (int j = 0; j < D4; ++j)
-      *reinterpret_cast<float4*>(o_s + row * D + ((j ^ (row & (D4 - 1))) << 2)) =
-          make_float4(o_reg[4 * j], o_reg[4 * j + 1], o_reg[4 * j + 2], o_reg[4 * j + 3]);
-    asm volatile("bar.sync 2, 128;\n" ::: "memory");
-    // merge the R replicas of every row; consecutive threads take consecutive float4 of a row (coalesced stores)
-    const int st = (warp - 2) * 32 + lane;
-    for (int slot = st; slot < M_rt * D4; slot += 128) {
-      const int m_local = slot / D4, d4 = slot - m_local * D4;
+          for (int d = 0; d < D; d += 8) {
+            uint4 w;
+            w.x = pack_bf16(o_reg[d] * inv, o_reg[d + 1] * inv);
+            w.y = pack_bf16(o_reg[d + 2] * inv, o_reg[d + 3] * inv);
+            w.z = pack_bf16(o_reg[d + 4] * inv, o_reg[d + 5] * inv);
+            w.w = pack_bf16(o_reg[d + 6] * inv, o_reg[d + 7] * inv);
+            *reinterpret_cast<uint4*>(o + d) = w;
+          }
+          if (p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (m_run + log2f(l_run)) * kLn2;
+        } else {
+          const int64_t prow = (unit * p.splits + split) * 128 + m_local;
+          float* o = p.part_o + prow * D;
+#pragma unroll
+          for (int d = 0; d < D; d += 4)
+            *reinterpret_cast<float4*>(o + d) = make_float4(o_reg[d], o_reg[d + 1], o_reg[d + 2], o_reg[d + 3]);
+          reinterpret_cast<float2*>(p.part_ml)[prow] = make_float2(m_run, l_run);
+        }
+      }
+    } else {
+      // The R replicas of a query row sit in different accumulator rows: merge them through shared memory. The ring
+      // is idle now (every load was consumed, the last PV has landed), so it serves as scratch:
+      //   o_s [128][D] fp32, the float4 index XOR-swizzled by the row; ml_s [128]; lm_s [rows_rep].
+      float* o_s = reinterpret_cast<float*>(stage0);
+      float2* ml_s = reinterpret_cast<float2*>(stage0 + 128 * D * 4);
+      float2* lm_s = ml_s + 128;
+      if (do_scores) asm volatile("bar.sync 3, 192;\n" ::: "memory");    // the saliency warps have left the ring
+      ml_s[row] = make_float2(m_run, l_run);
+      asm volatile("bar.sync 2, 128;\n" ::: "memory");
       float mstar = -INFINITY;
-      for (int rep = 0; rep < R; ++rep) {
-        const float2 x = ml_s[rep * rows_rep + m_local];
+      for (int r2 = 0; r2 < R; ++r2) {
+        const float2 x = ml_s[r2 * rows_rep + m_local];
         if (x.y > 0.f) mstar = fmaxf(mstar, x.x);
       }
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      float l = 0.f;
-      for (int rep = 0; rep < R; ++rep) {
-        const int rr = rep * rows_rep + m_local;
-        const float2 x = ml_s[rr];
-        if (!(x.y > 0.f)) continue;
-        const float w = fast_exp2(x.x - mstar);
-        l = fmaf(x.y, w, l);
-        const float4 o = *reinterpret_cast<const float4*>(o_s + rr * D + ((d4 ^ (rr & (D4 - 1))) << 2));
-        acc.x = fmaf(o.x, w, acc.x); acc.y = fmaf(o.y, w, acc.y); acc.z = fmaf(o.z, w, acc.z); acc.w = fmaf(o.w, w, acc.w);
+      float lsum = 0.f;
+      for (int r2 = 0; r2 < R; ++r2) {
+        const float2 x = ml_s[r2 * rows_rep + m_local];
+        if (x.y > 0.f) lsum = fmaf(x.y, fast_exp2(x.x - mstar), lsum);
       }
-      const int m = rt * 128 + m_local;                // row within the KV head: m = head_in_group * b + i
-      const int hg = m / p.b, i = m - hg * p.b;
-      if (p.splits == 1) {
-        const float inv = l > 0.f ? 1.f / l : 0.f;
-        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
-                           (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
-        uint2 w2;
-        w2.x = pack_bf16(acc.x * inv, acc.y * inv);
-        w2.y = pack_bf16(acc.z * inv, acc.w * inv);
-        *reinterpret_cast<uint2*>(o) = w2;
-        if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
-      } else {
-        const int64_t prow = (unit * p.splits + split) * 128 + m_local;
-        *reinterpret_cast<float4*>(p.part_o + prow * D + d4 * 4) = acc;
-        if (d4 == 0) reinterpret_cast<float2*>(p.part_ml)[prow] = make_float2(mstar, l);
+      const float w = l_run > 0.f ? fast_exp2(m_run - mstar) : 0.f;   // this replica's weight in the merged row
+      if (rep == 0) lm_s[m_local] = make_float2(mstar, lsum);
+#pragma unroll
+      for (int j = 0; j < D4; ++j)
+        *reinterpret_cast<float4*>(o_s + row * D + ((j ^ (row & (D4 - 1))) << 2)) =
+            make_float4(o_reg[4 * j] * w, o_reg[4 * j + 1] * w, o_reg[4 * j + 2] * w, o_reg[4 * j + 3] * w);
+      asm volatile("bar.sync 2, 128;\n" ::: "memory");
+      // consecutive threads take consecutive float4 of a row: coalesced stores
+      const int st = (warp - 2) * 32 + lane;
+      if (!*abort_flag) {
+#pragma unroll 4
+        for (int slot = st; slot < M_rt * D4; slot += 128) {
+          const int ml = slot / D4, d4 = slot - ml * D4;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int r2 = 0; r2 < R; ++r2) {
+            const int rr = r2 * rows_rep + ml;
+            const float4 o = *reinterpret_cast<const float4*>(o_s + rr * D + ((d4 ^ (rr & (D4 - 1))) << 2));
+            acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+          }
+          const float2 x = lm_s[ml];
+          const int m = rt * 128 + ml;
+          const int hg = m / p.b, i = m - hg * p.b;
+          if (p.splits == 1) {
+            const float inv = x.y > 0.f ? 1.f / x.y : 0.f;
+            __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
+                               (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
+            uint2 w2;
+            w2.x = pack_bf16(acc.x * inv, acc.y * inv);
+            w2.y = pack_bf16(acc.z * inv, acc.w * inv);
+            *reinterpret_cast<uint2*>(o) = w2;
+            if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (x.x + log2f(x.y)) * kLn2;
+          } else {
+            const int64_t prow = (unit * p.splits + split) * 128 + ml;
+            *reinterpret_cast<float4*>(p.part_o + prow * D + d4 * 4) = acc;
+            if (d4 == 0) reinterpret_cast<float2*>(p.part_ml)[prow] = x;
+          }
+        }
       }
     }
   }
@@ -688,7 +769,6 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         // stage the head's raw saliency in shared memory (the ring is free), then pool from there
         float* a_s = reinterpret_cast<float*>(stage0);
         const float* a = p.raw_scores + (int64_t)(bi * p.Hkv + g) * p.n1_max;
-        __syncthreads();
         for (int i = tid; i < n1; i += UM_THREADS) a_s[i] = __ldcg(a + i);
         __syncthreads();
         for (int pos = tid; pos < p.n1_max; pos += UM_THREADS)
@@ -701,7 +781,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   // ---- free the tensor memory ----
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == 1) {
     __syncwarp();
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
