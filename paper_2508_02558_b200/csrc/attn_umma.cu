@@ -312,7 +312,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   const uint32_t bars = smem_u32(smem);
   auto BAR = [&](int i) { return bars + 8u * (uint32_t)i; };
   const int Q_FULL = 0, FULL_K = 1, FULL_V = 1 + NS, EMPTY_K = 1 + 2 * NS, EMPTY_V = 1 + 3 * NS;
-  const int S_FULL = 1 + 4 * NS, P_FULL = S_FULL + 2, PV_DONE = S_FULL + 4, DRAIN = S_FULL + 5;
+  const int S_FULL = 1 + 4 * NS, P_FULL = S_FULL + 2, PV_DONE = S_FULL + 4, DRAIN = S_FULL + 6;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 260);
   int* last_flag = reinterpret_cast<int*>(smem + 264);
@@ -376,8 +376,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     for (int i = 0; i < 2; ++i) {
       mbar_init(BAR(S_FULL + i), 1);
       mbar_init(BAR(P_FULL + i), 4);
+      mbar_init(BAR(PV_DONE + i), 1);
     }
-    mbar_init(BAR(PV_DONE), 1);
     mbar_init(BAR(DRAIN), 1);
     *abort_flag = 0;
     *last_flag = 0;
@@ -442,7 +442,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         for (int ks = 0; ks < x.n_mma / 16; ++ks)
           mma_ts(tmem_base + O_COL, a_t + ks * 8, smem_desc(vsm + ks * 2048, (uint32_t)half_bytes, 1024u), idesc_pv,
                  (j > 0 || ks > 0) ? 1u : 0u);
-        tc_commit(BAR(PV_DONE));       // phase j of this barrier completes when O holds tiles 0..j
+        tc_commit(BAR(PV_DONE + pb));  // two alternating barriers: a waiter is never a whole phase ahead of either
         tc_commit(BAR(EMPTY_V + s));
         return true;
       };
@@ -523,7 +523,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         }
         if (it > 0 && __any_sync(0xffffffffu, grow)) {
           // every PV issued so far must have landed before the rows are rewritten; PV of this tile waits for our arrive
-          if (!wait_bar_warp(BAR(PV_DONE), (it - 1) & 1, abort_flag, p.status, 8)) { ok = false; break; }
+          if (!wait_bar_warp(BAR(PV_DONE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag, p.status, 8)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll
           for (int c = 0; c < D / 32; ++c) {
@@ -583,7 +583,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
       // ---- the finished accumulator row: TMEM -> registers ----
 #pragma unroll
       for (int d = 0; d < D; ++d) o_reg[d] = 0.f;
-      if (ok && it > 0 && wait_bar_warp(BAR(PV_DONE), (it - 1) & 1, abort_flag, p.status, 6)) {
+      if (ok && it > 0 && wait_bar_warp(BAR(PV_DONE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag, p.status, 6)) {
         tc_fence_after();
 #pragma unroll
         for (int c = 0; c < D / 32; ++c) {

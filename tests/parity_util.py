@@ -44,6 +44,12 @@ def assert_close(got: np.ndarray, ref: np.ndarray, dtype: str, what: str):
     lim = a + r * np.abs(ref)
     bad = err > lim
     assert not bad.any(), f"{what}: {bad.sum()} of {bad.size} outside tolerance, max err {err.max():.3e}"
+    # The stated tolerance is loose against outputs that average many small values; what the arithmetic allows
+    # (bf16 P and output rounding, fp32 accumulation) is an error of a few percent of the output's own scale.
+    scale = np.sqrt(np.mean(np.square(ref))) + 1e-30
+    tight = (1e-6 if dtype == "f32" else 1e-2) * np.abs(ref) + (1e-5 if dtype == "f32" else 3e-2) * scale
+    worse = err > tight
+    assert not worse.any(), f"{what}: {worse.sum()} of {worse.size} beyond the arithmetic's own error, max err {err.max():.3e}, scale {scale:.3e}"
 
 
 @dataclass
