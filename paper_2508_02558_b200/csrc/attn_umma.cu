@@ -282,6 +282,22 @@ __global__ void __launch_bounds__(256) umma_tail_kernel(const UmmaParams up, con
   p.pooled[idx] = pool_at(p, p.raw_scores + bh * p.n1_max, L, p.block_off[bi], pos);
 }
 
+// Optional timeline of CTA (0,0,0): built with -DSDLLM_TRACE, each point stores the global timer in the 8-byte slot
+// `slot` (1..31) of the workspace's 256-byte status block. Compiled out by default.
+#ifdef SDLLM_TRACE
+__device__ __forceinline__ void trace_point(int32_t* status, int slot) {
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    reinterpret_cast<unsigned long long*>(status)[slot] = t;
+    if (slot == 1 || slot == 15) reinterpret_cast<long long*>(status)[slot == 1 ? 30 : 31] = clock64();
+  }
+}
+#define TRACE(slot) trace_point(p.status, slot)
+#else
+#define TRACE(slot) do { } while (0)
+#endif
+
 template <int D>
 __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __grid_constant__ UmmaMaps tm, const UmmaParams up) {
   constexpr int H = D / 64;            // 128-byte column halves of a row
@@ -296,6 +312,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   const int bi = blockIdx.z;
   const int g = blockIdx.y / up.row_tiles, rt = blockIdx.y - g * up.row_tiles;
   const int split = blockIdx.x;
+  if (tid == 0) TRACE(1);
   const int tiles1 = (p.n1_max + KT - 1) / KT;
   const int tiles2 = (p.n2 + KT2 - 1) / KT2;
   const int tiles_all = tiles1 + tiles2;
@@ -382,11 +399,14 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     *abort_flag = 0;
     *last_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    TRACE(2);
     if (!zero_q && (do_attn || do_scores)) {
       grid_dependency_wait();          // the loads below read what earlier kernels in the stream wrote
       prod_n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
       prod_n1 = min(max(prod_n1, 0), p.n1_max);
+      TRACE(4);
       produce(NS);                     // the first NS slots are free: no waiting here
+      TRACE(5);
     }
   }
   if (zero_q)
@@ -400,6 +420,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (tid == 0) TRACE(3);
 
   grid_dependency_wait();              // everything below may read what earlier kernels in the stream wrote
   grid_launch_dependents();
@@ -408,8 +429,9 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   n1 = min(max(n1, 0), p.n1_max);
 
   // softmax state of this thread's accumulator row (softmax warps only)
-  float o_reg[D];
   float m_run = -INFINITY, l_run = 0.f;
+  bool sm_ok = true;
+  int sm_tiles = 0;
 
   if (warp == 0) {
     // ======================================= TMA producer =======================================
@@ -435,7 +457,9 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
       auto issue_pv = [&](const Tile& x, int j) -> bool {
         const int s = j % NS, pb = j & 1;
         if (!wait_bar(BAR(P_FULL + pb), (j >> 1) & 1, abort_flag, p.status, 4)) return false;
+        if (j == 0) TRACE(8);
         if (!wait_bar(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 5)) return false;
+        if (j == 0) TRACE(9);
         tc_fence_after();
         const uint32_t vsm = smem_u32(stage0 + (size_t)s * stage_bytes) + kv_bytes;
         const uint32_t a_t = tmem_base + (uint32_t)pb * 128u;
@@ -455,6 +479,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
           if (!wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 3)) { ok = false; break; }
           have_q = true;
         }
+        if (it == 0) TRACE(7);
         tc_fence_after();
         const uint32_t ksm = smem_u32(stage0 + (size_t)s * stage_bytes);
         const uint32_t qsm = smem_u32(q_s);
@@ -495,6 +520,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         // columns of this tile owned by this replica
         const int c_lo = min(rep * chunk_keys, x.nv), c_hi = min((rep + 1) * chunk_keys, x.nv);
         if (!wait_bar_warp(BAR(S_FULL + sb), (it >> 1) & 1, abort_flag, p.status, 9)) { ok = false; break; }
+        if (tid == 64) TRACE(it == 0 ? 10 : (it == 1 ? 16 : 18));
         tc_fence_after();
         const uint32_t s_addr = lane_addr + (uint32_t)sb * 128u;
         // ---- the owned part of the S row, all loads in flight together ----
@@ -503,10 +529,16 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         for (int c = 0; c < 4; ++c)
           if (c * 32 < c_hi && c * 32 + 32 > c_lo) tmem_ld32(s_addr + c * 32, sv[c]);
         tc_wait_ld();
+        if (tid == 64 && it == 1) TRACE(23);
         float mx = -INFINITY;
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-          if (c * 32 < c_hi && c * 32 + 32 > c_lo) {
+          if (c * 32 >= c_lo && c * 32 + 32 <= c_hi) {        // whole chunk owned and valid
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(sv[c][i]));
+            mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
+          } else if (c * 32 < c_hi && c * 32 + 32 > c_lo) {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
               if (c * 32 + i >= c_lo && c * 32 + i < c_hi) mx = fmaxf(mx, __uint_as_float(sv[c][i]));
@@ -541,13 +573,24 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
           }
         }
         const float mu = (m_run == -INFINITY) ? 0.f : m_run;
+        if (tid == 64 && it == 1) TRACE(24);
         // ---- P = exp2(S * scale_log2 - mu) as bf16 over the S columns; zero outside the owned slice ----
         float psum = 0.f;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           if (c * 32 >= x.n_mma) continue;
           uint32_t pk[16];
-          if (c * 32 < c_hi && c * 32 + 32 > c_lo) {
+          if (c * 32 >= c_lo && c * 32 + 32 <= c_hi) {        // whole chunk owned and valid
+            float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float e0 = fast_exp2(fmaf(__uint_as_float(sv[c][2 * i]), p.scale_log2, -mu));
+              const float e1 = fast_exp2(fmaf(__uint_as_float(sv[c][2 * i + 1]), p.scale_log2, -mu));
+              ps4[i & 3] += e0 + e1;
+              pk[i] = pack_bf16(e0, e1);
+            }
+            psum += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
+          } else if (c * 32 < c_hi && c * 32 + 32 > c_lo) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
               const int j0 = c * 32 + 2 * i;
@@ -563,6 +606,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
           tmem_st16(s_addr + c * 16, pk);
         }
         l_run += psum;
+        if (tid == 64 && it == 1) TRACE(25);
         // ---- V rows past the source's count may hold anything: zero them so that 0 * V stays 0 ----
         if (x.nv < x.n_mma) {
           if (!wait_bar_warp(BAR(FULL_V + s), (it / NS) & 1, abort_flag, p.status, 10)) { ok = false; break; }
@@ -575,25 +619,15 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
           fence_proxy_async();
         }
         tc_wait_st();
+        if (tid == 64 && it == 1) TRACE(26);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(BAR(P_FULL + sb));
+        if (tid == 64) TRACE(it == 0 ? 11 : (it == 1 ? 17 : 19));
         ++it;
       }
-      // ---- the finished accumulator row: TMEM -> registers ----
-#pragma unroll
-      for (int d = 0; d < D; ++d) o_reg[d] = 0.f;
-      if (ok && it > 0 && wait_bar_warp(BAR(PV_DONE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag, p.status, 6)) {
-        tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t ov[32];
-          tmem_ld32(lane_addr + O_COL + c * 32, ov);
-          tc_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o_reg[c * 32 + i] = __uint_as_float(ov[i]);
-        }
-      }
+      if (tid == 64) TRACE(12);
+      sm_ok = ok; sm_tiles = it;
     }
   } else {
     // ======================================= saliency warps (refresh) =======================================
@@ -643,107 +677,98 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(BAR(EMPTY_K + s));
+        if (tid == 192) TRACE(it == 0 ? 20 : (it == 1 ? 21 : 22));
         ++it;
       }
       // the softmax warps reuse the ring as scratch once they are done: tell them the K tiles are no longer read
-      if (do_attn && R > 1) asm volatile("bar.sync 3, 192;\n" ::: "memory");
+      if (do_attn) asm volatile("bar.sync 3, 192;\n" ::: "memory");
     }
   }
 
   // ======================================= epilogue =======================================
+  // The ring is idle now (every load was consumed), so it serves as scratch for the way out of TMEM:
+  //   o_s [128][D] fp32, the float4 index XOR-swizzled by the row; ml_s [128]; lm_s [rows_rep].
+  // Each accumulator row is weighted for the merge of the R replicas while it moves from TMEM to shared memory;
+  // then consecutive threads store consecutive float4 of a row, so every global store is coalesced.
   const int64_t unit = (int64_t)(bi * p.Hkv + g) * up.row_tiles + rt;      // (sequence, KV head, row tile)
   if (do_attn && warp >= 2 && warp < 6) {
     constexpr int D4 = D / 4;
-    const int row = (warp & 3) * 32 + lane;
+    const int q4 = warp & 3;
+    const int row = q4 * 32 + lane;
     const int rep = row / rows_rep, m_local = row - rep * rows_rep;
-    if (R == 1) {
-      // one accumulator row per query row: straight from registers
-      if (m_local < M_rt && !*abort_flag) {
-        const int m = rt * 128 + m_local;              // row within the KV head: m = head_in_group * b + i
+    float* o_s = reinterpret_cast<float*>(stage0);
+    float2* ml_s = reinterpret_cast<float2*>(stage0 + 128 * D * 4);
+    float2* lm_s = ml_s + 128;
+    if (do_scores) asm volatile("bar.sync 3, 192;\n" ::: "memory");      // the saliency warps have left the ring
+    ml_s[row] = make_float2(m_run, l_run);
+    asm volatile("bar.sync 2, 128;\n" ::: "memory");
+    float mstar = -INFINITY;
+    for (int r2 = 0; r2 < R; ++r2) {
+      const float2 x = ml_s[r2 * rows_rep + m_local];
+      if (x.y > 0.f) mstar = fmaxf(mstar, x.x);
+    }
+    float lsum = 0.f;
+    for (int r2 = 0; r2 < R; ++r2) {
+      const float2 x = ml_s[r2 * rows_rep + m_local];
+      if (x.y > 0.f) lsum = fmaf(x.y, fast_exp2(x.x - mstar), lsum);
+    }
+    const float w = l_run > 0.f ? fast_exp2(m_run - mstar) : 0.f;       // this replica's weight in the merged row
+    if (rep == 0) lm_s[m_local] = make_float2(mstar, lsum);
+    // the finished accumulator row: TMEM -> weight -> shared memory, 32 columns at a time
+    const bool have_o = sm_ok && sm_tiles > 0 &&
+                        wait_bar_warp(BAR(PV_DONE + ((sm_tiles - 1) & 1)), ((sm_tiles - 1) >> 1) & 1, abort_flag, p.status, 6);
+    tc_fence_after();
+#pragma unroll 1
+    for (int c = 0; c < D / 32; ++c) {
+      uint32_t ov[32];
+      if (have_o) {
+        tmem_ld32(tmem_base + ((uint32_t)(q4 * 32) << 16) + O_COL + c * 32, ov);
+        tc_wait_ld();
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) ov[i] = 0u;
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        *reinterpret_cast<float4*>(o_s + row * D + (((c * 8 + j) ^ (row & (D4 - 1))) << 2)) =
+            make_float4(__uint_as_float(ov[4 * j]) * w, __uint_as_float(ov[4 * j + 1]) * w, __uint_as_float(ov[4 * j + 2]) * w,
+                        __uint_as_float(ov[4 * j + 3]) * w);
+    }
+    if (tid == 64) TRACE(27);
+    asm volatile("bar.sync 2, 128;\n" ::: "memory");
+    if (tid == 64) TRACE(29);
+    const int st = (warp - 2) * 32 + lane;
+    if (!*abort_flag) {
+#pragma unroll 2
+      for (int slot = st; slot < M_rt * D4; slot += 128) {
+        const int ml = slot / D4, d4 = slot - ml * D4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int r2 = 0; r2 < R; ++r2) {
+          const int rr = r2 * rows_rep + ml;
+          const float4 o = *reinterpret_cast<const float4*>(o_s + rr * D + ((d4 ^ (rr & (D4 - 1))) << 2));
+          acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+        }
+        const float2 x = lm_s[ml];
+        const int m = rt * 128 + ml;                   // row within the KV head: m = head_in_group * b + i
         const int hg = m / p.b, i = m - hg * p.b;
         if (p.splits == 1) {
-          const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+          const float inv = x.y > 0.f ? 1.f / x.y : 0.f;
           __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
-                             (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2];
-#pragma unroll
-          for (int d = 0; d < D; d += 8) {
-            uint4 w;
-            w.x = pack_bf16(o_reg[d] * inv, o_reg[d + 1] * inv);
-            w.y = pack_bf16(o_reg[d + 2] * inv, o_reg[d + 3] * inv);
-            w.z = pack_bf16(o_reg[d + 4] * inv, o_reg[d + 5] * inv);
-            w.w = pack_bf16(o_reg[d + 6] * inv, o_reg[d + 7] * inv);
-            *reinterpret_cast<uint4*>(o + d) = w;
-          }
-          if (p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (m_run + log2f(l_run)) * kLn2;
+                             (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
+          uint2 w2;
+          w2.x = pack_bf16(acc.x * inv, acc.y * inv);
+          w2.y = pack_bf16(acc.z * inv, acc.w * inv);
+          *reinterpret_cast<uint2*>(o) = w2;
+          if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (x.x + log2f(x.y)) * kLn2;
         } else {
-          const int64_t prow = (unit * p.splits + split) * 128 + m_local;
-          float* o = p.part_o + prow * D;
-#pragma unroll
-          for (int d = 0; d < D; d += 4)
-            *reinterpret_cast<float4*>(o + d) = make_float4(o_reg[d], o_reg[d + 1], o_reg[d + 2], o_reg[d + 3]);
-          reinterpret_cast<float2*>(p.part_ml)[prow] = make_float2(m_run, l_run);
-        }
-      }
-    } else {
-      // The R replicas of a query row sit in different accumulator rows: merge them through shared memory. The ring
-      // is idle now (every load was consumed, the last PV has landed), so it serves as scratch:
-      //   o_s [128][D] fp32, the float4 index XOR-swizzled by the row; ml_s [128]; lm_s [rows_rep].
-      float* o_s = reinterpret_cast<float*>(stage0);
-      float2* ml_s = reinterpret_cast<float2*>(stage0 + 128 * D * 4);
-      float2* lm_s = ml_s + 128;
-      if (do_scores) asm volatile("bar.sync 3, 192;\n" ::: "memory");    // the saliency warps have left the ring
-      ml_s[row] = make_float2(m_run, l_run);
-      asm volatile("bar.sync 2, 128;\n" ::: "memory");
-      float mstar = -INFINITY;
-      for (int r2 = 0; r2 < R; ++r2) {
-        const float2 x = ml_s[r2 * rows_rep + m_local];
-        if (x.y > 0.f) mstar = fmaxf(mstar, x.x);
-      }
-      float lsum = 0.f;
-      for (int r2 = 0; r2 < R; ++r2) {
-        const float2 x = ml_s[r2 * rows_rep + m_local];
-        if (x.y > 0.f) lsum = fmaf(x.y, fast_exp2(x.x - mstar), lsum);
-      }
-      const float w = l_run > 0.f ? fast_exp2(m_run - mstar) : 0.f;   // this replica's weight in the merged row
-      if (rep == 0) lm_s[m_local] = make_float2(mstar, lsum);
-#pragma unroll
-      for (int j = 0; j < D4; ++j)
-        *reinterpret_cast<float4*>(o_s + row * D + ((j ^ (row & (D4 - 1))) << 2)) =
-            make_float4(o_reg[4 * j] * w, o_reg[4 * j + 1] * w, o_reg[4 * j + 2] * w, o_reg[4 * j + 3] * w);
-      asm volatile("bar.sync 2, 128;\n" ::: "memory");
-      // consecutive threads take consecutive float4 of a row: coalesced stores
-      const int st = (warp - 2) * 32 + lane;
-      if (!*abort_flag) {
-#pragma unroll 4
-        for (int slot = st; slot < M_rt * D4; slot += 128) {
-          const int ml = slot / D4, d4 = slot - ml * D4;
-          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-          for (int r2 = 0; r2 < R; ++r2) {
-            const int rr = r2 * rows_rep + ml;
-            const float4 o = *reinterpret_cast<const float4*>(o_s + rr * D + ((d4 ^ (rr & (D4 - 1))) << 2));
-            acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
-          }
-          const float2 x = lm_s[ml];
-          const int m = rt * 128 + ml;
-          const int hg = m / p.b, i = m - hg * p.b;
-          if (p.splits == 1) {
-            const float inv = x.y > 0.f ? 1.f / x.y : 0.f;
-            __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
-                               (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
-            uint2 w2;
-            w2.x = pack_bf16(acc.x * inv, acc.y * inv);
-            w2.y = pack_bf16(acc.z * inv, acc.w * inv);
-            *reinterpret_cast<uint2*>(o) = w2;
-            if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (x.x + log2f(x.y)) * kLn2;
-          } else {
-            const int64_t prow = (unit * p.splits + split) * 128 + ml;
-            *reinterpret_cast<float4*>(p.part_o + prow * D + d4 * 4) = acc;
-            if (d4 == 0) reinterpret_cast<float2*>(p.part_ml)[prow] = x;
-          }
+          const int64_t prow = (unit * p.splits + split) * 128 + ml;
+          *reinterpret_cast<float4*>(p.part_o + prow * D + d4 * 4) = acc;
+          if (d4 == 0) reinterpret_cast<float2*>(p.part_ml)[prow] = x;
         }
       }
     }
   }
+  if (tid == 64) TRACE(13);
 
   // ---- fused tail: the last CTA of the unit merges the key splits and pools the saliency; nobody waits ----
   const bool tail_merge = do_attn && p.splits > 1;
@@ -779,6 +804,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   }
 
   // ---- free the tensor memory ----
+  if (tid == 64) TRACE(14);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -786,6 +812,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
+  if (tid == 0) TRACE(15);
 }
 
 // ---------------------------------------------------------------------------------------------------------
