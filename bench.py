@@ -268,7 +268,9 @@ def run_ours(args):
                 dist.barrier()
         return e0.elapsed_time(e1) / 1e3
 
-    launches_per_step = n_layers * (4 + 2 * reuse_steps)
+    d0 = caches[0].desc
+    launches_per_step = n_layers * (B.launch_count(d0, B.OP_REFRESH_SCORES) + B.launch_count(d0, B.OP_SELECT_TOPK) +
+                                    B.launch_count(d0, B.OP_COMPACT_KV) + reuse_steps * B.launch_count(d0, B.OP_SPARSE_BLOCK_ATTN))
     step_runner = make_runner(one_step)
     sampler = ClockSampler(local) if rank == 0 else None
     sec = timed(step_runner, args.steps, max(args.warmup, 3))
@@ -288,7 +290,7 @@ def run_ours(args):
     rf_sec = timed(rf_runner, max(3, args.steps // 2), 3) / max(3, args.steps // 2) / n_layers
     peak, peak_kind = peaks()
     achieved = ab["sparse"] / sp_sec / 1e9
-    roofline = {"bound": "hbm", "kernel": "sdllm_sparse_block_attn (split-K partial + merge)", "achieved": achieved,
+    roofline = {"bound": "hbm", "kernel": "sdllm_sparse_block_attn (attn_umma_bf16_kernel<128>: tcgen05 attention, fused split merge)", "achieved": achieved,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                 "frac_of_8TBps": achieved / 8000.0, "algorithmic_bytes_per_launch": ab["sparse"], "us_per_launch": sp_sec * 1e6,
                 "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),

@@ -116,6 +116,10 @@ sdllm_status sdllm_keep_count(const sdllm_desc* desc, int32_t seq_len, int32_t b
  * 0 = dense step (cache unused), 1 = refresh (run Algorithm 1), 2 = reuse the compacted cache. */
 int32_t sdllm_cache_state(int32_t step_in_block, int32_t delay);
 
+/* Host-only. Number of kernels one call of `op` launches for this description (refresh with all outputs requested);
+ * -1 for an invalid description or op. Lets a caller account for its launches without tracing them. */
+int32_t sdllm_launch_count(const sdllm_desc* desc, int op);
+
 /* Reads the device status word kept in the first 4 bytes of an attention workspace. The kernels bound every wait
  * on a shared-memory barrier; if one ever expires they record a non-zero code there and run to the end instead of
  * hanging (the outputs of that call are then invalid). The caller zeroes those 4 bytes once after allocating the

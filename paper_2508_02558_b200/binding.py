@@ -20,7 +20,7 @@ POOL_MAX, POOL_AVG = 0, 1
 SELECT_JOINT_FLOOR, SELECT_PER_REGION_CEIL, SELECT_PREFIX_ONLY = 0, 1, 2
 OP_REFRESH_SCORES, OP_SELECT_TOPK, OP_COMPACT_KV, OP_SPARSE_BLOCK_ATTN = range(4)
 
-EXPORTS = ("sdllm_version", "sdllm_status_string", "sdllm_workspace_bytes", "sdllm_keep_count", "sdllm_cache_state",
+EXPORTS = ("sdllm_version", "sdllm_status_string", "sdllm_workspace_bytes", "sdllm_keep_count", "sdllm_cache_state", "sdllm_launch_count",
            "sdllm_read_status",
            "sdllm_refresh_scores", "sdllm_select_topk", "sdllm_compact_kv", "sdllm_sparse_block_attn")
 
@@ -63,6 +63,8 @@ def lib() -> ctypes.CDLL:
         L.sdllm_workspace_bytes.argtypes = [dp, ctypes.c_int]
         L.sdllm_keep_count.restype = ctypes.c_int
         L.sdllm_keep_count.argtypes = [dp, ctypes.c_int32, ctypes.c_int32] + [ctypes.POINTER(ctypes.c_int32)] * 3
+        L.sdllm_launch_count.restype = ctypes.c_int32
+        L.sdllm_launch_count.argtypes = [ctypes.POINTER(Desc), ctypes.c_int]
         L.sdllm_cache_state.restype = ctypes.c_int32
         L.sdllm_cache_state.argtypes = [ctypes.c_int32, ctypes.c_int32]
         L.sdllm_read_status.restype = ctypes.c_int
@@ -153,6 +155,10 @@ def keep_count(desc: Desc, seq_len: int, block_off: int):
     _check(lib().sdllm_keep_count(ctypes.byref(desc), int(seq_len), int(block_off), *[ctypes.byref(x) for x in n]),
            "sdllm_keep_count")
     return n[0].value, n[1].value, n[2].value
+
+
+def launch_count(desc: Desc, op: int) -> int:
+    return int(lib().sdllm_launch_count(ctypes.byref(desc), int(op)))
 
 
 def cache_state(step_in_block: int, delay: int = 1) -> int:

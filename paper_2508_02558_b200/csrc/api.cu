@@ -139,6 +139,21 @@ sdllm_status sdllm_keep_count(const sdllm_desc* d, int32_t seq_len, int32_t bloc
   return SDLLM_OK;
 }
 
+int32_t sdllm_launch_count(const sdllm_desc* d, int op) {
+  if (check_desc(d) != SDLLM_OK) return -1;
+  if (op == SDLLM_OP_SELECT_TOPK) return 1;
+  if (op == SDLLM_OP_COMPACT_KV) return d->n_keep_max > 0 ? 1 : 0;
+  if (op != SDLLM_OP_REFRESH_SCORES && op != SDLLM_OP_SPARSE_BLOCK_ATTN) return -1;
+  const bool refresh = op == SDLLM_OP_REFRESH_SCORES;
+  const AttnPlan pl = plan_for(d, op);
+  const int M = d->n_q_heads / d->n_kv_heads * d->block_len;
+  if (pl.kind == 2) {
+    const bool tail_work = pl.splits > 1 || refresh;
+    return 1 + ((tail_work && !umma_tail_is_fused(pl, d->head_dim, M, refresh ? d->seq_len_max : d->n_keep_max, refresh)) ? 1 : 0);
+  }
+  return 1 + ((refresh || pl.splits > 1) ? 1 : 0);
+}
+
 int32_t sdllm_cache_state(int32_t i, int32_t delay) { return i > delay ? 2 : (i == delay ? 1 : 0); }
 
 sdllm_status sdllm_read_status(const void* workspace, void* cuda_stream, int32_t* device_status) {

@@ -891,6 +891,15 @@ bool umma_supported(int dtype, int D, int M, int b) {
   return M <= 128 || 128 % b == 0;
 }
 
+// The last CTA of a unit does the tail itself while that is a small job; otherwise a second launch spreads it over
+// the whole GPU.
+bool umma_tail_is_fused(const AttnPlan& pl, int D, int M, int n1_max, bool pool) {
+  const size_t merge_bytes = pl.splits > 1 ? (size_t)pl.splits * (M < 128 ? M : 128) * D * 4 : 0;
+  bool fused = merge_bytes <= 256 * 1024 && (!pool || n1_max <= 8192);
+  if (const char* e = getenv("SDLLM_FUSED_TAIL")) fused = e[0] == '1' && (!pool || n1_max <= 8192);   // tuning aid
+  return fused;
+}
+
 AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, int n2) {
   AttnPlan pl{};
   pl.kind = 2; pl.tma = true; pl.cluster = 1; pl.fused_tail = true;
@@ -930,12 +939,8 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
   up.a.splits = pl.splits;
   up.KT = pl.key_tile; up.KT2 = pl.key_tile2; up.R = pl.rep; up.row_tiles = pl.row_tiles;
   up.heads_rt = pl.row_tiles == 1 ? p.G : 128 / p.b;
-  // The last CTA of a unit does the tail itself while that is a small job; otherwise a second launch spreads it
-  // over the whole GPU.
-  const size_t merge_bytes = pl.splits > 1 ? (size_t)pl.splits * (p.M < 128 ? p.M : 128) * D * 4 : 0;
   const bool pool = p.want_scores && p.pooled != nullptr;
-  up.fused_tail = (merge_bytes <= 256 * 1024 && (!pool || p.n1_max <= 8192)) ? 1 : 0;
-  if (const char* e = getenv("SDLLM_FUSED_TAIL")) up.fused_tail = e[0] == '1' && (!pool || p.n1_max <= 8192);   // tuning aid
+  up.fused_tail = umma_tail_is_fused(pl, D, p.M, p.n1_max, pool) ? 1 : 0;
   memset(&tm, 0, sizeof(tm));
   bool ok = true;
   if (p.out != nullptr) ok = make_map(&tm.q, p.q, D, p.b, p.Hq, p.B, p.q_stride, p.b, up.heads_rt);

@@ -95,6 +95,7 @@ struct CompactParams {
 
 AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_max, int n2);
 
+bool umma_tail_is_fused(const AttnPlan& pl, int D, int M, int n1_max, bool pool);
 cudaError_t launch_attn_partial(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st);
 cudaError_t launch_merge_pool(const MergeParams& p, cudaStream_t st);
 cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st);
