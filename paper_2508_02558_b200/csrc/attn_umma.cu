@@ -122,6 +122,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
@@ -523,26 +530,32 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         if (tid == 64) TRACE(it == 0 ? 10 : (it == 1 ? 16 : 18));
         tc_fence_after();
         const uint32_t s_addr = lane_addr + (uint32_t)sb * 128u;
-        // ---- the owned part of the S row, all loads in flight together ----
+        // ---- the owned part of the S row. Chunks of 32 columns that are owned and valid as a whole go through the
+        //      unrolled register path, all their loads in flight together; the one chunk the end of the slice may cut
+        //      (cp) takes a small predicated path of its own, so the common code stays short ----
+        const int cf_lo = c_lo >> 5, cf_hi = c_hi >> 5;          // full chunks [cf_lo, cf_hi); c_lo is a multiple of 32
+        const int cp = (c_hi & 31) && c_lo < c_hi ? cf_hi : -1;  // partial chunk, if any
         uint32_t sv[4][32];
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-          if (c * 32 < c_hi && c * 32 + 32 > c_lo) tmem_ld32(s_addr + c * 32, sv[c]);
+          if (c >= cf_lo && c < cf_hi) tmem_ld32(s_addr + c * 32, sv[c]);
+        uint32_t tv[32];
+        if (cp >= 0) tmem_ld32(s_addr + cp * 32, tv);
         tc_wait_ld();
-        if (tid == 64 && it == 1) TRACE(23);
         float mx = -INFINITY;
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-          if (c * 32 >= c_lo && c * 32 + 32 <= c_hi) {        // whole chunk owned and valid
+          if (c >= cf_lo && c < cf_hi) {
             float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
             for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(sv[c][i]));
             mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
-          } else if (c * 32 < c_hi && c * 32 + 32 > c_lo) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (c * 32 + i >= c_lo && c * 32 + i < c_hi) mx = fmaxf(mx, __uint_as_float(sv[c][i]));
           }
+        if (cp >= 0) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (cp * 32 + i >= c_lo && cp * 32 + i < c_hi) mx = fmaxf(mx, __uint_as_float(tv[i]));
+        }
         // ---- running maximum: O (in TMEM) and l are rescaled only when the maximum grows by more than 2^8, so P stays
         //      below 2^8 and the accumulator is touched on very few tiles ----
         const float m_new = fmaxf(m_run, mx * p.scale_log2);
@@ -557,30 +570,23 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
           // every PV issued so far must have landed before the rows are rewritten; PV of this tile waits for our arrive
           if (!wait_bar_warp(BAR(PV_DONE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag, p.status, 8)) { ok = false; break; }
           tc_fence_after();
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t ov[32];
-            tmem_ld32(lane_addr + O_COL + c * 32, ov);
+#pragma unroll 1
+          for (int c = 0; c < D / 16; ++c) {
+            uint32_t ov[16];
+            tmem_ld16(lane_addr + O_COL + c * 16, ov);
             tc_wait_ld();
-            uint32_t lo[16], hi[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              lo[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-              hi[i] = __float_as_uint(__uint_as_float(ov[16 + i]) * alpha);
-            }
-            tmem_st16(lane_addr + O_COL + c * 32, lo);
-            tmem_st16(lane_addr + O_COL + c * 32 + 16, hi);
+            for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+            tmem_st16(lane_addr + O_COL + c * 16, ov);
           }
         }
         const float mu = (m_run == -INFINITY) ? 0.f : m_run;
-        if (tid == 64 && it == 1) TRACE(24);
         // ---- P = exp2(S * scale_log2 - mu) as bf16 over the S columns; zero outside the owned slice ----
         float psum = 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          if (c * 32 >= x.n_mma) continue;
-          uint32_t pk[16];
-          if (c * 32 >= c_lo && c * 32 + 32 <= c_hi) {        // whole chunk owned and valid
+        for (int c = 0; c < 4; ++c)
+          if (c >= cf_lo && c < cf_hi) {
+            uint32_t pk[16];
             float ps4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
@@ -590,23 +596,29 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
               pk[i] = pack_bf16(e0, e1);
             }
             psum += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
-          } else if (c * 32 < c_hi && c * 32 + 32 > c_lo) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const int j0 = c * 32 + 2 * i;
-              const float e0 = (j0 >= c_lo && j0 < c_hi) ? fast_exp2(fmaf(__uint_as_float(sv[c][2 * i]), p.scale_log2, -mu)) : 0.f;
-              const float e1 = (j0 + 1 >= c_lo && j0 + 1 < c_hi) ? fast_exp2(fmaf(__uint_as_float(sv[c][2 * i + 1]), p.scale_log2, -mu)) : 0.f;
-              psum += e0 + e1;
-              pk[i] = pack_bf16(e0, e1);
-            }
-          } else {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+            tmem_st16(s_addr + c * 16, pk);
           }
-          tmem_st16(s_addr + c * 16, pk);
+        if (cp >= 0) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int j0 = cp * 32 + 2 * i;
+            const float e0 = (j0 >= c_lo && j0 < c_hi) ? fast_exp2(fmaf(__uint_as_float(tv[2 * i]), p.scale_log2, -mu)) : 0.f;
+            const float e1 = (j0 + 1 >= c_lo && j0 + 1 < c_hi) ? fast_exp2(fmaf(__uint_as_float(tv[2 * i + 1]), p.scale_log2, -mu)) : 0.f;
+            psum += e0 + e1;
+            pk[i] = pack_bf16(e0, e1);
+          }
+          tmem_st16(s_addr + cp * 16, pk);
+        }
+        if (R > 1) {                                    // the other replicas' slices of this tile read as zero
+          uint32_t zz[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) zz[i] = 0u;
+#pragma unroll 1
+          for (int c = 0; c * 32 < x.n_mma; ++c)
+            if (!(c >= cf_lo && c < cf_hi) && c != cp) tmem_st16(s_addr + c * 16, zz);
         }
         l_run += psum;
-        if (tid == 64 && it == 1) TRACE(25);
         // ---- V rows past the source's count may hold anything: zero them so that 0 * V stays 0 ----
         if (x.nv < x.n_mma) {
           if (!wait_bar_warp(BAR(FULL_V + s), (it / NS) & 1, abort_flag, p.status, 10)) { ok = false; break; }
