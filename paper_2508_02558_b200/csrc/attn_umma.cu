@@ -219,11 +219,12 @@ __device__ __forceinline__ float pool_at(const AttnParams& p, const float* a, in
 template <int D>
 __device__ __forceinline__ void merge_slot(const AttnParams& p, int64_t unit, int bi, int g, int rt, int m_local, int d4) {
   const int P = p.splits;
-  const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + unit * P * 128 + m_local;
-  const float4* po = reinterpret_cast<const float4*>(p.part_o + (unit * P * 128 + m_local) * D) + d4;
+  const int prt = min(p.M, 128);                      // rows of one partial
+  const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + unit * P * prt + m_local;
+  const float4* po = reinterpret_cast<const float4*>(p.part_o + (unit * P * prt + m_local) * D) + d4;
   float mstar = -INFINITY;
   for (int pi = 0; pi < P; ++pi) {
-    const float2 x = __ldcg(ml + (int64_t)pi * 128);
+    const float2 x = __ldcg(ml + (int64_t)pi * prt);
     if (x.y > 0.f) mstar = fmaxf(mstar, x.x);
   }
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -234,8 +235,8 @@ __device__ __forceinline__ void merge_slot(const AttnParams& p, int64_t unit, in
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int pi = min(p0 + u, P - 1);
-      x[u] = __ldcg(ml + (int64_t)pi * 128);
-      o[u] = __ldcg(po + (int64_t)pi * 128 * (D / 4));
+      x[u] = __ldcg(ml + (int64_t)pi * prt);
+      o[u] = __ldcg(po + (int64_t)pi * prt * (D / 4));
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
@@ -773,7 +774,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
           *reinterpret_cast<uint2*>(o) = w2;
           if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (x.x + log2f(x.y)) * kLn2;
         } else {
-          const int64_t prow = (unit * p.splits + split) * 128 + ml;
+          const int64_t prow = (unit * p.splits + split) * min(p.M, 128) + ml;
           *reinterpret_cast<float4*>(p.part_o + prow * D + d4 * 4) = acc;
           if (d4 == 0) reinterpret_cast<float2*>(p.part_ml)[prow] = x;
         }
@@ -938,7 +939,7 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
   pl.splits = (int)want;
   pl.parts = pl.splits;                 // replicas are merged inside the CTA
   pl.rows_rep = 128 / pl.rep;
-  pl.part_rows = pl.splits > 1 ? (size_t)pl.row_tiles * pl.splits * 128 : 0;
+  pl.part_rows = pl.splits > 1 ? (size_t)pl.row_tiles * pl.splits * (M < 128 ? M : 128) : 0;
   pl.n_counters = (size_t)B * Hkv * pl.row_tiles;
   pl.smem_bytes = umma_smem_bytes(D, pl.key_tile);
   return pl;
