@@ -157,6 +157,25 @@ sdllm_status sdllm_sparse_block_attn(const sdllm_desc* desc, const void* q_blk, 
                                      const int32_t* kept_cnt, const void* k_blk, const void* v_blk, void* out,
                                      void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The reuse step for callers that cannot allocate device memory. The paper has no counterpart for this call: it
+ * computes exactly what sdllm_sparse_block_attn computes, but takes no workspace. Some hosts of this library run under
+ * a fixed memory plan - an inference server that sized every buffer at start-up, a plug-in whose host owns the
+ * allocator - and must not call cudaMalloc (or any allocating library routine) once they are running; they have
+ * nowhere to get the workspace from. For them the scratch (status word, completion counters, key-split partials) is a
+ * 8 MiB array built into the library image; every GPU that loads the library holds one copy until the process exits.
+ *   - Shapes whose workspace (sdllm_workspace_bytes(desc, SDLLM_OP_SPARSE_BLOCK_ATTN)) exceeds 8 MiB are refused with
+ *     SDLLM_ERR_WORKSPACE; use sdllm_sparse_block_attn with a caller-owned workspace for those.
+ *   - The call allocates and frees nothing. The first call on each device looks the array's device address up
+ *     (cudaGetSymbolAddress, with that device current); make that first call before any stream capture.
+ *   - All calls on a device share the one array and it keeps what the last call left; each call clears the part that
+ *     has to start at zero on its stream. Two calls that overlap on the GPU (different streams) race on it: keep the
+ *     calls of one device in one stream order.
+ *   - There is no workspace pointer to hand to sdllm_read_status; a bounded wait that expired shows as wrong output.
+ * Inputs, outputs, layouts and errors are otherwise those of sdllm_sparse_block_attn. */
+sdllm_status sdllm_sparse_block_attn_static(const sdllm_desc* desc, const void* q_blk, const void* k_c, const void* v_c,
+                                            const int32_t* kept_cnt, const void* k_blk, const void* v_blk, void* out,
+                                            void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,7 +22,8 @@ OP_REFRESH_SCORES, OP_SELECT_TOPK, OP_COMPACT_KV, OP_SPARSE_BLOCK_ATTN = range(4
 
 EXPORTS = ("sdllm_version", "sdllm_status_string", "sdllm_workspace_bytes", "sdllm_keep_count", "sdllm_cache_state", "sdllm_launch_count",
            "sdllm_read_status",
-           "sdllm_refresh_scores", "sdllm_select_topk", "sdllm_compact_kv", "sdllm_sparse_block_attn")
+           "sdllm_refresh_scores", "sdllm_select_topk", "sdllm_compact_kv", "sdllm_sparse_block_attn",
+           "sdllm_sparse_block_attn_static")
 
 
 class Desc(ctypes.Structure):
@@ -71,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.sdllm_read_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
         L.sdllm_refresh_scores.restype = ctypes.c_int
         L.sdllm_refresh_scores.argtypes = [dp, vp, vp, vp, i32p, i32p, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.sdllm_sparse_block_attn_static.restype = ctypes.c_int
+        L.sdllm_sparse_block_attn_static.argtypes = [dp, vp, vp, vp, i32p, vp, vp, vp, vp]
         L.sdllm_select_topk.restype = ctypes.c_int
         L.sdllm_select_topk.argtypes = [dp, vp, i32p, i32p, vp, vp, vp, ctypes.c_size_t, vp]
         L.sdllm_compact_kv.restype = ctypes.c_int
@@ -195,3 +198,10 @@ def sparse_block_attn(desc: Desc, q_blk, k_c, v_c, kept_cnt, k_blk, v_blk, out, 
     _check(lib().sdllm_sparse_block_attn(ctypes.byref(desc), _ptr(q_blk), _ptr(k_c), _ptr(v_c), _ptr(kept_cnt),
                                          _ptr(k_blk), _ptr(v_blk), _ptr(out), _ptr(workspace), _nbytes(workspace),
                                          _stream(stream)), "sdllm_sparse_block_attn")
+
+
+def sparse_block_attn_static(desc: Desc, q_blk, k_c, v_c, kept_cnt, k_blk, v_blk, out, stream=None):
+    """The reuse step without a caller workspace (scratch built into the library; shapes above its 8 MiB are refused)."""
+    _check(lib().sdllm_sparse_block_attn_static(ctypes.byref(desc), _ptr(q_blk), _ptr(k_c), _ptr(v_c), _ptr(kept_cnt),
+                                                _ptr(k_blk), _ptr(v_blk), _ptr(out), _stream(stream)),
+           "sdllm_sparse_block_attn_static")

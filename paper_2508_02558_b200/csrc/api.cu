@@ -3,6 +3,8 @@
 #include <stdio.h>
 #include <stdlib.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 using namespace sdllm;
@@ -99,6 +101,28 @@ void fill_common(AttnParams& p, const sdllm_desc* d, const AttnPlan& pl) {
   p.scale = scale_of(d);
   p.scale_log2 = p.scale * kLog2e;
   for (int i = 0; i < 3; ++i) { p.q_stride[i] = d->q_stride[i]; p.o_stride[i] = d->o_stride[i]; }
+}
+
+// Built-in scratch of sdllm_sparse_block_attn_static: lives in the library image, one copy per GPU that loads it.
+constexpr size_t kStaticScratchBytes = (size_t)8 << 20;
+constexpr int kMaxDevices = 64;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+std::mutex g_static_mutex;
+void* g_static_scratch_ptr[kMaxDevices] = {};      // device address of g_static_scratch on each device, once looked up
+
+// The array's name is only a handle on the host; the address a kernel can use comes from the runtime, per device.
+sdllm_status static_scratch_address(void** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SDLLM_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return SDLLM_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_scratch_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cuda_failed(cudaGetSymbolAddress(&ptr, g_static_scratch), "cudaGetSymbolAddress") || ptr == nullptr) return SDLLM_ERR_CUDA;
+    g_static_scratch_ptr[dev] = ptr;
+  }
+  *out = g_static_scratch_ptr[dev];
+  return SDLLM_OK;
 }
 
 }  // namespace
@@ -284,6 +308,20 @@ sdllm_status sdllm_sparse_block_attn(const sdllm_desc* d, const void* q_blk, con
     if (cuda_failed(launch_merge_pool(m, stream), "merge/pool launch")) return SDLLM_ERR_CUDA;
   }
   return SDLLM_OK;
+}
+
+sdllm_status sdllm_sparse_block_attn_static(const sdllm_desc* d, const void* q_blk, const void* k_c, const void* v_c,
+                                            const int32_t* kept_cnt, const void* k_blk, const void* v_blk, void* out, void* cuda_stream) {
+  sdllm_status st = check_desc(d);
+  if (st != SDLLM_OK) return st;
+  const WsLayout w = attn_ws(d, plan_for(d, SDLLM_OP_SPARSE_BLOCK_ATTN), false);
+  if (w.total > kStaticScratchBytes) return SDLLM_ERR_WORKSPACE;       // this shape needs more than the built-in scratch
+  if ((st = check_device()) != SDLLM_OK) return st;
+  void* scratch = nullptr;
+  if ((st = static_scratch_address(&scratch)) != SDLLM_OK) return st;
+  // the status word and the completion counters must start at zero whatever the last call left behind
+  if (cuda_failed(cudaMemsetAsync(scratch, 0, w.part_o, reinterpret_cast<cudaStream_t>(cuda_stream)), "scratch clear")) return SDLLM_ERR_CUDA;
+  return sdllm_sparse_block_attn(d, q_blk, k_c, v_c, kept_cnt, k_blk, v_blk, out, scratch, kStaticScratchBytes, cuda_stream);
 }
 
 }  // extern "C"
