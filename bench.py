@@ -35,7 +35,7 @@ METRIC = "cached_kv_tokens_per_s_per_layer"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the sparse-attention kernel pair on this workload,
 # from the ncu capture summarised under profiles/ (None until a capture exists for the workload).
-NCU_TRAFFIC_BYTES = {"c2_llada": None}
+NCU_TRAFFIC_BYTES = {"c2_llada": 11113472}
 
 
 def parse_args():
@@ -44,7 +44,10 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2_llada", choices=["c2_llada", "c3_dream"])
+    ap.add_argument("--workload", default="c2_llada", choices=["c2_llada", "c3_dream", "c4_long", "c5_serving"])
+    ap.add_argument("--batch", type=int, default=1, help="sequences per call (c5_serving: ragged prompt lengths)")
+    ap.add_argument("--phase", default="all", choices=["all", "refresh", "sparse"],
+                    help="profiling aid: run only the refresh chain or only the reuse steps in the timed step")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (0 = the workload's)")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-e2e", action="store_true")
@@ -60,20 +63,24 @@ def peaks():
 
 
 # ------------------------------------------------------------------------------------------------ workload
-def tokens_per_step(cfg: W.WorkloadConfig, n_layers: int, n_keep: int) -> int:
+def tokens_per_step(cfg: W.WorkloadConfig, n_layers: int, seq_lens, n_keeps, phase: str = "all") -> int:
     reuse_steps = cfg.steps_per_block - 2
-    return n_layers * (cfg.seq_len + reuse_steps * (n_keep + cfg.block_len))
+    refresh = sum(seq_lens) if phase in ("all", "refresh") else 0
+    sparse = reuse_steps * sum(n + cfg.block_len for n in n_keeps) if phase in ("all", "sparse") else 0
+    return n_layers * (refresh + sparse)
 
 
-def algorithmic_bytes(cfg: W.WorkloadConfig, n_keep: int):
-    """Bytes each call must move (K and V once, Q and O once, scores / indices), per layer."""
+def algorithmic_bytes(cfg: W.WorkloadConfig, seq_lens, n_keeps):
+    """Bytes each call must move (K and V once, Q and O once, scores / indices), per layer, summed over the batch."""
     e = 2 if cfg.dtype == "bf16" else 4
-    L, b, Hq, Hkv, D = cfg.seq_len, cfg.block_len, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
-    refresh = 2 * L * Hkv * D * e + 2 * b * Hq * D * e + 4 * (L - b) * Hkv
-    topk = 4 * (L - b) * Hkv + 4 * n_keep * Hkv
-    compact = 2 * (2 * n_keep * Hkv * D * e) + 4 * n_keep * Hkv
-    sparse = 2 * (n_keep + b) * Hkv * D * e + 2 * b * Hq * D * e
-    return {"refresh": refresh, "topk": topk, "compact": compact, "sparse": sparse}
+    b, Hq, Hkv, D = cfg.block_len, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    out = {"refresh": 0, "topk": 0, "compact": 0, "sparse": 0}
+    for L, n_keep in zip(seq_lens, n_keeps):
+        out["refresh"] += 2 * L * Hkv * D * e + 2 * b * Hq * D * e + 4 * (L - b) * Hkv
+        out["topk"] += 4 * (L - b) * Hkv + 4 * n_keep * Hkv
+        out["compact"] += 2 * (2 * n_keep * Hkv * D * e) + 4 * n_keep * Hkv
+        out["sparse"] += 2 * (n_keep + b) * Hkv * D * e + 2 * b * Hq * D * e
+    return out
 
 
 class ClockSampler:
@@ -183,7 +190,7 @@ def run_ours(args):
 
     cfg = W.CONFIGS[args.workload]
     n_layers = args.layers or cfg.n_layers
-    Hq, Hkv, D, L, b = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.seq_len, cfg.block_len
+    Hq, Hkv, D, b = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.block_len
     reuse_steps = cfg.steps_per_block - 2
     tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
     bdt = B.BF16 if cfg.dtype == "bf16" else B.F32
@@ -194,30 +201,41 @@ def run_ours(args):
         return torch.from_numpy(x).to(dev)
 
     # ---- inputs: base tensors from the seeded host generator (one (layer, block=0) each); per-step drift on the device
+    Bn = max(1, args.batch)
+    if cfg.name == "c5_serving":
+        prompt_lens = W.serving_prompt_lengths(Bn, seed=5 + rank)
+    else:
+        prompt_lens = [cfg.prompt_len] * Bn
+    seq_lens = [p_ + cfg.gen_len for p_ in prompt_lens]
+    L = max(seq_lens)
     caches, Ks, Vs, Qr = [], [], [], []
     gen = torch.Generator(device=dev); gen.manual_seed(1234 + rank)
     for l in range(n_layers):
-        s = W.make_sequence(cfg, seed=rank, layer=l, block=0)
-        q, k, v = s.refresh_inputs(1)
-        Ks.append(to_dev(k)[None]); Vs.append(to_dev(v)[None]); Qr.append(to_dev(q)[None])
-        caches.append(LayerCache(batch=1, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, seq_len_max=L, block_len=b, dtype=bdt,
+        bw = W.make_batch(cfg, prompt_lens, seed=rank, layer=l, block=0)
+        q, k, v = bw.refresh_inputs(1)
+        Ks.append(to_dev(k)); Vs.append(to_dev(v)); Qr.append(to_dev(q))
+        caches.append(LayerCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, seq_len_max=L, block_len=b, dtype=bdt,
                                  retention=cfg.retention, pool_window=cfg.pool_window, device=str(dev),
                                  share_scratch_with=caches[0] if caches else None))
-    o = cfg.prompt_len
-    n_keep = B.keep_count(caches[0].desc, L, o)[0]
-    block_off = torch.tensor([o], dtype=torch.int32, device=dev)
+    n_keeps = [B.keep_count(caches[0].desc, Li, pi)[0] for Li, pi in zip(seq_lens, prompt_lens)]
+    n_keep = max(n_keeps)
+    seq_len_t = torch.tensor(seq_lens, dtype=torch.int32, device=dev)
+    block_off = torch.tensor(prompt_lens, dtype=torch.int32, device=dev)
     drift = cfg.drift_std / np.sqrt(D)
     # fresh block rows for every (reuse step, layer): Q_b', K_n, V_n = base + drift, rounded to the compute dtype
-    Qs = torch.empty((reuse_steps, n_layers, 1, Hq, b, D), dtype=tdt, device=dev)
-    Kn = torch.empty((reuse_steps, n_layers, 1, Hkv, b, D), dtype=tdt, device=dev)
+    Qs = torch.empty((reuse_steps, n_layers, Bn, Hq, b, D), dtype=tdt, device=dev)
+    Kn = torch.empty((reuse_steps, n_layers, Bn, Hkv, b, D), dtype=tdt, device=dev)
     Vn = torch.empty_like(Kn)
+    rows = torch.stack([torch.arange(o_, o_ + b, device=dev) for o_ in prompt_lens])          # [B, b] block positions
+    gather = rows[:, None, :, None].expand(Bn, Hkv, b, D)
     for l in range(n_layers):
+        kb, vb = Ks[l].gather(2, gather).float(), Vs[l].gather(2, gather).float()
         for t in range(reuse_steps):
             Qs[t, l] = (Qr[l].float() + drift * torch.randn(Qr[l].shape, device=dev, generator=gen)).to(tdt)
-            Kn[t, l] = (Ks[l][:, :, o:o + b].float() + drift * torch.randn((1, Hkv, b, D), device=dev, generator=gen)).to(tdt)
-            Vn[t, l] = (Vs[l][:, :, o:o + b].float() + drift * torch.randn((1, Hkv, b, D), device=dev, generator=gen)).to(tdt)
-    out_r = torch.empty((n_layers, 1, Hq, b, D), dtype=tdt, device=dev)
-    out_s = torch.empty((reuse_steps, n_layers, 1, Hq, b, D), dtype=tdt, device=dev)
+            Kn[t, l] = (kb + drift * torch.randn((Bn, Hkv, b, D), device=dev, generator=gen)).to(tdt)
+            Vn[t, l] = (vb + drift * torch.randn((Bn, Hkv, b, D), device=dev, generator=gen)).to(tdt)
+    out_r = torch.empty((n_layers, Bn, Hq, b, D), dtype=tdt, device=dev)
+    out_s = torch.empty((reuse_steps, n_layers, Bn, Hq, b, D), dtype=tdt, device=dev)
 
     stream = torch.cuda.Stream(device=dev)
     torch.cuda.synchronize(dev)                     # the inputs above were produced on the default stream
@@ -225,7 +243,7 @@ def run_ours(args):
     def one_step():
         """One decoding block: refresh every layer, then every reuse step over every layer (model order)."""
         for l in range(n_layers):
-            caches[l].refresh(Qr[l], Ks[l], Vs[l], None, block_off, out=out_r[l], stream=stream)
+            caches[l].refresh(Qr[l], Ks[l], Vs[l], seq_len_t, block_off, out=out_r[l], stream=stream)
         for t in range(reuse_steps):
             for l in range(n_layers):
                 caches[l].sparse_step(Qs[t, l], Kn[t, l], Vn[t, l], out_s[t, l], stream=stream)
@@ -237,7 +255,7 @@ def run_ours(args):
 
     def refresh_only():
         for l in range(n_layers):
-            caches[l].refresh(Qr[l], Ks[l], Vs[l], None, block_off, out=out_r[l], stream=stream)
+            caches[l].refresh(Qr[l], Ks[l], Vs[l], seq_len_t, block_off, out=out_r[l], stream=stream)
 
     def make_runner(fn):
         if args.no_graph:
@@ -268,10 +286,13 @@ def run_ours(args):
                 dist.barrier()
         return e0.elapsed_time(e1) / 1e3
 
+    with torch.cuda.stream(stream):
+        refresh_only()                              # every layer's cache exists before any reuse step runs
+    stream.synchronize()
     d0 = caches[0].desc
     launches_per_step = n_layers * (B.launch_count(d0, B.OP_REFRESH_SCORES) + B.launch_count(d0, B.OP_SELECT_TOPK) +
                                     B.launch_count(d0, B.OP_COMPACT_KV) + reuse_steps * B.launch_count(d0, B.OP_SPARSE_BLOCK_ATTN))
-    step_runner = make_runner(one_step)
+    step_runner = make_runner({"all": one_step, "refresh": refresh_only, "sparse": sparse_only}[args.phase])
     sampler = ClockSampler(local) if rank == 0 else None
     sec = timed(step_runner, args.steps, max(args.warmup, 3))
     clocks = sampler.stop() if sampler else None
@@ -279,11 +300,11 @@ def run_ours(args):
         t = torch.tensor([sec], device=dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         sec = float(t.item())
-    tok = tokens_per_step(cfg, n_layers, n_keep)
+    tok = tokens_per_step(cfg, n_layers, seq_lens, n_keeps, args.phase)
     value = world * tok * args.steps / sec
 
     # ---- roofline of the dominant call (sparse block attention: 30 of the 31 calls per layer per block)
-    ab = algorithmic_bytes(cfg, n_keep)
+    ab = algorithmic_bytes(cfg, seq_lens, n_keeps)
     sp_runner = make_runner(sparse_only)
     sp_sec = timed(sp_runner, max(3, args.steps // 2), 3) / max(3, args.steps // 2) / (n_layers * reuse_steps)
     rf_runner = make_runner(refresh_only)
@@ -311,7 +332,7 @@ def run_ours(args):
             with torch.cuda.stream(stream):
                 for l in range(n_layers):
                     dQ.copy_(hQ[l], non_blocking=True); dK.copy_(hK[l], non_blocking=True); dV.copy_(hV[l], non_blocking=True)
-                    caches[l].refresh(dQ, dK, dV, None, block_off, out=out_r[l], stream=stream)
+                    caches[l].refresh(dQ, dK, dV, seq_len_t, block_off, out=out_r[l], stream=stream)
                     h_out_r[l].copy_(out_r[l], non_blocking=True)
                 for t in range(reuse_steps):
                     for l in range(n_layers):
@@ -325,8 +346,8 @@ def run_ours(args):
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             e2e_sec = float(t.item())
         esz = Ks[0].element_size()
-        h2d = n_layers * ((2 * Hkv * L * D + Hq * b * D) * esz + reuse_steps * (2 * Hkv * b * D + Hq * b * D) * esz)
-        d2h = n_layers * (1 + reuse_steps) * Hq * b * D * esz
+        h2d = n_layers * Bn * ((2 * Hkv * L * D + Hq * b * D) * esz + reuse_steps * (2 * Hkv * b * D + Hq * b * D) * esz)
+        d2h = n_layers * Bn * (1 + reuse_steps) * Hq * b * D * esz
         e2e = {"value": world * tok * e2e_iters / e2e_sec, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "ms_per_step": 1e3 * e2e_sec / e2e_iters}
 
@@ -344,11 +365,11 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": cfg.dtype, "data": "synthetic",
-            "config": {"workload": cfg.name, "layers": n_layers, "seq_len": L, "block_len": b, "n_q_heads": Hq, "n_kv_heads": Hkv,
+            "config": {"workload": cfg.name, "batch": Bn, "phase": args.phase, "layers": n_layers, "seq_len": L, "block_len": b, "n_q_heads": Hq, "n_kv_heads": Hkv,
                        "head_dim": D, "retention": cfg.retention, "pool_window": cfg.pool_window, "n_keep": n_keep,
                        "step": "1 decoding block: %d layers x (1 refresh chain + %d reuse steps)" % (n_layers, reuse_steps),
                        "l2": "no flush: one step streams %.0f MB of K/V and caches across layers, larger than L2" % (
-                           n_layers * (ab["refresh"] + reuse_steps * 0 + 2 * n_keep * Hkv * D * 2) / 1e6),
+                           n_layers * (ab["refresh"] + ab["compact"] / 2) / 1e6),
                        "launch": "eager" if args.no_graph else "cuda_graph_replay", "parallelism": "replicas" if world > 1 else "1gpu"},
             "block_steps_per_s": world * n_layers * (1 + reuse_steps) * args.steps / sec,
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks,
