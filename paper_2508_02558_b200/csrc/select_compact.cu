@@ -16,18 +16,50 @@ __device__ __forceinline__ uint32_t score_key(float x) {
 
 constexpr int SEL_THREADS = 1024;
 constexpr int SEL_WARPS = SEL_THREADS / 32;
+constexpr int SEL_HIST = 8;               // histogram copies, one per group of warps, to spread shared-memory atomics
 
 struct Segment { int c_lo, c_hi, n; };   // candidate range and how many to keep
 
-// One CTA per (sequence, KV head). Radix select (4 passes of 8 bits, most significant first) finds the key of the
-// n-th largest candidate and how many candidates are strictly greater; a final ordered pass writes, in ascending
-// position order, every candidate above the threshold plus the lowest-index candidates equal to it. No step depends
-// on the order in which threads run, so the result is deterministic.
+// Exclusive prefix sum of one value per thread over the whole CTA (thread order); `total` receives the sum.
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* warp_tot, uint32_t* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t incl = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += y;
+  }
+  __syncthreads();                        // warp_tot may still be read from a previous scan
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const uint32_t t = warp_tot[lane];
+    uint32_t ti = t;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, ti, d);
+      if (lane >= d) ti += y;
+    }
+    warp_tot[lane] = ti - t;              // exclusive offset of each warp
+    if (lane == 31) warp_tot[32] = ti;    // grand total
+  }
+  __syncthreads();
+  *total = warp_tot[32];
+  return warp_tot[warp] + incl - v;
+}
+
+// One CTA per (sequence, KV head). The candidate keys are staged once in shared memory (coalesced loads, one padding
+// word per 32 so that a thread can walk its own contiguous run of candidates without bank conflicts). A radix select
+// (4 passes of 8 bits, most significant first, histograms by shared-memory atomics) finds the key of the n-th largest
+// candidate and how many candidates equal to it are still to be kept; then every thread counts the survivors of its run,
+// two CTA-wide prefix sums turn the counts into output offsets, and the kept positions are written in ascending
+// order, ties going to the lowest positions. Counts are integers, so nothing depends on the order in which threads or
+// atomics run: the result is deterministic.
 __global__ void __launch_bounds__(SEL_THREADS) select_topk_kernel(const SelectParams p) {
-  extern __shared__ uint32_t keys_s[];                 // optional cache of the candidate keys
-  __shared__ uint32_t hist[SEL_WARPS][256];
-  __shared__ uint32_t warp_cnt[2][SEL_WARPS];
-  __shared__ uint32_t sh_prefix, sh_remaining, sh_run_eq, sh_run_out;
+  extern __shared__ uint32_t keys_s[];                 // optional cache of the candidate keys, index c + c / 32
+  __shared__ uint32_t hist[SEL_HIST][256];
+  __shared__ uint32_t warp_tot[SEL_WARPS + 1];
+  __shared__ uint32_t sh_prefix, sh_remaining;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = blockIdx.x, bi = blockIdx.y;
@@ -42,10 +74,10 @@ __global__ void __launch_bounds__(SEL_THREADS) select_topk_kernel(const SelectPa
   const bool cached = C <= p.smem_keys;
 
   auto cand_pos = [&](int c) { return c < o ? c : c + b; };
-  auto key_at = [&](int c) -> uint32_t { return cached ? keys_s[c] : score_key(sc[cand_pos(c)]); };
+  auto key_at = [&](int c) -> uint32_t { return cached ? keys_s[c + (c >> 5)] : score_key(sc[cand_pos(c)]); };
 
   if (cached)
-    for (int c = tid; c < C; c += SEL_THREADS) keys_s[c] = score_key(sc[cand_pos(c)]);
+    for (int c = tid; c < C; c += SEL_THREADS) keys_s[c + (c >> 5)] = score_key(sc[cand_pos(c)]);
 
   int n_pre, n_suf;
   const int n_total = keep_count_total(o, C - o, p.retention, p.mode, &n_pre, &n_suf);
@@ -60,13 +92,15 @@ __global__ void __launch_bounds__(SEL_THREADS) select_topk_kernel(const SelectPa
     seg[1] = {o, C, min(n_suf, p.n_keep_max - np)};
     n_seg = 2;
   }
-  if (tid == 0) { sh_run_out = 0; }
+  uint32_t run_out = 0;                                // entries written so far (same value in every thread)
   __syncthreads();
 
   for (int si = 0; si < n_seg; ++si) {
     const int c_lo = seg[si].c_lo, c_hi = seg[si].c_hi, n = seg[si].n;
     const int len = c_hi - c_lo;
     if (n <= 0 || len <= 0) continue;
+    const int kpt = (len + SEL_THREADS - 1) / SEL_THREADS;   // candidates per thread, a contiguous run
+    const int my_lo = min(c_lo + tid * kpt, c_hi), my_hi = min(my_lo + kpt, c_hi);
     uint32_t thr = 0u, need_eq = 0u;
     const bool take_all = n >= len;
     if (!take_all) {
@@ -74,29 +108,21 @@ __global__ void __launch_bounds__(SEL_THREADS) select_topk_kernel(const SelectPa
       if (tid == 0) { sh_prefix = 0u; sh_remaining = (uint32_t)n; }
       for (int pass = 0; pass < 4; ++pass) {
         const int shift = 24 - 8 * pass;
-        for (int i = tid; i < SEL_WARPS * 256; i += SEL_THREADS) (&hist[0][0])[i] = 0u;
+        for (int i = tid; i < SEL_HIST * 256; i += SEL_THREADS) (&hist[0][0])[i] = 0u;
         __syncthreads();
         const uint32_t prefix = sh_prefix;
         const uint32_t remaining = sh_remaining;
         const uint32_t himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
-        for (int c0 = c_lo; c0 < c_hi; c0 += SEL_THREADS) {
-          const int c = c0 + tid;
-          const bool in = c < c_hi;
-          const uint32_t k = in ? key_at(c) : 0u;
-          const bool match = in && ((k & himask) == prefix);
-          const uint32_t digit = (k >> shift) & 0xFFu;
-          // aggregate equal digits inside the warp, one shared-memory add per distinct digit
-          const uint32_t active = __ballot_sync(0xffffffffu, match);
-          if (match) {
-            const uint32_t peers = __match_any_sync(active, digit);
-            if ((int)(__ffs(peers) - 1) == lane) hist[warp][digit] += __popc(peers);
-          }
+        uint32_t* my_hist = hist[warp & (SEL_HIST - 1)];
+        for (int c = my_lo; c < my_hi; ++c) {
+          const uint32_t k = key_at(c);
+          if ((k & himask) == prefix) atomicAdd(&my_hist[(k >> shift) & 0xFFu], 1u);
         }
         __syncthreads();
-        // column sums of the per-warp histograms, then a scan from the top bin by warp 0
         if (tid < 256) {
           uint32_t s = 0;
-          for (int w = 0; w < SEL_WARPS; ++w) s += hist[w][tid];
+#pragma unroll
+          for (int w = 0; w < SEL_HIST; ++w) s += hist[w][tid];
           hist[0][tid] = s;
         }
         __syncthreads();
@@ -129,40 +155,31 @@ __global__ void __launch_bounds__(SEL_THREADS) select_topk_kernel(const SelectPa
       thr = sh_prefix;
       need_eq = sh_remaining;                     // how many candidates equal to thr are still to be kept (>= 1)
     }
-    // ---- ordered emission ----
-    if (tid == 0) sh_run_eq = 0u;
-    __syncthreads();
-    for (int c0 = c_lo; c0 < c_hi; c0 += SEL_THREADS) {
-      const int c = c0 + tid;
-      const bool in = c < c_hi;
-      const uint32_t k = in ? key_at(c) : 0u;
-      const bool gt = in && (take_all || k > thr);
-      const bool eq = in && !take_all && k == thr;
-      const uint32_t beq = __ballot_sync(0xffffffffu, eq);
-      if (lane == 0) warp_cnt[0][warp] = __popc(beq);
-      __syncthreads();
-      uint32_t eq_before = sh_run_eq;
-      for (int w = 0; w < warp; ++w) eq_before += warp_cnt[0][w];
-      eq_before += __popc(beq & ((1u << lane) - 1u));
-      const bool keep = gt || (eq && eq_before < need_eq);
-      const uint32_t bk = __ballot_sync(0xffffffffu, keep);
-      if (lane == 0) warp_cnt[1][warp] = __popc(bk);
-      __syncthreads();
-      uint32_t out_before = sh_run_out;
-      for (int w = 0; w < warp; ++w) out_before += warp_cnt[1][w];
-      out_before += __popc(bk & ((1u << lane) - 1u));
-      if (keep && out_before < (uint32_t)p.n_keep_max) out[out_before] = cand_pos(c);
-      __syncthreads();
-      if (tid == 0) {
-        uint32_t te = 0, tk = 0;
-        for (int w = 0; w < SEL_WARPS; ++w) { te += warp_cnt[0][w]; tk += warp_cnt[1][w]; }
-        sh_run_eq += te; sh_run_out += tk;
-      }
-      __syncthreads();
+    // ---- ordered emission: a thread's run is contiguous, so thread order is position order ----
+    uint32_t my_eq = 0, my_gt = 0;
+    for (int c = my_lo; c < my_hi; ++c) {
+      const uint32_t k = key_at(c);
+      my_gt += (take_all || k > thr) ? 1u : 0u;
+      my_eq += (!take_all && k == thr) ? 1u : 0u;
     }
+    uint32_t total_eq, total_keep;
+    const uint32_t eq_before = block_exclusive_scan(my_eq, warp_tot, &total_eq);
+    const uint32_t eq_quota = need_eq > eq_before ? min(need_eq - eq_before, my_eq) : 0u;   // ties kept from this run: its first ones
+    const uint32_t out_before = block_exclusive_scan(my_gt + eq_quota, warp_tot, &total_keep);
+    uint32_t w = run_out + out_before, eq_seen = 0;
+    for (int c = my_lo; c < my_hi; ++c) {
+      const uint32_t k = key_at(c);
+      bool keep = take_all || k > thr;
+      if (!take_all && k == thr) { keep = eq_seen < eq_quota; ++eq_seen; }
+      if (keep) {
+        if (w < (uint32_t)p.n_keep_max) out[w] = cand_pos(c);
+        ++w;
+      }
+    }
+    run_out += total_keep;
   }
   __syncthreads();
-  const int kept = min((int)sh_run_out, p.n_keep_max);
+  const int kept = min((int)run_out, p.n_keep_max);
   for (int i = kept + tid; i < p.n_keep_max; i += SEL_THREADS) out[i] = -1;
   if (g == 0 && tid == 0) p.kept_cnt[bi] = kept;
 }
@@ -212,7 +229,7 @@ __global__ void __launch_bounds__(256) compact_kv_kernel(const CompactParams p) 
 
 cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st) {
   static size_t configured = 0;
-  const size_t smem = (size_t)p.smem_keys * 4;
+  const size_t smem = ((size_t)p.smem_keys + p.smem_keys / 32 + 1) * 4;
   if (smem > configured) {
     const cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
