@@ -152,7 +152,13 @@ sdllm_status sdllm_compact_kv(const sdllm_desc* desc, const void* k, const void*
                               const int32_t* kept_cnt, void* k_c, void* v_c, void* cuda_stream);
 
 /* Reuse step (cache_state 2, Algorithm 3): out = softmax(scale * Q_b' [K_c ; K_n]^T) [V_c ; V_n] over the first
- * kept_cnt[i] rows of the compacted cache followed by the block's b fresh rows k_blk, v_blk. */
+ * kept_cnt[i] rows of the compacted cache followed by the block's b fresh rows k_blk, v_blk.
+ * The compacted cache is older than the step that reuses it, and the call takes advantage of that: it starts streaming
+ * k_c, v_c (and reads kept_cnt) while the kernel in front of it in the stream may still be finishing. This is safe
+ * after every call of this library and after any kernel that holds its dependents back until it has completed (the
+ * default). Only a caller's own kernel that releases its dependents early (programmatic dependent launch) must not be
+ * the one that writes k_c, v_c or kept_cnt directly in front of this call. q_blk, k_blk and v_blk are read only
+ * after the preceding kernel has completed. */
 sdllm_status sdllm_sparse_block_attn(const sdllm_desc* desc, const void* q_blk, const void* k_c, const void* v_c,
                                      const int32_t* kept_cnt, const void* k_blk, const void* v_blk, void* out,
                                      void* workspace, size_t workspace_bytes, void* cuda_stream);

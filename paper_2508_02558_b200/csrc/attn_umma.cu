@@ -49,6 +49,7 @@ struct UmmaParams {
   int row_tiles;     // 128-row tiles of the b*G rows
   int heads_rt;      // query heads per row tile
   int fused_tail;    // 1: the last CTA of a unit merges and pools; 0: umma_tail_kernel does
+  int early_src1;    // 1: source 1 and its count are older than the previous kernel in the stream (reuse step)
 };
 
 // ---------------------------------------------------------------------------------------------------------
@@ -359,9 +360,21 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   // before the rest of the CTA is ready: the loads need nothing but the barriers.
   int prod_it = 0, prod_t = t_begin, prod_n1 = 0;
   bool prod_ok = true;
-  auto produce = [&](int limit) {     // issue loads for up to `limit` further tiles (producer lane only)
+  bool q_issued = false;
+  auto issue_q = [&]() {              // the Q tile (replicated R times along the accumulator rows)
+    q_issued = true;
+    if (!do_attn) return;
+    mbar_expect_tx(BAR(Q_FULL), (uint32_t)(R * H * p.b * up.heads_rt * 128));
+    for (int rep = 0; rep < R; ++rep)
+      for (int h = 0; h < H; ++h)
+        tma_load_4d(smem_u32(q_s + h * 128 * 128 + rep * rows_rep * 128), &tm.q, BAR(Q_FULL), h * 64, 0,
+                    g * p.G + rt * up.heads_rt, bi);
+  };
+  // issue loads for up to `limit` further tiles (producer lane only); with src1_only, stop in front of source 2
+  auto produce = [&](int limit, bool src1_only) {
     while (prod_t < t_end && limit > 0 && prod_ok) {
       const Tile x = tile_of(prod_t, tiles1, KT, KT2, prod_n1, n2);
+      if (src1_only && !x.src1) break;
       ++prod_t;
       if (x.nv == 0) continue;
       const int it = prod_it, s = it % NS;
@@ -373,13 +386,6 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
       if (it >= NS && !wait_bar(BAR(EMPTY_K + s), ph, abort_flag, p.status, 1)) { prod_ok = false; break; }
       mbar_expect_tx(BAR(FULL_K + s), tile_tx);
       for (int h = 0; h < H; ++h) tma_load_4d(kdst + h * half_bytes, mk, BAR(FULL_K + s), h * 64, x.row0, g, bi);
-      if (it == 0 && do_attn) {        // the Q tile right after the first K tile: S_0 needs both
-        mbar_expect_tx(BAR(Q_FULL), (uint32_t)(R * H * p.b * up.heads_rt * 128));
-        for (int rep = 0; rep < R; ++rep)
-          for (int h = 0; h < H; ++h)
-            tma_load_4d(smem_u32(q_s + h * 128 * 128 + rep * rows_rep * 128), &tm.q, BAR(Q_FULL), h * 64, 0,
-                        g * p.G + rt * up.heads_rt, bi);
-      }
       if (do_attn) {
         if (it >= NS && !wait_bar(BAR(EMPTY_V + s), ph, abort_flag, p.status, 2)) { prod_ok = false; break; }
         mbar_expect_tx(BAR(FULL_V + s), tile_tx);
@@ -409,11 +415,21 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     TRACE(2);
     if (!zero_q && (do_attn || do_scores)) {
+      if (up.early_src1) {
+        // Reuse step: the compacted cache and its count were written before the previous kernel in the stream even
+        // started, so their tiles may stream in while that kernel is still finishing.
+        prod_n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
+        prod_n1 = min(max(prod_n1, 0), p.n1_max);
+        produce(NS, true);             // the first NS slots are free: no waiting here
+      }
       grid_dependency_wait();          // the loads below read what earlier kernels in the stream wrote
-      prod_n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
-      prod_n1 = min(max(prod_n1, 0), p.n1_max);
+      if (!up.early_src1) {
+        prod_n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
+        prod_n1 = min(max(prod_n1, 0), p.n1_max);
+      }
       TRACE(4);
-      produce(NS);                     // the first NS slots are free: no waiting here
+      issue_q();
+      produce(NS - prod_it, false);
       TRACE(5);
     }
   }
@@ -445,14 +461,15 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     // ======================================= TMA producer =======================================
     if (lane == 0 && (do_attn || do_scores)) {
       prod_n1 = n1;
-      produce(1 << 30);
+      if (!q_issued) issue_q();
+      produce(1 << 30, false);
       if (*abort_flag) {
         // let the copies that were issued land before the CTA retires
         for (int j = max(prod_it - NS, 0); j < prod_it; ++j) {
           drain_bar(BAR(FULL_K + j % NS), (j / NS) & 1);
           if (do_attn) drain_bar(BAR(FULL_V + j % NS), (j / NS) & 1);
         }
-        if (do_attn && prod_it > 0) drain_bar(BAR(Q_FULL), 0);
+        if (do_attn && q_issued) drain_bar(BAR(Q_FULL), 0);
       }
     }
   } else if (warp == 1) {
@@ -953,6 +970,10 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
   up.KT = pl.key_tile; up.KT2 = pl.key_tile2; up.R = pl.rep; up.row_tiles = pl.row_tiles;
   up.heads_rt = pl.row_tiles == 1 ? p.G : 128 / p.b;
   const bool pool = p.want_scores && p.pooled != nullptr;
+  {
+    const char* e = getenv("SDLLM_EARLY_LOADS");   // SDLLM_EARLY_LOADS=0: no loads before the grid dependency (test aid)
+    up.early_src1 = (p.n2 > 0 && p.n1_max > 0 && !(e && e[0] == '0')) ? 1 : 0;
+  }
   up.fused_tail = umma_tail_is_fused(pl, D, p.M, p.n1_max, pool) ? 1 : 0;
   memset(&tm, 0, sizeof(tm));
   bool ok = true;
