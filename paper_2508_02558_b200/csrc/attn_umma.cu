@@ -215,34 +215,37 @@ __device__ __forceinline__ float pool_at(const AttnParams& p, const float* a, in
   return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
 }
 
-// Merge of the key-split partials of one (row, float4 column) slot of a unit and the final store. Loads of four
-// partials are issued together so that their latencies overlap.
-template <int D>
+// Merge of the key-split partials of one (row, float4 column) slot of a unit and the final store. The partials are
+// read in batches of MB with all loads of a batch in flight together (one L2 latency per batch) and folded with a
+// running maximum, so that four splits cost a single round trip.
+template <int D, int MB>
 __device__ __forceinline__ void merge_slot(const AttnParams& p, int64_t unit, int bi, int g, int rt, int m_local, int d4) {
   const int P = p.splits;
   const int prt = min(p.M, 128);                      // rows of one partial
   const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + unit * P * prt + m_local;
   const float4* po = reinterpret_cast<const float4*>(p.part_o + (unit * P * prt + m_local) * D) + d4;
-  float mstar = -INFINITY;
-  for (int pi = 0; pi < P; ++pi) {
-    const float2 x = __ldcg(ml + (int64_t)pi * prt);
-    if (x.y > 0.f) mstar = fmaxf(mstar, x.x);
-  }
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  float l = 0.f;
-  for (int p0 = 0; p0 < P; p0 += 4) {
-    float2 x[4];
-    float4 o[4];
+  float l = 0.f, m_run = -INFINITY;
+  for (int p0 = 0; p0 < P; p0 += MB) {
+    float2 x[MB];
+    float4 o[MB];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < MB; ++u) {
       const int pi = min(p0 + u, P - 1);
       x[u] = __ldcg(ml + (int64_t)pi * prt);
       o[u] = __ldcg(po + (int64_t)pi * prt * (D / 4));
     }
+    float bm = m_run;
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < MB; ++u)
+      if (p0 + u < P && x[u].y > 0.f) bm = fmaxf(bm, x[u].x);
+    const float a = (bm == -INFINITY) ? 1.f : fast_exp2(m_run - bm);    // 0 on the first batch with data
+    acc.x *= a; acc.y *= a; acc.z *= a; acc.w *= a; l *= a;
+    m_run = bm;
+#pragma unroll
+    for (int u = 0; u < MB; ++u) {
       if (p0 + u >= P || !(x[u].y > 0.f)) continue;
-      const float w = fast_exp2(x[u].x - mstar);
+      const float w = fast_exp2(x[u].x - m_run);
       l = fmaf(x[u].y, w, l);
       acc.x = fmaf(o[u].x, w, acc.x); acc.y = fmaf(o[u].y, w, acc.y); acc.z = fmaf(o[u].z, w, acc.z); acc.w = fmaf(o[u].w, w, acc.w);
     }
@@ -256,7 +259,7 @@ __device__ __forceinline__ void merge_slot(const AttnParams& p, int64_t unit, in
   w2.x = pack_bf16(acc.x * inv, acc.y * inv);
   w2.y = pack_bf16(acc.z * inv, acc.w * inv);
   *reinterpret_cast<uint2*>(out) = w2;
-  if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
+  if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (m_run + log2f(l)) * kLn2;
 }
 
 // Deferred tail (large partial volumes or long sequences): one launch that merges the key splits, one thread per
@@ -278,7 +281,7 @@ __global__ void __launch_bounds__(256) umma_tail_kernel(const UmmaParams up, con
     const int64_t bg = unit / up.row_tiles;
     const int g = (int)(bg % p.Hkv), bi = (int)(bg / p.Hkv);
     if (m_local >= min(p.M - rt * 128, 128)) return;
-    merge_slot<D>(p, unit, bi, g, rt, m_local, d4);
+    merge_slot<D, 8>(p, unit, bi, g, rt, m_local, d4);
     return;
   }
   const int64_t idx = (int64_t)(blockIdx.x - merge_blocks) * 256 + threadIdx.x;
@@ -303,8 +306,18 @@ __device__ __forceinline__ void trace_point(int32_t* status, int slot) {
   }
 }
 #define TRACE(slot) trace_point(p.status, slot)
+__device__ __forceinline__ void trace_all(int32_t* status, int slot, bool is_min) {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  unsigned long long* a = reinterpret_cast<unsigned long long*>(status) + slot;
+  if (is_min) atomicMin(a, t); else atomicMax(a, t);
+}
+#define TRACE_MIN(slot) trace_all(p.status, slot, true)
+#define TRACE_MAX(slot) trace_all(p.status, slot, false)
 #else
 #define TRACE(slot) do { } while (0)
+#define TRACE_MIN(slot) do { } while (0)
+#define TRACE_MAX(slot) do { } while (0)
 #endif
 
 template <int D>
@@ -321,7 +334,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   const int bi = blockIdx.z;
   const int g = blockIdx.y / up.row_tiles, rt = blockIdx.y - g * up.row_tiles;
   const int split = blockIdx.x;
-  if (tid == 0) TRACE(1);
+  if (tid == 0) { TRACE(1); TRACE_MAX(24); }
   const int tiles1 = (p.n1_max + KT - 1) / KT;
   const int tiles2 = (p.n2 + KT2 - 1) / KT2;
   const int tiles_all = tiles1 + tiles2;
@@ -767,38 +780,51 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     if (tid == 64) TRACE(27);
     asm volatile("bar.sync 2, 128;\n" ::: "memory");
     if (tid == 64) TRACE(29);
+    // consecutive threads take consecutive float4 of a row; a thread keeps its column and walks down the rows, four
+    // rows per step with all their shared-memory reads in flight together
     const int st = (warp - 2) * 32 + lane;
     if (!*abort_flag) {
-#pragma unroll 2
-      for (int slot = st; slot < M_rt * D4; slot += 128) {
-        const int ml = slot / D4, d4 = slot - ml * D4;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int r2 = 0; r2 < R; ++r2) {
-          const int rr = r2 * rows_rep + ml;
-          const float4 o = *reinterpret_cast<const float4*>(o_s + rr * D + ((d4 ^ (rr & (D4 - 1))) << 2));
-          acc.x += o.x; acc.y += o.y; acc.z += o.z; acc.w += o.w;
+      const int d4 = st % D4, r_first = st / D4, r_step = 128 / D4;
+      const int m_first = rt * 128;
+      for (int mb = r_first; mb < M_rt; mb += 4 * r_step) {
+        float4 acc[4];
+        float2 x[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int ml = min(mb + u * r_step, M_rt - 1);
+          acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+          x[u] = lm_s[ml];
+          for (int r2 = 0; r2 < R; ++r2) {
+            const int rr = r2 * rows_rep + ml;
+            const float4 o = *reinterpret_cast<const float4*>(o_s + rr * D + ((d4 ^ (rr & (D4 - 1))) << 2));
+            acc[u].x += o.x; acc[u].y += o.y; acc[u].z += o.z; acc[u].w += o.w;
+          }
         }
-        const float2 x = lm_s[ml];
-        const int m = rt * 128 + ml;                   // row within the KV head: m = head_in_group * b + i
-        const int hg = m / p.b, i = m - hg * p.b;
-        if (p.splits == 1) {
-          const float inv = x.y > 0.f ? 1.f / x.y : 0.f;
-          __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
-                             (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
-          uint2 w2;
-          w2.x = pack_bf16(acc.x * inv, acc.y * inv);
-          w2.y = pack_bf16(acc.z * inv, acc.w * inv);
-          *reinterpret_cast<uint2*>(o) = w2;
-          if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (x.x + log2f(x.y)) * kLn2;
-        } else {
-          const int64_t prow = (unit * p.splits + split) * min(p.M, 128) + ml;
-          *reinterpret_cast<float4*>(p.part_o + prow * D + d4 * 4) = acc;
-          if (d4 == 0) reinterpret_cast<float2*>(p.part_ml)[prow] = x;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int ml = mb + u * r_step;
+          if (ml >= M_rt) break;
+          const int m = m_first + ml;                  // row within the KV head: m = head_in_group * b + i
+          const int hg = m / p.b, i = m - hg * p.b;
+          if (p.splits == 1) {
+            const float inv = x[u].y > 0.f ? 1.f / x[u].y : 0.f;
+            __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
+                               (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
+            uint2 w2;
+            w2.x = pack_bf16(acc[u].x * inv, acc[u].y * inv);
+            w2.y = pack_bf16(acc[u].z * inv, acc[u].w * inv);
+            *reinterpret_cast<uint2*>(o) = w2;
+            if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (x[u].x + log2f(x[u].y)) * kLn2;
+          } else {
+            const int64_t prow = (unit * p.splits + split) * min(p.M, 128) + ml;
+            *reinterpret_cast<float4*>(p.part_o + prow * D + d4 * 4) = acc[u];
+            if (d4 == 0) reinterpret_cast<float2*>(p.part_ml)[prow] = x[u];
+          }
         }
       }
     }
   }
-  if (tid == 64) TRACE(13);
+  if (tid == 64) { TRACE(13); TRACE_MAX(25); }
 
   // ---- fused tail: the last CTA of the unit merges the key splits and pools the saliency; nobody waits ----
   const bool tail_merge = do_attn && p.splits > 1;
@@ -819,7 +845,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
       __threadfence();
       if (tail_merge)
         for (int slot = tid; slot < M_rt * (D / 4); slot += UM_THREADS)
-          merge_slot<D>(p, unit, bi, g, rt, slot / (D / 4), slot % (D / 4));
+          merge_slot<D, 4>(p, unit, bi, g, rt, slot / (D / 4), slot % (D / 4));
       if (tail_pool) {
         // stage the head's raw saliency in shared memory (the ring is free), then pool from there
         float* a_s = reinterpret_cast<float*>(stage0);
@@ -842,7 +868,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
-  if (tid == 0) TRACE(15);
+  if (tid == 0) { TRACE(15); TRACE_MAX(26); TRACE_MAX(16 + (int)blockIdx.x); }
 }
 
 // ---------------------------------------------------------------------------------------------------------
