@@ -215,51 +215,70 @@ __device__ __forceinline__ float pool_at(const AttnParams& p, const float* a, in
   return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
 }
 
-// Merge of the key-split partials of one (row, float4 column) slot of a unit and the final store. The partials are
-// read in batches of MB with all loads of a batch in flight together (one L2 latency per batch) and folded with a
-// running maximum, so that four splits cost a single round trip.
-template <int D, int MB>
-__device__ __forceinline__ void merge_slot(const AttnParams& p, int64_t unit, int bi, int g, int rt, int m_local, int d4) {
+// Merge of the key-split partials of S (row, float4 column) slots of a unit and the final stores. slot[s] < 0 marks
+// an unused entry. The partials are read in batches of MB per slot with the loads of all slots and of the whole batch
+// in flight together (one L2 latency per batch) and folded with a running maximum, so that four splits cost a single
+// round trip for everything a thread merges.
+template <int D, int MB, int S>
+__device__ __forceinline__ void merge_slots(const AttnParams& p, int64_t unit, int bi, int g, int rt, const int (&slot)[S]) {
+  constexpr int D4 = D / 4;
   const int P = p.splits;
   const int prt = min(p.M, 128);                      // rows of one partial
-  const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + unit * P * prt + m_local;
-  const float4* po = reinterpret_cast<const float4*>(p.part_o + (unit * P * prt + m_local) * D) + d4;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  float l = 0.f, m_run = -INFINITY;
+  const float2* ml_base = reinterpret_cast<const float2*>(p.part_ml) + unit * P * prt;
+  const float4* po_base = reinterpret_cast<const float4*>(p.part_o + unit * P * prt * D);
+  float4 acc[S];
+  float l[S], m_run[S];
+  int m_local[S], d4[S];
+#pragma unroll
+  for (int s = 0; s < S; ++s) {
+    acc[s] = make_float4(0.f, 0.f, 0.f, 0.f); l[s] = 0.f; m_run[s] = -INFINITY;
+    const int sl = max(slot[s], 0);
+    m_local[s] = sl / D4; d4[s] = sl - m_local[s] * D4;
+  }
   for (int p0 = 0; p0 < P; p0 += MB) {
-    float2 x[MB];
-    float4 o[MB];
+    float2 x[S][MB];
+    float4 o[S][MB];
 #pragma unroll
-    for (int u = 0; u < MB; ++u) {
-      const int pi = min(p0 + u, P - 1);
-      x[u] = __ldcg(ml + (int64_t)pi * prt);
-      o[u] = __ldcg(po + (int64_t)pi * prt * (D / 4));
-    }
-    float bm = m_run;
+    for (int s = 0; s < S; ++s)
 #pragma unroll
-    for (int u = 0; u < MB; ++u)
-      if (p0 + u < P && x[u].y > 0.f) bm = fmaxf(bm, x[u].x);
-    const float a = (bm == -INFINITY) ? 1.f : fast_exp2(m_run - bm);    // 0 on the first batch with data
-    acc.x *= a; acc.y *= a; acc.z *= a; acc.w *= a; l *= a;
-    m_run = bm;
+      for (int u = 0; u < MB; ++u) {
+        const int pi = min(p0 + u, P - 1);
+        x[s][u] = __ldcg(ml_base + (int64_t)pi * prt + m_local[s]);
+        o[s][u] = __ldcg(po_base + ((int64_t)pi * prt + m_local[s]) * D4 + d4[s]);
+      }
 #pragma unroll
-    for (int u = 0; u < MB; ++u) {
-      if (p0 + u >= P || !(x[u].y > 0.f)) continue;
-      const float w = fast_exp2(x[u].x - m_run);
-      l = fmaf(x[u].y, w, l);
-      acc.x = fmaf(o[u].x, w, acc.x); acc.y = fmaf(o[u].y, w, acc.y); acc.z = fmaf(o[u].z, w, acc.z); acc.w = fmaf(o[u].w, w, acc.w);
+    for (int s = 0; s < S; ++s) {
+      float bm = m_run[s];
+#pragma unroll
+      for (int u = 0; u < MB; ++u)
+        if (p0 + u < P && x[s][u].y > 0.f) bm = fmaxf(bm, x[s][u].x);
+      const float a = (bm == -INFINITY) ? 1.f : fast_exp2(m_run[s] - bm);    // 0 on the first batch with data
+      acc[s].x *= a; acc[s].y *= a; acc[s].z *= a; acc[s].w *= a; l[s] *= a;
+      m_run[s] = bm;
+#pragma unroll
+      for (int u = 0; u < MB; ++u) {
+        if (p0 + u >= P || !(x[s][u].y > 0.f)) continue;
+        const float w = fast_exp2(x[s][u].x - bm);
+        l[s] = fmaf(x[s][u].y, w, l[s]);
+        acc[s].x = fmaf(o[s][u].x, w, acc[s].x); acc[s].y = fmaf(o[s][u].y, w, acc[s].y);
+        acc[s].z = fmaf(o[s][u].z, w, acc[s].z); acc[s].w = fmaf(o[s][u].w, w, acc[s].w);
+      }
     }
   }
-  const float inv = l > 0.f ? 1.f / l : 0.f;
-  const int m = rt * 128 + m_local;
-  const int hg = m / p.b, i = m - hg * p.b;
-  __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
-                       (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
-  uint2 w2;
-  w2.x = pack_bf16(acc.x * inv, acc.y * inv);
-  w2.y = pack_bf16(acc.z * inv, acc.w * inv);
-  *reinterpret_cast<uint2*>(out) = w2;
-  if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (m_run + log2f(l)) * kLn2;
+#pragma unroll
+  for (int s = 0; s < S; ++s) {
+    if (slot[s] < 0) continue;
+    const float inv = l[s] > 0.f ? 1.f / l[s] : 0.f;
+    const int m = rt * 128 + m_local[s];
+    const int hg = m / p.b, i = m - hg * p.b;
+    __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
+                         (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4[s] * 4;
+    uint2 w2;
+    w2.x = pack_bf16(acc[s].x * inv, acc[s].y * inv);
+    w2.y = pack_bf16(acc[s].z * inv, acc[s].w * inv);
+    *reinterpret_cast<uint2*>(out) = w2;
+    if (d4[s] == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (m_run[s] + log2f(l[s])) * kLn2;
+  }
 }
 
 // Deferred tail (large partial volumes or long sequences): one launch that merges the key splits, one thread per
@@ -281,7 +300,8 @@ __global__ void __launch_bounds__(256) umma_tail_kernel(const UmmaParams up, con
     const int64_t bg = unit / up.row_tiles;
     const int g = (int)(bg % p.Hkv), bi = (int)(bg / p.Hkv);
     if (m_local >= min(p.M - rt * 128, 128)) return;
-    merge_slot<D, 8>(p, unit, bi, g, rt, m_local, d4);
+    const int one[1] = {m_local * D4 + d4};
+    merge_slots<D, 8, 1>(p, unit, bi, g, rt, one);
     return;
   }
   const int64_t idx = (int64_t)(blockIdx.x - merge_blocks) * 256 + threadIdx.x;
@@ -844,8 +864,12 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     if (last && !*abort_flag) {
       __threadfence();
       if (tail_merge)
-        for (int slot = tid; slot < M_rt * (D / 4); slot += UM_THREADS)
-          merge_slot<D, 4>(p, unit, bi, g, rt, slot / (D / 4), slot % (D / 4));
+        for (int s0 = tid; s0 < M_rt * (D / 4); s0 += 4 * UM_THREADS) {
+          int four[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) four[u] = s0 + u * UM_THREADS < M_rt * (D / 4) ? s0 + u * UM_THREADS : -1;
+          merge_slots<D, 4, 4>(p, unit, bi, g, rt, four);
+        }
       if (tail_pool) {
         // stage the head's raw saliency in shared memory (the ring is free), then pool from there
         float* a_s = reinterpret_cast<float*>(stage0);
