@@ -798,13 +798,18 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
                         __uint_as_float(ov[4 * j + 3]) * w);
     }
     if (tid == 64) TRACE(27);
-    asm volatile("bar.sync 2, 128;\n" ::: "memory");
+  }
+  if (do_attn) {
+    // all eight warps share the stores: consecutive threads take consecutive float4 of a row; a thread keeps its column
+    // and walks down the rows, four rows per step with all their shared-memory reads in flight together
+    constexpr int D4 = D / 4;
+    const float* o_s = reinterpret_cast<const float*>(stage0);
+    const float2* lm_s = reinterpret_cast<const float2*>(stage0 + 128 * D * 4) + 128;
+    __syncthreads();
     if (tid == 64) TRACE(29);
-    // consecutive threads take consecutive float4 of a row; a thread keeps its column and walks down the rows, four
-    // rows per step with all their shared-memory reads in flight together
-    const int st = (warp - 2) * 32 + lane;
+    const int st = tid;
     if (!*abort_flag) {
-      const int d4 = st % D4, r_first = st / D4, r_step = 128 / D4;
+      const int d4 = st % D4, r_first = st / D4, r_step = UM_THREADS / D4;
       const int m_first = rt * 128;
       for (int mb = r_first; mb < M_rt; mb += 4 * r_step) {
         float4 acc[4];
@@ -852,6 +857,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   if (up.fused_tail && (tail_merge || tail_pool)) {
     __threadfence();
     __syncthreads();
+    if (tid == 0) TRACE_MAX(20);
     bool last = true;
     if (p.splits > 1) {
       if (tid == 0) {
@@ -861,6 +867,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
       __syncthreads();
       last = *last_flag != 0;
     }
+    if (tid == 0) TRACE_MAX(21);
     if (last && !*abort_flag) {
       __threadfence();
       if (tail_merge)
@@ -879,6 +886,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         for (int pos = tid; pos < p.n1_max; pos += UM_THREADS)
           p.pooled[(int64_t)(bi * p.Hkv + g) * p.n1_max + pos] = pool_at(p, a_s, n1, p.block_off[bi], pos);
       }
+      if (tid == 0) TRACE_MAX(22);
       if (p.splits > 1 && tid == 0) p.counters[unit] = 0;      // ready for the next call
     }
   }
