@@ -170,6 +170,23 @@ def run_reference(args):
     }))
 
 
+# ------------------------------------------------------------------------------------------------ replicas over ranks
+def slowest_rank_seconds(sec: float, device=None) -> float:
+    """Timed seconds of the slowest rank (the ranks run independent replicas: no data-path collective)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return sec
+    t = torch.tensor([sec], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_rank: float, world: int, slowest_sec: float) -> float:
+    """Whole-job throughput: every rank processed tokens_per_rank in at most slowest_sec."""
+    return world * tokens_per_rank / slowest_sec
+
+
 # ------------------------------------------------------------------------------------------------ CUDA arm
 def run_ours(args):
     import torch
@@ -296,12 +313,9 @@ def run_ours(args):
     sampler = ClockSampler(local) if rank == 0 else None
     sec = timed(step_runner, args.steps, max(args.warmup, 3))
     clocks = sampler.stop() if sampler else None
-    if world > 1:
-        t = torch.tensor([sec], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        sec = float(t.item())
+    sec = slowest_rank_seconds(sec, dev)
     tok = tokens_per_step(cfg, n_layers, seq_lens, n_keeps, args.phase)
-    value = world * tok * args.steps / sec
+    value = whole_job_value(tok * args.steps, world, sec)
 
     # ---- roofline of the dominant call (sparse block attention: 30 of the 31 calls per layer per block)
     ab = algorithmic_bytes(cfg, seq_lens, n_keeps)
@@ -341,14 +355,11 @@ def run_ours(args):
                         h_out_s[t, l].copy_(out_s[t, l], non_blocking=True)
         e2e_iters = max(2, min(args.steps, 5))
         e2e_sec = timed(e2e_step, e2e_iters, 1)
-        if world > 1:
-            t = torch.tensor([e2e_sec], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_sec = float(t.item())
+        e2e_sec = slowest_rank_seconds(e2e_sec, dev)
         esz = Ks[0].element_size()
         h2d = n_layers * Bn * ((2 * Hkv * L * D + Hq * b * D) * esz + reuse_steps * (2 * Hkv * b * D + Hq * b * D) * esz)
         d2h = n_layers * Bn * (1 + reuse_steps) * Hq * b * D * esz
-        e2e = {"value": world * tok * e2e_iters / e2e_sec, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+        e2e = {"value": whole_job_value(tok * e2e_iters, world, e2e_sec), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "ms_per_step": 1e3 * e2e_sec / e2e_iters}
 
     cpu_baseline = None
