@@ -108,14 +108,22 @@ def test_pool_windows(window):
     assert stats["set_mismatch"] == 0
 
 
-@pytest.mark.parametrize("env", [{"SDLLM_NO_TMA": "1"}, {"SDLLM_CLUSTER": "1", "SDLLM_SPLITS": "3"}, {"SDLLM_PDL": "0"},
-                                 {"SDLLM_SPLITS": "7"}, {"SDLLM_SPLITS": "1"}])
+@pytest.mark.parametrize("env", [
+    {"SDLLM_KERNEL": "cpasync"},                          # cp.async + mma.sync kernels, separate merge launch
+    {"SDLLM_KERNEL": "tma", "SDLLM_SPLITS": "3"},         # TMA + mma.sync kernel
+    {"SDLLM_PDL": "0"},                                   # no programmatic dependent launch
+    {"SDLLM_SPLITS": "7"}, {"SDLLM_SPLITS": "1"},         # other key-split counts of the tcgen05 kernel
+    {"SDLLM_SPLITS": "5", "SDLLM_FUSED_TAIL": "0"},       # split merge and pooling in the second launch
+    {"SDLLM_EARLY_LOADS": "0"},                           # no loads ahead of the grid dependency
+    {"SDLLM_KEY_TILE": "64", "SDLLM_SPLITS": "2"},        # 64-key tiles
+])
 def test_alternative_launch_plans_agree_with_oracle(env, monkeypatch):
-    """The cp.async kernel, the global-workspace merge (no cluster), and other split counts give the same answers."""
+    """Every kernel family, tail placement, tile size and split count gives the same answers."""
     for k, v in env.items():
         monkeypatch.setenv(k, v)
     _run_sequence_case(_small("alt_mha", "bf16", 4, 4, 128, 403, 130, salient_frac=0.02), seed=12, block=1)
     _run_sequence_case(_small("alt_gqa", "bf16", 8, 2, 128, 300, 64, retention=0.3, salient_frac=0.02), seed=13, block=0)
+    _run_sequence_case(_small("alt_gqa7", "bf16", 14, 2, 128, 260, 96, retention=0.4, salient_frac=0.02), seed=14, block=1)
 
 
 def test_ragged_batch():
