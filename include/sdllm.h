@@ -46,7 +46,9 @@ typedef enum { SDLLM_F32 = 0, SDLLM_BF16 = 1 } sdllm_dtype;
 
 /* Saliency of a candidate key (Algorithm 1, "Calculate attention scores").
  * LOGIT_MEAN: a_c = scale * <Mean(Q_b), k_c>, the pre-softmax score of the paper's equation and pseudocode.
- * PROB_MEAN : a_c = mean over the block queries of softmax(scale * Q_b K^T)[., c], normalised over all keys. */
+ * PROB_MEAN : a_c = mean over the block queries of softmax(scale * Q_b K^T)[., c], normalised over all keys. It costs a
+ *             second pass over K, needs `out` (the attention output) to be requested with the scores, and is available
+ *             for bf16 with block lengths that are multiples of 16 (other shapes: SDLLM_ERR_UNSUPPORTED). */
 typedef enum { SDLLM_SCORE_LOGIT_MEAN = 0, SDLLM_SCORE_PROB_MEAN = 1 } sdllm_score_kind;
 
 /* Key-axis pooling (Algorithm 1, MaxPool1D with kernel_size = s, padding = s/2, stride 1). AVG is the

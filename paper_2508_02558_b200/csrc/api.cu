@@ -41,7 +41,10 @@ sdllm_status check_desc(const sdllm_desc* d) {
   if (d->head_dim != 64 && d->head_dim != 128) return SDLLM_ERR_UNSUPPORTED;
   if ((int64_t)d->block_len * (d->n_q_heads / d->n_kv_heads) > kMaxRows) return SDLLM_ERR_UNSUPPORTED;
   if (d->batch > 65535 || d->n_kv_heads > 65535) return SDLLM_ERR_UNSUPPORTED;
-  if (d->score == SDLLM_SCORE_PROB_MEAN) return SDLLM_ERR_UNSUPPORTED;
+  // the softmax-probability saliency exists in the tcgen05 kernel only
+  if (d->score == SDLLM_SCORE_PROB_MEAN &&
+      !umma_supported(d->dtype, d->head_dim, d->n_q_heads / d->n_kv_heads * d->block_len, d->block_len))
+    return SDLLM_ERR_UNSUPPORTED;
   return SDLLM_OK;
 }
 
@@ -65,7 +68,7 @@ bool cuda_failed(cudaError_t e, const char* what) {
 float scale_of(const sdllm_desc* d) { return d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / sqrtf((float)d->head_dim); }
 
 struct WsLayout {
-  size_t status, counters, part_o, part_ml, raw, total;
+  size_t status, counters, part_o, part_ml, raw, lse, total;
 };
 
 WsLayout attn_ws(const sdllm_desc* d, const AttnPlan& pl, bool scores) {
@@ -82,7 +85,10 @@ WsLayout attn_ws(const sdllm_desc* d, const AttnPlan& pl, bool scores) {
   w.part_ml = off;
   off += align_up((size_t)d->batch * d->n_kv_heads * pl.part_rows * 2 * 4, 256);
   w.raw = off;
-  if (scores) off += align_up((size_t)d->batch * d->n_kv_heads * d->seq_len_max * 4, 256);
+  const bool prob = d->score == SDLLM_SCORE_PROB_MEAN;
+  if (scores) off += align_up((size_t)d->batch * d->n_kv_heads * d->seq_len_max * 4 * (prob ? pl.row_tiles : 1), 256);
+  w.lse = off;                         // probability saliency: the rows' log-sum-exp between its two passes
+  if (scores && prob) off += align_up((size_t)d->batch * d->n_q_heads * d->block_len * 4, 256);
   w.total = off;
   return w;
 }
@@ -172,8 +178,12 @@ int32_t sdllm_launch_count(const sdllm_desc* d, int op) {
   const AttnPlan pl = plan_for(d, op);
   const int M = d->n_q_heads / d->n_kv_heads * d->block_len;
   if (pl.kind == 2) {
+    const int n1 = refresh ? d->seq_len_max : d->n_keep_max;
+    if (refresh && d->score == SDLLM_SCORE_PROB_MEAN)     // attention pass (+ its merge) and saliency pass (+ its pooling)
+      return 1 + ((pl.splits > 1 && !umma_tail_is_fused(pl, d->head_dim, M, n1, false, true)) ? 1 : 0) + 1 +
+             (umma_tail_is_fused(pl, d->head_dim, M, n1, true, false) ? 0 : 1);
     const bool tail_work = pl.splits > 1 || refresh;
-    return 1 + ((tail_work && !umma_tail_is_fused(pl, d->head_dim, M, refresh ? d->seq_len_max : d->n_keep_max, refresh)) ? 1 : 0);
+    return 1 + ((tail_work && !umma_tail_is_fused(pl, d->head_dim, M, n1, refresh, true)) ? 1 : 0);
   }
   return 1 + ((refresh || pl.splits > 1) ? 1 : 0);
 }
@@ -221,6 +231,19 @@ sdllm_status sdllm_refresh_scores(const sdllm_desc* d, const void* q_blk, const 
   p.pooled = pooled_scores; p.window = d->pool_window; p.pool_kind = d->pool;
   p.per_region = d->select != SDLLM_SELECT_JOINT_FLOOR;
   for (int i = 0; i < 3; ++i) { p.k1_stride[i] = d->kv_stride[i]; p.k2_stride[i] = 0; }
+  if (d->score == SDLLM_SCORE_PROB_MEAN && pooled_scores != nullptr) {
+    // Softmax-probability saliency: the probabilities need each row's final normaliser, so the scores come from a
+    // second pass over K once the attention pass has left the rows' log-sum-exp.
+    if (!out) return SDLLM_ERR_INVALID_ARG;
+    AttnParams a = p;
+    a.want_scores = 0; a.pooled = nullptr; a.raw_scores = nullptr;
+    if (!a.lse) a.lse = reinterpret_cast<float*>(wsb + w.lse);
+    if (cuda_failed(launch_attn_partial(a, pl, d->dtype, d->head_dim, stream), "attention launch")) return SDLLM_ERR_CUDA;
+    AttnParams s2 = p;
+    s2.out = nullptr; s2.lse = nullptr; s2.lse_in = a.lse; s2.prob_pass = 1; s2.want_scores = 0;
+    if (cuda_failed(launch_attn_partial(s2, pl, d->dtype, d->head_dim, stream), "saliency launch")) return SDLLM_ERR_CUDA;
+    return SDLLM_OK;
+  }
   if (cuda_failed(launch_attn_partial(p, pl, d->dtype, d->head_dim, stream), "attention launch")) return SDLLM_ERR_CUDA;
   if (pl.fused_tail) return SDLLM_OK;
 

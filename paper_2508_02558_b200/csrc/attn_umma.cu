@@ -50,6 +50,7 @@ struct UmmaParams {
   int heads_rt;      // query heads per row tile
   int fused_tail;    // 1: the last CTA of a unit merges and pools; 0: umma_tail_kernel does
   int early_src1;    // 1: source 1 and its count are older than the previous kernel in the stream (reuse step)
+  int prob_pass;     // 1: second pass of the probability saliency: S and the rows' log-sum-exp give column means of P
 };
 
 // ---------------------------------------------------------------------------------------------------------
@@ -197,7 +198,8 @@ __device__ __forceinline__ void drain_bar(uint32_t bar, uint32_t parity) {
 // Importance of one absolute position: Algorithm 1, MaxPool1D(A, kernel_size = s, padding = s/2) over the candidate
 // axis Concat(prefix, suffix) (AvgPool for the ablation); block positions and padding get -inf. `a` holds the raw
 // saliency by absolute position.
-__device__ __forceinline__ float pool_at(const AttnParams& p, const float* a, int L, int o_in, int pos) {
+__device__ __forceinline__ float pool_at(const AttnParams& p, const float* a, int L, int o_in, int pos, int n_arr = 1,
+                                         int64_t arr_stride = 0) {
   const int b = p.b;
   const int o = min(max(o_in, 0), max(L - b, 0));
   if (pos >= L || (pos >= o && pos < o + b)) return -INFINITY;
@@ -208,7 +210,8 @@ __device__ __forceinline__ float pool_at(const AttnParams& p, const float* a, in
   float mx = -INFINITY, sum = 0.f;
   for (int t = c - w; t <= c + w; ++t) {
     if (t < lo || t >= hi) continue;
-    const float x = a[t < o ? t : t + b];
+    float x = a[t < o ? t : t + b];
+    for (int r2 = 1; r2 < n_arr; ++r2) x += a[r2 * arr_stride + (t < o ? t : t + b)];   // one array per row tile
     mx = fmaxf(mx, x);
     sum += x;
   }
@@ -311,7 +314,8 @@ __global__ void __launch_bounds__(256) umma_tail_kernel(const UmmaParams up, con
   const int bi = (int)(bh / p.Hkv);
   int L = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
   L = min(max(L, 0), p.n1_max);
-  p.pooled[idx] = pool_at(p, p.raw_scores + bh * p.n1_max, L, p.block_off[bi], pos);
+  p.pooled[idx] = pool_at(p, p.raw_scores + bh * p.n1_max, L, p.block_off[bi], pos, up.prob_pass ? up.row_tiles : 1,
+                          (int64_t)p.B * p.Hkv * p.n1_max);
 }
 
 // Optional timeline of CTA (0,0,0): built with -DSDLLM_TRACE, each point stores the global timer in the 8-byte slot
@@ -361,8 +365,10 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   const int t_begin = (int)(((long long)split * tiles_all) / p.splits);
   const int t_end = (int)(((long long)(split + 1) * tiles_all) / p.splits);
   const int M_rt = min(p.M - rt * 128, 128);          // valid query rows of this row tile (<= rows_rep when R > 1)
-  const bool do_attn = p.out != nullptr;
-  const bool do_scores = p.want_scores && rt == 0;
+  const bool prob_pass = up.prob_pass != 0;            // no V, no PV: S tiles only, reduced over the query rows
+  const bool do_attn = p.out != nullptr && !prob_pass;
+  const bool do_s = do_attn || prob_pass;              // Q and the S = Q K^T tiles are needed
+  const bool do_scores = p.want_scores && rt == 0 && !prob_pass;   // mean-query logit saliency (saliency warps)
   const int n2 = p.n2;
 
   // ---- shared memory carve-up (1024-byte aligned for the 128-byte swizzle) ----
@@ -382,11 +388,11 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   const int kv_bytes = H * half_bytes;                 // a whole K (or V) tile
   const int stage_bytes = 2 * kv_bytes;
   // Q rows that no TMA box covers must not hold non-finite garbage; only shapes with b*G below the replica's rows need it
-  const bool zero_q = do_attn && p.b * up.heads_rt < rows_rep;
+  const bool zero_q = do_s && p.b * up.heads_rt < rows_rep;
   if (tid == 0) {                        // the descriptors live in the kernel parameters: fetch them while the CTA sets up
     prefetch_tmap(&tm.k1); prefetch_tmap(&tm.v1);
     if (n2 > 0) { prefetch_tmap(&tm.k2); prefetch_tmap(&tm.v2); }
-    if (do_attn) prefetch_tmap(&tm.q);
+    if (do_s) prefetch_tmap(&tm.q);
   }
 
   // The producer lane sets the barriers up and, unless the Q tile has to be cleared first, starts the first loads
@@ -396,7 +402,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   bool q_issued = false;
   auto issue_q = [&]() {              // the Q tile (replicated R times along the accumulator rows)
     q_issued = true;
-    if (!do_attn) return;
+    if (!do_s) return;
     mbar_expect_tx(BAR(Q_FULL), (uint32_t)(R * H * p.b * up.heads_rt * 128));
     for (int rep = 0; rep < R; ++rep)
       for (int h = 0; h < H; ++h)
@@ -434,7 +440,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     for (int s = 0; s < NS; ++s) {
       mbar_init(BAR(FULL_K + s), 1);
       mbar_init(BAR(FULL_V + s), 1);
-      mbar_init(BAR(EMPTY_K + s), max((do_attn ? 1 : 0) + (do_scores ? 2 : 0), 1));
+      mbar_init(BAR(EMPTY_K + s), max((do_s ? 1 : 0) + (do_scores ? 2 : 0), 1));
       mbar_init(BAR(EMPTY_V + s), 1);
     }
     for (int i = 0; i < 2; ++i) {
@@ -447,7 +453,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     *last_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     TRACE(2);
-    if (!zero_q && (do_attn || do_scores)) {
+    if (!zero_q && (do_s || do_scores)) {
       if (up.early_src1) {
         // Reuse step: the compacted cache and its count were written before the previous kernel in the stream even
         // started, so their tiles may stream in while that kernel is still finishing.
@@ -492,7 +498,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
 
   if (warp == 0) {
     // ======================================= TMA producer =======================================
-    if (lane == 0 && (do_attn || do_scores)) {
+    if (lane == 0 && (do_s || do_scores)) {
       prod_n1 = n1;
       if (!q_issued) issue_q();
       produce(1 << 30, false);
@@ -502,12 +508,12 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
           drain_bar(BAR(FULL_K + j % NS), (j / NS) & 1);
           if (do_attn) drain_bar(BAR(FULL_V + j % NS), (j / NS) & 1);
         }
-        if (do_attn && q_issued) drain_bar(BAR(Q_FULL), 0);
+        if (do_s && q_issued) drain_bar(BAR(Q_FULL), 0);
       }
     }
   } else if (warp == 1) {
     // ======================================= MMA issuer =======================================
-    if (lane == 0 && do_attn) {
+    if (lane == 0 && do_s) {
       const uint32_t idesc_pv = instr_desc(D, true);
       bool ok = true, have_q = false;
       int it = 0;
@@ -537,6 +543,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
           if (!wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 3)) { ok = false; break; }
           have_q = true;
         }
+        // without PV nothing else orders the reuse of an S buffer: wait until the softmax warps have read tile it - 2
+        if (prob_pass && it >= 2 && !wait_bar(BAR(P_FULL + sb), ((it >> 1) - 1) & 1, abort_flag, p.status, 12)) { ok = false; break; }
         if (it == 0) TRACE(7);
         tc_fence_after();
         const uint32_t ksm = smem_u32(stage0 + (size_t)s * stage_bytes);
@@ -551,11 +559,11 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         }
         tc_commit(BAR(S_FULL + sb));
         tc_commit(BAR(EMPTY_K + s));
-        if (prev_it >= 0 && !issue_pv(prev, prev_it)) { ok = false; break; }
+        if (do_attn && prev_it >= 0 && !issue_pv(prev, prev_it)) { ok = false; break; }
         prev = x; prev_it = it;
         ++it;
       }
-      if (ok && prev_it >= 0) ok = issue_pv(prev, prev_it);
+      if (do_attn && ok && prev_it >= 0) ok = issue_pv(prev, prev_it);
       if (*abort_flag) {               // wait for the tensor pipe to finish what was issued before TMEM is freed
         tc_commit(BAR(DRAIN));
         drain_bar(BAR(DRAIN), 0);
@@ -563,7 +571,75 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     }
   } else if (warp < 6) {
     // ======================================= softmax warps =======================================
-    if (do_attn) {
+    if (prob_pass) {
+      // Probability saliency, second pass: with the rows' log-sum-exp known, P_ij = exp(S_ij - lse_i) is final, and
+      // the saliency of key j is the mean of column j over the b*G query rows. Each warp sums its 32 rows of a
+      // 32-column chunk with a shuffle transpose (lane i ends up with column i); the four warps' sums meet in shared
+      // memory (the V half of ring slot 0, never loaded in this pass), double-buffered by tile parity.
+      const int q4 = warp & 3;
+      const int row = q4 * 32 + lane;
+      const int rep = row / rows_rep, m_local = row - rep * rows_rep;
+      const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16);
+      const int chunk_keys = KT / R;
+      float* colsum = reinterpret_cast<float*>(stage0 + kv_bytes);          // [2][4][KT]
+      float lse2 = INFINITY;                           // rows outside the tile contribute exp2(-inf) = 0
+      if (m_local < M_rt) {
+        const int m = rt * 128 + m_local;
+        const int hg = m / p.b, i = m - hg * p.b;
+        lse2 = p.lse_in[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] * kLog2e;
+      }
+      const float inv_rows = 1.f / (float)p.M;
+      float* raw = p.raw_scores + ((int64_t)rt * p.B * p.Hkv + (int64_t)(bi * p.Hkv + g)) * p.n1_max;
+      const int st = (warp - 2) * 32 + lane;
+      int it = 0;
+      bool dead = false;
+      for (int t = t_begin; t < t_end; ++t) {
+        const Tile x = tile_of(t, tiles1, KT, KT2, n1, n2);
+        if (x.nv == 0) continue;
+        const int sb = it & 1;
+        const int c_lo = min(rep * chunk_keys, x.nv), c_hi = min((rep + 1) * chunk_keys, x.nv);
+        // a warp that gave up keeps walking the tiles so that the four warps meet at every barrier below
+        if (!dead && !wait_bar_warp(BAR(S_FULL + sb), (it >> 1) & 1, abort_flag, p.status, 9)) dead = true;
+        tc_fence_after();
+        float* cs = colsum + (size_t)sb * 4 * KT + (size_t)(warp - 2) * KT;
+#pragma unroll 1
+        for (int c = 0; c * 32 < KT && !dead; ++c) {
+          float v[32];
+          if (c * 32 < c_hi && c * 32 + 32 > c_lo) {
+            uint32_t sv[32];
+            tmem_ld32(lane_addr + (uint32_t)sb * 128u + c * 32, sv);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const bool in = c * 32 + i >= c_lo && c * 32 + i < c_hi;
+              v[i] = in ? fast_exp2(fmaf(__uint_as_float(sv[i]), p.scale_log2, -lse2)) : 0.f;
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) {
+              const bool up_half = (lane & off) != 0;
+#pragma unroll
+              for (int k = 0; k < off; ++k) {
+                const float send = up_half ? v[k] : v[k + off];
+                const float keep = up_half ? v[k + off] : v[k];
+                v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+              }
+            }
+          } else {
+            v[0] = 0.f;
+          }
+          cs[c * 32 + lane] = v[0];
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(P_FULL + sb));        // the S buffer may be overwritten
+        asm volatile("bar.sync 2, 128;\n" ::: "memory");
+        if (st < x.nv && x.src1 && !dead) {
+          const float* c4 = colsum + (size_t)sb * 4 * KT + st;
+          raw[x.row0 + st] = ((c4[0] + c4[KT]) + (c4[2 * KT] + c4[3 * KT])) * inv_rows;
+        }
+        ++it;
+      }
+    } else if (do_attn) {
       const int q4 = warp & 3;                         // TMEM lane quadrant this warp may access
       const int row = q4 * 32 + lane;
       const int rep = row / rows_rep;                  // warp-uniform
@@ -853,16 +929,20 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
 
   // ---- fused tail: the last CTA of the unit merges the key splits and pools the saliency; nobody waits ----
   const bool tail_merge = do_attn && p.splits > 1;
-  const bool tail_pool = do_scores && p.pooled != nullptr;
+  const bool tail_pool = (do_scores || prob_pass) && p.pooled != nullptr;
+  // who counts: the key splits of a unit; in the probability pass all row tiles of the head as well (its pooling
+  // needs every row tile's column sums), on the counter of the head's first unit
+  const int expected = prob_pass ? p.splits * up.row_tiles : p.splits;
+  int32_t* counter = p.counters + (prob_pass ? unit - rt : unit);
   if (up.fused_tail && (tail_merge || tail_pool)) {
     __threadfence();
     __syncthreads();
     if (tid == 0) TRACE_MAX(20);
     bool last = true;
-    if (p.splits > 1) {
+    if (expected > 1) {
       if (tid == 0) {
-        const int old = atomicAdd(p.counters + unit, 1);
-        *last_flag = (old == p.splits - 1) ? 1 : 0;
+        const int old = atomicAdd(counter, 1);
+        *last_flag = (old == expected - 1) ? 1 : 0;
       }
       __syncthreads();
       last = *last_flag != 0;
@@ -881,13 +961,18 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         // stage the head's raw saliency in shared memory (the ring is free), then pool from there
         float* a_s = reinterpret_cast<float*>(stage0);
         const float* a = p.raw_scores + (int64_t)(bi * p.Hkv + g) * p.n1_max;
-        for (int i = tid; i < n1; i += UM_THREADS) a_s[i] = __ldcg(a + i);
+        const int n_arr = prob_pass ? up.row_tiles : 1;          // the probability pass left one array per row tile
+        for (int i = tid; i < n1; i += UM_THREADS) {
+          float x = 0.f;
+          for (int r2 = 0; r2 < n_arr; ++r2) x += __ldcg(a + (int64_t)r2 * p.B * p.Hkv * p.n1_max + i);
+          a_s[i] = x;
+        }
         __syncthreads();
         for (int pos = tid; pos < p.n1_max; pos += UM_THREADS)
           p.pooled[(int64_t)(bi * p.Hkv + g) * p.n1_max + pos] = pool_at(p, a_s, n1, p.block_off[bi], pos);
       }
       if (tid == 0) TRACE_MAX(22);
-      if (p.splits > 1 && tid == 0) p.counters[unit] = 0;      // ready for the next call
+      if (expected > 1 && tid == 0) *counter = 0;               // ready for the next call
     }
   }
 
@@ -981,8 +1066,8 @@ bool umma_supported(int dtype, int D, int M, int b) {
 
 // The last CTA of a unit does the tail itself while that is a small job; otherwise a second launch spreads it over
 // the whole GPU.
-bool umma_tail_is_fused(const AttnPlan& pl, int D, int M, int n1_max, bool pool) {
-  const size_t merge_bytes = pl.splits > 1 ? (size_t)pl.splits * (M < 128 ? M : 128) * D * 4 : 0;
+bool umma_tail_is_fused(const AttnPlan& pl, int D, int M, int n1_max, bool pool, bool merge) {
+  const size_t merge_bytes = merge && pl.splits > 1 ? (size_t)pl.splits * (M < 128 ? M : 128) * D * 4 : 0;
   bool fused = merge_bytes <= 256 * 1024 && (!pool || n1_max <= 8192);
   if (const char* e = getenv("SDLLM_FUSED_TAIL")) fused = e[0] == '1' && (!pool || n1_max <= 8192);   // tuning aid
   return fused;
@@ -1032,10 +1117,11 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
     const char* e = getenv("SDLLM_EARLY_LOADS");   // SDLLM_EARLY_LOADS=0: no loads before the grid dependency (test aid)
     up.early_src1 = (p.n2 > 0 && p.n1_max > 0 && !(e && e[0] == '0')) ? 1 : 0;
   }
-  up.fused_tail = umma_tail_is_fused(pl, D, p.M, p.n1_max, pool) ? 1 : 0;
+  up.prob_pass = p.prob_pass;
+  up.fused_tail = umma_tail_is_fused(pl, D, p.M, p.n1_max, pool || p.prob_pass, p.out != nullptr && !p.prob_pass) ? 1 : 0;
   memset(&tm, 0, sizeof(tm));
   bool ok = true;
-  if (p.out != nullptr) ok = make_map(&tm.q, p.q, D, p.b, p.Hq, p.B, p.q_stride, p.b, up.heads_rt);
+  if (p.out != nullptr || p.prob_pass) ok = make_map(&tm.q, p.q, D, p.b, p.Hq, p.B, p.q_stride, p.b, up.heads_rt);
   if (p.n1_max > 0) {
     ok = ok && make_map(&tm.k1, p.k1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, pl.key_tile, 1);
     ok = ok && make_map(&tm.v1, p.v1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, pl.key_tile, 1);
@@ -1050,10 +1136,11 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
   if (!ok) return cudaErrorInvalidValue;
   cudaError_t err = D == 128 ? launch_umma_d<128>(tm, up, pl, st) : launch_umma_d<64>(tm, up, pl, st);
   if (err != cudaSuccess || up.fused_tail) return err;
-  const bool merge = p.out != nullptr && pl.splits > 1;
-  if (!merge && !pool) return cudaSuccess;
+  const bool merge = p.out != nullptr && !p.prob_pass && pl.splits > 1;
+  const bool pool_tail = pool || (p.prob_pass && p.pooled != nullptr);
+  if (!merge && !pool_tail) return cudaSuccess;
   const long long merge_threads = merge ? (long long)p.B * p.Hkv * pl.row_tiles * 128 * (D / 4) : 0;
-  const long long pool_threads = pool ? (long long)p.B * p.Hkv * p.n1_max : 0;
+  const long long pool_threads = pool_tail ? (long long)p.B * p.Hkv * p.n1_max : 0;
   const int merge_blocks = (int)((merge_threads + 255) / 256);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(merge_blocks + (pool_threads + 255) / 256));

@@ -60,6 +60,8 @@ struct AttnParams {
   int32_t* counters;           // completion counters (tcgen05 kernel), zero between calls
   float* pooled;               // refresh with a fused tail: pooled scores [B][Hkv][n1_max], else null
   int window, pool_kind, per_region;
+  const float* lse_in;         // probability saliency, second pass: log-sum-exp of every block row [B][Hq][b]
+  int prob_pass;               // 1: this launch is that second pass (tcgen05 kernel only)
   int want_scores;             // compute mean-query logit scores for src1 keys
   float scale;                 // softmax scale
   float scale_log2;            // scale * log2(e)
@@ -95,7 +97,8 @@ struct CompactParams {
 
 AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_max, int n2);
 
-bool umma_tail_is_fused(const AttnPlan& pl, int D, int M, int n1_max, bool pool);
+bool umma_tail_is_fused(const AttnPlan& pl, int D, int M, int n1_max, bool pool, bool merge);
+bool umma_supported(int dtype, int D, int M, int b);
 cudaError_t launch_attn_partial(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st);
 cudaError_t launch_merge_pool(const MergeParams& p, cudaStream_t st);
 cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st);

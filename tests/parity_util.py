@@ -87,7 +87,8 @@ def gpu_refresh(q, k, v, seq_len: Sequence[int], block_off: Sequence[int], dtype
 
 def check_refresh_against_oracle(g: GpuRefresh, q, k, v, seq_len, block_off, dtype, retention, window, *,
                                  heads: Optional[List[int]] = None, select=oracle.SELECT_JOINT_FLOOR,
-                                 pool_kind=oracle.POOL_MAX, score_rtol: float = 1e-4, seqs: Optional[List[int]] = None):
+                                 pool_kind=oracle.POOL_MAX, score_rtol: float = 1e-4, seqs: Optional[List[int]] = None,
+                                 score=oracle.SCORE_LOGIT_MEAN):
     """Element-by-element comparison of one refresh (all sequences; optionally a subset of KV heads)."""
     Bn, Hq, b, D = q.shape
     Hkv = k.shape[1]
@@ -97,7 +98,8 @@ def check_refresh_against_oracle(g: GpuRefresh, q, k, v, seq_len, block_off, dty
         L, o = int(seq_len[i]), int(block_off[i])
         hs = list(range(Hkv)) if heads is None else heads
         qh = np.concatenate([q[i, h * G:(h + 1) * G] for h in hs])
-        r = oracle.refresh(qh, k[i, hs, :L], v[i, hs, :L], o, retention, window, select=select, pool_kind=pool_kind)
+        r = oracle.refresh(qh, k[i, hs, :L], v[i, hs, :L], o, retention, window, select=select, pool_kind=pool_kind,
+                           score=score)
         n = r.n_keep
         assert int(g.kept_cnt[i]) == min(n, g.cache.n_keep_max), (g.kept_cnt[i], n)
         pos = oracle.candidate_positions(L, b, o)

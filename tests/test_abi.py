@@ -72,7 +72,7 @@ def test_workspace_sizes():
     (dict(n_q_heads=30), B.ERR_INVALID_ARG), (dict(dtype=7), B.ERR_INVALID_ARG),
     (dict(head_dim=96), B.ERR_UNSUPPORTED), (dict(n_kv_heads=1, block_len=32), B.ERR_UNSUPPORTED),
     (dict(kv_stride=(1, 2, 3)), B.ERR_INVALID_ARG), (dict(softmax_scale=-1.0), B.ERR_INVALID_ARG),
-    (dict(score=B.SCORE_PROB_MEAN), B.ERR_UNSUPPORTED),
+    (dict(score=B.SCORE_PROB_MEAN, dtype=B.F32), B.ERR_UNSUPPORTED),
 ])
 def test_bad_descriptions_are_rejected_before_any_launch(bad, status):
     d = _desc(**bad)

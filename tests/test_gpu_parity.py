@@ -27,9 +27,10 @@ def _run_sequence_case(cfg: W.WorkloadConfig, seed: int, block: int, n_sparse: i
     L, o = s.seq_len, s.block_off
     sel = policy.get("select", oracle.SELECT_JOINT_FLOOR)
     pk = policy.get("pool", oracle.POOL_MAX)
+    sk = policy.get("score", oracle.SCORE_LOGIT_MEAN)
     g = U.gpu_refresh(q[None], k[None], v[None], [L], [o], cfg.dtype, cfg.retention, cfg.pool_window, **policy)
     stats = U.check_refresh_against_oracle(g, q[None], k[None], v[None], [L], [o], cfg.dtype, cfg.retention,
-                                           cfg.pool_window, heads=heads, select=sel, pool_kind=pk)
+                                           cfg.pool_window, heads=heads, select=sel, pool_kind=pk, score=sk)
     U.check_compaction_bit_exact(g, g.k_dev, g.v_dev)
     for step in range(2, 2 + n_sparse):
         q2, kn, vn = s.sparse_inputs(step)
@@ -124,6 +125,20 @@ def test_alternative_launch_plans_agree_with_oracle(env, monkeypatch):
     _run_sequence_case(_small("alt_mha", "bf16", 4, 4, 128, 403, 130, salient_frac=0.02), seed=12, block=1)
     _run_sequence_case(_small("alt_gqa", "bf16", 8, 2, 128, 300, 64, retention=0.3, salient_frac=0.02), seed=13, block=0)
     _run_sequence_case(_small("alt_gqa7", "bf16", 14, 2, 128, 260, 96, retention=0.4, salient_frac=0.02), seed=14, block=1)
+
+
+@pytest.mark.parametrize("cfg,block", [
+    (_small("prob_mha", "bf16", 4, 4, 128, 403, 130, salient_frac=0.02), 1),            # replicated rows, ragged tail
+    (_small("prob_gqa4", "bf16", 8, 2, 128, 517, 64, retention=0.3, salient_frac=0.01), 0),   # one full 128-row tile
+    (_small("prob_gqa7", "bf16", 14, 2, 128, 300, 96, retention=0.25, salient_frac=0.01, sink_tokens=4), 2),   # two row tiles
+    (_small("prob_d64", "bf16", 4, 2, 64, 150, 64, salient_frac=0.02), 1),
+])
+@pytest.mark.parametrize("env", [{}, {"SDLLM_SPLITS": "3", "SDLLM_FUSED_TAIL": "0"}, {"SDLLM_SPLITS": "1"}])
+def test_softmax_probability_saliency(cfg, block, env, monkeypatch):
+    """The second reading of "attention scores": mean softmax probability per key (two passes over K)."""
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    _run_sequence_case(cfg, seed=15, block=block, n_sparse=1, score=B.SCORE_PROB_MEAN)
 
 
 def test_ragged_batch():
