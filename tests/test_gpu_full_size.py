@@ -38,15 +38,15 @@ def _check_all_heads_properties(g, seq_len, block_off, b):
                 assert pooled[h][kept].min() >= pooled[h][cand & ~kept].max()
 
 
-def _run(cfg, seed, heads, retention=None, window=None):
+def _run(cfg, seed, heads, retention=None, window=None, score=oracle.SCORE_LOGIT_MEAN):
     import parity_util as U
     r = cfg.retention if retention is None else retention
     s_ = cfg.pool_window if window is None else window
     s = W.make_sequence(cfg, seed=seed, layer=0, block=0)
     q, k, v = s.refresh_inputs(1)
     L, o = s.seq_len, s.block_off
-    g = U.gpu_refresh(q[None], k[None], v[None], [L], [o], cfg.dtype, r, s_)
-    U.check_refresh_against_oracle(g, q[None], k[None], v[None], [L], [o], cfg.dtype, r, s_, heads=heads)
+    g = U.gpu_refresh(q[None], k[None], v[None], [L], [o], cfg.dtype, r, s_, score=score)
+    U.check_refresh_against_oracle(g, q[None], k[None], v[None], [L], [o], cfg.dtype, r, s_, heads=heads, score=score)
     _check_all_heads_properties(g, [L], [o], cfg.block_len)
     U.check_compaction_bit_exact(g, g.k_dev, g.v_dev)
     q2, kn, vn = s.sparse_inputs(2)
@@ -66,6 +66,11 @@ def test_c3_dream_layer_full_size():
 @pytest.mark.parametrize("r,window", [(0.1, 7), (0.5, 3)])
 def test_c4_long_context_full_size(r, window):
     _run(W.CONFIGS["c4_long"], seed=23, heads=[5], retention=r, window=window)
+
+
+@pytest.mark.parametrize("name,heads,r,window", [("c3_dream", [1], None, None), ("c4_long", [2], 0.25, 1)])
+def test_softmax_probability_saliency_full_size(name, heads, r, window):
+    _run(W.CONFIGS[name], seed=25, heads=heads, retention=r, window=window, score=oracle.SCORE_PROB_MEAN)
 
 
 @pytest.mark.parametrize("batch", [4, 16])
