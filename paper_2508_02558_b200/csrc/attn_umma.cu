@@ -51,6 +51,7 @@ struct UmmaParams {
   int fused_tail;    // 1: the last CTA of a unit merges and pools; 0: umma_tail_kernel does
   int early_src1;    // 1: source 1 and its count are older than the previous kernel in the stream (reuse step)
   int prob_pass;     // 1: second pass of the probability saliency: S and the rows' log-sum-exp give column means of P
+  int cluster;       // > 1: the key splits of a unit form a thread-block cluster and merge through distributed shared memory
 };
 
 // ---------------------------------------------------------------------------------------------------------
@@ -143,6 +144,26 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];\n" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+  return v;
+}
+
 // Shared-memory matrix descriptor of tcgen05.mma: 128-byte swizzle, start address / leading / stride offsets in
 // 16-byte units, descriptor version 1 in bits 46-47, swizzle mode 2 (128 B) in bits 61-63.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -212,6 +233,25 @@ __device__ __forceinline__ float pool_at(const AttnParams& p, const float* a, in
     if (t < lo || t >= hi) continue;
     float x = a[t < o ? t : t + b];
     for (int r2 = 1; r2 < n_arr; ++r2) x += a[r2 * arr_stride + (t < o ? t : t + b)];   // one array per row tile
+    mx = fmaxf(mx, x);
+    sum += x;
+  }
+  return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
+}
+
+// The same, reading the raw saliency from global memory through L2 (other CTAs wrote it during this launch).
+__device__ __forceinline__ float pool_at_ldcg(const AttnParams& p, const float* a, int L, int o_in, int pos) {
+  const int b = p.b;
+  const int o = min(max(o_in, 0), max(L - b, 0));
+  if (pos >= L || (pos >= o && pos < o + b)) return -INFINITY;
+  const int C = max(L - b, 0), w = (p.window - 1) / 2;
+  const int c = pos < o ? pos : pos - b;
+  int lo = 0, hi = C;
+  if (p.per_region) { if (c < o) hi = o; else lo = o; }
+  float mx = -INFINITY, sum = 0.f;
+  for (int t = c - w; t <= c + w; ++t) {
+    if (t < lo || t >= hi) continue;
+    const float x = __ldcg(a + (t < o ? t : t + b));
     mx = fmaxf(mx, x);
     sum += x;
   }
@@ -916,6 +956,9 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
             w2.y = pack_bf16(acc[u].z * inv, acc[u].w * inv);
             *reinterpret_cast<uint2*>(o) = w2;
             if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (x[u].x + log2f(x[u].y)) * kLn2;
+          } else if (up.cluster > 1) {
+            // this split's partial stays on chip: pm_s [M_rt][D] next to lm_s, read by the cluster peers below
+            *reinterpret_cast<float4*>(reinterpret_cast<float*>(stage0 + 128 * D * 4 + 2048) + ml * D + d4 * 4) = acc[u];
           } else {
             const int64_t prow = (unit * p.splits + split) * min(p.M, 128) + ml;
             *reinterpret_cast<float4*>(p.part_o + prow * D + d4 * 4) = acc[u];
@@ -934,7 +977,63 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   // needs every row tile's column sums), on the counter of the head's first unit
   const int expected = prob_pass ? p.splits * up.row_tiles : p.splits;
   int32_t* counter = p.counters + (prob_pass ? unit - rt : unit);
-  if (up.fused_tail && (tail_merge || tail_pool)) {
+  if (up.cluster > 1) {
+    // ---- cluster tail: the key splits of the unit are the CTAs of one cluster. After a cluster barrier every split's
+    //      partial (in its shared memory) and raw saliency (in global memory) is visible to all of them; each CTA then
+    //      merges a share of the rows straight out of its peers' shared memory and pools a share of the positions.
+    //      No partial touches global memory, no counter, no CTA is left to do the whole tail alone. ----
+    constexpr int D4 = D / 4;
+    const int S = up.cluster;
+    __threadfence();
+    __syncthreads();                     // also brings the lanes of the producer and MMA warps back together
+    cluster_sync_all();
+    if (tail_merge && !*abort_flag) {
+      const uint32_t lm_a = smem_u32(stage0 + 128 * D * 4) + 128 * 8;      // lm_s
+      const uint32_t pm_a = smem_u32(stage0 + 128 * D * 4 + 2048);         // pm_s
+      const int r_lo = (int)(((long long)split * M_rt) / S), r_hi = (int)(((long long)(split + 1) * M_rt) / S);
+      for (int slot = tid; slot < (r_hi - r_lo) * D4; slot += UM_THREADS) {
+        const int ml = r_lo + slot / D4, d4 = slot % D4;
+        float2 x[8];
+        float4 o[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint32_t peer = (uint32_t)min(c, S - 1);
+          x[c] = ld_cluster_f2(map_to_cta(lm_a + ml * 8, peer));
+          o[c] = ld_cluster_f4(map_to_cta(pm_a + (uint32_t)(ml * D + d4 * 4) * 4u, peer));
+        }
+        float mstar = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          if (c < S && x[c].y > 0.f) mstar = fmaxf(mstar, x[c].x);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float l = 0.f;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          if (c >= S || !(x[c].y > 0.f)) continue;
+          const float w = fast_exp2(x[c].x - mstar);
+          l = fmaf(x[c].y, w, l);
+          acc.x = fmaf(o[c].x, w, acc.x); acc.y = fmaf(o[c].y, w, acc.y); acc.z = fmaf(o[c].z, w, acc.z); acc.w = fmaf(o[c].w, w, acc.w);
+        }
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        const int m = rt * 128 + ml;
+        const int hg = m / p.b, i = m - hg * p.b;
+        __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
+                             (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
+        uint2 w2;
+        w2.x = pack_bf16(acc.x * inv, acc.y * inv);
+        w2.y = pack_bf16(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2*>(out) = w2;
+        if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
+      }
+    }
+    if (tail_pool && !*abort_flag) {
+      const float* a = p.raw_scores + (int64_t)(bi * p.Hkv + g) * p.n1_max;
+      const int p_lo = (int)(((long long)split * p.n1_max) / S), p_hi = (int)(((long long)(split + 1) * p.n1_max) / S);
+      for (int pos = p_lo + tid; pos < p_hi; pos += UM_THREADS)
+        p.pooled[(int64_t)(bi * p.Hkv + g) * p.n1_max + pos] = pool_at_ldcg(p, a, n1, p.block_off[bi], pos);
+    }
+    cluster_sync_all();                  // nobody leaves while a peer may still read its shared memory
+  } else if (up.fused_tail && (tail_merge || tail_pool)) {
     __threadfence();
     __syncthreads();
     if (tid == 0) TRACE_MAX(20);
@@ -1042,12 +1141,17 @@ cudaError_t launch_umma_d(const UmmaMaps& tm, const UmmaParams& up, const AttnPl
   cfg.blockDim = dim3(UM_THREADS);
   cfg.dynamicSmemBytes = pl.smem_bytes;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   int na = 0;
   const char* e = getenv("SDLLM_PDL");       // SDLLM_PDL=0 turns programmatic dependent launch off (tuning and test aid)
   if (!(e && e[0] == '0')) {
     attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  if (up.cluster > 1) {                      // the key splits (grid x) of a unit form one cluster
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = up.cluster; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
     ++na;
   }
   cfg.attrs = attr; cfg.numAttrs = na;
@@ -1102,6 +1206,17 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
   pl.part_rows = pl.splits > 1 ? (size_t)pl.row_tiles * pl.splits * (M < 128 ? M : 128) : 0;
   pl.n_counters = (size_t)B * Hkv * pl.row_tiles;
   pl.smem_bytes = umma_smem_bytes(D, pl.key_tile);
+  // Few key splits of a small problem: make them one thread-block cluster, so that they merge through distributed shared
+  // memory instead of the workspace. Only where the whole grid is one wave (a cluster needs all its SMs at once).
+  {
+    const char* e = getenv("SDLLM_CLUSTER");           // SDLLM_CLUSTER=0: never (tuning and test aid)
+    const char* f = getenv("SDLLM_FUSED_TAIL");
+    const bool off = (e && e[0] == '0') || (f && f[0] == '0');
+    const size_t merge_bytes = (size_t)pl.splits * (M < 128 ? M : 128) * D * 4;
+    if (!off && pl.splits >= 2 && pl.splits <= 8 && pl.row_tiles == 1 && pl.key_tile == 128 && units * pl.splits <= kNumSMs &&
+        merge_bytes <= 256 * 1024 && n1_max <= 8192)
+      pl.cluster = pl.splits;
+  }
   return pl;
 }
 
@@ -1118,7 +1233,9 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
     up.early_src1 = (p.n2 > 0 && p.n1_max > 0 && !(e && e[0] == '0')) ? 1 : 0;
   }
   up.prob_pass = p.prob_pass;
-  up.fused_tail = umma_tail_is_fused(pl, D, p.M, p.n1_max, pool || p.prob_pass, p.out != nullptr && !p.prob_pass) ? 1 : 0;
+  up.cluster = pl.cluster;
+  if (up.cluster > 1) up.fused_tail = 1;     // set again below; the cluster tail never needs the second launch
+  up.fused_tail = (pl.cluster > 1 || umma_tail_is_fused(pl, D, p.M, p.n1_max, pool || p.prob_pass, p.out != nullptr && !p.prob_pass)) ? 1 : 0;
   memset(&tm, 0, sizeof(tm));
   bool ok = true;
   if (p.out != nullptr || p.prob_pass) ok = make_map(&tm.q, p.q, D, p.b, p.Hq, p.B, p.q_stride, p.b, up.heads_rt);
