@@ -384,7 +384,9 @@ __device__ __forceinline__ void trace_all(int32_t* status, int slot, bool is_min
 #define TRACE_MAX(slot) do { } while (0)
 #endif
 
-template <int D>
+// PROB selects the second pass of the probability saliency; it is a template parameter so that the attention kernel proper
+// does not carry that pass's code.
+template <int D, bool PROB>
 __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __grid_constant__ UmmaMaps tm, const UmmaParams up) {
   constexpr int H = D / 64;            // 128-byte column halves of a row
   constexpr int NS = UM_STAGES;
@@ -405,7 +407,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   const int t_begin = (int)(((long long)split * tiles_all) / p.splits);
   const int t_end = (int)(((long long)(split + 1) * tiles_all) / p.splits);
   const int M_rt = min(p.M - rt * 128, 128);          // valid query rows of this row tile (<= rows_rep when R > 1)
-  const bool prob_pass = up.prob_pass != 0;            // no V, no PV: S tiles only, reduced over the query rows
+  constexpr bool prob_pass = PROB;                      // no V, no PV: S tiles only, reduced over the query rows
   const bool do_attn = p.out != nullptr && !prob_pass;
   const bool do_s = do_attn || prob_pass;              // Q and the S = Q K^T tiles are needed
   const bool do_scores = p.want_scores && rt == 0 && !prob_pass;   // mean-query logit saliency (saliency warps)
@@ -611,7 +613,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     }
   } else if (warp < 6) {
     // ======================================= softmax warps =======================================
-    if (prob_pass) {
+    if constexpr (PROB) {
       // Probability saliency, second pass: with the rows' log-sum-exp known, P_ij = exp(S_ij - lse_i) is final, and
       // the saliency of key j is the mean of column j over the b*G query rows. Each warp sums its 32 rows of a
       // 32-column chunk with a shuffle transpose (lane i ends up with column i); the four warps' sums meet in shared
@@ -1126,9 +1128,9 @@ size_t umma_smem_bytes(int D, int KT) {
   return need > 120 * 1024 ? need : 120 * 1024;
 }
 
-template <int D>
+template <int D, bool PROB>
 cudaError_t launch_umma_d(const UmmaMaps& tm, const UmmaParams& up, const AttnPlan& pl, cudaStream_t st) {
-  auto kern = attn_umma_bf16_kernel<D>;
+  auto kern = attn_umma_bf16_kernel<D, PROB>;
   static size_t configured = 0;
   if (pl.smem_bytes > configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
@@ -1251,7 +1253,9 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
     tm.k2 = tm.k1; tm.v2 = tm.v1;
   }
   if (!ok) return cudaErrorInvalidValue;
-  cudaError_t err = D == 128 ? launch_umma_d<128>(tm, up, pl, st) : launch_umma_d<64>(tm, up, pl, st);
+  cudaError_t err;
+  if (up.prob_pass) err = D == 128 ? launch_umma_d<128, true>(tm, up, pl, st) : launch_umma_d<64, true>(tm, up, pl, st);
+  else err = D == 128 ? launch_umma_d<128, false>(tm, up, pl, st) : launch_umma_d<64, false>(tm, up, pl, st);
   if (err != cudaSuccess || up.fused_tail) return err;
   const bool merge = p.out != nullptr && !p.prob_pass && pl.splits > 1;
   const bool pool_tail = pool || (p.prob_pass && p.pooled != nullptr);
