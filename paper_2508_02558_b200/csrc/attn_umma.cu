@@ -1280,4 +1280,27 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
                   : cudaLaunchKernelEx(&cfg, umma_tail_kernel<64>, up, merge_blocks);
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Dispatch between the kernel families
+AttnPlan plan_attention_legacy(int dtype, int D, int M, int B, int Hkv, int n_keys_max);
+cudaError_t launch_attn_legacy(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st);
+
+AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_max, int n2) {
+  // bf16 goes to the tcgen05 kernel wherever it applies; fp32 and the remaining bf16 shapes to the cp.async kernels.
+  // SDLLM_KERNEL=cpasync forces the latter (test aid).
+  const char* kern = getenv("SDLLM_KERNEL");
+  if (!(kern && kern[0] == 'c') && umma_supported(dtype, D, M, b)) return plan_attention_umma(D, M, b, B, Hkv, n1_max, n2);
+  AttnPlan pl = plan_attention_legacy(dtype, D, M, B, Hkv, n1_max + n2);
+  pl.tma = false; pl.cluster = 1; pl.warp_keys = 32; pl.kind = 0;
+  pl.part_rows = pl.splits > 1 ? (size_t)pl.splits * M : 0;      // partial rows the kernels leave per (sequence, KV head)
+  pl.n_counters = 0; pl.fused_tail = false;
+  pl.rep = 1; pl.row_tiles = 1; pl.parts = pl.splits; pl.rows_rep = M; pl.key_tile2 = pl.key_tile;
+  return pl;
+}
+
+cudaError_t launch_attn_partial(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st) {
+  if (plan.kind == 2) return launch_attn_umma(p, plan, D, st);
+  return launch_attn_legacy(p, plan, dtype, D, st);
+}
+
 }  // namespace sdllm

@@ -20,14 +20,14 @@ struct AttnPlan {
   int key_tile;     // keys per pipeline stage
   int m_warps;      // warps along the query rows (16 rows each, bf16) / row chunks (32 rows each, fp32)
   int c_warps;      // warps along the keys of a tile (bf16 only)
-  int warp_keys;    // keys per warp per tile (bf16 TMA kernel: 16, 32 or 64)
+  int warp_keys;    // keys per warp per tile (cp.async bf16 kernel)
   int stages;       // shared-memory pipeline depth
-  int cluster;      // CTAs of one (sequence, KV head) that merge through distributed shared memory
+  int cluster;      // > 1: the key splits of a unit form a thread-block cluster and merge through distributed shared memory
   int splits;       // partials per (sequence, KV head) left in the workspace (1 = final output written directly)
   int threads;
-  bool tma;         // bf16 TMA kernel (else the cp.async kernels)
+  bool tma;         // the kernel is fed by TMA (tcgen05 kernel), else by cp.async
   size_t smem_bytes;
-  int kind;         // 0: cp.async kernels, 1: TMA + mma.sync kernel, 2: TMA + tcgen05 kernel
+  int kind;         // 0: cp.async kernels (fp32 FMA / bf16 mma.sync), 2: TMA + tcgen05 kernel
   int key_tile2;    // tcgen05 kernel: keys per tile of source 2
   int rep;          // tcgen05 kernel: replicas of the query rows along the 128 accumulator rows
   int row_tiles;    // tcgen05 kernel: 128-row tiles of the b*G rows

@@ -111,11 +111,13 @@ def test_pool_windows(window):
 
 @pytest.mark.parametrize("env", [
     {"SDLLM_KERNEL": "cpasync"},                          # cp.async + mma.sync kernels, separate merge launch
-    {"SDLLM_KERNEL": "tma", "SDLLM_SPLITS": "3"},         # TMA + mma.sync kernel
+    {"SDLLM_KERNEL": "cpasync", "SDLLM_SPLITS": "3"},
     {"SDLLM_PDL": "0"},                                   # no programmatic dependent launch
     {"SDLLM_SPLITS": "7"}, {"SDLLM_SPLITS": "1"},         # other key-split counts of the tcgen05 kernel
     {"SDLLM_SPLITS": "5", "SDLLM_FUSED_TAIL": "0"},       # split merge and pooling in the second launch
     {"SDLLM_EARLY_LOADS": "0"},                           # no loads ahead of the grid dependency
+    {"SDLLM_CLUSTER": "0", "SDLLM_SPLITS": "4"},          # key splits merged by the last CTA instead of a cluster
+    {"SDLLM_SPLITS": "4"},                                # ... and by a cluster of four
     {"SDLLM_KEY_TILE": "64", "SDLLM_SPLITS": "2"},        # 64-key tiles
 ])
 def test_alternative_launch_plans_agree_with_oracle(env, monkeypatch):
