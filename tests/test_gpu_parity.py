@@ -94,6 +94,40 @@ def test_retention_extremes(r):
         np.testing.assert_allclose(out, g.out, rtol=0, atol=1e-5)
 
 
+@pytest.mark.parametrize("r", [0.0, 1.0, 0.03])
+def test_retention_extremes_bf16(r):
+    """Nothing kept (the reuse step attends over the block alone), everything kept, and a handful kept, on the tcgen05 path."""
+    cfg = _small("rext16", "bf16", 4, 2, 128, 230, 96, retention=r, salient_frac=0.02)
+    stats = _run_sequence_case(cfg, seed=16, block=1)
+    assert stats["set_mismatch"] == 0 or r not in (0.0, 1.0)
+
+
+@pytest.mark.parametrize("cfg,block", [
+    (_small("gqa8_two_full_row_tiles", "bf16", 16, 2, 128, 200, 64, retention=0.4, salient_frac=0.02), 1),   # b*G = 256
+    (_small("blk128", "bf16", 2, 2, 128, 150, 256, block_len=128, salient_frac=0.02), 1),                    # b = 128
+    (_small("blk48_fallback", "bf16", 2, 2, 128, 150, 96, block_len=48, salient_frac=0.02), 1),              # not a multiple of 16
+    (_small("gqa2_two_replicas", "bf16", 4, 2, 128, 333, 64, salient_frac=0.02), 0),                         # b*G = 64
+    (_small("one_tile", "bf16", 4, 4, 128, 40, 64, salient_frac=0.05), 0),                                   # shorter than one key tile
+])
+def test_more_shapes(cfg, block):
+    _run_sequence_case(cfg, seed=17, block=block)
+
+
+def test_batch_with_an_empty_cache_and_a_full_one():
+    """Ragged batch in which one sequence is nothing but its block (no candidates at all) beside ordinary ones."""
+    import parity_util as U
+    cfg = _small("rag0", "bf16", 4, 4, 128, 64, 32, salient_frac=0.02)
+    bw = W.make_batch(cfg, [0, 300, 37], seed=18, block=0)
+    q, k, v = bw.refresh_inputs(1, pad_value=np.nan)
+    g = U.gpu_refresh(q, k, v, bw.seq_len, bw.block_off, "bf16", 0.5, 3)
+    k0, v0 = np.nan_to_num(k), np.nan_to_num(v)
+    U.check_refresh_against_oracle(g, q, k0, v0, bw.seq_len, bw.block_off, "bf16", 0.5, 3)
+    assert int(g.kept_cnt[0]) == 0
+    q2, kn, vn = bw.sparse_inputs(2)
+    out = U.gpu_sparse_step(g, q2, kn, vn, "bf16")
+    U.check_sparse_against_oracle(g, out, q2, kn, vn, "bf16")
+
+
 @pytest.mark.parametrize("policy", [
     dict(select=B.SELECT_PER_REGION_CEIL), dict(select=B.SELECT_PREFIX_ONLY), dict(pool=B.POOL_AVG),
 ])
