@@ -386,11 +386,17 @@ __device__ __forceinline__ void trace_all(int32_t* status, int slot, bool is_min
 
 // PROB selects the second pass of the probability saliency; it is a template parameter so that the attention kernel proper
 // does not carry that pass's code.
-template <int D, bool PROB>
-__global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __grid_constant__ UmmaMaps tm, const UmmaParams up) {
+// DUAL is the small-footprint variant for grids of several waves: 64-key tiles, a two-slot ring, 256 TMEM columns and at
+// most 128 registers per thread, so that two CTAs share an SM and one's set-up and way out overlap the other's streaming.
+template <int D, bool PROB, bool DUAL>
+__global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kernel(const __grid_constant__ UmmaMaps tm, const UmmaParams up) {
   constexpr int H = D / 64;            // 128-byte column halves of a row
-  constexpr int NS = UM_STAGES;
-  constexpr uint32_t O_COL = 256;      // TMEM columns: S/P buffers at 0 and 128, the O accumulator at 256
+  constexpr int NS = DUAL ? 2 : UM_STAGES;
+  constexpr int NCH = DUAL ? 2 : 4;    // 32-column chunks of a key tile
+  constexpr uint32_t S_STRIDE = DUAL ? 64 : 128;   // TMEM columns: the two S/P buffers, then the O accumulator
+  constexpr uint32_t O_COL = 2 * S_STRIDE;
+  constexpr uint32_t TMEM_COLS = DUAL ? 256 : 512;
+  constexpr int CTRL = DUAL ? 4096 : 1024;         // control block: barriers, flags, qbar (and the merge scratch if DUAL)
   const AttnParams& p = up.a;
   extern __shared__ unsigned char smem_raw[];
 
@@ -424,7 +430,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 260);
   int* last_flag = reinterpret_cast<int*>(smem + 264);
   float* qbar_s = reinterpret_cast<float*>(smem + 512);
-  unsigned char* q_s = smem + 1024;
+  unsigned char* q_s = smem + CTRL;
   unsigned char* stage0 = q_s + H * 128 * 128;
   const int half_bytes = KT * 128;                     // one 64-column half of a K or V tile
   const int kv_bytes = H * half_bytes;                 // a whole K (or V) tile
@@ -517,7 +523,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   if (zero_q)
     for (int i = tid; i < H * 128 * 128 / 16; i += UM_THREADS) reinterpret_cast<uint4*>(q_s)[i] = make_uint4(0u, 0u, 0u, 0u);
   if (warp == 1) {                     // the MMA warp owns the tensor memory
-    tmem_alloc(smem_u32(tmem_slot), 512);
+    tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
     tmem_relinquish();
   }
   fence_proxy_async();
@@ -568,7 +574,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         if (j == 0) TRACE(9);
         tc_fence_after();
         const uint32_t vsm = smem_u32(stage0 + (size_t)s * stage_bytes) + kv_bytes;
-        const uint32_t a_t = tmem_base + (uint32_t)pb * 128u;
+        const uint32_t a_t = tmem_base + (uint32_t)pb * S_STRIDE;
         for (int ks = 0; ks < x.n_mma / 16; ++ks)
           mma_ts(tmem_base + O_COL, a_t + ks * 8, smem_desc(vsm + ks * 2048, (uint32_t)half_bytes, 1024u), idesc_pv,
                  (j > 0 || ks > 0) ? 1u : 0u);
@@ -592,7 +598,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         const uint32_t ksm = smem_u32(stage0 + (size_t)s * stage_bytes);
         const uint32_t qsm = smem_u32(q_s);
         const uint32_t idesc_s = instr_desc(x.n_mma, false);
-        const uint32_t d_t = tmem_base + (uint32_t)sb * 128u;
+        const uint32_t d_t = tmem_base + (uint32_t)sb * S_STRIDE;
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const uint32_t hq = (ks >> 2) * (128 * 128) + (ks & 3) * 32;
@@ -649,7 +655,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
           float v[32];
           if (c * 32 < c_hi && c * 32 + 32 > c_lo) {
             uint32_t sv[32];
-            tmem_ld32(lane_addr + (uint32_t)sb * 128u + c * 32, sv);
+            tmem_ld32(lane_addr + (uint32_t)sb * S_STRIDE + c * 32, sv);
             tc_wait_ld();
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
@@ -693,27 +699,29 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         const Tile x = tile_of(t, tiles1, KT, KT2, n1, n2);
         if (x.nv == 0) continue;
         const int s = it % NS, sb = it & 1;
-        // columns of this tile owned by this replica
-        const int c_lo = min(rep * chunk_keys, x.nv), c_hi = min((rep + 1) * chunk_keys, x.nv);
+        // columns of this tile owned by this replica; a warp whose 32 accumulator rows all lie beyond the valid rows of
+        // its replica owns nothing
+        const bool idle = q4 * 32 - rep * rows_rep >= M_rt;
+        const int c_lo = idle ? x.nv : min(rep * chunk_keys, x.nv), c_hi = min((rep + 1) * chunk_keys, x.nv);
         if (!wait_bar_warp(BAR(S_FULL + sb), (it >> 1) & 1, abort_flag, p.status, 9)) { ok = false; break; }
-        if (tid == 64) TRACE(it == 0 ? 10 : (it == 1 ? 16 : 18));
+        if (tid == 64 && it == 0) TRACE(10);
         tc_fence_after();
-        const uint32_t s_addr = lane_addr + (uint32_t)sb * 128u;
+        const uint32_t s_addr = lane_addr + (uint32_t)sb * S_STRIDE;
         // ---- the owned part of the S row. Chunks of 32 columns that are owned and valid as a whole go through the
         //      unrolled register path, all their loads in flight together; the one chunk the end of the slice may cut
         //      (cp) takes a small predicated path of its own, so the common code stays short ----
         const int cf_lo = c_lo >> 5, cf_hi = c_hi >> 5;          // full chunks [cf_lo, cf_hi); c_lo is a multiple of 32
         const int cp = (c_hi & 31) && c_lo < c_hi ? cf_hi : -1;  // partial chunk, if any
-        uint32_t sv[4][32];
+        uint32_t sv[NCH][32];
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < NCH; ++c)
           if (c >= cf_lo && c < cf_hi) tmem_ld32(s_addr + c * 32, sv[c]);
         uint32_t tv[32];
         if (cp >= 0) tmem_ld32(s_addr + cp * 32, tv);
         tc_wait_ld();
         float mx = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < NCH; ++c)
           if (c >= cf_lo && c < cf_hi) {
             float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -753,7 +761,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         // ---- P = exp2(S * scale_log2 - mu) as bf16 over the S columns; zero outside the owned slice ----
         float psum = 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < NCH; ++c)
           if (c >= cf_lo && c < cf_hi) {
             uint32_t pk[16];
             float ps4[4] = {0.f, 0.f, 0.f, 0.f};
@@ -800,11 +808,10 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
           fence_proxy_async();
         }
         tc_wait_st();
-        if (tid == 64 && it == 1) TRACE(26);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(BAR(P_FULL + sb));
-        if (tid == 64) TRACE(it == 0 ? 11 : (it == 1 ? 17 : 19));
+        if (tid == 64 && it == 0) TRACE(11);
         ++it;
       }
       if (tid == 64) TRACE(12);
@@ -824,11 +831,13 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
         qbar_s[d] = acc / (float)p.M;
       }
       asm volatile("bar.sync 1, 64;\n" ::: "memory");
-      float qb[D];                                       // the whole mean query in registers
+      float qb[DUAL ? 8 : D];                            // the whole mean query in registers (DUAL: read per use)
+      if constexpr (!DUAL) {
 #pragma unroll
-      for (int d = 0; d < D; d += 4) {
-        const float4 v4 = *reinterpret_cast<const float4*>(qbar_s + d);
-        qb[d] = v4.x; qb[d + 1] = v4.y; qb[d + 2] = v4.z; qb[d + 3] = v4.w;
+        for (int d = 0; d < D; d += 4) {
+          const float4 v4 = *reinterpret_cast<const float4*>(qbar_s + d);
+          qb[d] = v4.x; qb[d + 1] = v4.y; qb[d + 2] = v4.z; qb[d + 3] = v4.w;
+        }
       }
       int it = 0;
       for (int t = t_begin; t < t_end; ++t) {
@@ -844,21 +853,25 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
 #pragma unroll
             for (int c = 0; c < H * 8; ++c) {
               const uint4 raw = *reinterpret_cast<const uint4*>(kst + (c >> 3) * half_bytes + kk * 128 + (((c & 7) ^ (kk & 7)) << 4));
-              a0 = fmaf(qb[c * 8 + 0], __uint_as_float(raw.x << 16), a0);
-              a1 = fmaf(qb[c * 8 + 1], __uint_as_float(raw.x & 0xffff0000u), a1);
-              a2 = fmaf(qb[c * 8 + 2], __uint_as_float(raw.y << 16), a2);
-              a3 = fmaf(qb[c * 8 + 3], __uint_as_float(raw.y & 0xffff0000u), a3);
-              a0 = fmaf(qb[c * 8 + 4], __uint_as_float(raw.z << 16), a0);
-              a1 = fmaf(qb[c * 8 + 5], __uint_as_float(raw.z & 0xffff0000u), a1);
-              a2 = fmaf(qb[c * 8 + 6], __uint_as_float(raw.w << 16), a2);
-              a3 = fmaf(qb[c * 8 + 7], __uint_as_float(raw.w & 0xffff0000u), a3);
+              if constexpr (DUAL) {
+                const float4 qa = *reinterpret_cast<const float4*>(qbar_s + c * 8), qc = *reinterpret_cast<const float4*>(qbar_s + c * 8 + 4);
+                qb[0] = qa.x; qb[1] = qa.y; qb[2] = qa.z; qb[3] = qa.w; qb[4] = qc.x; qb[5] = qc.y; qb[6] = qc.z; qb[7] = qc.w;
+              }
+              constexpr int QO = DUAL ? 0 : 1;       // qb index = QO * c * 8 + j
+              a0 = fmaf(qb[QO * c * 8 + 0], __uint_as_float(raw.x << 16), a0);
+              a1 = fmaf(qb[QO * c * 8 + 1], __uint_as_float(raw.x & 0xffff0000u), a1);
+              a2 = fmaf(qb[QO * c * 8 + 2], __uint_as_float(raw.y << 16), a2);
+              a3 = fmaf(qb[QO * c * 8 + 3], __uint_as_float(raw.y & 0xffff0000u), a3);
+              a0 = fmaf(qb[QO * c * 8 + 4], __uint_as_float(raw.z << 16), a0);
+              a1 = fmaf(qb[QO * c * 8 + 5], __uint_as_float(raw.z & 0xffff0000u), a1);
+              a2 = fmaf(qb[QO * c * 8 + 6], __uint_as_float(raw.w << 16), a2);
+              a3 = fmaf(qb[QO * c * 8 + 7], __uint_as_float(raw.w & 0xffff0000u), a3);
             }
             p.raw_scores[(int64_t)(bi * p.Hkv + g) * p.n1_max + x.row0 + kk] = ((a0 + a1) + (a2 + a3)) * p.scale;
           }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(BAR(EMPTY_K + s));
-        if (tid == 192) TRACE(it == 0 ? 20 : (it == 1 ? 21 : 22));
         ++it;
       }
       // the softmax warps reuse the ring as scratch once they are done: tell them the K tiles are no longer read
@@ -878,7 +891,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     const int row = q4 * 32 + lane;
     const int rep = row / rows_rep, m_local = row - rep * rows_rep;
     float* o_s = reinterpret_cast<float*>(stage0);
-    float2* ml_s = reinterpret_cast<float2*>(stage0 + 128 * D * 4);
+    float2* ml_s = reinterpret_cast<float2*>(DUAL ? smem + 1024 : stage0 + 128 * D * 4);   // DUAL: the ring is all o_s
     float2* lm_s = ml_s + 128;
     if (do_scores) asm volatile("bar.sync 3, 192;\n" ::: "memory");      // the saliency warps have left the ring
     ml_s[row] = make_float2(m_run, l_run);
@@ -922,7 +935,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
     // and walks down the rows, four rows per step with all their shared-memory reads in flight together
     constexpr int D4 = D / 4;
     const float* o_s = reinterpret_cast<const float*>(stage0);
-    const float2* lm_s = reinterpret_cast<const float2*>(stage0 + 128 * D * 4) + 128;
+    const float2* lm_s = reinterpret_cast<const float2*>(DUAL ? smem + 1024 : stage0 + 128 * D * 4) + 128;
     __syncthreads();
     if (tid == 64) TRACE(29);
     const int st = tid;
@@ -1084,7 +1097,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_bf16_kernel(const __g
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
+    tmem_dealloc(tmem_base, TMEM_COLS);
   }
   if (tid == 0) { TRACE(15); TRACE_MAX(26); TRACE_MAX(16 + (int)blockIdx.x); }
 }
@@ -1121,16 +1134,17 @@ bool make_map(CUtensorMap* m, const void* base, int D, int rows, int heads, int 
              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-size_t umma_smem_bytes(int D, int KT) {
+size_t umma_smem_bytes(int D, int KT, bool dual) {
   const size_t H = D / 64;
+  if (dual) return 1024 /*alignment slack*/ + 4096 /*control block*/ + H * 128 * 128 + (size_t)2 * 2 * H * 64 * 128;
   const size_t need = 1024 /*alignment slack*/ + 1024 /*barriers, qbar*/ + H * 128 * 128 + (size_t)UM_STAGES * 2 * H * KT * 128;
   // every CTA allocates all 512 TMEM columns, so two CTAs must never share an SM: ask for more than half its shared memory
   return need > 120 * 1024 ? need : 120 * 1024;
 }
 
-template <int D, bool PROB>
+template <int D, bool PROB, bool DUAL>
 cudaError_t launch_umma_d(const UmmaMaps& tm, const UmmaParams& up, const AttnPlan& pl, cudaStream_t st) {
-  auto kern = attn_umma_bf16_kernel<D, PROB>;
+  auto kern = attn_umma_bf16_kernel<D, PROB, DUAL>;
   static size_t configured = 0;
   if (pl.smem_bytes > configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
@@ -1187,6 +1201,11 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
   pl.row_tiles = M <= 128 ? 1 : (G + 128 / b - 1) / (128 / b);
   pl.rep = M <= 32 ? 4 : (M <= 64 ? 2 : 1);
   const long long units = (long long)B * Hkv * pl.row_tiles;
+  // Several waves of CTAs: the small-footprint variant puts two of them on an SM, so that one's set-up and way out
+  // overlap the other's streaming. It works on 64-key tiles, which leaves room for two replicas of the rows at most.
+  pl.dual = units >= 2 * kNumSMs;
+  if (const char* e = getenv("SDLLM_DUAL")) pl.dual = e[0] == '1';      // tuning and test aid
+  if (pl.dual && pl.rep > 2) pl.rep = 2;
   long long want = kNumSMs / units;
   if (want < 1) want = 1;
   if (const char* e = getenv("SDLLM_SPLITS")) { if (atoi(e) >= 1) want = atoi(e); }   // tuning aid
@@ -1197,6 +1216,7 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
     if (atoi(e) == 64 && pl.rep <= 2) pl.key_tile = 64;
     if (atoi(e) == 128) pl.key_tile = 128;
   }
+  if (pl.dual) { pl.key_tile = 64; pl.stages = 2; }
   pl.key_tile2 = kt2 > 0 ? (kt2 < pl.key_tile ? kt2 : pl.key_tile) : pl.key_tile;
   const int tiles = (n1_max + pl.key_tile - 1) / pl.key_tile + (n2 > 0 ? (n2 + pl.key_tile2 - 1) / pl.key_tile2 : 0);
   if (want > tiles) want = tiles;
@@ -1207,7 +1227,7 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
   pl.rows_rep = 128 / pl.rep;
   pl.part_rows = pl.splits > 1 ? (size_t)pl.row_tiles * pl.splits * (M < 128 ? M : 128) : 0;
   pl.n_counters = (size_t)B * Hkv * pl.row_tiles;
-  pl.smem_bytes = umma_smem_bytes(D, pl.key_tile);
+  pl.smem_bytes = umma_smem_bytes(D, pl.key_tile, pl.dual);
   // Few key splits of a small problem: make them one thread-block cluster, so that they merge through distributed shared
   // memory instead of the workspace. Only where the whole grid is one wave (a cluster needs all its SMs at once).
   {
@@ -1254,8 +1274,13 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
   }
   if (!ok) return cudaErrorInvalidValue;
   cudaError_t err;
-  if (up.prob_pass) err = D == 128 ? launch_umma_d<128, true>(tm, up, pl, st) : launch_umma_d<64, true>(tm, up, pl, st);
-  else err = D == 128 ? launch_umma_d<128, false>(tm, up, pl, st) : launch_umma_d<64, false>(tm, up, pl, st);
+  if (pl.dual) {
+    if (up.prob_pass) err = D == 128 ? launch_umma_d<128, true, true>(tm, up, pl, st) : launch_umma_d<64, true, true>(tm, up, pl, st);
+    else err = D == 128 ? launch_umma_d<128, false, true>(tm, up, pl, st) : launch_umma_d<64, false, true>(tm, up, pl, st);
+  } else {
+    if (up.prob_pass) err = D == 128 ? launch_umma_d<128, true, false>(tm, up, pl, st) : launch_umma_d<64, true, false>(tm, up, pl, st);
+    else err = D == 128 ? launch_umma_d<128, false, false>(tm, up, pl, st) : launch_umma_d<64, false, false>(tm, up, pl, st);
+  }
   if (err != cudaSuccess || up.fused_tail) return err;
   const bool merge = p.out != nullptr && !p.prob_pass && pl.splits > 1;
   const bool pool_tail = pool || (p.prob_pass && p.pooled != nullptr);

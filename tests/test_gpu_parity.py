@@ -152,6 +152,8 @@ def test_pool_windows(window):
     {"SDLLM_EARLY_LOADS": "0"},                           # no loads ahead of the grid dependency
     {"SDLLM_CLUSTER": "0", "SDLLM_SPLITS": "4"},          # key splits merged by the last CTA instead of a cluster
     {"SDLLM_SPLITS": "4"},                                # ... and by a cluster of four
+    {"SDLLM_DUAL": "1", "SDLLM_SPLITS": "1"},             # small-footprint variant (two CTAs per SM)
+    {"SDLLM_DUAL": "1", "SDLLM_SPLITS": "3"},
     {"SDLLM_KEY_TILE": "64", "SDLLM_SPLITS": "2"},        # 64-key tiles
 ])
 def test_alternative_launch_plans_agree_with_oracle(env, monkeypatch):
@@ -169,7 +171,7 @@ def test_alternative_launch_plans_agree_with_oracle(env, monkeypatch):
     (_small("prob_gqa7", "bf16", 14, 2, 128, 300, 96, retention=0.25, salient_frac=0.01, sink_tokens=4), 2),   # two row tiles
     (_small("prob_d64", "bf16", 4, 2, 64, 150, 64, salient_frac=0.02), 1),
 ])
-@pytest.mark.parametrize("env", [{}, {"SDLLM_SPLITS": "3", "SDLLM_FUSED_TAIL": "0"}, {"SDLLM_SPLITS": "1"}])
+@pytest.mark.parametrize("env", [{}, {"SDLLM_SPLITS": "3", "SDLLM_FUSED_TAIL": "0"}, {"SDLLM_SPLITS": "1"}, {"SDLLM_DUAL": "1"}])
 def test_softmax_probability_saliency(cfg, block, env, monkeypatch):
     """The second reading of "attention scores": mean softmax probability per key (two passes over K)."""
     for k, v in env.items():
