@@ -1203,7 +1203,7 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
   const long long units = (long long)B * Hkv * pl.row_tiles;
   // Several waves of CTAs: the small-footprint variant puts two of them on an SM, so that one's set-up and way out
   // overlap the other's streaming. It works on 64-key tiles, which leaves room for two replicas of the rows at most.
-  pl.dual = units >= 2 * kNumSMs;
+  pl.dual = units >= 2 * kNumSMs && n2 > 0;          // measured: pays for the reuse step, not for the refresh step
   if (const char* e = getenv("SDLLM_DUAL")) pl.dual = e[0] == '1';      // tuning and test aid
   if (pl.dual && pl.rep > 2) pl.rep = 2;
   long long want = kNumSMs / units;
