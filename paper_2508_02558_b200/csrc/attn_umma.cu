@@ -435,8 +435,13 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
   const int half_bytes = KT * 128;                     // one 64-column half of a K or V tile
   const int kv_bytes = H * half_bytes;                 // a whole K (or V) tile
   const int stage_bytes = 2 * kv_bytes;
-  // Q rows that no TMA box covers must not hold non-finite garbage; only shapes with b*G below the replica's rows need it
-  const bool zero_q = do_s && p.b * up.heads_rt < rows_rep;
+  // The Q box (b rows x the row tile's heads) is loaded as many times as it fits into the 128 accumulator rows: every
+  // replica starts on a copy, and rows past the valid ones hold real data whose results are simply not used. Only a box
+  // that does not divide 128 leaves rows uncovered; those must not hold non-finite garbage and are cleared first.
+  const int q_rows = p.b * up.heads_rt;
+  const int q_copies = (128 % q_rows == 0) ? 128 / q_rows : R;
+  const int q_step = (128 % q_rows == 0) ? q_rows : rows_rep;
+  const bool zero_q = do_s && 128 % q_rows != 0 && q_rows < rows_rep;
   if (tid == 0) {                        // the descriptors live in the kernel parameters: fetch them while the CTA sets up
     prefetch_tmap(&tm.k1); prefetch_tmap(&tm.v1);
     if (n2 > 0) { prefetch_tmap(&tm.k2); prefetch_tmap(&tm.v2); }
@@ -451,10 +456,10 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
   auto issue_q = [&]() {              // the Q tile (replicated R times along the accumulator rows)
     q_issued = true;
     if (!do_s) return;
-    mbar_expect_tx(BAR(Q_FULL), (uint32_t)(R * H * p.b * up.heads_rt * 128));
-    for (int rep = 0; rep < R; ++rep)
+    mbar_expect_tx(BAR(Q_FULL), (uint32_t)(q_copies * H * q_rows * 128));
+    for (int c = 0; c < q_copies; ++c)
       for (int h = 0; h < H; ++h)
-        tma_load_4d(smem_u32(q_s + h * 128 * 128 + rep * rows_rep * 128), &tm.q, BAR(Q_FULL), h * 64, 0,
+        tma_load_4d(smem_u32(q_s + h * 128 * 128 + c * q_step * 128), &tm.q, BAR(Q_FULL), h * 64, 0,
                     g * p.G + rt * up.heads_rt, bi);
   };
   // issue loads for up to `limit` further tiles (producer lane only); with src1_only, stop in front of source 2
