@@ -52,6 +52,7 @@ struct UmmaParams {
   int early_src1;    // 1: source 1 and its count are older than the previous kernel in the stream (reuse step)
   int prob_pass;     // 1: second pass of the probability saliency: S and the rows' log-sum-exp give column means of P
   int cluster;       // > 1: the key splits of a unit form a thread-block cluster and merge through distributed shared memory
+  int lpt;           // 1: grid z counts the sequences from the longest to the shortest (several waves of ragged work)
 };
 
 // ---------------------------------------------------------------------------------------------------------
@@ -403,7 +404,24 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int KT = up.KT, KT2 = up.KT2, R = up.R;
   const int rows_rep = 128 / R;
-  const int bi = blockIdx.z;
+  // Which sequence: grid z itself, or, for ragged batches that take several waves, the sequence of that rank when the
+  // batch is ordered from the longest to the shortest - CTAs are handed out in grid order, so the long ones start first
+  // and the short ones fill the tail. Every warp ranks the (at most 64) lengths on its own: no shared memory, no barrier.
+  int bi = blockIdx.z;
+  if (up.lpt) {
+    if (!up.early_src1) grid_dependency_wait();        // the lengths may come from the kernel in front
+    const int lane_ = threadIdx.x & 31;
+    const int l0 = lane_ < p.B ? p.n1_per_seq[lane_] : -1, l1 = lane_ + 32 < p.B ? p.n1_per_seq[lane_ + 32] : -1;
+    int r0 = 0, r1 = 0;                                // how many sequences come before mine (longer, or equal and earlier)
+    for (int i = 0; i < p.B; ++i) {
+      const int li = __shfl_sync(0xffffffffu, i < 32 ? l0 : l1, i & 31);
+      r0 += (li > l0 || (li == l0 && i < lane_)) ? 1 : 0;
+      r1 += (li > l1 || (li == l1 && i < lane_ + 32)) ? 1 : 0;
+    }
+    const unsigned hit0 = __ballot_sync(0xffffffffu, lane_ < p.B && r0 == (int)blockIdx.z);
+    const unsigned hit1 = __ballot_sync(0xffffffffu, lane_ + 32 < p.B && r1 == (int)blockIdx.z);
+    bi = hit0 ? __ffs(hit0) - 1 : (hit1 ? __ffs(hit1) + 31 : (int)blockIdx.z);
+  }
   const int g = blockIdx.y / up.row_tiles, rt = blockIdx.y - g * up.row_tiles;
   const int split = blockIdx.x;
   if (tid == 0) { TRACE(1); TRACE_MAX(24); }
@@ -1261,6 +1279,12 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
   }
   up.prob_pass = p.prob_pass;
   up.cluster = pl.cluster;
+  {
+    const char* e = getenv("SDLLM_LPT");               // SDLLM_LPT=0/1 forces the ordering off/on (tuning and test aid)
+    const long long ctas = (long long)pl.splits * p.Hkv * pl.row_tiles * p.B;
+    up.lpt = (p.n1_per_seq != nullptr && p.B >= 4 && p.B <= 64 && ctas > kNumSMs) ? 1 : 0;
+    if (e) up.lpt = (e[0] == '1' && p.n1_per_seq != nullptr && p.B >= 2 && p.B <= 64) ? 1 : 0;
+  }
   if (up.cluster > 1) up.fused_tail = 1;     // set again below; the cluster tail never needs the second launch
   up.fused_tail = (pl.cluster > 1 || umma_tail_is_fused(pl, D, p.M, p.n1_max, pool || p.prob_pass, p.out != nullptr && !p.prob_pass)) ? 1 : 0;
   memset(&tm, 0, sizeof(tm));

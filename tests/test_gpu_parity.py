@@ -179,8 +179,11 @@ def test_softmax_probability_saliency(cfg, block, env, monkeypatch):
     _run_sequence_case(cfg, seed=15, block=block, n_sparse=1, score=B.SCORE_PROB_MEAN)
 
 
-def test_ragged_batch():
+@pytest.mark.parametrize("env", [{}, {"SDLLM_LPT": "1"}, {"SDLLM_LPT": "1", "SDLLM_DUAL": "1", "SDLLM_SPLITS": "1"}])
+def test_ragged_batch(env, monkeypatch):
     import parity_util as U
+    for k_, v_ in env.items():
+        monkeypatch.setenv(k_, v_)
     cfg = _small("rag", "bf16", 4, 4, 128, 64, 64, salient_frac=0.02)
     bw = W.make_batch(cfg, [40, 333, 64, 200], seed=7, block=1)
     q, k, v = bw.refresh_inputs(1, pad_value=np.nan)       # padding must never be read
