@@ -890,27 +890,21 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
               p.raw_scores[(int64_t)(bi * p.Hkv + g) * p.n1_max + x.row0 + kk] = ((a0 + a1) + (a2 + a3)) * p.scale;
             }
           } else {
-            // two keys per lane (rows kA and kA + 64 of the tile), interleaved so that their chains hide each other
-            const int kA = (warp - 6) * 32 + lane, kB = kA + 64;
-            if (kA < x.nv) {
-              const int kBc = min(kB, KT - 1);             // a row that exists; its result is dropped if kB >= nv
-              float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f, b0 = 0.f, b1 = 0.f, b2 = 0.f, b3 = 0.f;
+            for (int kk = (warp - 6) * 32 + lane; kk < x.nv; kk += 64) {
+              float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
               for (int c = 0; c < H * 8; ++c) {
-                const uint4 ra = *reinterpret_cast<const uint4*>(kst + (c >> 3) * half_bytes + kA * 128 + (((c & 7) ^ (kA & 7)) << 4));
-                const uint4 rb = *reinterpret_cast<const uint4*>(kst + (c >> 3) * half_bytes + kBc * 128 + (((c & 7) ^ (kBc & 7)) << 4));
-                a0 = fmaf(qb[c * 8 + 0], __uint_as_float(ra.x << 16), a0);          b0 = fmaf(qb[c * 8 + 0], __uint_as_float(rb.x << 16), b0);
-                a1 = fmaf(qb[c * 8 + 1], __uint_as_float(ra.x & 0xffff0000u), a1);  b1 = fmaf(qb[c * 8 + 1], __uint_as_float(rb.x & 0xffff0000u), b1);
-                a2 = fmaf(qb[c * 8 + 2], __uint_as_float(ra.y << 16), a2);          b2 = fmaf(qb[c * 8 + 2], __uint_as_float(rb.y << 16), b2);
-                a3 = fmaf(qb[c * 8 + 3], __uint_as_float(ra.y & 0xffff0000u), a3);  b3 = fmaf(qb[c * 8 + 3], __uint_as_float(rb.y & 0xffff0000u), b3);
-                a0 = fmaf(qb[c * 8 + 4], __uint_as_float(ra.z << 16), a0);          b0 = fmaf(qb[c * 8 + 4], __uint_as_float(rb.z << 16), b0);
-                a1 = fmaf(qb[c * 8 + 5], __uint_as_float(ra.z & 0xffff0000u), a1);  b1 = fmaf(qb[c * 8 + 5], __uint_as_float(rb.z & 0xffff0000u), b1);
-                a2 = fmaf(qb[c * 8 + 6], __uint_as_float(ra.w << 16), a2);          b2 = fmaf(qb[c * 8 + 6], __uint_as_float(rb.w << 16), b2);
-                a3 = fmaf(qb[c * 8 + 7], __uint_as_float(ra.w & 0xffff0000u), a3);  b3 = fmaf(qb[c * 8 + 7], __uint_as_float(rb.w & 0xffff0000u), b3);
+                const uint4 raw = *reinterpret_cast<const uint4*>(kst + (c >> 3) * half_bytes + kk * 128 + (((c & 7) ^ (kk & 7)) << 4));
+                a0 = fmaf(qb[c * 8 + 0], __uint_as_float(raw.x << 16), a0);
+                a1 = fmaf(qb[c * 8 + 1], __uint_as_float(raw.x & 0xffff0000u), a1);
+                a2 = fmaf(qb[c * 8 + 2], __uint_as_float(raw.y << 16), a2);
+                a3 = fmaf(qb[c * 8 + 3], __uint_as_float(raw.y & 0xffff0000u), a3);
+                a0 = fmaf(qb[c * 8 + 4], __uint_as_float(raw.z << 16), a0);
+                a1 = fmaf(qb[c * 8 + 5], __uint_as_float(raw.z & 0xffff0000u), a1);
+                a2 = fmaf(qb[c * 8 + 6], __uint_as_float(raw.w << 16), a2);
+                a3 = fmaf(qb[c * 8 + 7], __uint_as_float(raw.w & 0xffff0000u), a3);
               }
-              float* dst = p.raw_scores + (int64_t)(bi * p.Hkv + g) * p.n1_max + x.row0;
-              dst[kA] = ((a0 + a1) + (a2 + a3)) * p.scale;
-              if (kB < x.nv) dst[kB] = ((b0 + b1) + (b2 + b3)) * p.scale;
+              p.raw_scores[(int64_t)(bi * p.Hkv + g) * p.n1_max + x.row0 + kk] = ((a0 + a1) + (a2 + a3)) * p.scale;
             }
           }
         }
