@@ -1255,6 +1255,15 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
     if (atoi(e) == 128) pl.key_tile = 128;
   }
   if (pl.dual) { pl.key_tile = 64; pl.stages = 2; }
+  // A reuse step with few heads and a short cache: rather than many one-tile splits whose merge needs a second launch,
+  // take at most eight splits of 128-key tiles, which one cluster merges on chip.
+  const int tiles128 = (n1_max + 127) / 128 + (n2 > 0 ? 1 : 0);
+  const bool no_cluster = (getenv("SDLLM_CLUSTER") && getenv("SDLLM_CLUSTER")[0] == '0') ||
+                          (getenv("SDLLM_FUSED_TAIL") && getenv("SDLLM_FUSED_TAIL")[0] == '0');
+  if (!pl.dual && !no_cluster && !getenv("SDLLM_SPLITS") && !getenv("SDLLM_KEY_TILE") && n2 > 0 && want > 8 && tiles128 <= 16) {
+    pl.key_tile = 128;
+    want = tiles128 < 8 ? tiles128 : 8;
+  }
   pl.key_tile2 = kt2 > 0 ? (kt2 < pl.key_tile ? kt2 : pl.key_tile) : pl.key_tile;
   const int tiles = (n1_max + pl.key_tile - 1) / pl.key_tile + (n2 > 0 ? (n2 + pl.key_tile2 - 1) / pl.key_tile2 : 0);
   if (want > tiles) want = tiles;
@@ -1269,12 +1278,10 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
   // Few key splits of a small problem: make them one thread-block cluster, so that they merge through distributed shared
   // memory instead of the workspace. Only where the whole grid is one wave (a cluster needs all its SMs at once).
   {
-    const char* e = getenv("SDLLM_CLUSTER");           // SDLLM_CLUSTER=0: never (tuning and test aid)
-    const char* f = getenv("SDLLM_FUSED_TAIL");
-    const bool off = (e && e[0] == '0') || (f && f[0] == '0');
-    const size_t merge_bytes = (size_t)pl.splits * (M < 128 ? M : 128) * D * 4;
-    if (!off && pl.splits >= 2 && pl.splits <= 8 && pl.row_tiles == 1 && pl.key_tile == 128 && units * pl.splits <= kNumSMs &&
-        merge_bytes <= 256 * 1024 && n1_max <= 8192)
+    // SDLLM_CLUSTER=0 (or SDLLM_FUSED_TAIL=0): never (tuning and test aid). Several row tiles only at the reuse step:
+    // the probability pass of the refresh step pools over all row tiles of a head, which one cluster does not span.
+    if (!no_cluster && pl.splits >= 2 && pl.splits <= 8 && (pl.row_tiles == 1 || n2 > 0) && pl.key_tile == 128 &&
+        units * pl.splits <= kNumSMs && n1_max <= 8192)
       pl.cluster = pl.splits;
   }
   return pl;
