@@ -50,9 +50,9 @@ def test_static_scratch_variant_matches_the_workspace_variant_twice(Hq, Hkv, n_k
 
 
 def test_static_scratch_variant_refuses_shapes_beyond_its_scratch():
-    # a Dream-shaped layer: few KV heads, so many key splits, whose partials need more than the built-in 8 MiB
-    d = B.make_desc(batch=1, n_q_heads=28, n_kv_heads=4, head_dim=128, seq_len_max=4096, block_len=32, dtype=B.BF16,
-                    retention=0.25, n_keep_max=1016)
+    # a long-context GQA layer: few KV heads, so many key splits, whose partials need more than the built-in 8 MiB
+    d = B.make_desc(batch=1, n_q_heads=32, n_kv_heads=8, head_dim=128, seq_len_max=32768, block_len=32, dtype=B.BF16,
+                    retention=0.5, n_keep_max=16368)
     assert B.workspace_bytes(d, B.OP_SPARSE_BLOCK_ATTN) > (8 << 20)
     a = 0x1000      # never dereferenced: the size check comes first
     with pytest.raises(B.SdllmError) as e:
