@@ -35,7 +35,7 @@ METRIC = "cached_kv_tokens_per_s_per_layer"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the sparse-attention kernel pair on this workload,
 # from the ncu capture summarised under profiles/ (None until a capture exists for the workload).
-NCU_TRAFFIC_BYTES = {"c2_llada": 11114496}
+NCU_TRAFFIC_BYTES = {"c2_llada": 11117056}
 
 
 def parse_args():
@@ -325,7 +325,7 @@ def run_ours(args):
     rf_sec = timed(rf_runner, max(3, args.steps // 2), 3) / max(3, args.steps // 2) / n_layers
     peak, peak_kind = peaks()
     achieved = ab["sparse"] / sp_sec / 1e9
-    roofline = {"bound": "hbm", "kernel": "sdllm_sparse_block_attn (attn_umma_bf16_kernel<128, false>: tcgen05 attention, key splits merged through cluster shared memory)", "achieved": achieved,
+    roofline = {"bound": "hbm", "kernel": "sdllm_sparse_block_attn (attn_umma_bf16_kernel<128, false, false>: tcgen05 attention, key splits merged through cluster shared memory)", "achieved": achieved,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                 "frac_of_8TBps": achieved / 8000.0, "algorithmic_bytes_per_launch": ab["sparse"], "us_per_launch": sp_sec * 1e6,
                 "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
