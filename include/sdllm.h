@@ -66,7 +66,8 @@ typedef enum {
   SDLLM_OP_REFRESH_SCORES = 0,
   SDLLM_OP_SELECT_TOPK = 1,
   SDLLM_OP_COMPACT_KV = 2,
-  SDLLM_OP_SPARSE_BLOCK_ATTN = 3
+  SDLLM_OP_SPARSE_BLOCK_ATTN = 3,
+  SDLLM_OP_DENSE_ATTN = 4
 } sdllm_op;
 
 /* Problem description, filled by the caller. Plain data; set struct_size = sizeof(sdllm_desc). */
@@ -164,6 +165,21 @@ sdllm_status sdllm_compact_kv(const sdllm_desc* desc, const void* k, const void*
 sdllm_status sdllm_sparse_block_attn(const sdllm_desc* desc, const void* q_blk, const void* k_c, const void* v_c,
                                      const int32_t* kept_cnt, const void* k_blk, const void* v_blk, void* out,
                                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Dense step (cache_state 0, and the full-sequence part of cache_state 1; Algorithm 3, "all L rows"): bidirectional
+ * attention of every row of a sequence over all of its keys,
+ *   out[i, h, t, :] = softmax_u(scale * q[i, h, t, :] . k[i, h / G, u, :]) v[i, h / G, u, :],   t, u < seq_len[i].
+ *   q   [B, Hq, seq_len_max, D], strides q_stride[3] = (batch, head, row) in ELEMENTS, rows of D contiguous elements
+ *   k,v [B, Hkv, seq_len_max, D] with desc->kv_stride
+ *   out [B, Hq, seq_len_max, D] with o_stride[3]; rows t >= seq_len[i] are not written
+ *   lse [B, Hq, seq_len_max] fp32, nullable: log-sum-exp of the scaled logits per written row
+ * seq_len NULL means every sequence has seq_len_max rows. desc->block_len, retention and the selection fields are
+ * not used. bf16 only, D in {64, 128}, n_kv_heads * G * ceil(seq_len_max / 128) <= 65535; anything else returns
+ * SDLLM_ERR_UNSUPPORTED. The probability matrix is never written to memory. Workspace:
+ * sdllm_workspace_bytes(desc, SDLLM_OP_DENSE_ATTN), zeroed once by the caller like the other attention workspaces. */
+sdllm_status sdllm_dense_attn(const sdllm_desc* desc, const void* q, const int64_t* q_stride, const void* k, const void* v,
+                              const int32_t* seq_len, void* out, const int64_t* o_stride, float* lse, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream);
 
 /* The reuse step for callers that cannot allocate device memory. The paper has no counterpart for this call: it
  * computes exactly what sdllm_sparse_block_attn computes, but takes no workspace. Some hosts of this library run under

@@ -196,6 +196,16 @@ def sparse_block_attention(q, k_c, v_c, k_n, v_n, scale: Optional[float] = None)
     return attention(q, k, v, scale)
 
 
+def dense_attention(q, k, v, scale: Optional[float] = None, rows: Optional[Sequence[int]] = None):
+    """Dense step (Algorithm 3, cache_state 0 and the full-sequence part of cache_state 1): every row of the sequence
+    attends to all L keys, no mask. q [Hq,L,D], k/v [Hkv,L,D] -> out [Hq,L,D], lse [Hq,L]. The rows are independent,
+    so `rows` (query positions) restricts the work to a sample of them: out [Hq,len(rows),D]."""
+    q = _f64(q)
+    if rows is not None:
+        q = np.ascontiguousarray(q[:, np.asarray(list(rows), dtype=np.int64)])
+    return attention(q, k, v, scale)
+
+
 def positions_to_candidates(kept_idx: np.ndarray, block_len: int, block_off: int) -> np.ndarray:
     """Inverse of the candidate position map for kept absolute positions."""
     kept_idx = np.asarray(kept_idx)

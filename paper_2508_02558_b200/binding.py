@@ -18,12 +18,12 @@ F32, BF16 = 0, 1
 SCORE_LOGIT_MEAN, SCORE_PROB_MEAN = 0, 1
 POOL_MAX, POOL_AVG = 0, 1
 SELECT_JOINT_FLOOR, SELECT_PER_REGION_CEIL, SELECT_PREFIX_ONLY = 0, 1, 2
-OP_REFRESH_SCORES, OP_SELECT_TOPK, OP_COMPACT_KV, OP_SPARSE_BLOCK_ATTN = range(4)
+OP_REFRESH_SCORES, OP_SELECT_TOPK, OP_COMPACT_KV, OP_SPARSE_BLOCK_ATTN, OP_DENSE_ATTN = range(5)
 
 EXPORTS = ("sdllm_version", "sdllm_status_string", "sdllm_workspace_bytes", "sdllm_keep_count", "sdllm_cache_state", "sdllm_launch_count",
            "sdllm_read_status",
            "sdllm_refresh_scores", "sdllm_select_topk", "sdllm_compact_kv", "sdllm_sparse_block_attn",
-           "sdllm_sparse_block_attn_static")
+           "sdllm_sparse_block_attn_static", "sdllm_dense_attn")
 
 
 class Desc(ctypes.Structure):
@@ -80,6 +80,9 @@ def lib() -> ctypes.CDLL:
         L.sdllm_compact_kv.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp]
         L.sdllm_sparse_block_attn.restype = ctypes.c_int
         L.sdllm_sparse_block_attn.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.sdllm_dense_attn.restype = ctypes.c_int
+        L.sdllm_dense_attn.argtypes = [dp, vp, ctypes.POINTER(ctypes.c_int64), vp, vp, i32p, vp, ctypes.POINTER(ctypes.c_int64), vp, vp,
+                                       ctypes.c_size_t, vp]
         _lib = L
     return _lib
 
@@ -205,3 +208,11 @@ def sparse_block_attn_static(desc: Desc, q_blk, k_c, v_c, kept_cnt, k_blk, v_blk
     _check(lib().sdllm_sparse_block_attn_static(ctypes.byref(desc), _ptr(q_blk), _ptr(k_c), _ptr(v_c), _ptr(kept_cnt),
                                                 _ptr(k_blk), _ptr(v_blk), _ptr(out), _stream(stream)),
            "sdllm_sparse_block_attn_static")
+
+
+def dense_attn(desc: Desc, q, k, v, seq_len, out, lse, workspace, stream=None):
+    """Full-sequence bidirectional attention; q and out are [B, Hq, seq_len_max, D] tensors whose strides are passed on."""
+    qs = (ctypes.c_int64 * 3)(*q.stride()[:3])
+    os_ = (ctypes.c_int64 * 3)(*out.stride()[:3])
+    _check(lib().sdllm_dense_attn(ctypes.byref(desc), _ptr(q), qs, _ptr(k), _ptr(v), _ptr(seq_len), _ptr(out), os_, _ptr(lse),
+                                  _ptr(workspace), _nbytes(workspace), _stream(stream)), "sdllm_dense_attn")

@@ -37,6 +37,8 @@ struct AttnPlan {
   bool dual;        // tcgen05 kernel, small-footprint variant: two CTAs per SM
   size_t part_rows; // partial rows per (sequence, KV head) in the workspace (0: none)
   size_t n_counters;// completion counters in the workspace
+  int nqb;          // full-sequence attention (tcgen05 kernel): 128-row query blocks per head, one row tile each; else 0
+  int lq_max;       // full-sequence attention: query rows per head in the tensors
 };
 
 // Key sources of one attention launch. The virtual key axis is [src1 rows 0..n1) ++ [src2 rows 0..n2).
@@ -100,6 +102,7 @@ AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_m
 
 bool umma_tail_is_fused(const AttnPlan& pl, int D, int M, int n1_max, bool pool, bool merge);
 bool umma_supported(int dtype, int D, int M, int b);
+AttnPlan plan_attention_dense(int D, int G, int B, int Hkv, int L);
 cudaError_t launch_attn_partial(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st);
 cudaError_t launch_merge_pool(const MergeParams& p, cudaStream_t st);
 cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st);

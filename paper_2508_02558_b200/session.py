@@ -1,6 +1,6 @@
 """Device-memory plumbing around the C ABI: one object per (layer, batch shape) that owns the
 compacted cache, the index/score buffers and the workspace (all torch CUDA tensors) and issues the
-four libsdllm calls in the order of the paper's Algorithm 3. It allocates and passes pointers; every
+libsdllm calls in the order of the paper's Algorithm 3. It allocates and passes pointers; every
 arithmetic step runs inside libsdllm.
 """
 from __future__ import annotations
@@ -48,7 +48,7 @@ class LayerCache:
             self.pooled, self.workspace = share_scratch_with.pooled, share_scratch_with.workspace
         else:
             self.pooled = torch.empty((batch, n_kv_heads, seq_len_max), dtype=torch.float32, device=dev)
-            ws = max(B.workspace_bytes(self.desc, op) for op in range(4))
+            ws = max(B.workspace_bytes(self.desc, op) for op in range(5))
             self.workspace = torch.zeros((max(ws, 256),), dtype=torch.uint8, device=dev)   # status word starts at 0
 
     # cache_state 1: dense block attention + Algorithm 1
@@ -63,4 +63,10 @@ class LayerCache:
     # cache_state 2: attention over Concat(K_c, K_n)
     def sparse_step(self, q_blk, k_blk, v_blk, out, stream=None):
         B.sparse_block_attn(self.desc, q_blk, self.k_c, self.v_c, self.kept_cnt, k_blk, v_blk, out, self.workspace, stream)
+        return out
+
+    # cache_state 0 (and the full-sequence part of cache_state 1): every row over all keys
+    def dense_step(self, q, k, v, seq_len, out, lse=None, stream=None):
+        """q/out [B,Hq,Lmax,D], k/v [B,Hkv,Lmax,D]; bf16 only."""
+        B.dense_attn(self.desc, q, k, v, seq_len, out, lse, self.workspace, stream)
         return out

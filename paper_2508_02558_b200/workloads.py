@@ -151,6 +151,17 @@ class SequenceWorkload:
         return round_to_dtype(q, c.dtype), round_to_dtype(kb, c.dtype), round_to_dtype(vb, c.dtype)
 
 
+    def dense_inputs(self, step: int = 0) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+        """(Q, K, V) of a dense step: query rows for all L positions (the block's rows are that step's Q_b), and the
+        K, V of `refresh_inputs(step)`."""
+        c = self.cfg
+        qb, k, v = self.refresh_inputs(step)
+        inv = np.float32(1.0 / np.sqrt(c.head_dim))
+        q = self._rng(step, 6).standard_normal((c.n_q_heads, c.seq_len, c.head_dim), dtype=np.float32) * inv
+        q[:, self.block_off:self.block_off + c.block_len] = qb
+        return round_to_dtype(q, c.dtype), k, v
+
+
 def _mix(*vals: int) -> int:
     """Small integer hash so (seed, layer, block) give unrelated Philox keys."""
     h = 0x9E3779B97F4A7C15

@@ -177,3 +177,43 @@ def check_sparse_against_oracle(g: GpuRefresh, out_gpu, q2, kn, vn, dtype, heads
         ref, _ = oracle.sparse_block_attention(qh, kc, vc, kn[i, hs], vn[i, hs])
         for j, h in enumerate(hs):
             assert_close(out_gpu[i, h * G:(h + 1) * G], ref[j * G:(j + 1) * G], dtype, f"sparse out seq {i} head {h}")
+
+
+def gpu_dense(q, k, v, seq_len: Optional[Sequence[int]], dtype: str = "bf16", want_lse: bool = True):
+    """Dense step through the C ABI. q [B,Hq,Lmax,D], k/v [B,Hkv,Lmax,D] float32 host arrays -> (out, lse) with NaN
+    wherever the call did not write."""
+    Bn, Hq, Lmax, D = q.shape
+    Hkv = k.shape[1]
+    d = B.make_desc(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, seq_len_max=Lmax, block_len=min(32, Lmax),
+                    dtype=B.BF16 if dtype == "bf16" else B.F32)
+    qd, kd, vd = to_dev(q, dtype), to_dev(k, dtype), to_dev(v, dtype)
+    sl = None if seq_len is None else torch.tensor(list(seq_len), dtype=torch.int32, device=DEV)
+    out = torch.full((Bn, Hq, Lmax, D), float("nan"), dtype=qd.dtype, device=DEV)
+    lse = torch.full((Bn, Hq, Lmax), float("nan"), dtype=torch.float32, device=DEV) if want_lse else None
+    ws = torch.zeros((max(B.workspace_bytes(d, B.OP_DENSE_ATTN), 256),), dtype=torch.uint8, device=DEV)
+    torch.cuda.synchronize()
+    for _ in range(2):               # the second call runs on the counters the first one left behind
+        B.dense_attn(d, qd, kd, vd, sl, out, lse, ws)
+    torch.cuda.synchronize()
+    assert B.read_status(ws) == 0, "a bounded device-side wait expired"
+    return to_host_f32(out), (lse.cpu().numpy() if want_lse else None)
+
+
+def check_dense_against_oracle(out, lse, q, k, v, seq_len: Optional[Sequence[int]], rows=None, heads=None):
+    """Element by element on the rows t < seq_len[i] (all of them, or the sample `rows`); rows past the length must
+    not have been written."""
+    Bn, Hq, Lmax, D = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    for i in range(Bn):
+        L = Lmax if seq_len is None else int(seq_len[i])
+        assert np.isnan(out[i, :, L:]).all(), f"dense out seq {i}: rows past the length were written"
+        if L == 0:
+            continue
+        rs = list(range(L)) if rows is None else [t for t in rows if t < L]
+        for g in (range(Hkv) if heads is None else heads):
+            ref, ref_lse = oracle.dense_attention(q[i, g * G:(g + 1) * G, :L], k[i, g:g + 1, :L], v[i, g:g + 1, :L], rows=rs)
+            assert_close(out[i, g * G:(g + 1) * G][:, rs], ref, "bf16", f"dense out seq {i} kv head {g}")
+            if lse is not None:
+                np.testing.assert_allclose(lse[i, g * G:(g + 1) * G][:, rs], ref_lse, atol=1e-4, rtol=0,
+                                           err_msg=f"dense lse seq {i} kv head {g}")

@@ -264,3 +264,57 @@ def test_scores_only_and_attention_only_calls():
     torch.cuda.synchronize()
     assert torch.equal(pooled2, torch.from_numpy(g.pooled).cuda())
     np.testing.assert_array_equal(U.to_host_f32(out2), g.out)
+
+
+# ------------------------------------------------------------------ dense step (all rows over all keys)
+def _dense_case(Hq, Hkv, D, lens, seed, pad=np.nan):
+    """Padded batch of full-sequence inputs: q [B,Hq,Lmax,D], k/v [B,Hkv,Lmax,D]; the padding must never matter."""
+    Lmax = max(max(lens), 1)
+    q = np.full((len(lens), Hq, Lmax, D), pad, np.float32)
+    k = np.full((len(lens), Hkv, Lmax, D), pad, np.float32)
+    v = np.full((len(lens), Hkv, Lmax, D), pad, np.float32)
+    for i, L in enumerate(lens):
+        if L == 0:
+            continue
+        cfg = _small("dense", "bf16", Hq, Hkv, D, L - 16, 16, block_len=16, salient_frac=0.02)
+        s = W.make_sequence(cfg, seed=seed + i)
+        q[i, :, :L], k[i, :, :L], v[i, :, :L] = s.dense_inputs(0)
+    return q, k, v
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,lens", [
+    (2, 2, 128, [333]),                 # several query blocks and key tiles with ragged tails, key splits merged
+    (8, 2, 64, [200]),                  # grouped heads, D = 64
+    (4, 1, 128, [128]),                 # exactly one tile each way
+    (2, 1, 128, [17]),                  # shorter than a tile
+    (4, 2, 128, [300, 40, 0, 257]),     # ragged batch with an empty sequence
+])
+def test_dense_step(Hq, Hkv, D, lens):
+    import parity_util as U
+    q, k, v = _dense_case(Hq, Hkv, D, lens, seed=21)
+    out, lse = U.gpu_dense(q, k, v, lens)
+    U.check_dense_against_oracle(out, lse, np.nan_to_num(q), np.nan_to_num(k), np.nan_to_num(v), lens)
+
+
+@pytest.mark.parametrize("env", [{"SDLLM_FUSED_TAIL": "0"}, {"SDLLM_SPLITS": "1"}, {"SDLLM_SPLITS": "3", "SDLLM_KEY_TILE": "64"}])
+def test_dense_step_launch_plans(env, monkeypatch):
+    import parity_util as U
+    for k_, v_ in env.items():
+        monkeypatch.setenv(k_, v_)
+    q, k, v = _dense_case(4, 2, 128, [300, 129], seed=22)
+    out, lse = U.gpu_dense(q, k, v, [300, 129])
+    U.check_dense_against_oracle(out, lse, np.nan_to_num(q), np.nan_to_num(k), np.nan_to_num(v), [300, 129])
+
+
+def test_dense_step_without_lengths_and_refusals():
+    import parity_util as U
+    q, k, v = _dense_case(2, 2, 64, [256], seed=23)
+    out, _ = U.gpu_dense(q, k, v, None, want_lse=False)
+    U.check_dense_against_oracle(out, None, q, k, v, None)
+    d = B.make_desc(batch=1, n_q_heads=2, n_kv_heads=2, head_dim=64, seq_len_max=256, block_len=32, dtype=B.F32)
+    assert B.workspace_bytes(d, B.OP_DENSE_ATTN) == 0
+    t = torch.zeros((1, 2, 256, 64), device="cuda:0")
+    ws = torch.zeros((4096,), dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(B.SdllmError) as e:
+        B.dense_attn(d, t, t, t, None, t, None, ws)
+    assert e.value.status == B.ERR_UNSUPPORTED

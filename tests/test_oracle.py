@@ -274,6 +274,37 @@ def test_full_retention_reproduces_dense_attention():
     np.testing.assert_allclose(lse, r.lse, atol=1e-13)
 
 
+def test_dense_step_brute_force_closed_form_and_row_sampling():
+    """The dense step (all L rows over all L keys, Algorithm 3) against loops written out, a closed form and the
+    block rows of the refresh step."""
+    rng = np.random.default_rng(11)
+    Hq, Hkv, L, D = 4, 2, 7, 3
+    q, k, v = rng.standard_normal((Hq, L, D)), rng.standard_normal((Hkv, L, D)), rng.standard_normal((Hkv, L, D))
+    out, lse = oracle.dense_attention(q, k, v, scale=0.7)
+    for h in range(Hq):
+        g = h // (Hq // Hkv)                       # query heads of a group share one KV head
+        for t in range(L):
+            w = [np.exp(0.7 * sum(q[h, t, d] * k[g, u, d] for d in range(D))) for u in range(L)]
+            z = sum(w)
+            for d in range(D):
+                assert abs(out[h, t, d] - sum(w[u] * v[g, u, d] for u in range(L)) / z) < 1e-12
+            assert abs(lse[h, t] - np.log(z)) < 1e-12
+    # no mask of any kind: with zero queries every row is the plain mean of V over the whole sequence
+    out0, lse0 = oracle.dense_attention(np.zeros_like(q), k, v)
+    np.testing.assert_allclose(out0, np.repeat(v.mean(axis=1), Hq // Hkv, axis=0)[:, None, :].repeat(L, axis=1), atol=1e-13)
+    np.testing.assert_allclose(lse0, np.log(L), atol=1e-13)
+    # a sample of rows gives those rows; the block's rows are what the refresh step computes for the block
+    cfg = W.CONFIGS["c1_tiny"]
+    s = W.make_sequence(cfg, seed=5)
+    qf, kf, vf = s.dense_inputs(1)
+    full, _ = oracle.dense_attention(qf, kf, vf)
+    some, _ = oracle.dense_attention(qf, kf, vf, rows=[0, 5, cfg.seq_len - 1])
+    np.testing.assert_array_equal(some, full[:, [0, 5, cfg.seq_len - 1]])
+    qb, kb, vb = s.refresh_inputs(1)
+    blk, _ = oracle.attention(qb, kb, vb)
+    np.testing.assert_allclose(full[:, s.block_off:s.block_off + cfg.block_len], blk, atol=1e-13)
+
+
 def test_sparse_attention_equals_dense_over_kept_subset():
     cfg = W.CONFIGS["c1_tiny"]
     s = W.make_sequence(cfg, seed=5)
