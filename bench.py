@@ -5,7 +5,7 @@ A "step" is one decoding block of the workload's attention stack: for every laye
 (dense block attention + saliency + pooling, top-k, K/V compaction) followed by the block's
 cache-reuse steps (sparse block attention over [K_c ; K_n]), issued in model order (step-major,
 layer-minor), so consecutive calls touch different layers' K/V and caches. The dense step 0 of each
-block (cache_state 0) is not part of this path and is not timed. "Cached-KV tokens" of a call are the
+block (cache_state 0) is not part of this path; `--phase dense` times it on its own, with its own metric. "Cached-KV tokens" of a call are the
 key/value positions it consumes: L for a refresh, n + b for a reuse step.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2_llada] [--impl ours|reference]
@@ -46,8 +46,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_llada", choices=["c2_llada", "c3_dream", "c4_long", "c5_serving"])
     ap.add_argument("--batch", type=int, default=1, help="sequences per call (c5_serving: ragged prompt lengths)")
-    ap.add_argument("--phase", default="all", choices=["all", "refresh", "sparse"],
-                    help="profiling aid: run only the refresh chain or only the reuse steps in the timed step")
+    ap.add_argument("--phase", default="all", choices=["all", "refresh", "sparse", "dense"],
+                    help="profiling aid: run only the refresh chain or only the reuse steps in the timed step; "
+                         "dense: time the full-sequence dense step (cache_state 0) of every layer instead, on its own metric")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (0 = the workload's)")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-e2e", action="store_true")
@@ -60,6 +61,15 @@ def peaks():
     if os.path.exists(path):
         return float(json.load(open(path))["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def tensor_peaks():
+    """(burst, sustained) dense bf16 TFLOP/s of a library GEMM on this machine."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        m = json.load(open(path))
+        return float(m["bf16_tflops"]), float(m.get("bf16_tflops_sustained", m["bf16_tflops"])), "measured"
+    return 1590.0, 1400.0, "fallback"
 
 
 # ------------------------------------------------------------------------------------------------ workload
@@ -302,6 +312,42 @@ def run_ours(args):
             if world > 1:
                 dist.barrier()
         return e0.elapsed_time(e1) / 1e3
+
+    if args.phase == "dense":
+        # ---- the dense step on its own: every row of every sequence over all of its keys, layer after layer
+        nq = min(n_layers, max(1, int(4e9 // (2 * Bn * Hq * L * D * 2))))        # distinct Q / output sets (a few GB)
+        inv = 1.0 / np.sqrt(D)
+        Qf = [(torch.randn((Bn, Hq, L, D), device=dev, generator=gen) * inv).to(tdt) for _ in range(nq)]
+        Of = [torch.empty((Bn, Hq, L, D), dtype=tdt, device=dev) for _ in range(nq)]
+        torch.cuda.synchronize(dev)
+
+        def dense_only():
+            for l in range(n_layers):
+                caches[l].dense_step(Qf[l % nq], Ks[l], Vs[l], seq_len_t, Of[l % nq], stream=stream)
+        sampler = ClockSampler(local) if rank == 0 else None
+        sec = slowest_rank_seconds(timed(make_runner(dense_only), args.steps, max(args.warmup, 3)), dev)
+        clocks = sampler.stop() if sampler else None
+        flops = 4.0 * sum(float(x) * x for x in seq_lens) * Hq * D * n_layers
+        burst, sustained, kind = tensor_peaks()
+        tflops = world * flops * args.steps / sec / 1e12
+        per_gpu = tflops / world
+        if rank == 0:
+            print(json.dumps({
+                "metric": "dense_step_query_tokens_per_s_per_layer", "value": whole_job_value(sum(seq_lens) * n_layers * args.steps, world, sec),
+                "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": 1e3 * sec / args.steps,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+                "config": {"workload": cfg.name, "batch": Bn, "phase": "dense", "layers": n_layers, "seq_len": L, "n_q_heads": Hq,
+                           "n_kv_heads": Hkv, "head_dim": D, "step": "the dense step (all rows x all keys) of %d layers" % n_layers,
+                           "launch": "eager" if args.no_graph else "cuda_graph_replay", "parallelism": "replicas" if world > 1 else "1gpu"},
+                "roofline": {"bound": "tensor", "kernel": "sdllm_dense_attn (attn_umma_bf16_kernel, one row tile per query head and 128-row block)",
+                             "achieved": per_gpu, "peak": sustained, "peak_kind": kind + ", sustained library GEMM", "unit": "TFLOP/s",
+                             "frac": per_gpu / sustained, "frac_of_burst": per_gpu / burst, "flops_per_step": flops,
+                             "us_per_launch": 1e6 * sec / args.steps / n_layers, "traffic": None},
+                "clocks": clocks, "gpu_launches": n_layers * B.launch_count(caches[0].desc, B.OP_DENSE_ATTN) * args.steps,
+            }))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     with torch.cuda.stream(stream):
         refresh_only()                              # every layer's cache exists before any reuse step runs

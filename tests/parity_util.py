@@ -185,7 +185,7 @@ def gpu_dense(q, k, v, seq_len: Optional[Sequence[int]], dtype: str = "bf16", wa
     Bn, Hq, Lmax, D = q.shape
     Hkv = k.shape[1]
     d = B.make_desc(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, seq_len_max=Lmax, block_len=min(32, Lmax),
-                    dtype=B.BF16 if dtype == "bf16" else B.F32)
+                    dtype=B.BF16 if dtype == "bf16" else B.F32, retention=0.5)
     qd, kd, vd = to_dev(q, dtype), to_dev(k, dtype), to_dev(v, dtype)
     sl = None if seq_len is None else torch.tensor(list(seq_len), dtype=torch.int32, device=DEV)
     out = torch.full((Bn, Hq, Lmax, D), float("nan"), dtype=qd.dtype, device=DEV)

@@ -89,3 +89,31 @@ def test_c5_serving_ragged_batch_full_size(batch):
     out = U.gpu_sparse_step(g, q2, kn, vn, "bf16")
     U.check_sparse_against_oracle(g, out, q2, kn, vn, "bf16", heads=[7, 30], seqs=seqs)
     assert np.isfinite(out).all()
+
+
+@pytest.mark.parametrize("name,heads", [("c2_llada", [0, 17]), ("c3_dream", [3]), ("c4_long", [5])])
+def test_dense_step_full_size(name, heads):
+    """All L rows over all L keys at the workload's size; the oracle recomputes a sample of rows of a sample of heads."""
+    import parity_util as U
+    cfg = W.CONFIGS[name]
+    s = W.make_sequence(cfg, seed=31)
+    q, k, v = s.dense_inputs(0)
+    L = s.seq_len
+    out, lse = U.gpu_dense(q[None], k[None], v[None], [L])
+    rows = sorted({0, 1, 127, 128, L // 2 + 3, s.block_off, s.block_off + cfg.block_len - 1, L - 129, L - 1})
+    U.check_dense_against_oracle(out, lse, q[None], k[None], v[None], [L], rows=rows, heads=heads)
+    assert np.isfinite(out).all() and np.isfinite(lse).all()
+
+
+def test_dense_step_ragged_serving_batch_full_size():
+    import parity_util as U
+    cfg = W.CONFIGS["c5_serving"]
+    lens = W.serving_prompt_lengths(4, seed=5)
+    bw = W.make_batch(cfg, lens, seed=25)
+    Lm = bw.seq_len_max
+    q = np.zeros((4, cfg.n_q_heads, Lm, cfg.head_dim), np.float32)
+    k, v = np.zeros((4, cfg.n_kv_heads, Lm, cfg.head_dim), np.float32), np.zeros((4, cfg.n_kv_heads, Lm, cfg.head_dim), np.float32)
+    for i, s in enumerate(bw.seqs):
+        q[i, :, :s.seq_len], k[i, :, :s.seq_len], v[i, :, :s.seq_len] = s.dense_inputs(0)
+    out, lse = U.gpu_dense(q, k, v, bw.seq_len)
+    U.check_dense_against_oracle(out, lse, q, k, v, bw.seq_len, rows=[0, 130, 700, 2049, 4000], heads=[9])

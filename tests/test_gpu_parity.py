@@ -311,7 +311,7 @@ def test_dense_step_without_lengths_and_refusals():
     q, k, v = _dense_case(2, 2, 64, [256], seed=23)
     out, _ = U.gpu_dense(q, k, v, None, want_lse=False)
     U.check_dense_against_oracle(out, None, q, k, v, None)
-    d = B.make_desc(batch=1, n_q_heads=2, n_kv_heads=2, head_dim=64, seq_len_max=256, block_len=32, dtype=B.F32)
+    d = B.make_desc(batch=1, n_q_heads=2, n_kv_heads=2, head_dim=64, seq_len_max=256, block_len=32, dtype=B.F32, retention=0.5)
     assert B.workspace_bytes(d, B.OP_DENSE_ATTN) == 0
     t = torch.zeros((1, 2, 256, 64), device="cuda:0")
     ws = torch.zeros((4096,), dtype=torch.uint8, device="cuda:0")
