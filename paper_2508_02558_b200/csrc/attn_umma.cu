@@ -280,6 +280,16 @@ __device__ __forceinline__ int rows_of_tile(const UmmaParams& up, int rt, int n_
   return min(up.a.M - rt * 128, 128);
 }
 
+// Keys of source 1 that a CTA of sequence bi works on. Full-sequence mode: a query block past the end of its sequence
+// has no rows, so it takes no keys either.
+__device__ __forceinline__ int keys_of_seq(const UmmaParams& up, int bi, int rt) {
+  const AttnParams& p = up.a;
+  int n = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
+  n = min(max(n, 0), p.n1_max);
+  if (up.nqb > 0 && (rt % up.nqb) * 128 >= n) n = 0;
+  return n;
+}
+
 // Merge of the key-split partials of S (row, float4 column) slots of a unit and the final stores. slot[s] < 0 marks
 // an unused entry. The partials are read in batches of MB per slot with the loads of all slots and of the whole batch
 // in flight together (one L2 latency per batch) and folded with a running maximum, so that four splits cost a single
@@ -555,14 +565,12 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
       if (up.early_src1) {
         // Reuse step: the compacted cache and its count were written before the previous kernel in the stream even
         // started, so their tiles may stream in while that kernel is still finishing.
-        prod_n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
-        prod_n1 = min(max(prod_n1, 0), p.n1_max);
+        prod_n1 = keys_of_seq(up, bi, rt);
         produce(NS, true);             // the first NS slots are free: no waiting here
       }
       grid_dependency_wait();          // the loads below read what earlier kernels in the stream wrote
       if (!up.early_src1) {
-        prod_n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
-        prod_n1 = min(max(prod_n1, 0), p.n1_max);
+        prod_n1 = keys_of_seq(up, bi, rt);
       }
       TRACE(4);
       issue_q();
@@ -586,8 +594,7 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
   grid_dependency_wait();              // everything below may read what earlier kernels in the stream wrote
   grid_launch_dependents();
 
-  int n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
-  n1 = min(max(n1, 0), p.n1_max);
+  const int n1 = keys_of_seq(up, bi, rt);
   M_rt = rows_of_tile(up, rt, n1);     // full-sequence mode: the sequence has as many query rows as keys
 
   // softmax state of this thread's accumulator row (softmax warps only)
