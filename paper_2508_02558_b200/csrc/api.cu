@@ -188,6 +188,7 @@ int32_t sdllm_launch_count(const sdllm_desc* d, int op) {
   if (op == SDLLM_OP_COMPACT_KV) return d->n_keep_max > 0 ? 1 : 0;
   if (op == SDLLM_OP_DENSE_ATTN) {
     if (!dense_supported(d)) return -1;
+    if (dense_pair_kernel_wanted(d->batch, d->n_q_heads, d->seq_len_max)) return 1;
     const AttnPlan pl = dense_plan(d);
     return 1 + ((pl.splits > 1 && !umma_tail_is_fused(pl, d->head_dim, 128, d->seq_len_max, false, true)) ? 1 : 0);
   }
@@ -365,6 +366,13 @@ sdllm_status sdllm_dense_attn(const sdllm_desc* d, const void* q, const int64_t*
   if (w.total > 0 && (ws == nullptr || ws_bytes < w.total || (reinterpret_cast<uintptr_t>(ws) & 255u))) return SDLLM_ERR_WORKSPACE;
   if ((st = check_device()) != SDLLM_OK) return st;
   char* wsb = reinterpret_cast<char*>(ws);
+  if (dense_pair_kernel_wanted(d->batch, d->n_q_heads, d->seq_len_max)) {
+    if (cuda_failed(launch_dense_pair(q, q_stride, k, v, d->kv_stride, seq_len, out, o_stride, lse, reinterpret_cast<int32_t*>(wsb + w.status),
+                                      d->batch, d->n_q_heads, d->n_kv_heads, d->seq_len_max, d->head_dim, scale_of(d),
+                                      reinterpret_cast<cudaStream_t>(cuda_stream)), "dense attention launch"))
+      return SDLLM_ERR_CUDA;
+    return SDLLM_OK;
+  }
 
   AttnParams p{};
   fill_common(p, d, pl);

@@ -103,6 +103,11 @@ AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_m
 bool umma_tail_is_fused(const AttnPlan& pl, int D, int M, int n1_max, bool pool, bool merge);
 bool umma_supported(int dtype, int D, int M, int b);
 AttnPlan plan_attention_dense(int D, int G, int B, int Hkv, int L);
+// Full-sequence attention, two query tiles per CTA (attn_dense.cu): whether it is the kernel of choice, and its launch.
+bool dense_pair_kernel_wanted(int B, int Hq, int L);
+cudaError_t launch_dense_pair(const void* q, const int64_t* q_stride, const void* k, const void* v, const int64_t* kv_stride,
+                              const int32_t* seq_len, void* out, const int64_t* o_stride, float* lse, int32_t* status, int B, int Hq,
+                              int Hkv, int L, int D, float scale, cudaStream_t st);
 cudaError_t launch_attn_partial(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st);
 cudaError_t launch_merge_pool(const MergeParams& p, cudaStream_t st);
 cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st);

@@ -289,8 +289,11 @@ def _dense_case(Hq, Hkv, D, lens, seed, pad=np.nan):
     (2, 1, 128, [17]),                  # shorter than a tile
     (4, 2, 128, [300, 40, 0, 257]),     # ragged batch with an empty sequence
 ])
-def test_dense_step(Hq, Hkv, D, lens):
+@pytest.mark.parametrize("kernel", ["tile", "pair"])
+def test_dense_step(Hq, Hkv, D, lens, kernel, monkeypatch):
+    """Both kernels of the dense step: the block kernel's full-sequence mode and the two-query-tile kernel."""
     import parity_util as U
+    monkeypatch.setenv("SDLLM_DENSE", kernel)
     q, k, v = _dense_case(Hq, Hkv, D, lens, seed=21)
     out, lse = U.gpu_dense(q, k, v, lens)
     U.check_dense_against_oracle(out, lse, np.nan_to_num(q), np.nan_to_num(k), np.nan_to_num(v), lens)
@@ -299,6 +302,7 @@ def test_dense_step(Hq, Hkv, D, lens):
 @pytest.mark.parametrize("env", [{"SDLLM_FUSED_TAIL": "0"}, {"SDLLM_SPLITS": "1"}, {"SDLLM_SPLITS": "3", "SDLLM_KEY_TILE": "64"}])
 def test_dense_step_launch_plans(env, monkeypatch):
     import parity_util as U
+    monkeypatch.setenv("SDLLM_DENSE", "tile")
     for k_, v_ in env.items():
         monkeypatch.setenv(k_, v_)
     q, k, v = _dense_case(4, 2, 128, [300, 129], seed=22)
@@ -318,3 +322,12 @@ def test_dense_step_without_lengths_and_refusals():
     with pytest.raises(B.SdllmError) as e:
         B.dense_attn(d, t, t, t, None, t, None, ws)
     assert e.value.status == B.ERR_UNSUPPORTED
+
+
+def test_dense_step_two_tile_kernel_many_key_tiles():
+    """Enough key tiles for every barrier phase and ring slot to wrap several times; odd number of query blocks."""
+    import parity_util as U
+    q, k, v = _dense_case(8, 2, 128, [1100, 640], seed=24)
+    out, lse = U.gpu_dense(q, k, v, [1100, 640])
+    U.check_dense_against_oracle(out, lse, np.nan_to_num(q), np.nan_to_num(k), np.nan_to_num(v), [1100, 640],
+                                 rows=[0, 127, 128, 300, 639, 640, 1023, 1024, 1099])
