@@ -5,10 +5,9 @@
 //   warp 0      TMA producer: the two Q tiles, then K and V tiles (128 keys, 128-byte swizzle) into a two-slot ring
 //   warp 1      one thread issues tcgen05.mma. Per key tile j:  S0 = Q0 K_j^T,  O1 += P1(j-1) V_(j-1),  S1 = Q1 K_j^T,
 //               O0 += P0(j) V_j  -  while the softmax warps of one query tile work, the tensor pipe serves the other
-//   warps 4-7   softmax of query tile 0, warps 8-11 of query tile 1: a thread owns one accumulator row (TMEM lane),
+//   warps 2-5   softmax of query tile 0, warps 6-9 of query tile 1: a thread owns one accumulator row (TMEM lane),
 //               reads its S row, keeps the running max / sum and writes P (bf16) over S in TMEM; O accumulates in
 //               TMEM and is rescaled in place only when the row's maximum grows by more than 2^8
-//   warps 2-3   idle: they fill the first warpgroup, which gives most of its registers to the softmax warpgroups
 // Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 columns each (D = 64 uses half of an O region).
 // The finished rows go from TMEM through registers straight to global memory (bf16), normalised by the row sum.
 // Every wait on an mbarrier is bounded; on expiry the CTA sets an abort flag, records a code in the status word and
@@ -24,7 +23,7 @@ namespace sdllm {
 using namespace dev;
 namespace {
 
-constexpr int DN_THREADS = 384;
+constexpr int DN_THREADS = 320;
 constexpr int DN_STAGES = 2;
 
 struct DenseMaps {
@@ -103,11 +102,6 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
 
   auto tile_nv = [&](int j) { return min(n - j * KT, KT); };     // valid keys of tile j (> 0 for j < nt)
 
-  // Register budget by role: the first warpgroup (producer, MMA issuer, two idle warps) hands most of its registers
-  // to the two softmax warpgroups, whose threads each hold a whole 128-column S row.
-
-  if (warp < 4) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 56;\n");
   if (warp == 0) {
     // ======================================= TMA producer =======================================
     if (lane == 0) {
@@ -192,11 +186,9 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
         drain_bar(BAR(DRAIN), 0);
       }
     }
-  }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;\n");
     // ======================================= softmax warps =======================================
-    const int t = (warp - 4) >> 2;                     // query tile of this warp
+    const int t = (warp - 2) >> 2;                     // query tile of this warp
     const int q4 = warp & 3;                           // TMEM lane quadrant this warp may access
     const int row = q4 * 32 + lane;
     if (t == 0 || act1) {
@@ -209,90 +201,65 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
         const int nv = tile_nv(j);
         if (!wait_bar_warp(BAR(S_FULL + t), j & 1, abort_flag, p.status, 27)) { ok = false; break; }
         tc_fence_after();
-        // ---- one pass over the S row: P = exp2(S * scale_log2 - m_run) with the maximum the row had BEFORE this tile,
-        //      while the tile's own maximum is found on the side. The result stands unless the maximum grew by more than
-        //      2^8 (rare once a few tiles have passed); then O and l are rescaled and the pass runs again on the S row,
-        //      which is still intact in tensor memory because P is stored last. The first tile and a ragged last tile
-        //      find their maximum first. ----
-        const bool pre = (j == 0) || (nv < KT);          // warp-uniform
-        uint32_t pk[4][16];
-        float psum = 0.f, alpha = 1.f;
-        bool grow = false;
-#pragma unroll 1
-        for (int attempt = 0; attempt < 2; ++attempt) {
-          uint32_t sv[4][32];
+        uint32_t sv[4][32];
 #pragma unroll
-          for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sv[c]);
-          tc_wait_ld();
-          if (pre) {
-            if (nv < KT) {                               // the ragged last tile: keys past the end count as -inf
+        for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sv[c]);
+        tc_wait_ld();
+        if (nv < KT) {                                   // the ragged last tile: keys past the end count as -inf
 #pragma unroll
-              for (int c = 0; c < 4; ++c)
+          for (int c = 0; c < 4; ++c)
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                  if (c * 32 + i >= nv) sv[c][i] = __float_as_uint(-INFINITY);
-            }
-            float mx = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-              for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(sv[c][i]));
-              mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
-            }
-            const float m_new = fmaxf(m_run, mx * p.scale_log2);
-            grow = m_new > m_run + 8.f;                  // also true on the first finite maximum
-            if (grow) {
-              alpha = fast_exp2(m_run - m_new);          // 0 when m_run is -inf
-              m_run = m_new;
-              l_run *= alpha;
-            }
-          }
-          if (j > 0 && __any_sync(0xffffffffu, grow)) {
-            // the running maximum grew: every PV of this query tile issued so far must have landed before O is rewritten
-            if (!wait_bar_warp(BAR(PV_DONE + t), (j - 1) & 1, abort_flag, p.status, 28)) { ok = false; break; }
-            tc_fence_after();
-#pragma unroll 1
-            for (int c = 0; c < D / 16; ++c) {
-              uint32_t ov[16];
-              tmem_ld16(o_addr + c * 16, ov);
-              tc_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-              tmem_st16(o_addr + c * 16, ov);
-            }
-            tc_wait_st();
-          }
-          const float mu = (m_run == -INFINITY) ? 0.f : m_run;
-          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-          psum = 0.f;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            float ps4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float s0 = __uint_as_float(sv[c][2 * i]), s1 = __uint_as_float(sv[c][2 * i + 1]);
-              mx4[i & 3] = fmaxf(mx4[i & 3], fmaxf(s0, s1));
-              const float e0 = fast_exp2(fmaf(s0, p.scale_log2, -mu));
-              const float e1 = fast_exp2(fmaf(s1, p.scale_log2, -mu));
-              ps4[i & 3] += e0 + e1;
-              pk[c][i] = pack_bf16(e0, e1);
-            }
-            psum += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
-          }
-          const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2);
-          grow = m_new > m_run + 8.f;
-          alpha = 1.f;
-          if (grow) {
-            alpha = fast_exp2(m_run - m_new);
-            m_run = m_new;
-            l_run *= alpha;
-          }
-          if (!__any_sync(0xffffffffu, grow)) break;    // the usual case: P stands
+            for (int i = 0; i < 32; ++i)
+              if (c * 32 + i >= nv) sv[c][i] = __float_as_uint(-INFINITY);
         }
-        if (!ok) break;
+        float mx = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_st16(s_addr + c * 16, pk[c]);     // bf16 P over the first 64 columns of the S region
+        for (int c = 0; c < 4; ++c) {
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(sv[c][i]));
+          mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
+        }
+        // running maximum: O (in TMEM) and l are rescaled only when the maximum grows by more than 2^8
+        const float m_new = fmaxf(m_run, mx * p.scale_log2);
+        const bool grow = m_new > m_run + 8.f;          // also true on the first finite maximum
+        float alpha = 1.f;
+        if (grow) {
+          alpha = fast_exp2(m_run - m_new);             // 0 when m_run is -inf
+          m_run = m_new;
+          l_run *= alpha;
+        }
+        if (j > 0 && __any_sync(0xffffffffu, grow)) {
+          // every PV of this query tile issued so far must have landed before its rows are rewritten
+          if (!wait_bar_warp(BAR(PV_DONE + t), (j - 1) & 1, abort_flag, p.status, 28)) { ok = false; break; }
+          tc_fence_after();
+#pragma unroll 1
+          for (int c = 0; c < D / 16; ++c) {
+            uint32_t ov[16];
+            tmem_ld16(o_addr + c * 16, ov);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+            tmem_st16(o_addr + c * 16, ov);
+          }
+        }
+        const float mu = (m_run == -INFINITY) ? 0.f : m_run;
+        // P = exp2(S * scale_log2 - mu) as bf16 over the first 64 columns of the S region
+        float psum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t pk[16];
+          float ps4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float e0 = fast_exp2(fmaf(__uint_as_float(sv[c][2 * i]), p.scale_log2, -mu));
+            const float e1 = fast_exp2(fmaf(__uint_as_float(sv[c][2 * i + 1]), p.scale_log2, -mu));
+            ps4[i & 3] += e0 + e1;
+            pk[i] = pack_bf16(e0, e1);
+          }
+          psum += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
+          tmem_st16(s_addr + c * 16, pk);
+        }
         l_run += psum;
         // V rows past the sequence's end may hold anything: query tile 0 zeroes them so that 0 * V stays 0
         const int n_mma = (nv + 15) & ~15;
@@ -301,7 +268,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
           if (!wait_bar_warp(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 29)) { ok = false; break; }
           unsigned char* vs = stage0 + (size_t)s * 2 * TILE + TILE;
           const int nz = (n_mma - nv) * H * 8;           // 16-byte chunks to clear
-          for (int i = (warp - 4) * 32 + lane; i < nz; i += 128) {
+          for (int i = (warp - 2) * 32 + lane; i < nz; i += 128) {
             const int rr = nv + i / (H * 8), c = i % (H * 8);
             *reinterpret_cast<uint4*>(vs + (c >> 3) * HALF + rr * 128 + (((c & 7) ^ (rr & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
           }
