@@ -339,7 +339,7 @@ def run_ours(args):
                 "config": {"workload": cfg.name, "batch": Bn, "phase": "dense", "layers": n_layers, "seq_len": L, "n_q_heads": Hq,
                            "n_kv_heads": Hkv, "head_dim": D, "step": "the dense step (all rows x all keys) of %d layers" % n_layers,
                            "launch": "eager" if args.no_graph else "cuda_graph_replay", "parallelism": "replicas" if world > 1 else "1gpu"},
-                "roofline": {"bound": "tensor", "kernel": "sdllm_dense_attn (attn_umma_bf16_kernel, one row tile per query head and 128-row block)",
+                "roofline": {"bound": "tensor", "kernel": "sdllm_dense_attn (dense_attn_bf16_kernel: tcgen05, two 128-row query tiles per CTA share one pass over K/V)",
                              "achieved": per_gpu, "peak": sustained, "peak_kind": kind + ", sustained library GEMM", "unit": "TFLOP/s",
                              "frac": per_gpu / sustained, "frac_of_burst": per_gpu / burst, "flops_per_step": flops,
                              "us_per_launch": 1e6 * sec / args.steps / n_layers, "traffic": None},
