@@ -44,7 +44,10 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2_llada", choices=["c2_llada", "c3_dream", "c4_long", "c5_serving"])
+    ap.add_argument("--workload", default="c2_llada",
+                    choices=["c2_llada", "c3_dream", "c4_long", "c5_serving", "c6_gen512", "c7_long4k"])
+    ap.add_argument("--retention", type=float, default=None, help="override the workload's retention ratio r")
+    ap.add_argument("--pool-window", type=int, default=None, help="override the workload's pooling kernel size (odd)")
     ap.add_argument("--batch", type=int, default=1, help="sequences per call (c5_serving: ragged prompt lengths)")
     ap.add_argument("--phase", default="all", choices=["all", "refresh", "sparse", "dense"],
                     help="profiling aid: run only the refresh chain or only the reuse steps in the timed step; "
@@ -73,6 +76,17 @@ def tensor_peaks():
 
 
 # ------------------------------------------------------------------------------------------------ workload
+def workload_config(args) -> W.WorkloadConfig:
+    """The named workload, with the retention ratio and pooling kernel size overridden when asked (perf sweeps)."""
+    import dataclasses
+    cfg = W.CONFIGS[args.workload]
+    if args.retention is not None:
+        cfg = dataclasses.replace(cfg, retention=float(args.retention))
+    if args.pool_window is not None:
+        cfg = dataclasses.replace(cfg, pool_window=int(args.pool_window))
+    return cfg
+
+
 def tokens_per_step(cfg: W.WorkloadConfig, n_layers: int, seq_lens, n_keeps, phase: str = "all") -> int:
     reuse_steps = cfg.steps_per_block - 2
     refresh = sum(seq_lens) if phase in ("all", "refresh") else 0
@@ -158,7 +172,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    cfg = W.CONFIGS[args.workload]
+    cfg = workload_config(args)
     import oracle
     oracle.build()
     for i in range(args.warmup):
@@ -215,7 +229,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
     B.lib()
 
-    cfg = W.CONFIGS[args.workload]
+    cfg = workload_config(args)
     n_layers = args.layers or cfg.n_layers
     Hq, Hkv, D, b = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.block_len
     reuse_steps = cfg.steps_per_block - 2

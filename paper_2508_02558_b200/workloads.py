@@ -93,6 +93,10 @@ CONFIGS: Dict[str, WorkloadConfig] = {
                               salient_spans=16, salient_span_len=64),
     # one LLaDA-shaped layer for the ragged batched sweep (prompt length overridden per sequence)
     "c5_serving": WorkloadConfig("c5_serving", "bf16", 32, 32, 128, 4096, 256, salient_frac=0.02),
+    # second workload shapes (LLaDA-shaped stack): generation length 512 after a 512-token prompt, and a prompt
+    # truncated to 4k tokens followed by 512 generated tokens; block length 32, one denoising step per token
+    "c6_gen512": WorkloadConfig("c6_gen512", "bf16", 32, 32, 128, 512, 512, n_layers=32, salient_frac=0.02),
+    "c7_long4k": WorkloadConfig("c7_long4k", "bf16", 32, 32, 128, 4096, 512, n_layers=32, salient_frac=0.02),
 }
 
 

@@ -38,11 +38,11 @@ def _check_all_heads_properties(g, seq_len, block_off, b):
                 assert pooled[h][kept].min() >= pooled[h][cand & ~kept].max()
 
 
-def _run(cfg, seed, heads, retention=None, window=None, score=oracle.SCORE_LOGIT_MEAN):
+def _run(cfg, seed, heads, retention=None, window=None, score=oracle.SCORE_LOGIT_MEAN, block=0):
     import parity_util as U
     r = cfg.retention if retention is None else retention
     s_ = cfg.pool_window if window is None else window
-    s = W.make_sequence(cfg, seed=seed, layer=0, block=0)
+    s = W.make_sequence(cfg, seed=seed, layer=0, block=block)
     q, k, v = s.refresh_inputs(1)
     L, o = s.seq_len, s.block_off
     g = U.gpu_refresh(q[None], k[None], v[None], [L], [o], cfg.dtype, r, s_, score=score)
@@ -61,6 +61,12 @@ def test_c2_llada_layer_full_size():
 
 def test_c3_dream_layer_full_size():
     _run(W.CONFIGS["c3_dream"], seed=22, heads=[0, 3])
+
+
+@pytest.mark.parametrize("name,block,r,window", [("c6_gen512", 9, 0.3, 5), ("c7_long4k", 15, None, None)])
+def test_second_workload_shapes_full_size(name, block, r, window):
+    """Generation length 512 (a block in the middle: prefix and suffix both long) and the 4k-prompt shape (last block)."""
+    _run(W.CONFIGS[name], seed=26, heads=[4, 29], retention=r, window=window, block=block)
 
 
 @pytest.mark.parametrize("r,window", [(0.1, 7), (0.5, 3)])
