@@ -212,7 +212,7 @@ def sparse_block_attn_static(desc: Desc, q_blk, k_c, v_c, kept_cnt, k_blk, v_blk
 
 def dense_attn(desc: Desc, q, k, v, seq_len, out, lse, workspace, stream=None):
     """Full-sequence bidirectional attention; q and out are [B, Hq, seq_len_max, D] tensors whose strides are passed on."""
-    qs = (ctypes.c_int64 * 3)(*q.stride()[:3])
-    os_ = (ctypes.c_int64 * 3)(*out.stride()[:3])
+    qs = (ctypes.c_int64 * 3)(*(q.stride()[:3] if q is not None else (0, 0, 0)))
+    os_ = (ctypes.c_int64 * 3)(*(out.stride()[:3] if out is not None else (0, 0, 0)))
     _check(lib().sdllm_dense_attn(ctypes.byref(desc), _ptr(q), qs, _ptr(k), _ptr(v), _ptr(seq_len), _ptr(out), os_, _ptr(lse),
                                   _ptr(workspace), _nbytes(workspace), _stream(stream)), "sdllm_dense_attn")

@@ -331,3 +331,39 @@ def test_dense_step_two_tile_kernel_many_key_tiles():
     out, lse = U.gpu_dense(q, k, v, [1100, 640])
     U.check_dense_against_oracle(out, lse, np.nan_to_num(q), np.nan_to_num(k), np.nan_to_num(v), [1100, 640],
                                  rows=[0, 127, 128, 300, 639, 640, 1023, 1024, 1099])
+
+
+@pytest.mark.parametrize("kernel", ["tile", "pair"])
+def test_dense_step_strided_tensors_and_argument_checks(kernel, monkeypatch):
+    """q and out as column slices of wider tensors (row stride 2D), heads-last-but-one layouts left to the strides; the
+    untouched half of the output buffer must stay as it was. Then the argument checks of the entry point."""
+    import parity_util as U
+    monkeypatch.setenv("SDLLM_DENSE", kernel)
+    Hq, Hkv, D, L = 4, 2, 64, 200
+    q, k, v = _dense_case(Hq, Hkv, D, [L], seed=27, pad=0.0)
+    d = B.make_desc(batch=1, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, seq_len_max=L, block_len=32, dtype=B.BF16, retention=0.5)
+    wide_q = torch.zeros((1, Hq, L, 2 * D), dtype=torch.bfloat16, device="cuda:0")
+    wide_q[..., :D] = U.to_dev(q, "bf16")
+    wide_o = torch.full((1, Hq, L, 2 * D), 7.0, dtype=torch.bfloat16, device="cuda:0")
+    kd, vd = U.to_dev(k, "bf16"), U.to_dev(v, "bf16")
+    ws = torch.zeros((max(B.workspace_bytes(d, B.OP_DENSE_ATTN), 256),), dtype=torch.uint8, device="cuda:0")
+    assert B.launch_count(d, B.OP_DENSE_ATTN) >= 1
+    B.dense_attn(d, wide_q[..., :D], kd, vd, None, wide_o[..., :D], None, ws)
+    torch.cuda.synchronize()
+    assert B.read_status(ws) == 0
+    got = U.to_host_f32(wide_o)
+    assert (got[..., D:] == 7.0).all()
+    U.check_dense_against_oracle(np.ascontiguousarray(got[..., :D]), None, q, k, v, None)
+    # argument checks: missing tensors, a workspace that is too small, a misaligned pointer
+    qd = U.to_dev(q, "bf16")
+    out = torch.empty_like(qd)
+    for args in [(None, kd, vd, None, out, None, ws), (qd, kd, vd, None, None, None, ws)]:
+        with pytest.raises(B.SdllmError) as e:
+            B.dense_attn(d, *args)
+        assert e.value.status == B.ERR_INVALID_ARG
+    with pytest.raises(B.SdllmError) as e:
+        B.dense_attn(d, qd, kd, vd, None, out, None, ws[:128])
+    assert e.value.status == B.ERR_WORKSPACE
+    with pytest.raises(B.SdllmError) as e:
+        B.dense_attn(d, qd, kd.view(-1)[4:].view(-1), vd, None, out, None, ws)
+    assert e.value.status == B.ERR_INVALID_ARG
