@@ -1,16 +1,14 @@
 // Full-sequence bf16 attention on tcgen05 (the dense step: every row of a sequence over all of its keys).
 //
 // A dense contraction, bound by the tensor pipe and, in front of it, by the softmax. One CTA owns TWO 128-row query
-// tiles of one query head and streams the head's K/V once for both, in tiles of 64 keys:
-//   warp 0      TMA producer: the two Q tiles, then K and V tiles (128-byte swizzle) into a four-slot ring
-//   warp 1      one thread issues tcgen05.mma: S_t(j) = Q_t K_j^T into one of two S buffers per query tile t, two key
-//               tiles ahead of the softmax, and O_t += P_t(j) V_j as soon as the softmax warps have written P_t(j)
+// tiles of one query head and streams the head's K/V once for both:
+//   warp 0      TMA producer: the two Q tiles, then K and V tiles (128 keys, 128-byte swizzle) into a two-slot ring
+//   warp 1      one thread issues tcgen05.mma. Per key tile j:  S0 = Q0 K_j^T,  O1 += P1(j-1) V_(j-1),  S1 = Q1 K_j^T,
+//               O0 += P0(j) V_j  -  while the softmax warps of one query tile work, the tensor pipe serves the other
 //   warps 2-5   softmax of query tile 0, warps 6-9 of query tile 1: a thread owns one accumulator row (TMEM lane),
 //               reads its S row, keeps the running max / sum and writes P (bf16) over S in TMEM; O accumulates in
-//               TMEM and is rescaled in place only when the row's maximum grows by more than 2^8. With S(j+1)
-//               already waiting when tile j is done, the softmax warps never wait for the tensor pipe.
-// Tensor memory (512 columns): per query tile two S buffers of 64 columns, then O0 | O1 of 128 columns each
-// (D = 64 uses half of an O region).
+//               TMEM and is rescaled in place only when the row's maximum grows by more than 2^8
+// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 columns each (D = 64 uses half of an O region).
 // The finished rows go from TMEM through registers straight to global memory (bf16), normalised by the row sum.
 // Every wait on an mbarrier is bounded; on expiry the CTA sets an abort flag, records a code in the status word and
 // runs to its end (freeing its TMEM); the outputs of that call are then invalid.
@@ -26,7 +24,7 @@ using namespace dev;
 namespace {
 
 constexpr int DN_THREADS = 320;
-constexpr int DN_STAGES = 4;
+constexpr int DN_STAGES = 2;
 
 struct DenseMaps {
   CUtensorMap q, k, v;
@@ -48,14 +46,11 @@ template <int D>
 __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __grid_constant__ DenseMaps tm, const DenseParams p) {
   extern __shared__ unsigned char smem_raw[];
   constexpr int H = D / 64;                 // 64-column halves of a row (128 bytes each: one swizzle atom wide)
-  constexpr int KT = 64;                    // keys per tile
+  constexpr int KT = 128;                   // keys per tile
   constexpr int NS = DN_STAGES;
-  constexpr int QHALF = 128 * 128;          // bytes of one 64-column half of a 128-row Q tile
-  constexpr int QTILE = H * QHALF;          // bytes of a Q tile
-  constexpr int HALF = KT * 128;            // bytes of one 64-column half of a K or V tile
-  constexpr int TILE = H * HALF;            // bytes of a K or V tile
-  // tensor memory: per query tile t two S buffers of KT columns at t*128 + {0, KT}; O_t at 256 + t*128
-  constexpr uint32_t O_COL0 = 256, T_STRIDE = 128;
+  constexpr int HALF = KT * 128;            // bytes of one 64-column half of a 128-row tile
+  constexpr int TILE = H * HALF;            // bytes of a Q, K or V tile
+  constexpr uint32_t S_COL0 = 0, O_COL0 = 256, T_STRIDE = 128;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bi = blockIdx.z, h = blockIdx.y, g = h / p.G, jp = blockIdx.x;
 
@@ -73,11 +68,11 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
   const uint32_t bars = smem_u32(smem);
   auto BAR = [&](int i) { return bars + 8u * (uint32_t)i; };
   const int Q_FULL = 0, FULL_K = 1, FULL_V = 1 + NS, EMPTY_K = 1 + 2 * NS, EMPTY_V = 1 + 3 * NS;
-  const int S_FULL = 1 + 4 * NS, P_FULL = S_FULL + 4, PV_DONE = S_FULL + 8, DRAIN = S_FULL + 10;   // S/P: [query tile][buffer]
+  const int S_FULL = 1 + 4 * NS, P_FULL = S_FULL + 2, PV_DONE = S_FULL + 4, DRAIN = S_FULL + 6;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 260);
   unsigned char* q_s = smem + 1024;
-  unsigned char* stage0 = q_s + 2 * QTILE;
+  unsigned char* stage0 = q_s + 2 * TILE;
 
   if (tid == 0) {
     prefetch_tmap(&tm.q); prefetch_tmap(&tm.k); prefetch_tmap(&tm.v);
@@ -86,11 +81,11 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
       mbar_init(BAR(FULL_K + i), 1); mbar_init(BAR(FULL_V + i), 1);
       mbar_init(BAR(EMPTY_K + i), 1); mbar_init(BAR(EMPTY_V + i), 1);
     }
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < 2; ++i) {
       mbar_init(BAR(S_FULL + i), 1);
       mbar_init(BAR(P_FULL + i), 4);       // the four softmax warps of a query tile
+      mbar_init(BAR(PV_DONE + i), 1);
     }
-    for (int i = 0; i < 2; ++i) mbar_init(BAR(PV_DONE + i), 1);
     mbar_init(BAR(DRAIN), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -110,10 +105,10 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
   if (warp == 0) {
     // ======================================= TMA producer =======================================
     if (lane == 0) {
-      mbar_expect_tx(BAR(Q_FULL), (uint32_t)((act1 ? 2 : 1) * QTILE));
+      mbar_expect_tx(BAR(Q_FULL), (uint32_t)((act1 ? 2 : 1) * TILE));
       for (int t = 0; t < (act1 ? 2 : 1); ++t)
         for (int hh = 0; hh < H; ++hh)
-          tma_load_4d(smem_u32(q_s + t * QTILE + hh * QHALF), &tm.q, BAR(Q_FULL), hh * 64, row00 + t * 128, h, bi);
+          tma_load_4d(smem_u32(q_s + t * TILE + hh * HALF), &tm.q, BAR(Q_FULL), hh * 64, row00 + t * 128, h, bi);
       int issued = 0;
       bool ok = true;
       for (int j = 0; j < nt && ok; ++j) {
@@ -145,25 +140,26 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
       const uint32_t idesc_pv = instr_desc(D, true);
       const uint32_t qsm = smem_u32(q_s);
       bool ok = wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 23);
-      // S_t(j) = Q_t K_j^T into buffer j & 1 of query tile t
+      // S_t = Q_t K_j^T into the S region of query tile t
       auto issue_s = [&](int t, int j) {
         const uint32_t ksm = smem_u32(stage0 + (size_t)(j % NS) * 2 * TILE);
         const uint32_t idesc_s = instr_desc((tile_nv(j) + 15) & ~15, false);
-        const uint32_t d_t = tmem_base + (uint32_t)t * T_STRIDE + (uint32_t)(j & 1) * KT;
+        const uint32_t d_t = tmem_base + S_COL0 + (uint32_t)t * T_STRIDE;
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks)
-          mma_ss(d_t, smem_desc(qsm + t * QTILE + (ks >> 2) * QHALF + (ks & 3) * 32, 16u, 1024u),
-                 smem_desc(ksm + (ks >> 2) * HALF + (ks & 3) * 32, 16u, 1024u), idesc_s, ks > 0 ? 1u : 0u);
-        tc_commit(BAR(S_FULL + t * 2 + (j & 1)));
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t off = (ks >> 2) * HALF + (ks & 3) * 32;
+          mma_ss(d_t, smem_desc(qsm + t * TILE + off, 16u, 1024u), smem_desc(ksm + off, 16u, 1024u), idesc_s, ks > 0 ? 1u : 0u);
+        }
+        tc_commit(BAR(S_FULL + t));
       };
-      // O_t += P_t(j) V_j once the softmax warps of query tile t have written P_t(j); `release` frees the V slot afterwards
+      // O_t += P_t V_j once the softmax warps of query tile t have written P_t; `release` frees the V slot afterwards
       auto issue_pv = [&](int t, int j, bool release) -> bool {
         const int s = j % NS;
-        if (!wait_bar(BAR(P_FULL + t * 2 + (j & 1)), (j >> 1) & 1, abort_flag, p.status, 24)) return false;
+        if (!wait_bar(BAR(P_FULL + t), j & 1, abort_flag, p.status, 24)) return false;
         if (!wait_bar(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 25)) return false;
         tc_fence_after();
         const uint32_t vsm = smem_u32(stage0 + (size_t)s * 2 * TILE) + TILE;
-        const uint32_t a_t = tmem_base + (uint32_t)t * T_STRIDE + (uint32_t)(j & 1) * KT;
+        const uint32_t a_t = tmem_base + S_COL0 + (uint32_t)t * T_STRIDE;
         const int n_mma = (tile_nv(j) + 15) & ~15;
         for (int ks = 0; ks < n_mma / 16; ++ks)
           mma_ts(tmem_base + O_COL0 + (uint32_t)t * T_STRIDE, a_t + ks * 8, smem_desc(vsm + ks * 2048, (uint32_t)HALF, 1024u), idesc_pv,
@@ -172,24 +168,19 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
         if (release) tc_commit(BAR(EMPTY_V + s));
         return true;
       };
-      // S of key tile j for both query tiles, as soon as its K has landed; then K's slot is free
-      auto issue_s_both = [&](int j) -> bool {
+      for (int j = 0; j < nt && ok; ++j) {
         const int s = j % NS;
-        if (!wait_bar(BAR(FULL_K + s), (j / NS) & 1, abort_flag, p.status, 26)) return false;
+        if (!wait_bar(BAR(FULL_K + s), (j / NS) & 1, abort_flag, p.status, 26)) { ok = false; break; }
         tc_fence_after();
         issue_s(0, j);
-        if (act1) issue_s(1, j);
+        if (act1) {
+          if (j > 0 && !issue_pv(1, j - 1, true)) { ok = false; break; }
+          issue_s(1, j);
+        }
         tc_commit(BAR(EMPTY_K + s));
-        return true;
-      };
-      // The S tiles run two key tiles ahead of the softmax (two buffers per query tile), so a softmax warp that has
-      // finished tile j finds S(j+1) waiting; S(j+2) goes into the buffer that P(j) V_j has just read.
-      for (int j = 0; j < min(nt, 2) && ok; ++j) ok = issue_s_both(j);
-      for (int j = 0; j < nt && ok; ++j) {
         if (!issue_pv(0, j, !act1)) { ok = false; break; }
-        if (act1 && !issue_pv(1, j, true)) { ok = false; break; }
-        if (j + 2 < nt && !issue_s_both(j + 2)) { ok = false; break; }
       }
+      if (ok && act1) ok = issue_pv(1, nt - 1, true);
       if (*abort_flag) {                    // wait for the tensor pipe to finish what was issued before TMEM is freed
         tc_commit(BAR(DRAIN));
         drain_bar(BAR(DRAIN), 0);
@@ -202,29 +193,28 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
     const int row = q4 * 32 + lane;
     if (t == 0 || act1) {
       const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16);
+      const uint32_t s_addr = lane_addr + S_COL0 + (uint32_t)t * T_STRIDE;
       const uint32_t o_addr = lane_addr + O_COL0 + (uint32_t)t * T_STRIDE;
       float m_run = -INFINITY, l_run = 0.f;
       bool ok = true;
       for (int j = 0; j < nt && ok; ++j) {
         const int nv = tile_nv(j);
-        const uint32_t s_addr = lane_addr + (uint32_t)t * T_STRIDE + (uint32_t)(j & 1) * KT;
-        if (!wait_bar_warp(BAR(S_FULL + t * 2 + (j & 1)), (j >> 1) & 1, abort_flag, p.status, 27)) { ok = false; break; }
+        if (!wait_bar_warp(BAR(S_FULL + t), j & 1, abort_flag, p.status, 27)) { ok = false; break; }
         tc_fence_after();
-        constexpr int NC = KT / 32;                      // 32-column chunks of an S row
-        uint32_t sv[NC][32];
+        uint32_t sv[4][32];
 #pragma unroll
-        for (int c = 0; c < NC; ++c) tmem_ld32(s_addr + c * 32, sv[c]);
+        for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sv[c]);
         tc_wait_ld();
         if (nv < KT) {                                   // the ragged last tile: keys past the end count as -inf
 #pragma unroll
-          for (int c = 0; c < NC; ++c)
+          for (int c = 0; c < 4; ++c)
 #pragma unroll
             for (int i = 0; i < 32; ++i)
               if (c * 32 + i >= nv) sv[c][i] = __float_as_uint(-INFINITY);
         }
         float mx = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < NC; ++c) {
+        for (int c = 0; c < 4; ++c) {
           float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
           for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(sv[c][i]));
@@ -254,10 +244,10 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
           }
         }
         const float mu = (m_run == -INFINITY) ? 0.f : m_run;
-        // P = exp2(S * scale_log2 - mu) as bf16 over the first half of the S buffer's columns
+        // P = exp2(S * scale_log2 - mu) as bf16 over the first 64 columns of the S region
         float psum = 0.f;
 #pragma unroll
-        for (int c = 0; c < NC; ++c) {
+        for (int c = 0; c < 4; ++c) {
           uint32_t pk[16];
           float ps4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -287,7 +277,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(P_FULL + t * 2 + (j & 1)));
+        if (lane == 0) mbar_arrive(BAR(P_FULL + t));
       }
       // ---- the finished row: TMEM -> registers -> normalise -> bf16 -> global memory ----
       if (ok) ok = wait_bar_warp(BAR(PV_DONE + t), (nt - 1) & 1, abort_flag, p.status, 30);
@@ -330,8 +320,8 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
 }
 
 size_t dense_smem_bytes(int D) {
-  const size_t q_tile = (size_t)(D / 64) * 128 * 128, kv_tile = (size_t)(D / 64) * 64 * 128;
-  return 1024 /*alignment slack*/ + 1024 /*barriers*/ + 2 * q_tile + (size_t)DN_STAGES * 2 * kv_tile;
+  const size_t tile = (size_t)(D / 64) * 128 * 128;
+  return 1024 /*alignment slack*/ + 1024 /*barriers*/ + 2 * tile + (size_t)DN_STAGES * 2 * tile;
 }
 
 template <int D>
@@ -379,8 +369,8 @@ cudaError_t launch_dense_pair(const void* q, const int64_t* q_stride, const void
   DenseMaps tm;
   memset(&tm, 0, sizeof(tm));
   bool ok = umma_make_map(&tm.q, q, D, L, Hq, B, q_stride, 128, 1);
-  ok = ok && umma_make_map(&tm.k, k, D, L, Hkv, B, kv_stride, 64, 1);       // K and V travel in tiles of 64 keys
-  ok = ok && umma_make_map(&tm.v, v, D, L, Hkv, B, kv_stride, 64, 1);
+  ok = ok && umma_make_map(&tm.k, k, D, L, Hkv, B, kv_stride, 128, 1);
+  ok = ok && umma_make_map(&tm.v, v, D, L, Hkv, B, kv_stride, 128, 1);
   if (!ok) return cudaErrorInvalidValue;
   DenseParams p{};
   p.seq_len = seq_len; p.out = out; p.lse = lse; p.status = status;
