@@ -174,9 +174,10 @@ sdllm_status sdllm_sparse_block_attn(const sdllm_desc* desc, const void* q_blk, 
  *   out [B, Hq, seq_len_max, D] with o_stride[3]; rows t >= seq_len[i] are not written
  *   lse [B, Hq, seq_len_max] fp32, nullable: log-sum-exp of the scaled logits per written row
  * seq_len NULL means every sequence has seq_len_max rows. desc->block_len, retention and the selection fields are
- * not used. bf16 only, D in {64, 128}, n_kv_heads * G * ceil(seq_len_max / 128) <= 65535; anything else returns
+ * not used. bf16 only, D in {64, 128}, at most 65535 query heads; anything else returns
  * SDLLM_ERR_UNSUPPORTED. The probability matrix is never written to memory. Workspace:
- * sdllm_workspace_bytes(desc, SDLLM_OP_DENSE_ATTN), zeroed once by the caller like the other attention workspaces. */
+ * sdllm_workspace_bytes(desc, SDLLM_OP_DENSE_ATTN) bytes (the status word), zeroed once by the caller; a workspace of
+ * the other attention calls serves as well. */
 sdllm_status sdllm_dense_attn(const sdllm_desc* desc, const void* q, const int64_t* q_stride, const void* k, const void* v,
                               const int32_t* seq_len, void* out, const int64_t* o_stride, float* lse, void* workspace,
                               size_t workspace_bytes, void* cuda_stream);

@@ -109,16 +109,11 @@ void fill_common(AttnParams& p, const sdllm_desc* d, const AttnPlan& pl) {
   for (int i = 0; i < 3; ++i) { p.q_stride[i] = d->q_stride[i]; p.o_stride[i] = d->o_stride[i]; }
 }
 
-// Full-sequence attention runs on the tcgen05 kernel only: bf16, one grid row per (KV head, query head of its group,
-// 128-row query block).
+// Full-sequence attention runs on its own tcgen05 kernel: bf16, D in {64, 128}, one grid row per query head.
+// Its workspace is the status word alone.
+constexpr size_t kDenseWorkspaceBytes = 256;
 bool dense_supported(const sdllm_desc* d) {
-  const int G = d->n_q_heads / d->n_kv_heads;
-  if (!umma_supported(d->dtype, d->head_dim, 128, 128)) return false;
-  return (int64_t)d->n_kv_heads * G * ((d->seq_len_max + 127) / 128) <= 65535;
-}
-
-AttnPlan dense_plan(const sdllm_desc* d) {
-  return plan_attention_dense(d->head_dim, d->n_q_heads / d->n_kv_heads, d->batch, d->n_kv_heads, d->seq_len_max);
+  return umma_supported(d->dtype, d->head_dim, 128, 128) && d->n_q_heads <= 65535;
 }
 
 // Built-in scratch of sdllm_sparse_block_attn_static: lives in the library image, one copy per GPU that loads it.
@@ -165,7 +160,7 @@ size_t sdllm_workspace_bytes(const sdllm_desc* d, int op) {
   if (check_desc(d) != SDLLM_OK) return 0;
   if (op == SDLLM_OP_REFRESH_SCORES) return attn_ws(d, plan_for(d, op), true).total;
   if (op == SDLLM_OP_SPARSE_BLOCK_ATTN) return attn_ws(d, plan_for(d, op), false).total;
-  if (op == SDLLM_OP_DENSE_ATTN && dense_supported(d)) return attn_ws(d, dense_plan(d), false).total;
+  if (op == SDLLM_OP_DENSE_ATTN && dense_supported(d)) return kDenseWorkspaceBytes;
   return 0;
 }
 
@@ -186,12 +181,7 @@ int32_t sdllm_launch_count(const sdllm_desc* d, int op) {
   if (check_desc(d) != SDLLM_OK) return -1;
   if (op == SDLLM_OP_SELECT_TOPK) return 1;
   if (op == SDLLM_OP_COMPACT_KV) return d->n_keep_max > 0 ? 1 : 0;
-  if (op == SDLLM_OP_DENSE_ATTN) {
-    if (!dense_supported(d)) return -1;
-    if (dense_pair_kernel_wanted(d->batch, d->n_q_heads, d->seq_len_max)) return 1;
-    const AttnPlan pl = dense_plan(d);
-    return 1 + ((pl.splits > 1 && !umma_tail_is_fused(pl, d->head_dim, 128, d->seq_len_max, false, true)) ? 1 : 0);
-  }
+  if (op == SDLLM_OP_DENSE_ATTN) return dense_supported(d) ? 1 : -1;
   if (op != SDLLM_OP_REFRESH_SCORES && op != SDLLM_OP_SPARSE_BLOCK_ATTN) return -1;
   const bool refresh = op == SDLLM_OP_REFRESH_SCORES;
   const AttnPlan pl = plan_for(d, op);
@@ -361,36 +351,11 @@ sdllm_status sdllm_dense_attn(const sdllm_desc* d, const void* q, const int64_t*
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(lse)) return SDLLM_ERR_INVALID_ARG;
   if (!strides_ok(q_stride, elem_size(d->dtype)) || !strides_ok(o_stride, elem_size(d->dtype))) return SDLLM_ERR_INVALID_ARG;
   if (!dense_supported(d)) return SDLLM_ERR_UNSUPPORTED;
-  const AttnPlan pl = dense_plan(d);
-  const WsLayout w = attn_ws(d, pl, false);
-  if (w.total > 0 && (ws == nullptr || ws_bytes < w.total || (reinterpret_cast<uintptr_t>(ws) & 255u))) return SDLLM_ERR_WORKSPACE;
+  if (ws == nullptr || ws_bytes < kDenseWorkspaceBytes || (reinterpret_cast<uintptr_t>(ws) & 255u)) return SDLLM_ERR_WORKSPACE;
   if ((st = check_device()) != SDLLM_OK) return st;
-  char* wsb = reinterpret_cast<char*>(ws);
-  if (dense_pair_kernel_wanted(d->batch, d->n_q_heads, d->seq_len_max)) {
-    if (cuda_failed(launch_dense_pair(q, q_stride, k, v, d->kv_stride, seq_len, out, o_stride, lse, reinterpret_cast<int32_t*>(wsb + w.status),
-                                      d->batch, d->n_q_heads, d->n_kv_heads, d->seq_len_max, d->head_dim, scale_of(d),
-                                      reinterpret_cast<cudaStream_t>(cuda_stream)), "dense attention launch"))
-      return SDLLM_ERR_CUDA;
-    return SDLLM_OK;
-  }
-
-  AttnParams p{};
-  fill_common(p, d, pl);
-  p.b = 128; p.M = 128 * p.G * pl.nqb;          // every (query head, 128-row query block) is a row tile
-  for (int i = 0; i < 3; ++i) { p.q_stride[i] = q_stride[i]; p.o_stride[i] = o_stride[i]; }
-  p.q = q; p.k1 = k; p.v1 = v; p.k2 = nullptr; p.v2 = nullptr;
-  p.n1_per_seq = seq_len; p.block_off = nullptr;
-  p.out = out; p.lse = lse;
-  p.status = reinterpret_cast<int32_t*>(wsb + w.status);
-  p.part_o = reinterpret_cast<float*>(wsb + w.part_o);
-  p.part_ml = reinterpret_cast<float*>(wsb + w.part_ml);
-  p.raw_scores = nullptr;
-  p.n1_max = d->seq_len_max; p.n2 = 0;
-  p.want_scores = 0;
-  p.counters = reinterpret_cast<int32_t*>(wsb + w.counters);
-  p.pooled = nullptr;
-  for (int i = 0; i < 3; ++i) { p.k1_stride[i] = d->kv_stride[i]; p.k2_stride[i] = 0; }
-  if (cuda_failed(launch_attn_partial(p, pl, d->dtype, d->head_dim, reinterpret_cast<cudaStream_t>(cuda_stream)), "attention launch"))
+  if (cuda_failed(launch_dense_pair(q, q_stride, k, v, d->kv_stride, seq_len, out, o_stride, lse, reinterpret_cast<int32_t*>(ws),
+                                    d->batch, d->n_q_heads, d->n_kv_heads, d->seq_len_max, d->head_dim, scale_of(d),
+                                    reinterpret_cast<cudaStream_t>(cuda_stream)), "dense attention launch"))
     return SDLLM_ERR_CUDA;
   return SDLLM_OK;
 }

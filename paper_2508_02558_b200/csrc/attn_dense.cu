@@ -354,14 +354,6 @@ cudaError_t launch_dense_d(const DenseMaps& tm, const DenseParams& p, int nqb, c
 
 }  // namespace
 
-// The two-tile kernel pays once there are enough (head, pair of query blocks) CTAs to fill the GPU; smaller problems
-// go to the block kernel's full-sequence mode, which splits the key axis. SDLLM_DENSE=tile / pair forces either.
-bool dense_pair_kernel_wanted(int B, int Hq, int L) {
-  if (const char* e = getenv("SDLLM_DENSE")) return e[0] == 'p';
-  const long long ctas = (long long)B * Hq * (((L + 127) / 128 + 1) / 2);
-  return ctas >= 96;
-}
-
 cudaError_t launch_dense_pair(const void* q, const int64_t* q_stride, const void* k, const void* v, const int64_t* kv_stride,
                               const int32_t* seq_len, void* out, const int64_t* o_stride, float* lse, int32_t* status, int B, int Hq,
                               int Hkv, int L, int D, float scale, cudaStream_t st) {

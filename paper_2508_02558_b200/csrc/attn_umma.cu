@@ -48,8 +48,6 @@ struct UmmaParams {
   int R;             // replicas of the query rows along the 128 accumulator rows (1, 2, 4)
   int row_tiles;     // 128-row tiles of the b*G rows
   int heads_rt;      // query heads per row tile
-  int nqb;           // full-sequence attention: 128-row query blocks per head (a row tile is one block of one head); else 0
-  int lq_max;        // full-sequence attention: query rows per head in the tensors (the rows' log-sum-exp is [B,Hq,lq_max])
   int fused_tail;    // 1: the last CTA of a unit merges and pools; 0: umma_tail_kernel does
   int early_src1;    // 1: source 1 and its count are older than the previous kernel in the stream (reuse step)
   int prob_pass;     // 1: second pass of the probability saliency: S and the rows' log-sum-exp give column means of P
@@ -101,42 +99,12 @@ __device__ __forceinline__ float pool_at_ldcg(const AttnParams& p, const float* 
   return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
 }
 
-// Where accumulator row ml of row tile rt goes: the query head and the row inside that head's output. Block mode packs
-// the group's heads b rows each; full-sequence mode gives every (head, 128-row query block) a row tile of its own.
-__device__ __forceinline__ void row_target(const UmmaParams& up, int g, int rt, int ml, int& head, int& i, int& lse_rows) {
-  const AttnParams& p = up.a;
-  if (up.nqb > 0) {
-    const int hg = rt / up.nqb;
-    head = g * p.G + hg; i = (rt - hg * up.nqb) * 128 + ml; lse_rows = up.lq_max;
-  } else {
-    const int m = rt * 128 + ml, hg = m / p.b;
-    head = g * p.G + hg; i = m - hg * p.b; lse_rows = p.b;
-  }
-}
-
-// Valid query rows of a row tile; n_seq is the sequence's length (full-sequence mode: its query rows).
-__device__ __forceinline__ int rows_of_tile(const UmmaParams& up, int rt, int n_seq) {
-  if (up.nqb > 0) return min(max(n_seq - (rt % up.nqb) * 128, 0), 128);
-  return min(up.a.M - rt * 128, 128);
-}
-
-// Keys of source 1 that a CTA of sequence bi works on. Full-sequence mode: a query block past the end of its sequence
-// has no rows, so it takes no keys either.
-__device__ __forceinline__ int keys_of_seq(const UmmaParams& up, int bi, int rt) {
-  const AttnParams& p = up.a;
-  int n = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
-  n = min(max(n, 0), p.n1_max);
-  if (up.nqb > 0 && (rt % up.nqb) * 128 >= n) n = 0;
-  return n;
-}
-
 // Merge of the key-split partials of S (row, float4 column) slots of a unit and the final stores. slot[s] < 0 marks
 // an unused entry. The partials are read in batches of MB per slot with the loads of all slots and of the whole batch
 // in flight together (one L2 latency per batch) and folded with a running maximum, so that four splits cost a single
 // round trip for everything a thread merges.
 template <int D, int MB, int S>
-__device__ __forceinline__ void merge_slots(const UmmaParams& up, int64_t unit, int bi, int g, int rt, const int (&slot)[S]) {
-  const AttnParams& p = up.a;
+__device__ __forceinline__ void merge_slots(const AttnParams& p, int64_t unit, int bi, int g, int rt, const int (&slot)[S]) {
   constexpr int D4 = D / 4;
   const int P = p.splits;
   const int prt = min(p.M, 128);                      // rows of one partial
@@ -185,15 +153,15 @@ __device__ __forceinline__ void merge_slots(const UmmaParams& up, int64_t unit, 
   for (int s = 0; s < S; ++s) {
     if (slot[s] < 0) continue;
     const float inv = l[s] > 0.f ? 1.f / l[s] : 0.f;
-    int head, i, lse_rows;
-    row_target(up, g, rt, m_local[s], head, i, lse_rows);
+    const int m = rt * 128 + m_local[s];
+    const int hg = m / p.b, i = m - hg * p.b;
     __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
-                         (int64_t)head * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4[s] * 4;
+                         (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4[s] * 4;
     uint2 w2;
     w2.x = pack_bf16(acc[s].x * inv, acc[s].y * inv);
     w2.y = pack_bf16(acc[s].z * inv, acc[s].w * inv);
     *reinterpret_cast<uint2*>(out) = w2;
-    if (d4[s] == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + head) * lse_rows + i] = (m_run[s] + log2f(l[s])) * kLn2;
+    if (d4[s] == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (m_run[s] + log2f(l[s])) * kLn2;
   }
 }
 
@@ -215,10 +183,9 @@ __global__ void __launch_bounds__(256) umma_tail_kernel(const UmmaParams up, con
     const int rt = (int)(unit % up.row_tiles);
     const int64_t bg = unit / up.row_tiles;
     const int g = (int)(bg % p.Hkv), bi = (int)(bg / p.Hkv);
-    const int n_seq = p.n1_per_seq ? min(max(p.n1_per_seq[bi], 0), p.n1_max) : p.n1_max;
-    if (m_local >= rows_of_tile(up, rt, n_seq)) return;
+    if (m_local >= min(p.M - rt * 128, 128)) return;
     const int one[1] = {m_local * D4 + d4};
-    merge_slots<D, 8, 1>(up, unit, bi, g, rt, one);
+    merge_slots<D, 8, 1>(p, unit, bi, g, rt, one);
     return;
   }
   const int64_t idx = (int64_t)(blockIdx.x - merge_blocks) * 256 + threadIdx.x;
@@ -303,7 +270,7 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
   const int tiles_all = tiles1 + tiles2;
   const int t_begin = (int)(((long long)split * tiles_all) / p.splits);
   const int t_end = (int)(((long long)(split + 1) * tiles_all) / p.splits);
-  int M_rt = min(p.M - rt * 128, 128);                // valid query rows of this row tile (<= rows_rep when R > 1)
+  const int M_rt = min(p.M - rt * 128, 128);          // valid query rows of this row tile (<= rows_rep when R > 1)
   constexpr bool prob_pass = PROB;                      // no V, no PV: S tiles only, reduced over the query rows
   const bool do_attn = p.out != nullptr && !prob_pass;
   const bool do_s = do_attn || prob_pass;              // Q and the S = Q K^T tiles are needed
@@ -350,12 +317,8 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
     mbar_expect_tx(BAR(Q_FULL), (uint32_t)(q_copies * H * q_rows * 128));
     for (int c = 0; c < q_copies; ++c)
       for (int h = 0; h < H; ++h)
-        if (up.nqb > 0) {               // full-sequence mode: 128 rows of one head, rows past the tensor read as zero
-          tma_load_4d(smem_u32(q_s + h * 128 * 128), &tm.q, BAR(Q_FULL), h * 64, (rt % up.nqb) * 128, g * p.G + rt / up.nqb, bi);
-        } else {
-          tma_load_4d(smem_u32(q_s + h * 128 * 128 + c * q_step * 128), &tm.q, BAR(Q_FULL), h * 64, 0,
-                      g * p.G + rt * up.heads_rt, bi);
-        }
+        tma_load_4d(smem_u32(q_s + h * 128 * 128 + c * q_step * 128), &tm.q, BAR(Q_FULL), h * 64, 0,
+                    g * p.G + rt * up.heads_rt, bi);
   };
   // issue loads for up to `limit` further tiles (producer lane only); with src1_only, stop in front of source 2
   auto produce = [&](int limit, bool src1_only) {
@@ -405,12 +368,14 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
       if (up.early_src1) {
         // Reuse step: the compacted cache and its count were written before the previous kernel in the stream even
         // started, so their tiles may stream in while that kernel is still finishing.
-        prod_n1 = keys_of_seq(up, bi, rt);
+        prod_n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
+        prod_n1 = min(max(prod_n1, 0), p.n1_max);
         produce(NS, true);             // the first NS slots are free: no waiting here
       }
       grid_dependency_wait();          // the loads below read what earlier kernels in the stream wrote
       if (!up.early_src1) {
-        prod_n1 = keys_of_seq(up, bi, rt);
+        prod_n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
+        prod_n1 = min(max(prod_n1, 0), p.n1_max);
       }
       TRACE(4);
       issue_q();
@@ -434,8 +399,8 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
   grid_dependency_wait();              // everything below may read what earlier kernels in the stream wrote
   grid_launch_dependents();
 
-  const int n1 = keys_of_seq(up, bi, rt);
-  M_rt = rows_of_tile(up, rt, n1);     // full-sequence mode: the sequence has as many query rows as keys
+  int n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
+  n1 = min(max(n1, 0), p.n1_max);
 
   // softmax state of this thread's accumulator row (softmax warps only)
   float m_run = -INFINITY, l_run = 0.f;
@@ -856,6 +821,7 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
     const int st = tid;
     if (!*abort_flag) {
       const int d4 = st % D4, r_first = st / D4, r_step = UM_THREADS / D4;
+      const int m_first = rt * 128;
       for (int mb = r_first; mb < M_rt; mb += 4 * r_step) {
         float4 acc[4];
         float2 x[4];
@@ -874,17 +840,17 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
         for (int u = 0; u < 4; ++u) {
           const int ml = mb + u * r_step;
           if (ml >= M_rt) break;
-          int head, i, lse_rows;
-          row_target(up, g, rt, ml, head, i, lse_rows);
+          const int m = m_first + ml;                  // row within the KV head: m = head_in_group * b + i
+          const int hg = m / p.b, i = m - hg * p.b;
           if (p.splits == 1) {
             const float inv = x[u].y > 0.f ? 1.f / x[u].y : 0.f;
             __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
-                               (int64_t)head * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
+                               (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
             uint2 w2;
             w2.x = pack_bf16(acc[u].x * inv, acc[u].y * inv);
             w2.y = pack_bf16(acc[u].z * inv, acc[u].w * inv);
             *reinterpret_cast<uint2*>(o) = w2;
-            if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + head) * lse_rows + i] = (x[u].x + log2f(x[u].y)) * kLn2;
+            if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (x[u].x + log2f(x[u].y)) * kLn2;
           } else if (up.cluster > 1) {
             // this split's partial stays on chip: pm_s [M_rt][D] next to lm_s, read by the cluster peers below
             *reinterpret_cast<float4*>(reinterpret_cast<float*>(stage0 + 128 * D * 4 + 2048) + ml * D + d4 * 4) = acc[u];
@@ -944,15 +910,15 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
           acc.x = fmaf(o[c].x, w, acc.x); acc.y = fmaf(o[c].y, w, acc.y); acc.z = fmaf(o[c].z, w, acc.z); acc.w = fmaf(o[c].w, w, acc.w);
         }
         const float inv = l > 0.f ? 1.f / l : 0.f;
-        int head, i, lse_rows;
-        row_target(up, g, rt, ml, head, i, lse_rows);
+        const int m = rt * 128 + ml;
+        const int hg = m / p.b, i = m - hg * p.b;
         __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
-                             (int64_t)head * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
+                             (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i * p.o_stride[2] + d4 * 4;
         uint2 w2;
         w2.x = pack_bf16(acc.x * inv, acc.y * inv);
         w2.y = pack_bf16(acc.z * inv, acc.w * inv);
         *reinterpret_cast<uint2*>(out) = w2;
-        if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + head) * lse_rows + i] = (mstar + log2f(l)) * kLn2;
+        if (d4 == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
       }
     }
     if (tail_pool && !*abort_flag) {
@@ -983,7 +949,7 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
           int four[4];
 #pragma unroll
           for (int u = 0; u < 4; ++u) four[u] = s0 + u * UM_THREADS < M_rt * (D / 4) ? s0 + u * UM_THREADS : -1;
-          merge_slots<D, 4, 4>(up, unit, bi, g, rt, four);
+          merge_slots<D, 4, 4>(p, unit, bi, g, rt, four);
         }
       if (tail_pool) {
         // stage the head's raw saliency in shared memory (the ring is free), then pool from there
@@ -1168,15 +1134,6 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
   return pl;
 }
 
-// Full-sequence attention (every row of the sequence attends to every key: the dense steps around the block steps):
-// each (query head, 128-row query block) is a row tile of the same kernel, all row tiles of a KV head stream its keys.
-AttnPlan plan_attention_dense(int D, int G, int B, int Hkv, int L) {
-  const int nqb = (L + 127) / 128;
-  AttnPlan pl = plan_attention_umma(D, 128 * G * nqb, 128, B, Hkv, L, 0);
-  pl.nqb = nqb; pl.lq_max = L;
-  return pl;
-}
-
 cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cudaStream_t st) {
   UmmaMaps tm;
   UmmaParams up{};
@@ -1184,8 +1141,6 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
   up.a.splits = pl.splits;
   up.KT = pl.key_tile; up.KT2 = pl.key_tile2; up.R = pl.rep; up.row_tiles = pl.row_tiles;
   up.heads_rt = pl.row_tiles == 1 ? p.G : 128 / p.b;
-  up.nqb = pl.nqb; up.lq_max = pl.lq_max;
-  if (pl.nqb > 0) up.heads_rt = 1;
   const bool pool = p.want_scores && p.pooled != nullptr;
   {
     const char* e = getenv("SDLLM_EARLY_LOADS");   // SDLLM_EARLY_LOADS=0: no loads before the grid dependency (test aid)
@@ -1203,8 +1158,7 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
   up.fused_tail = (pl.cluster > 1 || umma_tail_is_fused(pl, D, p.M, p.n1_max, pool || p.prob_pass, p.out != nullptr && !p.prob_pass)) ? 1 : 0;
   memset(&tm, 0, sizeof(tm));
   bool ok = true;
-  if (pl.nqb > 0) ok = make_map(&tm.q, p.q, D, pl.lq_max, p.Hq, p.B, p.q_stride, 128, 1);
-  else if (p.out != nullptr || p.prob_pass) ok = make_map(&tm.q, p.q, D, p.b, p.Hq, p.B, p.q_stride, p.b, up.heads_rt);
+  if (p.out != nullptr || p.prob_pass) ok = make_map(&tm.q, p.q, D, p.b, p.Hq, p.B, p.q_stride, p.b, up.heads_rt);
   if (p.n1_max > 0) {
     ok = ok && make_map(&tm.k1, p.k1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, pl.key_tile, 1);
     ok = ok && make_map(&tm.v1, p.v1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, pl.key_tile, 1);

@@ -37,8 +37,6 @@ struct AttnPlan {
   bool dual;        // tcgen05 kernel, small-footprint variant: two CTAs per SM
   size_t part_rows; // partial rows per (sequence, KV head) in the workspace (0: none)
   size_t n_counters;// completion counters in the workspace
-  int nqb;          // full-sequence attention (tcgen05 kernel): 128-row query blocks per head, one row tile each; else 0
-  int lq_max;       // full-sequence attention: query rows per head in the tensors
 };
 
 // Key sources of one attention launch. The virtual key axis is [src1 rows 0..n1) ++ [src2 rows 0..n2).
@@ -102,9 +100,7 @@ AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_m
 
 bool umma_tail_is_fused(const AttnPlan& pl, int D, int M, int n1_max, bool pool, bool merge);
 bool umma_supported(int dtype, int D, int M, int b);
-AttnPlan plan_attention_dense(int D, int G, int B, int Hkv, int L);
-// Full-sequence attention, two query tiles per CTA (attn_dense.cu): whether it is the kernel of choice, and its launch.
-bool dense_pair_kernel_wanted(int B, int Hq, int L);
+// Full-sequence attention, two query tiles per CTA (attn_dense.cu).
 cudaError_t launch_dense_pair(const void* q, const int64_t* q_stride, const void* k, const void* v, const int64_t* kv_stride,
                               const int32_t* seq_len, void* out, const int64_t* o_stride, float* lse, int32_t* status, int B, int Hq,
                               int Hkv, int L, int D, float scale, cudaStream_t st);

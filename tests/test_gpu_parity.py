@@ -283,31 +283,17 @@ def _dense_case(Hq, Hkv, D, lens, seed, pad=np.nan):
 
 
 @pytest.mark.parametrize("Hq,Hkv,D,lens", [
-    (2, 2, 128, [333]),                 # several query blocks and key tiles with ragged tails, key splits merged
+    (2, 2, 128, [333]),                 # several query blocks (an odd number) and key tiles with ragged tails
     (8, 2, 64, [200]),                  # grouped heads, D = 64
     (4, 1, 128, [128]),                 # exactly one tile each way
     (2, 1, 128, [17]),                  # shorter than a tile
     (4, 2, 128, [300, 40, 0, 257]),     # ragged batch with an empty sequence
 ])
-@pytest.mark.parametrize("kernel", ["tile", "pair"])
-def test_dense_step(Hq, Hkv, D, lens, kernel, monkeypatch):
-    """Both kernels of the dense step: the block kernel's full-sequence mode and the two-query-tile kernel."""
+def test_dense_step(Hq, Hkv, D, lens):
     import parity_util as U
-    monkeypatch.setenv("SDLLM_DENSE", kernel)
     q, k, v = _dense_case(Hq, Hkv, D, lens, seed=21)
     out, lse = U.gpu_dense(q, k, v, lens)
     U.check_dense_against_oracle(out, lse, np.nan_to_num(q), np.nan_to_num(k), np.nan_to_num(v), lens)
-
-
-@pytest.mark.parametrize("env", [{"SDLLM_FUSED_TAIL": "0"}, {"SDLLM_SPLITS": "1"}, {"SDLLM_SPLITS": "3", "SDLLM_KEY_TILE": "64"}])
-def test_dense_step_launch_plans(env, monkeypatch):
-    import parity_util as U
-    monkeypatch.setenv("SDLLM_DENSE", "tile")
-    for k_, v_ in env.items():
-        monkeypatch.setenv(k_, v_)
-    q, k, v = _dense_case(4, 2, 128, [300, 129], seed=22)
-    out, lse = U.gpu_dense(q, k, v, [300, 129])
-    U.check_dense_against_oracle(out, lse, np.nan_to_num(q), np.nan_to_num(k), np.nan_to_num(v), [300, 129])
 
 
 def test_dense_step_without_lengths_and_refusals():
@@ -333,12 +319,10 @@ def test_dense_step_two_tile_kernel_many_key_tiles():
                                  rows=[0, 127, 128, 300, 639, 640, 1023, 1024, 1099])
 
 
-@pytest.mark.parametrize("kernel", ["tile", "pair"])
-def test_dense_step_strided_tensors_and_argument_checks(kernel, monkeypatch):
+def test_dense_step_strided_tensors_and_argument_checks():
     """q and out as column slices of wider tensors (row stride 2D), heads-last-but-one layouts left to the strides; the
     untouched half of the output buffer must stay as it was. Then the argument checks of the entry point."""
     import parity_util as U
-    monkeypatch.setenv("SDLLM_DENSE", kernel)
     Hq, Hkv, D, L = 4, 2, 64, 200
     q, k, v = _dense_case(Hq, Hkv, D, [L], seed=27, pad=0.0)
     d = B.make_desc(batch=1, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, seq_len_max=L, block_len=32, dtype=B.BF16, retention=0.5)
