@@ -1,5 +1,7 @@
 // Top-k selection over the pooled importance scores and the K/V gather-compaction
 // (Algorithm 1: "n <- floor(|I| r)", "TopKIndices(I, n)", "Select(K_f, I)", "Select(V_f, I)").
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace sdllm {
@@ -184,6 +186,190 @@ __global__ void __launch_bounds__(SEL_THREADS) select_topk_kernel(const SelectPa
   if (g == 0 && tid == 0) p.kept_cnt[bi] = kept;
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Long sequences: the same selection by a thread-block cluster. One CTA per (sequence, KV head) leaves the GPU to a
+// handful of SMs when there are few heads and tens of thousands of candidates, so here SELC_CTAS CTAs share a head:
+// each stages a contiguous slice of the candidates, the radix passes add the slices' histograms up through
+// distributed shared memory (every CTA ends up with the same global histogram and takes the same decision), and the
+// ordered emission gets its offsets from the counts of the CTAs before it in position order. All counts are
+// integers: the result is the single-CTA kernel's, bit for bit.
+constexpr int SELC_CTAS = 8;
+constexpr int SELC_SLICE = 8192;          // candidates one CTA can stage
+
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;\n" : "=r"(r));
+  return r;
+}
+// Reads the word that lives at `local` in the shared memory of CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t peer_ld_u32(const uint32_t* local, uint32_t rank) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(local);
+  uint32_t ra, v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(ra) : "r"(a), "r"(rank));
+  asm volatile("ld.shared::cluster.u32 %0, [%1];\n" : "=r"(v) : "r"(ra) : "memory");
+  return v;
+}
+
+__global__ void __launch_bounds__(SEL_THREADS) select_topk_cluster_kernel(const SelectParams p) {
+  __shared__ uint32_t keys_s[SELC_SLICE + SELC_SLICE / 32 + 1];   // this CTA's slice, index i + i / 32
+  __shared__ uint32_t hist[SEL_HIST][256];
+  __shared__ uint32_t fold[2][256];       // this CTA's histogram of a pass (two in turn), read by the peers
+  __shared__ uint32_t ghist[256];         // the cluster's histogram
+  __shared__ uint32_t warp_tot[SEL_WARPS + 1];
+  __shared__ uint32_t sh_prefix, sh_remaining;
+  __shared__ uint32_t pub_eq[2], pub_keep[2];   // per segment: this CTA's tie and keep counts, read by the peers
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int rank = (int)cluster_rank();
+  const int g = blockIdx.y, bi = blockIdx.z;
+  int L = p.seq_len ? p.seq_len[bi] : p.Lmax;
+  L = min(max(L, 0), p.Lmax);
+  const int b = p.b;
+  int o = p.block_off[bi];
+  o = min(max(o, 0), max(L - b, 0));
+  const int C = max(L - b, 0);
+  const float* sc = p.pooled + (int64_t)(bi * p.Hkv + g) * p.Lmax;
+  int32_t* out = p.kept_idx + (int64_t)(bi * p.Hkv + g) * p.n_keep_max;
+  auto cand_pos = [&](int c) { return c < o ? c : c + b; };
+
+  int n_pre, n_suf;
+  const int n_total = keep_count_total(o, C - o, p.retention, p.mode, &n_pre, &n_suf);
+  Segment seg[2];
+  int n_seg;
+  if (p.mode == SDLLM_SELECT_JOINT_FLOOR) {
+    seg[0] = {0, C, min(n_total, p.n_keep_max)};
+    n_seg = 1;
+  } else {
+    const int np = min(n_pre, p.n_keep_max);
+    seg[0] = {0, o, np};
+    seg[1] = {o, C, min(n_suf, p.n_keep_max - np)};
+    n_seg = 2;
+  }
+  uint32_t run_out = 0;                                // entries written so far (same value in every thread of every CTA)
+  int pass_id = 0;                                     // radix passes done so far (the same in every CTA)
+
+  for (int si = 0; si < n_seg; ++si) {
+    const int c_lo = seg[si].c_lo, c_hi = seg[si].c_hi, n = seg[si].n;
+    const int len = c_hi - c_lo;
+    if (n <= 0 || len <= 0) continue;                  // the same decision in every CTA of the cluster
+    // this CTA's slice of the segment (slices in rank order are in position order), staged in shared memory
+    const int chunk = (len + SELC_CTAS - 1) / SELC_CTAS;
+    const int s_lo = min(c_lo + rank * chunk, c_hi), s_hi = min(s_lo + chunk, c_hi);
+    const int slen = s_hi - s_lo;
+    __syncthreads();                                   // the previous segment's keys are no longer read
+    for (int i = tid; i < slen; i += SEL_THREADS) keys_s[i + (i >> 5)] = score_key(sc[cand_pos(s_lo + i)]);
+    const int kpt = (slen + SEL_THREADS - 1) / SEL_THREADS;   // candidates per thread, a contiguous run of the slice
+    const int my_lo = min(tid * kpt, slen), my_hi = min(my_lo + kpt, slen);
+    __syncthreads();
+    uint32_t thr = 0u, need_eq = 0u;
+    const bool take_all = n >= len;
+    if (!take_all) {
+      // ---- radix select of the n-th largest key of the whole segment ----
+      uint32_t prefix = 0u, remaining = (uint32_t)n;
+      for (int pass = 0; pass < 4; ++pass, ++pass_id) {
+        const int shift = 24 - 8 * pass;
+        for (int i = tid; i < SEL_HIST * 256; i += SEL_THREADS) (&hist[0][0])[i] = 0u;
+        __syncthreads();
+        const uint32_t himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+        uint32_t* my_hist = hist[warp & (SEL_HIST - 1)];
+        for (int i = my_lo; i < my_hi; ++i) {
+          const uint32_t k = keys_s[i + (i >> 5)];
+          if ((k & himask) == prefix) atomicAdd(&my_hist[(k >> shift) & 0xFFu], 1u);
+        }
+        __syncthreads();
+        if (tid < 256) {
+          uint32_t s2 = 0;
+#pragma unroll
+          for (int w = 0; w < SEL_HIST; ++w) s2 += hist[w][tid];
+          fold[pass_id & 1][tid] = s2;
+        }
+        // every CTA's histogram of this pass is complete (and everybody is done with the one of two passes ago)
+        cluster_barrier();
+        if (tid < 256) {
+          uint32_t s2 = 0;
+#pragma unroll
+          for (int q = 0; q < SELC_CTAS; ++q) s2 += peer_ld_u32(&fold[pass_id & 1][tid], (uint32_t)q);
+          ghist[tid] = s2;
+        }
+        __syncthreads();
+        if (warp == 0) {
+          // lane handles bins [255 - 8*lane - 7, 255 - 8*lane], scanning downward
+          uint32_t local[8], sum = 0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { local[i] = ghist[255 - (8 * lane + i)]; sum += local[i]; }
+          uint32_t incl = sum;
+#pragma unroll
+          for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += y;
+          }
+          uint32_t above = incl - sum;            // candidates in bins above this lane's range
+          if (above < remaining && incl >= remaining) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              if (above + local[i] >= remaining) {
+                sh_prefix = prefix | ((uint32_t)(255 - (8 * lane + i)) << shift);
+                sh_remaining = remaining - above;
+                break;
+              }
+              above += local[i];
+            }
+          }
+        }
+        __syncthreads();
+        prefix = sh_prefix;
+        remaining = sh_remaining;
+      }
+      thr = prefix;
+      need_eq = remaining;                        // how many candidates equal to thr are still to be kept (>= 1)
+    }
+    // ---- ordered emission: runs in thread order and slices in rank order are in position order ----
+    uint32_t my_eq = 0, my_gt = 0;
+    for (int i = my_lo; i < my_hi; ++i) {
+      const uint32_t k = keys_s[i + (i >> 5)];
+      my_gt += (take_all || k > thr) ? 1u : 0u;
+      my_eq += (!take_all && k == thr) ? 1u : 0u;
+    }
+    uint32_t total_eq, total_keep;
+    uint32_t eq_before = block_exclusive_scan(my_eq, warp_tot, &total_eq);
+    if (tid == 0) pub_eq[si] = total_eq;
+    cluster_barrier();
+    for (int q = 0; q < rank; ++q) eq_before += peer_ld_u32(&pub_eq[si], (uint32_t)q);
+    const uint32_t eq_quota = need_eq > eq_before ? min(need_eq - eq_before, my_eq) : 0u;   // ties kept from this run: its first ones
+    const uint32_t out_before = block_exclusive_scan(my_gt + eq_quota, warp_tot, &total_keep);
+    if (tid == 0) pub_keep[si] = total_keep;
+    cluster_barrier();
+    uint32_t keep_before = 0, keep_all = 0;
+#pragma unroll
+    for (int q = 0; q < SELC_CTAS; ++q) {
+      const uint32_t v = peer_ld_u32(&pub_keep[si], (uint32_t)q);
+      keep_all += v;
+      if (q < rank) keep_before += v;
+    }
+    uint32_t w = run_out + keep_before + out_before, eq_seen = 0;
+    for (int i = my_lo; i < my_hi; ++i) {
+      const uint32_t k = keys_s[i + (i >> 5)];
+      bool keep = take_all || k > thr;
+      if (!take_all && k == thr) { keep = eq_seen < eq_quota; ++eq_seen; }
+      if (keep) {
+        if (w < (uint32_t)p.n_keep_max) out[w] = cand_pos(s_lo + i);
+        ++w;
+      }
+    }
+    run_out += keep_all;
+  }
+  cluster_barrier();                                   // nobody leaves while a peer may still read its shared memory
+  if (rank == 0) {
+    const int kept = min((int)run_out, p.n_keep_max);
+    for (int i = kept + tid; i < p.n_keep_max; i += SEL_THREADS) out[i] = -1;
+    if (g == 0 && tid == 0) p.kept_cnt[bi] = kept;
+  }
+}
+
 // Gather of the kept rows: 16 bytes per thread, four rows of K and of V in flight per thread.
 constexpr int CP_ROWS_PER_THREAD = 4;
 
@@ -228,6 +414,22 @@ __global__ void __launch_bounds__(256) compact_kv_kernel(const CompactParams p) 
 }  // namespace
 
 cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st) {
+  // Tens of thousands of candidates per head: a cluster of CTAs per head (SDLLM_SELECT=cluster / single forces either
+  // wherever the cluster kernel applies: tuning and test aid).
+  const int cand = p.Lmax - p.b;
+  bool clustered = cand > 8192;
+  if (const char* e = getenv("SDLLM_SELECT")) clustered = e[0] == 'c';
+  if (clustered && cand >= 1 && cand <= SELC_CTAS * SELC_SLICE) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(SELC_CTAS, p.Hkv, p.B);
+    cfg.blockDim = dim3(SEL_THREADS);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = SELC_CTAS; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, select_topk_cluster_kernel, p);
+  }
   static size_t configured = 0;
   const size_t smem = ((size_t)p.smem_keys + p.smem_keys / 32 + 1) * 4;
   if (smem > configured) {

@@ -131,8 +131,10 @@ def test_batch_with_an_empty_cache_and_a_full_one():
 @pytest.mark.parametrize("policy", [
     dict(select=B.SELECT_PER_REGION_CEIL), dict(select=B.SELECT_PREFIX_ONLY), dict(pool=B.POOL_AVG),
 ])
-def test_policies(policy):
+def test_policies(policy, monkeypatch):
     cfg = _small("pol", "bf16", 4, 2, 128, 190, 96, retention=0.3, salient_frac=0.02)
+    _run_sequence_case(cfg, seed=5, block=1, **policy)
+    monkeypatch.setenv("SDLLM_SELECT", "cluster")        # two regions, each split over the CTAs of a cluster
     _run_sequence_case(cfg, seed=5, block=1, **policy)
 
 
@@ -155,6 +157,7 @@ def test_pool_windows(window):
     {"SDLLM_DUAL": "1", "SDLLM_SPLITS": "1"},             # small-footprint variant (two CTAs per SM)
     {"SDLLM_DUAL": "1", "SDLLM_SPLITS": "3"},
     {"SDLLM_KEY_TILE": "64", "SDLLM_SPLITS": "2"},        # 64-key tiles
+    {"SDLLM_SELECT": "cluster"},                          # top-k by a cluster of CTAs per head
 ])
 def test_alternative_launch_plans_agree_with_oracle(env, monkeypatch):
     """Every kernel family, tail placement, tile size and split count gives the same answers."""
@@ -179,7 +182,8 @@ def test_softmax_probability_saliency(cfg, block, env, monkeypatch):
     _run_sequence_case(cfg, seed=15, block=block, n_sparse=1, score=B.SCORE_PROB_MEAN)
 
 
-@pytest.mark.parametrize("env", [{}, {"SDLLM_LPT": "1"}, {"SDLLM_LPT": "1", "SDLLM_DUAL": "1", "SDLLM_SPLITS": "1"}])
+@pytest.mark.parametrize("env", [{}, {"SDLLM_LPT": "1"}, {"SDLLM_LPT": "1", "SDLLM_DUAL": "1", "SDLLM_SPLITS": "1"},
+                                 {"SDLLM_SELECT": "cluster"}])
 def test_ragged_batch(env, monkeypatch):
     import parity_util as U
     for k_, v_ in env.items():
@@ -196,8 +200,12 @@ def test_ragged_batch(env, monkeypatch):
     U.check_sparse_against_oracle(g, out, q2, kn, vn, "bf16")
 
 
-def test_select_topk_alone_heavy_ties_bit_exact():
-    """Plateaus of exactly equal scores (what max pooling produces) must resolve to the lowest positions."""
+@pytest.mark.parametrize("kernel", ["default", "cluster", "single"])
+def test_select_topk_alone_heavy_ties_bit_exact(kernel, monkeypatch):
+    """Plateaus of exactly equal scores (what max pooling produces) must resolve to the lowest positions. The selection
+    by one CTA per head and the one by a cluster of CTAs per head (long sequences) must both be exact."""
+    if kernel != "default":
+        monkeypatch.setenv("SDLLM_SELECT", kernel)
     rng = np.random.default_rng(8)
     for (Bn, Hkv, L, b, o, r) in [(2, 3, 300, 32, 100, 0.5), (1, 2, 2080, 32, 2048, 0.37), (1, 1, 40000, 32, 7, 0.25), (1, 1, 50000, 32, 49000, 0.6),
                                   (1, 2, 64, 32, 0, 0.5), (1, 2, 64, 32, 32, 0.99)]:
