@@ -414,10 +414,11 @@ __global__ void __launch_bounds__(256) compact_kv_kernel(const CompactParams p) 
 }  // namespace
 
 cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st) {
-  // Tens of thousands of candidates per head: a cluster of CTAs per head (SDLLM_SELECT=cluster / single forces either
-  // wherever the cluster kernel applies: tuning and test aid).
+  // Tens of thousands of candidates per head and few heads (all clusters resident at once): a cluster of CTAs per head;
+  // with many heads one CTA per head already fills the GPU and measured several times faster than clusters.
+  // SDLLM_SELECT=cluster / single forces either wherever the cluster kernel applies (tuning and test aid).
   const int cand = p.Lmax - p.b;
-  bool clustered = cand > 8192;
+  bool clustered = cand > 8192 && (long long)p.B * p.Hkv * SELC_CTAS <= kNumSMs;
   if (const char* e = getenv("SDLLM_SELECT")) clustered = e[0] == 'c';
   if (clustered && cand >= 1 && cand <= SELC_CTAS * SELC_SLICE) {
     cudaLaunchConfig_t cfg{};
