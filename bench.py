@@ -370,8 +370,10 @@ def run_ours(args):
         refresh_only()                              # every layer's cache exists before any reuse step runs
     stream.synchronize()
     d0 = caches[0].desc
-    launches_per_step = n_layers * (B.launch_count(d0, B.OP_REFRESH_SCORES) + B.launch_count(d0, B.OP_SELECT_TOPK) +
-                                    B.launch_count(d0, B.OP_COMPACT_KV) + reuse_steps * B.launch_count(d0, B.OP_SPARSE_BLOCK_ATTN))
+    refresh_launches = B.launch_count(d0, B.OP_REFRESH_SCORES) + B.launch_count(d0, B.OP_SELECT_TOPK) + B.launch_count(d0, B.OP_COMPACT_KV)
+    sparse_launches = reuse_steps * B.launch_count(d0, B.OP_SPARSE_BLOCK_ATTN)
+    launches_per_step = n_layers * ((refresh_launches if args.phase in ("all", "refresh") else 0) +
+                                    (sparse_launches if args.phase in ("all", "sparse") else 0))
     step_runner = make_runner({"all": one_step, "refresh": refresh_only, "sparse": sparse_only}[args.phase])
     sampler = ClockSampler(local) if rank == 0 else None
     sec = timed(step_runner, args.steps, max(args.warmup, 3))
