@@ -1094,6 +1094,14 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
   long long want = kNumSMs / units;
   if (want < 1) want = 1;
   if (const char* e = getenv("SDLLM_SPLITS")) { if (atoi(e) >= 1) want = atoi(e); }   // tuning aid
+  // Reuse step with replicated rows (few query rows per head, so a tile costs a softmax warp little): a CTA works
+  // best on about four 128-key tiles. With fewer, the set-up of the CTAs and the merge of their partials weigh more
+  // than the streaming they save (LLaDA-shaped layer, 6 tiles per head: 2 splits 11.5 us, 4 splits 12.5 us, 1 split
+  // 12.4 us; 18 tiles per head: 4 splits 17.6 us, 2 splits 20.0 us).
+  if (n2 > 0 && pl.rep > 1 && !pl.dual && !getenv("SDLLM_SPLITS")) {
+    const long long cap = ((n1_max + 127) / 128 + 1 + 3) / 4;
+    if (want > cap) want = cap;
+  }
   const int kt2 = n2 > 0 ? (n2 < 128 ? n2 : 128) : 0;
   pl.key_tile = 128;
   if (pl.rep <= 2 && (n1_max + 127) / 128 + (n2 > 0 ? 1 : 0) < want) pl.key_tile = 64;
