@@ -35,7 +35,7 @@ METRIC = "cached_kv_tokens_per_s_per_layer"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the sparse-attention kernel pair on this workload,
 # from the ncu capture summarised under profiles/ (None until a capture exists for the workload).
-NCU_TRAFFIC_BYTES = {"c2_llada": 11117312}
+NCU_TRAFFIC_BYTES = {"c2_llada": 11118080}
 
 
 def parse_args():
