@@ -54,6 +54,8 @@ def parse_args():
                          "dense: time the full-sequence dense step (cache_state 0) of every layer instead, on its own metric")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (0 = the workload's)")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
+    ap.add_argument("--tune", action="append", default=[], metavar="NAME=VALUE",
+                    help="override one decision of the library's launch planner (sdllm_tuning_set), e.g. --tune splits=4")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -228,6 +230,9 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     B.lib()
+    for item in args.tune:
+        name, _, val = item.partition("=")
+        B.tuning_set(name, int(val))
 
     cfg = workload_config(args)
     n_layers = args.layers or cfg.n_layers

@@ -39,7 +39,7 @@ typedef enum {
   SDLLM_ERR_UNSUPPORTED = 2, /* shape or mode outside what the kernels cover, or not an sm_100 device */
   SDLLM_ERR_WORKSPACE = 3,   /* workspace NULL or smaller than sdllm_workspace_bytes() */
   SDLLM_ERR_CUDA = 4,        /* a CUDA runtime call or launch failed */
-  SDLLM_ERR_TIMEOUT = 5      /* reserved: a bounded device-side wait gave up */
+  SDLLM_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up (sdllm_read_status) */
 } sdllm_status;
 
 typedef enum { SDLLM_F32 = 0, SDLLM_BF16 = 1 } sdllm_dtype;
@@ -105,7 +105,9 @@ const char* sdllm_status_string(sdllm_status status);
  * Returns 0 for an invalid description or when the op needs none. The workspace needs 256-byte alignment and the
  * caller zeroes ALL of it once after allocating it: its first 4 bytes are a status word (see sdllm_read_status) and
  * it holds completion counters that every call leaves at zero again; the rest is unspecified after a call. One
- * workspace may serve any number of calls that run one after another on the GPU, never two that overlap. */
+ * workspace may serve any number of calls that run one after another on the GPU, never two that overlap.
+ * After a call whose status word reads non-zero (SDLLM_ERR_TIMEOUT) zero the whole workspace again before reusing it:
+ * the status word is sticky, and the call that gave up may have left its counters anywhere. */
 size_t sdllm_workspace_bytes(const sdllm_desc* desc, int op);
 
 /* Host-only. Number of cache entries kept for a sequence of length seq_len whose block starts at block_off:
@@ -200,6 +202,25 @@ sdllm_status sdllm_dense_attn(const sdllm_desc* desc, const void* q, const int64
 sdllm_status sdllm_sparse_block_attn_static(const sdllm_desc* desc, const void* q_blk, const void* k_c, const void* v_c,
                                             const int32_t* kept_cnt, const void* k_blk, const void* v_blk, void* out,
                                             void* cuda_stream);
+
+/* Tuning and test aid; the paper has no counterpart. Overrides one decision of the launch planner, process-wide, until
+ * sdllm_tuning_reset(). The library never reads the environment: these overrides are the only hidden input of the
+ * planner, so sdllm_workspace_bytes, sdllm_launch_count and the launches agree as long as no override changes between
+ * them. Host-only, thread-safe; takes effect for calls made afterwards. `name` is a NUL-terminated host string:
+ *   "splits"      > 0: key splits per (sequence, KV head) of the attention calls
+ *   "kernel"      attention kernel family: 0 automatic, 1 cp.async, 2 tcgen05 with the queries on the accumulator rows,
+ *                 3 tcgen05 with the keys on the accumulator rows (only where that kernel covers the shape)
+ *   "pdl"         0: no programmatic dependent launch     "early_loads" 0: no loads ahead of the grid dependency
+ *   "cluster", "fused_tail", "dual", "key_tile", "lpt", "stages"   plan details of the tcgen05 kernels
+ *   "select"      top-k kernel: 1 one CTA per head, 2 one cluster per head
+ *   "wait_cycles" limit, in SM clock cycles, of every abortable device-side wait (default 400 000 000, ~0.2 s). A limit
+ *                 of a few cycles makes the first wait that is not already satisfied give up: the call still returns,
+ *                 its outputs are invalid and sdllm_read_status reports SDLLM_ERR_TIMEOUT (how the tests exercise
+ *                 that path without hanging anything).
+ *   "debug"       1: print the CUDA error behind an SDLLM_ERR_CUDA to stderr
+ * Returns SDLLM_ERR_INVALID_ARG for an unknown name. */
+sdllm_status sdllm_tuning_set(const char* name, int64_t value);
+void sdllm_tuning_reset(void);
 
 #ifdef __cplusplus
 }

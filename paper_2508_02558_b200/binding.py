@@ -23,7 +23,7 @@ OP_REFRESH_SCORES, OP_SELECT_TOPK, OP_COMPACT_KV, OP_SPARSE_BLOCK_ATTN, OP_DENSE
 EXPORTS = ("sdllm_version", "sdllm_status_string", "sdllm_workspace_bytes", "sdllm_keep_count", "sdllm_cache_state", "sdllm_launch_count",
            "sdllm_read_status",
            "sdllm_refresh_scores", "sdllm_select_topk", "sdllm_compact_kv", "sdllm_sparse_block_attn",
-           "sdllm_sparse_block_attn_static", "sdllm_dense_attn")
+           "sdllm_sparse_block_attn_static", "sdllm_dense_attn", "sdllm_tuning_set", "sdllm_tuning_reset")
 
 
 class Desc(ctypes.Structure):
@@ -83,6 +83,10 @@ def lib() -> ctypes.CDLL:
         L.sdllm_dense_attn.restype = ctypes.c_int
         L.sdllm_dense_attn.argtypes = [dp, vp, ctypes.POINTER(ctypes.c_int64), vp, vp, i32p, vp, ctypes.POINTER(ctypes.c_int64), vp, vp,
                                        ctypes.c_size_t, vp]
+        L.sdllm_tuning_set.restype = ctypes.c_int
+        L.sdllm_tuning_set.argtypes = [ctypes.c_char_p, ctypes.c_int64]
+        L.sdllm_tuning_reset.restype = None
+        L.sdllm_tuning_reset.argtypes = []
         _lib = L
     return _lib
 
@@ -216,3 +220,12 @@ def dense_attn(desc: Desc, q, k, v, seq_len, out, lse, workspace, stream=None):
     os_ = (ctypes.c_int64 * 3)(*(out.stride()[:3] if out is not None else (0, 0, 0)))
     _check(lib().sdllm_dense_attn(ctypes.byref(desc), _ptr(q), qs, _ptr(k), _ptr(v), _ptr(seq_len), _ptr(out), os_, _ptr(lse),
                                   _ptr(workspace), _nbytes(workspace), _stream(stream)), "sdllm_dense_attn")
+
+
+def tuning_set(name: str, value: int):
+    """Override one decision of the launch planner (tuning and test aid) until tuning_reset()."""
+    _check(lib().sdllm_tuning_set(name.encode(), int(value)), f"sdllm_tuning_set({name})")
+
+
+def tuning_reset():
+    lib().sdllm_tuning_reset()

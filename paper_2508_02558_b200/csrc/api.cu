@@ -6,6 +6,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "tuning.cuh"
 
 using namespace sdllm;
 
@@ -48,6 +49,16 @@ sdllm_status check_desc(const sdllm_desc* d) {
   return SDLLM_OK;
 }
 
+// Pointer checks of the reuse step (both entry points).
+sdllm_status check_sparse_args(const sdllm_desc* d, const void* q_blk, const void* k_c, const void* v_c, const int32_t* kept_cnt,
+                               const void* k_blk, const void* v_blk, const void* out) {
+  if (!q_blk || !k_blk || !v_blk || !out || !kept_cnt) return SDLLM_ERR_INVALID_ARG;
+  if (d->n_keep_max > 0 && (!k_c || !v_c)) return SDLLM_ERR_INVALID_ARG;
+  if (!aligned16(q_blk) || !aligned16(k_c) || !aligned16(v_c) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out))
+    return SDLLM_ERR_INVALID_ARG;
+  return SDLLM_OK;
+}
+
 // The kernels are built for sm_100a only.
 sdllm_status check_device() {
   int dev = 0, major = 0;
@@ -56,11 +67,10 @@ sdllm_status check_device() {
   return major == 10 ? SDLLM_OK : SDLLM_ERR_UNSUPPORTED;
 }
 
-// SDLLM_DEBUG=1 prints the CUDA error behind an SDLLM_ERR_CUDA to stderr.
+// With the tuning field "debug" set, the CUDA error behind an SDLLM_ERR_CUDA is printed to stderr.
 bool cuda_failed(cudaError_t e, const char* what) {
   if (e == cudaSuccess) return false;
-  const char* dbg = getenv("SDLLM_DEBUG");
-  if (dbg && dbg[0] == '1') fprintf(stderr, "libsdllm: %s: %s\n", what, cudaGetErrorString(e));
+  if (tuning().debug != 0) fprintf(stderr, "libsdllm: %s: %s\n", what, cudaGetErrorString(e));
   (void)cudaGetLastError();
   return true;
 }
@@ -97,7 +107,8 @@ AttnPlan plan_for(const sdllm_desc* d, int op) {
   const int G = d->n_q_heads / d->n_kv_heads;
   const bool refresh = op == SDLLM_OP_REFRESH_SCORES;
   return plan_attention(d->dtype, d->head_dim, G * d->block_len, d->block_len, d->batch, d->n_kv_heads,
-                        refresh ? d->seq_len_max : d->n_keep_max, refresh ? 0 : d->block_len);
+                        refresh ? d->seq_len_max : d->n_keep_max, refresh ? 0 : d->block_len,
+                        refresh && d->score == SDLLM_SCORE_PROB_MEAN);
 }
 
 void fill_common(AttnParams& p, const sdllm_desc* d, const AttnPlan& pl) {
@@ -106,6 +117,7 @@ void fill_common(AttnParams& p, const sdllm_desc* d, const AttnPlan& pl) {
   p.splits_total = pl.splits * pl.cluster;
   p.scale = scale_of(d);
   p.scale_log2 = p.scale * kLog2e;
+  p.wait_cycles = tuning().wait_cycles;
   for (int i = 0; i < 3; ++i) { p.q_stride[i] = d->q_stride[i]; p.o_stride[i] = d->o_stride[i]; }
 }
 
@@ -118,7 +130,6 @@ bool dense_supported(const sdllm_desc* d) {
 
 // Built-in scratch of sdllm_sparse_block_attn_static: lives in the library image, one copy per GPU that loads it.
 constexpr size_t kStaticScratchBytes = (size_t)8 << 20;
-constexpr int kMaxDevices = 64;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 std::mutex g_static_mutex;
 void* g_static_scratch_ptr[kMaxDevices] = {};      // device address of g_static_scratch on each device, once looked up
@@ -143,6 +154,12 @@ sdllm_status static_scratch_address(void** out) {
 extern "C" {
 
 int sdllm_version(void) { return SDLLM_VERSION; }
+
+sdllm_status sdllm_tuning_set(const char* name, int64_t value) {
+  return tuning_set(name, (long long)value) ? SDLLM_OK : SDLLM_ERR_INVALID_ARG;
+}
+
+void sdllm_tuning_reset(void) { tuning_reset(); }
 
 const char* sdllm_status_string(sdllm_status s) {
   switch (s) {
@@ -186,6 +203,7 @@ int32_t sdllm_launch_count(const sdllm_desc* d, int op) {
   const bool refresh = op == SDLLM_OP_REFRESH_SCORES;
   const AttnPlan pl = plan_for(d, op);
   const int M = d->n_q_heads / d->n_kv_heads * d->block_len;
+  if (pl.kind == 3) return 1;       // the key splits merge, and the scores are pooled, inside the one launch
   if (pl.kind == 2) {
     const int n1 = refresh ? d->seq_len_max : d->n_keep_max;
     if (refresh && d->score == SDLLM_SCORE_PROB_MEAN)     // attention pass (+ its merge) and saliency pass (+ its pooling)
@@ -306,10 +324,7 @@ sdllm_status sdllm_sparse_block_attn(const sdllm_desc* d, const void* q_blk, con
                                      const void* k_blk, const void* v_blk, void* out, void* ws, size_t ws_bytes, void* cuda_stream) {
   sdllm_status st = check_desc(d);
   if (st != SDLLM_OK) return st;
-  if (!q_blk || !k_blk || !v_blk || !out || !kept_cnt) return SDLLM_ERR_INVALID_ARG;
-  if (d->n_keep_max > 0 && (!k_c || !v_c)) return SDLLM_ERR_INVALID_ARG;
-  if (!aligned16(q_blk) || !aligned16(k_c) || !aligned16(v_c) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out))
-    return SDLLM_ERR_INVALID_ARG;
+  if ((st = check_sparse_args(d, q_blk, k_c, v_c, kept_cnt, k_blk, v_blk, out)) != SDLLM_OK) return st;
   const AttnPlan pl = plan_for(d, SDLLM_OP_SPARSE_BLOCK_ATTN);
   const WsLayout w = attn_ws(d, pl, false);
   if (w.total > 0 && (ws == nullptr || ws_bytes < w.total || (reinterpret_cast<uintptr_t>(ws) & 255u))) return SDLLM_ERR_WORKSPACE;
@@ -364,6 +379,7 @@ sdllm_status sdllm_sparse_block_attn_static(const sdllm_desc* d, const void* q_b
                                             const int32_t* kept_cnt, const void* k_blk, const void* v_blk, void* out, void* cuda_stream) {
   sdllm_status st = check_desc(d);
   if (st != SDLLM_OK) return st;
+  if ((st = check_sparse_args(d, q_blk, k_c, v_c, kept_cnt, k_blk, v_blk, out)) != SDLLM_OK) return st;
   const WsLayout w = attn_ws(d, plan_for(d, SDLLM_OP_SPARSE_BLOCK_ATTN), false);
   if (w.total > kStaticScratchBytes) return SDLLM_ERR_WORKSPACE;       // this shape needs more than the built-in scratch
   if ((st = check_device()) != SDLLM_OK) return st;

@@ -8,9 +8,9 @@
 // "A <- MatMul(qbar, K_f^T)"), so the L x b probability matrix and the logit matrix never exist in memory.
 //
 // bf16: QK^T and PV run on the tensor cores (mma.sync m16n8k16, fp32 accumulate); fp32: plain FMA.
-#include <stdlib.h>
 
 #include "attn_device.cuh"
+#include "tuning.cuh"
 
 namespace sdllm {
 using namespace dev;
@@ -549,13 +549,10 @@ __global__ void __launch_bounds__(256) merge_pool_kernel(const MergeParams p) {
   p.pooled[idx] = outv;
 }
 
-// Raise the dynamic shared-memory limit of a kernel once per (kernel, size high-water mark).
+// Raise the dynamic shared-memory limit of a kernel once per (kernel, device, size high-water mark).
 template <typename K>
-cudaError_t set_smem(K kernel, size_t bytes, size_t* configured) {
-  if (bytes <= *configured) return cudaSuccess;
-  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-  if (e == cudaSuccess) *configured = bytes;
-  return e;
+cudaError_t set_smem(K kernel, size_t bytes, SmemConfig* configured) {
+  return configure_smem(reinterpret_cast<const void*>(kernel), bytes, *configured, false);
 }
 
 template <int D, int STAGES>
@@ -565,7 +562,7 @@ cudaError_t launch_bf16(const AttnParams& p, const AttnPlan& plan, cudaStream_t 
 #define SDLLM_LAUNCH(NT, QR)                                                                          \
   do {                                                                                                \
     auto kern = attn_partial_bf16_kernel<D, STAGES, NT, QR>;                                          \
-    static size_t configured = 0;                                                                     \
+    static SmemConfig configured;                                                                     \
     if ((e = set_smem(kern, plan.smem_bytes, &configured)) != cudaSuccess) return e;                  \
     kern<<<grid, block, plan.smem_bytes, st>>>(p, plan.m_warps, plan.c_warps);                        \
   } while (0)
@@ -591,7 +588,7 @@ size_t attn_legacy_smem_bytes(int dtype, int D, const AttnPlan& plan) {
   return (32 * rs + 32 * (F32_KT + 1) + D + 2 * 2 * F32_KT * rs) * 4;
 }
 
-AttnPlan plan_attention_legacy(int dtype, int D, int M, int B, int Hkv, int n_keys_max) {
+AttnPlan plan_attention_legacy(int dtype, int D, int M, int B, int Hkv, int n_keys_max, const Tuning& tn) {
   AttnPlan pl{};
   pl.cluster = 1; pl.warp_keys = 32; pl.tma = false;
   const long long base = (long long)B * Hkv;
@@ -612,10 +609,11 @@ AttnPlan plan_attention_legacy(int dtype, int D, int M, int B, int Hkv, int n_ke
   }
   pl.smem_bytes = attn_legacy_smem_bytes(dtype, D, pl);
   const int n_tiles = (n_keys_max + pl.key_tile - 1) / pl.key_tile;
-  long long want = (kNumSMs + base - 1) / base;
+  const int sms = sm_count();
+  long long want = (sms + base - 1) / base;
   if (dtype != SDLLM_BF16) want = (want + pl.m_warps - 1) / pl.m_warps;
   long long splits = want < 1 ? 1 : want;
-  if (const char* e = getenv("SDLLM_SPLITS")) { if (atoi(e) >= 1) splits = atoi(e); }   // tuning aid
+  if (tn.splits > 0) splits = tn.splits;
   if (splits > n_tiles) splits = n_tiles;
   if (splits > kMaxSplits) splits = kMaxSplits;
   if (splits < 1) splits = 1;
@@ -636,7 +634,7 @@ cudaError_t launch_attn_legacy(const AttnParams& p, const AttnPlan& plan, int dt
   }
   const dim3 grid(plan.splits * plan.m_warps, p.Hkv, p.B), block(256);
   cudaError_t e;
-  static size_t configured128 = 0, configured64 = 0;
+  static SmemConfig configured128, configured64;
   if (D == 128) {
     if ((e = set_smem(attn_partial_f32_kernel<128>, plan.smem_bytes, &configured128)) != cudaSuccess) return e;
     attn_partial_f32_kernel<128><<<grid, block, plan.smem_bytes, st>>>(p, plan.m_warps);

@@ -13,10 +13,10 @@
 // Every wait on an mbarrier is bounded; on expiry the CTA sets an abort flag, records a code in the status word and
 // runs to its end (freeing its TMEM); the outputs of that call are then invalid.
 #include <cuda.h>
-#include <stdlib.h>
 #include <string.h>
 
 #include "attn_device.cuh"
+#include "tuning.cuh"
 #include "umma_host.cuh"
 
 namespace sdllm {
@@ -38,6 +38,7 @@ struct DenseParams {
   int B, Hq, G, L;
   float scale_log2;         // softmax scale * log2(e)
   int64_t o_stride[3];
+  long long wait_cycles;    // limit of every abortable mbarrier wait
 };
 
 #include "umma_ptx.cuh"
@@ -115,10 +116,10 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
         const int s = j % NS;
         const uint32_t ph = ((j / NS) - 1) & 1;
         const uint32_t kdst = smem_u32(stage0 + (size_t)s * 2 * TILE), vdst = kdst + TILE;
-        if (j >= NS && !wait_bar(BAR(EMPTY_K + s), ph, abort_flag, p.status, 21)) { ok = false; break; }
+        if (j >= NS && !wait_bar(BAR(EMPTY_K + s), ph, abort_flag, p.status, 21, p.wait_cycles)) { ok = false; break; }
         mbar_expect_tx(BAR(FULL_K + s), (uint32_t)TILE);
         for (int hh = 0; hh < H; ++hh) tma_load_4d(kdst + hh * HALF, &tm.k, BAR(FULL_K + s), hh * 64, j * KT, g, bi);
-        if (j >= NS && !wait_bar(BAR(EMPTY_V + s), ph, abort_flag, p.status, 22)) {
+        if (j >= NS && !wait_bar(BAR(EMPTY_V + s), ph, abort_flag, p.status, 22, p.wait_cycles)) {
           drain_bar(BAR(FULL_K + s), (j / NS) & 1);                 // the K half of this slot is already on its way
           ok = false; break;
         }
@@ -139,7 +140,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
     if (lane == 0) {
       const uint32_t idesc_pv = instr_desc(D, true);
       const uint32_t qsm = smem_u32(q_s);
-      bool ok = wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 23);
+      bool ok = wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 23, p.wait_cycles);
       // S_t = Q_t K_j^T into the S region of query tile t
       auto issue_s = [&](int t, int j) {
         const uint32_t ksm = smem_u32(stage0 + (size_t)(j % NS) * 2 * TILE);
@@ -155,8 +156,8 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
       // O_t += P_t V_j once the softmax warps of query tile t have written P_t; `release` frees the V slot afterwards
       auto issue_pv = [&](int t, int j, bool release) -> bool {
         const int s = j % NS;
-        if (!wait_bar(BAR(P_FULL + t), j & 1, abort_flag, p.status, 24)) return false;
-        if (!wait_bar(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 25)) return false;
+        if (!wait_bar(BAR(P_FULL + t), j & 1, abort_flag, p.status, 24, p.wait_cycles)) return false;
+        if (!wait_bar(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 25, p.wait_cycles)) return false;
         tc_fence_after();
         const uint32_t vsm = smem_u32(stage0 + (size_t)s * 2 * TILE) + TILE;
         const uint32_t a_t = tmem_base + S_COL0 + (uint32_t)t * T_STRIDE;
@@ -170,7 +171,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
       };
       for (int j = 0; j < nt && ok; ++j) {
         const int s = j % NS;
-        if (!wait_bar(BAR(FULL_K + s), (j / NS) & 1, abort_flag, p.status, 26)) { ok = false; break; }
+        if (!wait_bar(BAR(FULL_K + s), (j / NS) & 1, abort_flag, p.status, 26, p.wait_cycles)) { ok = false; break; }
         tc_fence_after();
         issue_s(0, j);
         if (act1) {
@@ -199,7 +200,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
       bool ok = true;
       for (int j = 0; j < nt && ok; ++j) {
         const int nv = tile_nv(j);
-        if (!wait_bar_warp(BAR(S_FULL + t), j & 1, abort_flag, p.status, 27)) { ok = false; break; }
+        if (!wait_bar_warp(BAR(S_FULL + t), j & 1, abort_flag, p.status, 27, p.wait_cycles)) { ok = false; break; }
         tc_fence_after();
         uint32_t sv[4][32];
 #pragma unroll
@@ -231,7 +232,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
         }
         if (j > 0 && __any_sync(0xffffffffu, grow)) {
           // every PV of this query tile issued so far must have landed before its rows are rewritten
-          if (!wait_bar_warp(BAR(PV_DONE + t), (j - 1) & 1, abort_flag, p.status, 28)) { ok = false; break; }
+          if (!wait_bar_warp(BAR(PV_DONE + t), (j - 1) & 1, abort_flag, p.status, 28, p.wait_cycles)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll 1
           for (int c = 0; c < D / 16; ++c) {
@@ -265,7 +266,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
         const int n_mma = (nv + 15) & ~15;
         if (t == 0 && nv < n_mma) {
           const int s = j % NS;
-          if (!wait_bar_warp(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 29)) { ok = false; break; }
+          if (!wait_bar_warp(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 29, p.wait_cycles)) { ok = false; break; }
           unsigned char* vs = stage0 + (size_t)s * 2 * TILE + TILE;
           const int nz = (n_mma - nv) * H * 8;           // 16-byte chunks to clear
           for (int i = (warp - 2) * 32 + lane; i < nz; i += 128) {
@@ -280,7 +281,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1) dense_attn_bf16_kernel(const __
         if (lane == 0) mbar_arrive(BAR(P_FULL + t));
       }
       // ---- the finished row: TMEM -> registers -> normalise -> bf16 -> global memory ----
-      if (ok) ok = wait_bar_warp(BAR(PV_DONE + t), (nt - 1) & 1, abort_flag, p.status, 30);
+      if (ok) ok = wait_bar_warp(BAR(PV_DONE + t), (nt - 1) & 1, abort_flag, p.status, 30, p.wait_cycles);
       tc_fence_after();
       const int r_glob = row00 + t * 128 + row;
       if (ok) {
@@ -327,14 +328,10 @@ size_t dense_smem_bytes(int D) {
 template <int D>
 cudaError_t launch_dense_d(const DenseMaps& tm, const DenseParams& p, int nqb, cudaStream_t st) {
   auto kern = dense_attn_bf16_kernel<D>;
-  static bool configured = false;
+  static SmemConfig configured;
   const size_t smem = dense_smem_bytes(D);
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    (void)cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    configured = true;
-  }
+  const cudaError_t ce = configure_smem(reinterpret_cast<const void*>(kern), smem, configured, true);
+  if (ce != cudaSuccess) return ce;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((nqb + 1) / 2, p.Hq, p.B);
   cfg.blockDim = dim3(DN_THREADS);
@@ -342,8 +339,7 @@ cudaError_t launch_dense_d(const DenseMaps& tm, const DenseParams& p, int nqb, c
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   int na = 0;
-  const char* e = getenv("SDLLM_PDL");       // SDLLM_PDL=0 turns programmatic dependent launch off (tuning and test aid)
-  if (!(e && e[0] == '0')) {
+  if (tuning().pdl != 0) {
     attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[na].val.programmaticStreamSerializationAllowed = 1;
     ++na;
@@ -368,6 +364,7 @@ cudaError_t launch_dense_pair(const void* q, const int64_t* q_stride, const void
   p.seq_len = seq_len; p.out = out; p.lse = lse; p.status = status;
   p.B = B; p.Hq = Hq; p.G = Hq / Hkv; p.L = L;
   p.scale_log2 = scale * kLog2e;
+  p.wait_cycles = tuning().wait_cycles;
   for (int i = 0; i < 3; ++i) p.o_stride[i] = o_stride[i];
   const int nqb = (L + 127) / 128;
   return D == 128 ? launch_dense_d<128>(tm, p, nqb, st) : launch_dense_d<64>(tm, p, nqb, st);

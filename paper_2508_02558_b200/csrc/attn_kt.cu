@@ -1,0 +1,721 @@
+// bf16 block-query attention with the KEYS on the accumulator rows (tcgen05, sm_100a), for heads with few query rows.
+//
+// When a KV head has N = b*G <= 64 query rows (multi-head attention with a block of 32: N = 32), putting the queries on
+// the 128 accumulator rows wastes three quarters of every MMA and forces the rows to be replicated and merged again.
+// Here the score tile is transposed instead:
+//     S^T [128 keys x N queries] = K_tile [128 x D] . Q^T            (A = K tile, B = Q, both K-major in shared memory)
+//     O^T [D x N queries]       += V_tile^T [D x keys] . P^T [keys x N]   (A = V tile read MN-major, B = P^T MN-major)
+// so one thread of the four softmax warps owns one KEY of the tile (a TMEM lane) and sees that key's logits against all
+// N queries. What this buys:
+//   * nothing is replicated and nothing is merged inside the CTA; both MMAs are N/128 of the row-major ones;
+//   * the mean-query saliency of Algorithm 1 ("qbar <- Mean(Q_b)", "A <- MatMul(qbar, K_f^T)") is, by linearity, the
+//     mean of the key's N logits: the thread that owns the key already holds them, no separate pass over K;
+//   * the finished O^T has one head dimension per thread and N columns: key splits are merged column by column.
+// The softmax needs one reference value per query (column) that all keys share. It is taken once, from the column
+// maxima of the CTA's first tile (warp reductions and a shared-memory max), and afterwards only checked: a tile
+// whose logits exceed a reference by more than 2^8 makes the softmax threads raise the references and rescale O^T and
+// the partial sums (rare). P is bf16, whose exponent range is that of fp32, so a reference within 2^8 of the true
+// maximum loses nothing.
+//
+// The key axis is  [source 1 rows 0..n1) ++ [source 2 rows 0..n2)  cut into groups of 32 rows; a CTA takes a contiguous
+// range of groups and walks it in tiles of up to four groups (128 keys), so a tile may mix the two sources.
+//   refresh step : source 1 = the full K/V of the sequence, no source 2;
+//   reuse step   : source 1 = the compacted cache, source 2 = the block's fresh rows (Algorithm 3, Concat(K_c, K_n)).
+// The S key splits of a (sequence, KV head) are the CTAs of one thread-block cluster. Each split pushes, for every
+// query column, its un-normalised O^T column and its (reference, sum) pair into the shared memory of the CTA that owns
+// the column (st.shared::cluster); after ONE cluster barrier every CTA merges and stores the columns it owns and, at
+// the refresh step, pools its share of the head's saliency (Algorithm 1, MaxPool1D). Nothing goes through global
+// memory, there is no counter and no second launch.
+// Warp roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-5 softmax.
+// With N <= 32 a CTA needs about 110 KB of shared memory and 128 TMEM columns, so two CTAs share an SM and, with
+// programmatic dependent launch, the next call's CTAs load their first tiles while this call's CTAs finish.
+//
+// Every wait on an mbarrier is bounded. On expiry the thread sets an abort flag that all other waits poll, records a
+// code in the status word and the CTA runs to its end, still taking part in the cluster barriers (no peer is left
+// waiting) and freeing its TMEM; the outputs of that call are then invalid.
+#include <cuda.h>
+#include <string.h>
+
+#include "attn_device.cuh"
+#include "tuning.cuh"
+#include "umma_host.cuh"
+
+namespace sdllm {
+using namespace dev;
+namespace {
+
+constexpr int KT_THREADS = 192;
+constexpr int KT_MAX_STAGES = 3;
+constexpr int KT_CTRL = 4096;            // control block: barriers, flags, references, sums, received (reference, sum) pairs
+
+struct KtMaps {
+  CUtensorMap q, k1, v1, k2, v2;
+};
+
+struct KtParams {
+  AttnParams a;
+  int N;             // query columns of a KV head (b * G)
+  int S;             // key splits of a unit = CTAs of its cluster (1..8)
+  int NS;            // ring slots (128-key K tile + V tile each)
+  int PB;            // P^T buffers (1 or 2)
+  int QL;            // query columns a CTA owns in the merge: ceil(N / S)
+  int gr2;           // rows of a source-2 box: min(32, n2)
+  int early_src1;    // 1: source 1 and its count are older than every kernel that may still run (reuse step)
+  long long wait_cycles;   // limit of every abortable mbarrier wait
+};
+
+#include "umma_ptx.cuh"
+
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed;\n" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release;\n" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire;\n" ::: "memory"); }
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;\n" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void st_cluster_f2(uint32_t addr, float x, float y) {
+  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};\n" ::"r"(addr), "f"(x), "f"(y) : "memory");
+}
+__device__ __forceinline__ float warp_max_f32(float v) {
+  float r;
+  asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;\n" : "=f"(r) : "f"(v));
+  return r;
+}
+// barrier of the 128 softmax threads that also ORs a predicate over them
+__device__ __forceinline__ bool softmax_barrier_or(bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.or.pred p, 1, 128, q;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(r) : "r"((uint32_t)pred) : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 1, 128;\n" ::: "memory"); }
+
+// order-preserving fp32 <-> u32 (larger float <=> larger code), for the shared-memory max of the references
+__device__ __forceinline__ uint32_t f2ord(float x) {
+  const uint32_t u = __float_as_uint(x);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ord2f(uint32_t k) { return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k); }
+
+// Instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B, M = 128, N = n; A and B K-major or MN-major.
+__device__ __forceinline__ uint32_t kt_idesc(int n, bool a_mn, bool b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
+         ((128u >> 4) << 24);
+}
+
+// One group of 32 key rows: where it comes from and how many of its rows are real keys.
+struct Group {
+  int src1;     // 1: source 1, 0: source 2
+  int row0;     // first row inside its source
+  int nv;       // valid rows, 1..32
+};
+__device__ __forceinline__ Group group_of(int gi, int g1, int n1, int n2) {
+  Group x;
+  if (gi < g1) { x.src1 = 1; x.row0 = gi * 32; x.nv = min(n1 - x.row0, 32); }
+  else { x.src1 = 0; x.row0 = (gi - g1) * 32; x.nv = min(n2 - x.row0, 32); }
+  return x;
+}
+
+// Importance of one absolute position: Algorithm 1, MaxPool1D(A, kernel_size = s, padding = s/2) over the candidate
+// axis Concat(prefix, suffix) (AvgPool for the ablation); block positions and padding get -inf. `a` is the raw
+// saliency by absolute position in global memory, written by other CTAs during this launch (read through L2).
+__device__ __forceinline__ float kt_pool_at(const AttnParams& p, const float* a, int L, int o_in, int pos) {
+  const int b = p.b;
+  const int o = min(max(o_in, 0), max(L - b, 0));
+  if (pos >= L || (pos >= o && pos < o + b)) return -INFINITY;
+  const int C = max(L - b, 0), w = (p.window - 1) / 2;
+  const int c = pos < o ? pos : pos - b;
+  int lo = 0, hi = C;
+  if (p.per_region) { if (c < o) hi = o; else lo = o; }
+  float mx = -INFINITY, sum = 0.f;
+  for (int t = c - w; t <= c + w; ++t) {
+    if (t < lo || t >= hi) continue;
+    const float x = __ldcg(a + (t < o ? t : t + b));
+    mx = fmaxf(mx, x);
+    sum += x;
+  }
+  return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
+}
+
+template <int D, int NCH>
+__global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(const __grid_constant__ KtMaps tm, const KtParams kp) {
+  constexpr int H = D / 64;                  // 128-byte column halves of a K/V row
+  constexpr int NP = NCH * 32;               // query columns padded to the softmax chunking
+  constexpr int HALF = 128 * 128;            // bytes of one 64-column half of a 128-key tile
+  constexpr int KV_BYTES = H * HALF;         // one K (or V) tile
+  constexpr int SLOT = 2 * KV_BYTES;
+  constexpr int PBUF = 128 * 128;            // one P^T buffer: 128 key rows of 64 bf16
+  constexpr uint32_t O_COL = 2 * NP;         // TMEM columns: two S^T buffers of NP, then O^T (64 columns)
+  constexpr uint32_t TMEM_COLS = (2 * NP + 64 <= 128) ? 128 : 256;
+  const AttnParams& p = kp.a;
+  extern __shared__ unsigned char smem_raw[];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int NS = kp.NS, S = kp.S, N = kp.N;
+  const int bi = blockIdx.z, g = blockIdx.y, split = blockIdx.x;
+  const int n2 = p.n2;
+  const long long wlim = kp.wait_cycles;
+
+  // ---- shared memory carve-up (1024-byte aligned for the 128-byte swizzle; identical in every CTA of the cluster) ----
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  unsigned char* smem = smem_raw + (((raw_addr + 1023u) & ~1023u) - raw_addr);
+  const uint32_t bars = smem_u32(smem);
+  auto BAR = [&](int i) { return bars + 8u * (uint32_t)i; };
+  constexpr int Q_FULL = 0, FULL_K = 1, FULL_V = 1 + KT_MAX_STAGES, EMPTY_K = 1 + 2 * KT_MAX_STAGES, EMPTY_V = 1 + 3 * KT_MAX_STAGES;
+  constexpr int S_FULL = 1 + 4 * KT_MAX_STAGES, P_FULL = S_FULL + 2, PV_DONE = S_FULL + 4, DRAIN = S_FULL + 6;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 256);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 260);
+  uint32_t* m_enc = reinterpret_cast<uint32_t*>(smem + 512);        // [64] references (log2 units), order-preserving codes
+  uint32_t* m_old = reinterpret_cast<uint32_t*>(smem + 768);        // [64] references before a raise
+  float* l_tot = reinterpret_cast<float*>(smem + 1024);             // [64] sums of this split
+  float* alpha_s = reinterpret_cast<float*>(smem + 1280);           // [64] rescale factors of a raise
+  float* l_w = reinterpret_cast<float*>(smem + 1536);               // [4][64] per-warp sums
+  float2* ml_recv = reinterpret_cast<float2*>(smem + 2560);         // [S][QL] (reference, sum) pairs pushed by the splits
+  unsigned char* q_s = smem + KT_CTRL;                              // [H][NP rows][128 B]
+  unsigned char* p_s = q_s + H * NP * 128;                          // [PB][128 key rows][128 B]
+  unsigned char* ring = p_s + kp.PB * PBUF;                         // [NS][K tile | V tile]
+  float* recv = reinterpret_cast<float*>(ring + (size_t)NS * SLOT); // [S][QL][D] un-normalised O^T columns pushed by the splits
+
+  if (tid == 0) {                        // the descriptors live in the kernel parameters: fetch them while the CTA sets up
+    prefetch_tmap(&tm.k1); prefetch_tmap(&tm.v1);
+    if (n2 > 0) { prefetch_tmap(&tm.k2); prefetch_tmap(&tm.v2); }
+    prefetch_tmap(&tm.q);
+    mbar_init(BAR(Q_FULL), 1);
+    for (int s = 0; s < KT_MAX_STAGES; ++s) {
+      mbar_init(BAR(FULL_K + s), 1);
+      mbar_init(BAR(FULL_V + s), 1);
+      mbar_init(BAR(EMPTY_K + s), 1);
+      mbar_init(BAR(EMPTY_V + s), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(BAR(S_FULL + i), 1);
+      mbar_init(BAR(P_FULL + i), 4);
+      mbar_init(BAR(PV_DONE + i), 1);
+    }
+    mbar_init(BAR(DRAIN), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  if (tid >= 64 && tid < 128) m_enc[tid - 64] = f2ord(-INFINITY);
+  // query rows past N (N not a multiple of 32) take part in the MMAs: they must be finite
+  if (N < NP)
+    for (int i = tid; i < H * (NP - N) * 8; i += KT_THREADS) {
+      const int h = i / ((NP - N) * 8), r = i % ((NP - N) * 8);
+      reinterpret_cast<uint4*>(q_s + h * NP * 128 + N * 128)[r] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  if (warp == 1) {                       // the MMA warp owns the tensor memory
+    tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+    tmem_relinquish();
+  }
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // The next kernel in the stream may start its own set-up now; before it touches anything this kernel writes it
+  // waits for this grid to complete (griddepcontrol.wait below, in that kernel).
+  grid_launch_dependents();
+  if (S > 1) cluster_arrive_relaxed();   // phase 1 of the cluster barrier: "this CTA runs"; waited for before the pushes
+
+  // ---- this CTA's share of the key axis, in groups of 32 rows ----
+  // The count of source 1 is read before the grid dependency only at the reuse step (older than any running kernel).
+  int n1 = 0, g1 = 0, gb = 0, ge = 0, T = 0;
+  auto read_counts = [&]() {
+    n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
+    n1 = min(max(n1, 0), p.n1_max);
+    g1 = (n1 + 31) >> 5;
+    const int gt = g1 + ((n2 + 31) >> 5);
+    gb = (int)(((long long)split * gt) / S);
+    ge = (int)(((long long)(split + 1) * gt) / S);
+    T = (ge - gb + 3) >> 2;
+  };
+  if (kp.early_src1) read_counts();
+  // Everything but the first loads of the producer lane comes after the kernels in front of this one: the other
+  // threads read the counts, write global memory, or depend on Q.
+  if (tid != 0) {
+    grid_dependency_wait();
+    if (!kp.early_src1) read_counts();
+  }
+
+  float l_acc[NP];                       // softmax warps: this key row's share of every column's sum
+#pragma unroll
+  for (int c = 0; c < NP; ++c) l_acc[c] = 0.f;
+  bool dead = false;                     // softmax warps: a wait gave up; the warp keeps meeting the others at every barrier
+
+  if (warp == 0) {
+    // ======================================= TMA producer =======================================
+    if (lane == 0) {
+      bool dep = false, ok = true;
+      int k_issued = 0, v_issued = 0;    // tiles whose K / V loads are on their way
+      auto dependency = [&]() {          // everything loaded from here on may have been written by the previous kernels
+        if (dep) return;
+        grid_dependency_wait();
+        dep = true;
+        if (!kp.early_src1) read_counts();
+        mbar_expect_tx(BAR(Q_FULL), (uint32_t)(H * N * 128));
+        for (int h = 0; h < H; ++h) tma_load_4d(smem_u32(q_s + h * NP * 128), &tm.q, BAR(Q_FULL), h * 64, 0, g * p.G, bi);
+      };
+      if (!kp.early_src1) dependency();
+      for (int t = 0; t < T && ok; ++t) {
+        const int s = t % NS;
+        const uint32_t ph = ((t / NS) - 1) & 1;
+        const int gi0 = gb + 4 * t, ng = min(4, ge - gi0);
+        // a tile that needs the ring to turn, or holds rows of source 2, comes after the dependency (and after Q)
+        if (t >= NS || gi0 + ng > g1) dependency();
+        uint32_t bytes = 0;
+        for (int j = 0; j < ng; ++j) bytes += (uint32_t)(H * 128 * (gi0 + j < g1 ? 32 : kp.gr2));
+        const uint32_t kdst = smem_u32(ring + (size_t)s * SLOT), vdst = kdst + KV_BYTES;
+        for (int kv = 0; kv < 2; ++kv) {
+          const int full = kv == 0 ? FULL_K : FULL_V, empty = kv == 0 ? EMPTY_K : EMPTY_V;
+          if (t >= NS && !wait_bar(BAR(empty + s), ph, abort_flag, p.status, 1 + kv, wlim)) { ok = false; break; }
+          mbar_expect_tx(BAR(full + s), bytes);
+          for (int j = 0; j < ng; ++j) {
+            const Group x = group_of(gi0 + j, g1, n1, n2);
+            const CUtensorMap* m = kv == 0 ? (x.src1 ? &tm.k1 : &tm.k2) : (x.src1 ? &tm.v1 : &tm.v2);
+            for (int h = 0; h < H; ++h)
+              tma_load_4d((kv == 0 ? kdst : vdst) + h * HALF + j * 4096, m, BAR(full + s), h * 64, x.row0, g, bi);
+          }
+          if (kv == 0) k_issued = t + 1; else v_issued = t + 1;
+        }
+      }
+      dependency();                      // a CTA without tiles still loads Q: the MMA lane waits for it before it leaves
+      if (*abort_flag) {
+        // let the copies that were issued land before the CTA retires
+        for (int j = max(k_issued - NS, 0); j < k_issued; ++j) drain_bar(BAR(FULL_K + j % NS), (j / NS) & 1);
+        for (int j = max(v_issued - NS, 0); j < v_issued; ++j) drain_bar(BAR(FULL_V + j % NS), (j / NS) & 1);
+        drain_bar(BAR(Q_FULL), 0);
+      }
+    }
+  } else if (warp == 1) {
+    // ======================================= MMA issuer =======================================
+    if (lane == 0) {
+      const uint32_t idesc_s = kt_idesc(NP, false, false);
+      const uint32_t idesc_pv = kt_idesc(64, true, true);
+      const uint32_t qsm = smem_u32(q_s);
+      bool ok = wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 3, wlim);
+      auto issue_pv = [&](int j) -> bool {
+        const int s = j % NS, pb = j & 1;
+        const int ng = min(4, ge - (gb + 4 * j));
+        if (!wait_bar(BAR(P_FULL + pb), (j >> 1) & 1, abort_flag, p.status, 4, wlim)) return false;
+        if (!wait_bar(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 5, wlim)) return false;
+        tc_fence_after();
+        const uint32_t vsm = smem_u32(ring + (size_t)s * SLOT) + KV_BYTES;
+        const uint32_t psm = smem_u32(p_s + (size_t)(j % kp.PB) * PBUF);
+        // O^T += V^T P^T, 16 keys per instruction. A: the V tile read MN-major (the head dimension runs along M; its two
+        // 64-element halves lie HALF bytes apart; with D = 64 both halves alias the same data and rows 64..127 of O^T
+        // are duplicates nobody reads). B: P^T, MN-major, one 64-element half.
+        for (int ks = 0; ks < 2 * ng; ++ks)
+          mma_ss(tmem_base + O_COL, smem_desc(vsm + ks * 2048, H == 2 ? (uint32_t)HALF : 0u, 1024u),
+                 smem_desc(psm + ks * 2048, (uint32_t)PBUF, 1024u), idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+        tc_commit(BAR(PV_DONE + pb));    // two alternating barriers: a waiter is never a whole phase ahead of either
+        tc_commit(BAR(EMPTY_V + s));
+        return true;
+      };
+      for (int t = 0; t < T && ok; ++t) {
+        const int s = t % NS, sb = t & 1;
+        if (!wait_bar(BAR(FULL_K + s), (t / NS) & 1, abort_flag, p.status, 7, wlim)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t ksm = smem_u32(ring + (size_t)s * SLOT);
+        const uint32_t d_t = tmem_base + (uint32_t)sb * NP;
+        // S^T = K_tile Q^T: the S^T buffer of tile t - 2 is free, its softmax arrived before PV(t - 2) was issued
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t hk = (ks >> 2) * HALF + (ks & 3) * 32;
+          const uint32_t hq = (ks >> 2) * (NP * 128) + (ks & 3) * 32;
+          mma_ss(d_t, smem_desc(ksm + hk, 16u, 1024u), smem_desc(qsm + hq, 16u, 1024u), idesc_s, ks > 0 ? 1u : 0u);
+        }
+        tc_commit(BAR(S_FULL + sb));
+        tc_commit(BAR(EMPTY_K + s));
+        if (t > 0 && !issue_pv(t - 1)) { ok = false; break; }
+      }
+      if (ok && T > 0) ok = issue_pv(T - 1);
+      if (*abort_flag) {                 // wait for the tensor pipe to finish what was issued before TMEM is freed
+        tc_commit(BAR(DRAIN));
+        drain_bar(BAR(DRAIN), 0);
+      }
+    }
+  } else {
+    // ======================================= softmax warps =======================================
+    // A warp whose wait gave up (`dead`) keeps walking the tiles without touching data, so that the four warps meet at
+    // every named barrier below; the barrier pattern depends only on values all four warps share.
+    const int q4 = warp & 3;                           // TMEM lane quadrant this warp may access = its group of the tile
+    const int row = q4 * 32 + lane;                    // key row of the tile
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16);
+    const float sl2 = p.scale_log2;
+    const bool scores = p.want_scores != 0;
+    for (int t = 0; t < T; ++t) {
+      const int s = t % NS, sb = t & 1;
+      const int gi0 = gb + 4 * t, ng = min(4, ge - gi0);
+      const bool active = q4 < ng;                     // warp-uniform: this warp's group exists in the tile
+      Group x{1, 0, 0};
+      if (active) x = group_of(gi0 + q4, g1, n1, n2);
+      const bool valid = lane < x.nv;                  // this thread's row is a real key
+      if (!dead && !wait_bar_warp(BAR(S_FULL + sb), (t >> 1) & 1, abort_flag, p.status, 9, wlim)) dead = true;
+      tc_fence_after();
+      const bool work = active && !dead;
+      uint32_t sv[NP];
+      if (work) {
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) tmem_ld32(lane_addr + (uint32_t)sb * NP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
+        tc_wait_ld();
+      } else {
+#pragma unroll
+        for (int c = 0; c < NP; ++c) sv[c] = 0u;
+      }
+      // ---- the references: set from the first tile's column maxima, afterwards only checked ----
+      bool raise = t == 0;
+      if (t > 0) {
+        bool over = false;
+        if (work && valid) {
+#pragma unroll
+          for (int c = 0; c < NP; ++c) over |= __uint_as_float(sv[c]) * sl2 > ord2f(m_enc[c]) + 8.f;
+        }
+        raise = softmax_barrier_or(over);
+        if (raise) {
+          // (rare) every PV issued so far must have landed before O^T is rewritten; the PV of this tile waits for our arrive
+          if (!dead && !wait_bar_warp(BAR(PV_DONE + ((t - 1) & 1)), ((t - 1) >> 1) & 1, abort_flag, p.status, 8, wlim)) dead = true;
+          tc_fence_after();
+          if (tid - 64 < NP) m_old[tid - 64] = m_enc[tid - 64];
+          softmax_barrier();
+        }
+      }
+      if (raise) {
+        if (work) {
+          float mine[NCH];
+#pragma unroll
+          for (int c = 0; c < NP; ++c) {
+            const float r = warp_max_f32(valid ? __uint_as_float(sv[c]) : -INFINITY);
+            if ((c & 31) == lane) mine[c >> 5] = r;
+          }
+#pragma unroll
+          for (int c = 0; c < NCH; ++c) atomicMax(m_enc + c * 32 + lane, f2ord(mine[c] * sl2));
+        }
+        softmax_barrier();
+      }
+      if (raise && t > 0) {
+        if (tid - 64 < NP) alpha_s[tid - 64] = fast_exp2(ord2f(m_old[tid - 64]) - ord2f(m_enc[tid - 64]));
+        softmax_barrier();
+        // this thread's TMEM lane is a head dimension of O^T here, not a key: all four warps rescale their lanes
+        if (!dead) {
+#pragma unroll
+          for (int c = 0; c < NCH; ++c) {
+            uint32_t o32[32];
+            tmem_ld32(lane_addr + O_COL + c * 32, o32);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float a = alpha_s[c * 32 + i];
+              o32[i] = __float_as_uint(__uint_as_float(o32[i]) * a);
+              l_acc[c * 32 + i] *= a;
+            }
+            tmem_st16(lane_addr + O_COL + c * 32, *reinterpret_cast<uint32_t(*)[16]>(&o32[0]));
+            tmem_st16(lane_addr + O_COL + c * 32 + 16, *reinterpret_cast<uint32_t(*)[16]>(&o32[16]));
+          }
+          tc_wait_st();
+        }
+      }
+      // ---- saliency of this key (refresh step): scale * mean of its N logits ----
+      if (scores && work && valid && x.src1) {
+        float a4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int c = 0; c < NP; ++c)
+          if (c < N) a4[c & 3] += __uint_as_float(sv[c]);
+        p.raw_scores[(int64_t)(bi * p.Hkv + g) * p.n1_max + x.row0 + lane] = ((a4[0] + a4[1]) + (a4[2] + a4[3])) * (p.scale / (float)N);
+      }
+      // ---- P^T = exp2(S^T * scale_log2 - reference) as bf16, one 128-byte row per key (128-byte swizzle) ----
+      // the P^T buffer is free once the PV that read it has completed
+      if (!dead && t >= kp.PB &&
+          !wait_bar_warp(BAR(PV_DONE + ((t - kp.PB) & 1)), ((t - kp.PB) >> 1) & 1, abort_flag, p.status, 6, wlim))
+        dead = true;
+      if (active && !dead) {
+        unsigned char* prow = p_s + (size_t)(t % kp.PB) * PBUF + row * 128;
+#pragma unroll
+        for (int c8 = 0; c8 < NP / 8; ++c8) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int c = c8 * 8 + 2 * i;
+            const float e0 = valid ? fast_exp2(fmaf(__uint_as_float(sv[c]), sl2, -ord2f(m_enc[c]))) : 0.f;
+            const float e1 = valid ? fast_exp2(fmaf(__uint_as_float(sv[c + 1]), sl2, -ord2f(m_enc[c + 1]))) : 0.f;
+            l_acc[c] += e0; l_acc[c + 1] += e1;
+            pk[i] = pack_bf16(e0, e1);
+          }
+          *reinterpret_cast<uint4*>(prow + ((c8 ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+        // ---- V rows of this group past its count may hold anything: zero them so that 0 * V stays 0 ----
+        if (x.nv < 32) {
+          if (!wait_bar_warp(BAR(FULL_V + s), (t / NS) & 1, abort_flag, p.status, 10, wlim)) dead = true;
+          unsigned char* vs = ring + (size_t)s * SLOT + KV_BYTES;
+          const int nz = dead ? 0 : (32 - x.nv) * H * 8;          // 16-byte chunks to clear
+          for (int i = lane; i < nz; i += 32) {
+            const int rr = q4 * 32 + x.nv + i / (H * 8), c = i % (H * 8);
+            *reinterpret_cast<uint4*>(vs + (c >> 3) * HALF + rr * 128 + (((c & 7) ^ (rr & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+        fence_proxy_async();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0 && !dead) mbar_arrive(BAR(P_FULL + sb));
+    }
+  }
+
+  // ======================================= epilogue =======================================
+  const bool do_attn = p.out != nullptr;
+  uint32_t ov[NP];                       // softmax warps: this thread's head dimension of O^T, all columns
+  if (warp >= 2) {
+    const int q4 = warp & 3;
+    const int row = q4 * 32 + lane;
+    // ---- column sums over the 128 key rows: shuffle transpose inside a warp (lane i ends up with column i), then the
+    //      four warps' rows in a fixed order ----
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      float v[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = l_acc[c * 32 + i];
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) {
+        const bool up_half = (lane & off) != 0;
+#pragma unroll
+        for (int k = 0; k < off; ++k) {
+          const float send = up_half ? v[k] : v[k + off];
+          const float keep = up_half ? v[k + off] : v[k];
+          v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+      }
+      l_w[(warp - 2) * 64 + c * 32 + lane] = v[0];
+    }
+    softmax_barrier();
+    if (tid - 64 < NP) l_tot[tid - 64] = (l_w[tid - 64] + l_w[64 + tid - 64]) + (l_w[128 + tid - 64] + l_w[192 + tid - 64]);
+    softmax_barrier();
+    // ---- the finished accumulator row of this thread ----
+    const bool have_o = do_attn && !dead && T > 0 &&
+                        wait_bar_warp(BAR(PV_DONE + ((T - 1) & 1)), ((T - 1) >> 1) & 1, abort_flag, p.status, 6, wlim);
+    tc_fence_after();
+    if (have_o) {
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) tmem_ld32(tmem_base + ((uint32_t)(q4 * 32) << 16) + O_COL + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[c * 32]));
+      tc_wait_ld();
+    } else {
+#pragma unroll
+      for (int c = 0; c < NP; ++c) ov[c] = 0u;
+    }
+    if (S == 1 && do_attn && !*abort_flag) {
+      // one split: normalise and store; a warp writes 32 consecutive bf16 of one output row per column
+      if (row < D) {
+#pragma unroll
+        for (int c = 0; c < NP; ++c) {
+          if (c >= N) break;
+          const float l = l_tot[c];
+          const float inv = l > 0.f ? 1.f / l : 0.f;
+          const int hg = c / p.b, i = c - hg * p.b;
+          reinterpret_cast<__nv_bfloat16*>(p.out)[(int64_t)bi * p.o_stride[0] + (int64_t)(g * p.G + hg) * p.o_stride[1] +
+                                                   (int64_t)i * p.o_stride[2] + row] = __float2bfloat16_rn(__uint_as_float(ov[c]) * inv);
+        }
+      }
+      if (p.lse && tid - 64 < N) {
+        const int c = tid - 64;
+        const int hg = c / p.b, i = c - hg * p.b;
+        p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (ord2f(m_enc[c]) + log2f(l_tot[c])) * kLn2;
+      }
+    }
+  }
+
+  if (S > 1) {
+    // ---- cluster merge: every split pushes each column to the CTA that owns it; one barrier; owners merge and store ----
+    cluster_wait_acquire();              // phase 1: every CTA of the cluster runs, so its shared memory may be written
+    const int QL = kp.QL;
+    if (warp >= 2 && do_attn) {
+      const int row = (warp & 3) * 32 + lane;
+      const uint32_t recv_a = smem_u32(recv), ml_a = smem_u32(ml_recv);
+      if (row < D) {
+#pragma unroll
+        for (int c = 0; c < NP; ++c) {
+          if (c >= N) break;
+          const int owner = c / QL, ql = c - owner * QL;
+          st_cluster_f32(map_to_cta(recv_a + (uint32_t)(((split * QL + ql) * D + row) * 4), (uint32_t)owner), __uint_as_float(ov[c]));
+        }
+      }
+      if (tid - 64 < N) {
+        const int c = tid - 64;
+        const int owner = c / QL, ql = c - owner * QL;
+        st_cluster_f2(map_to_cta(ml_a + (uint32_t)((split * QL + ql) * 8), (uint32_t)owner), ord2f(m_enc[c]), l_tot[c]);
+      }
+    }
+    __threadfence();                     // the raw saliency of this split, for the peers that pool it
+    cluster_arrive_release();
+    cluster_wait_acquire();
+    if (warp >= 2 && do_attn && !*abort_flag) {
+      const int row = (warp & 3) * 32 + lane;
+      const int c_lo = split * QL, c_hi = min(c_lo + QL, N);
+      for (int c = c_lo; c < c_hi; ++c) {
+        const int ql = c - c_lo;
+        float mstar = -INFINITY;
+        for (int s2 = 0; s2 < S; ++s2) {
+          const float2 x = ml_recv[s2 * QL + ql];
+          if (x.y > 0.f) mstar = fmaxf(mstar, x.x);
+        }
+        float acc = 0.f, l = 0.f;
+        for (int s2 = 0; s2 < S; ++s2) {
+          const float2 x = ml_recv[s2 * QL + ql];
+          if (!(x.y > 0.f)) continue;
+          const float w = fast_exp2(x.x - mstar);
+          l = fmaf(x.y, w, l);
+          if (row < D) acc = fmaf(recv[(s2 * QL + ql) * D + row], w, acc);
+        }
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        const int hg = c / p.b, i = c - hg * p.b;
+        if (row < D)
+          reinterpret_cast<__nv_bfloat16*>(p.out)[(int64_t)bi * p.o_stride[0] + (int64_t)(g * p.G + hg) * p.o_stride[1] +
+                                                   (int64_t)i * p.o_stride[2] + row] = __float2bfloat16_rn(acc * inv);
+        if (row == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
+      }
+    }
+  } else {
+    __syncthreads();                     // the raw saliency of the whole head is visible to this CTA
+  }
+
+  // ---- pooling of the head's saliency (refresh step): this CTA's share of the positions ----
+  if (p.want_scores && p.pooled != nullptr && !*abort_flag) {
+    const float* a = p.raw_scores + (int64_t)(bi * p.Hkv + g) * p.n1_max;
+    const int p_lo = (int)(((long long)split * p.n1_max) / S), p_hi = (int)(((long long)(split + 1) * p.n1_max) / S);
+    const int o = p.block_off[bi];
+    for (int pos = p_lo + tid; pos < p_hi; pos += KT_THREADS)
+      p.pooled[(int64_t)(bi * p.Hkv + g) * p.n1_max + pos] = kt_pool_at(p, a, n1, o, pos);
+  }
+
+  // ---- free the tensor memory ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Host side
+size_t kt_smem_bytes(int D, int NP, int NS, int PB, int S, int QL) {
+  const size_t H = D / 64;
+  return 1024 /*alignment slack*/ + KT_CTRL + H * NP * 128 + (size_t)PB * 128 * 128 + (size_t)NS * 2 * H * 128 * 128 +
+         (S > 1 ? (size_t)S * QL * D * 4 : 0);
+}
+
+template <int D, int NCH>
+cudaError_t launch_kt_d(const KtMaps& tm, const KtParams& kp, const AttnPlan& pl, bool pdl, cudaStream_t st) {
+  auto kern = attn_kt_kernel<D, NCH>;
+  static SmemConfig configured;
+  cudaError_t e = configure_smem(reinterpret_cast<const void*>(kern), pl.smem_bytes, configured, true);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(kp.S, kp.a.Hkv, kp.a.B);
+  cfg.blockDim = dim3(KT_THREADS);
+  cfg.dynamicSmemBytes = pl.smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  if (pdl) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  if (kp.S > 1) {                            // the key splits (grid x) of a unit form one cluster
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = kp.S; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.attrs = attr; cfg.numAttrs = na;
+  return cudaLaunchKernelEx(&cfg, kern, tm, kp);
+}
+
+}  // namespace
+
+// Whether the key-row kernel covers a shape: bf16, D in {64, 128}, at most 64 query rows per KV head, block length a
+// multiple of 16.
+bool kt_supported(int dtype, int D, int M, int b) {
+  return umma_supported(dtype, D, M, b) && M <= 64;
+}
+
+AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int n2, const Tuning& tn) {
+  (void)b;
+  AttnPlan pl{};
+  pl.kind = 3; pl.tma = true; pl.fused_tail = true;
+  pl.threads = KT_THREADS;
+  pl.key_tile = 128; pl.key_tile2 = n2 < 32 ? n2 : 32;
+  pl.rep = 1; pl.row_tiles = 1; pl.rows_rep = M;
+  const int NP = M <= 32 ? 32 : 64;
+  const int groups = (n1_max + 31) / 32 + (n2 + 31) / 32;
+  const long long units = (long long)B * Hkv;
+  const int sms = sm_count();
+  // Key splits: enough CTAs to fill the SMs (two per SM with few query columns), but at least one full 128-key tile
+  // per CTA, and at most eight (one cluster).
+  long long want = (NP == 32 ? 2 : 1) * (long long)sms / units;
+  const long long by_tiles = (groups + 3) / 4;
+  if (want > by_tiles) want = by_tiles;
+  if (tn.splits > 0) want = tn.splits;
+  if (want > 8) want = 8;
+  if (want > M) want = M;
+  if (want < 1) want = 1;
+  const int S = (int)want;
+  const int QL = (M + S - 1) / S;
+  const int tiles_cta = ((groups + S - 1) / S + 3) / 4;
+  // Ring depth and P^T buffers. With few query columns, and either more CTAs than SMs or a single tile per CTA, the
+  // footprint is kept below half an SM, so that two CTAs are resident and the next call's CTAs can start loading while
+  // this call's finish; otherwise the CTA takes what one SM has.
+  const size_t half_sm = 113 * 1024;
+  int NS = 1, PB = 1;
+  const bool small = NP == 32 && (units * S > sms || tiles_cta <= 1);
+  if (small) {
+    while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, NP, NS + 1, PB, S, QL) <= half_sm) ++NS;
+  } else {
+    PB = 2;
+    while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, NP, NS + 1, PB, S, QL) <= 226 * 1024) ++NS;
+  }
+  if (tn.stages > 0) {
+    NS = tn.stages > KT_MAX_STAGES ? KT_MAX_STAGES : tn.stages;
+    while (NS > 1 && kt_smem_bytes(D, NP, NS, PB, S, QL) > 226 * 1024) --NS;
+  }
+  pl.splits = 1;                        // nothing is left in the workspace: the splits merge inside their cluster
+  pl.parts = 1;
+  pl.cluster = S;
+  pl.stages = NS;
+  pl.m_warps = PB;                      // (field reused: P^T buffers)
+  pl.part_rows = 0;
+  pl.n_counters = 0;
+  pl.smem_bytes = kt_smem_bytes(D, NP, NS, PB, S, QL);
+  return pl;
+}
+
+cudaError_t launch_attn_kt(const AttnParams& p, const AttnPlan& pl, int D, cudaStream_t st) {
+  const Tuning tn = tuning();
+  KtMaps tm;
+  KtParams kp{};
+  kp.a = p;
+  kp.a.wait_cycles = tn.wait_cycles;
+  kp.N = p.M; kp.S = pl.cluster; kp.NS = pl.stages; kp.PB = pl.m_warps;
+  kp.QL = (p.M + kp.S - 1) / kp.S;
+  kp.gr2 = p.n2 < 32 ? p.n2 : 32;
+  kp.early_src1 = (p.n2 > 0 && p.n1_max > 0 && tn.early_loads != 0) ? 1 : 0;
+  kp.wait_cycles = tn.wait_cycles;
+  memset(&tm, 0, sizeof(tm));
+  bool ok = umma_make_map(&tm.q, p.q, D, p.b, p.Hq, p.B, p.q_stride, p.b, p.G);
+  if (p.n1_max > 0) {
+    ok = ok && umma_make_map(&tm.k1, p.k1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 32, 1);
+    ok = ok && umma_make_map(&tm.v1, p.v1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 32, 1);
+  }
+  if (p.n2 > 0) {
+    ok = ok && umma_make_map(&tm.k2, p.k2, D, p.n2, p.Hkv, p.B, p.k2_stride, kp.gr2, 1);
+    ok = ok && umma_make_map(&tm.v2, p.v2, D, p.n2, p.Hkv, p.B, p.k2_stride, kp.gr2, 1);
+    if (p.n1_max <= 0) { tm.k1 = tm.k2; tm.v1 = tm.v2; }
+  } else {
+    tm.k2 = tm.k1; tm.v2 = tm.v1;
+  }
+  if (!ok) return cudaErrorInvalidValue;
+  const bool pdl = tn.pdl != 0;
+  const int NP = p.M <= 32 ? 32 : 64;
+  if (NP == 32) return D == 128 ? launch_kt_d<128, 1>(tm, kp, pl, pdl, st) : launch_kt_d<64, 1>(tm, kp, pl, pdl, st);
+  return D == 128 ? launch_kt_d<128, 2>(tm, kp, pl, pdl, st) : launch_kt_d<64, 2>(tm, kp, pl, pdl, st);
+}
+
+}  // namespace sdllm

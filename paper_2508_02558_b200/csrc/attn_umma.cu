@@ -24,10 +24,10 @@
 // Every wait on an mbarrier is bounded. On expiry the thread sets an abort flag that all other waits poll, records a
 // code in the status word and the CTA runs to its end (freeing its TMEM); the outputs of that call are then invalid.
 #include <cuda.h>
-#include <stdlib.h>
 #include <string.h>
 
 #include "attn_device.cuh"
+#include "tuning.cuh"
 #include "umma_host.cuh"
 
 namespace sdllm {
@@ -333,11 +333,11 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
       const CUtensorMap* mk = x.src1 ? &tm.k1 : &tm.k2;
       const CUtensorMap* mv = x.src1 ? &tm.v1 : &tm.v2;
       const uint32_t tile_tx = (uint32_t)(H * (x.src1 ? KT : KT2) * 128);
-      if (it >= NS && !wait_bar(BAR(EMPTY_K + s), ph, abort_flag, p.status, 1)) { prod_ok = false; break; }
+      if (it >= NS && !wait_bar(BAR(EMPTY_K + s), ph, abort_flag, p.status, 1, p.wait_cycles)) { prod_ok = false; break; }
       mbar_expect_tx(BAR(FULL_K + s), tile_tx);
       for (int h = 0; h < H; ++h) tma_load_4d(kdst + h * half_bytes, mk, BAR(FULL_K + s), h * 64, x.row0, g, bi);
       if (do_attn) {
-        if (it >= NS && !wait_bar(BAR(EMPTY_V + s), ph, abort_flag, p.status, 2)) { prod_ok = false; break; }
+        if (it >= NS && !wait_bar(BAR(EMPTY_V + s), ph, abort_flag, p.status, 2, p.wait_cycles)) { prod_ok = false; break; }
         mbar_expect_tx(BAR(FULL_V + s), tile_tx);
         for (int h = 0; h < H; ++h) tma_load_4d(vdst + h * half_bytes, mv, BAR(FULL_V + s), h * 64, x.row0, g, bi);
       }
@@ -431,9 +431,9 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
       Tile prev{}; int prev_it = -1;
       auto issue_pv = [&](const Tile& x, int j) -> bool {
         const int s = j % NS, pb = j & 1;
-        if (!wait_bar(BAR(P_FULL + pb), (j >> 1) & 1, abort_flag, p.status, 4)) return false;
+        if (!wait_bar(BAR(P_FULL + pb), (j >> 1) & 1, abort_flag, p.status, 4, p.wait_cycles)) return false;
         if (j == 0) TRACE(8);
-        if (!wait_bar(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 5)) return false;
+        if (!wait_bar(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 5, p.wait_cycles)) return false;
         if (j == 0) TRACE(9);
         tc_fence_after();
         const uint32_t vsm = smem_u32(stage0 + (size_t)s * stage_bytes) + kv_bytes;
@@ -449,13 +449,13 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
         const Tile x = tile_of(t, tiles1, KT, KT2, n1, n2);
         if (x.nv == 0) continue;
         const int s = it % NS, sb = it & 1;
-        if (!wait_bar(BAR(FULL_K + s), (it / NS) & 1, abort_flag, p.status, 7)) { ok = false; break; }
+        if (!wait_bar(BAR(FULL_K + s), (it / NS) & 1, abort_flag, p.status, 7, p.wait_cycles)) { ok = false; break; }
         if (!have_q) {
-          if (!wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 3)) { ok = false; break; }
+          if (!wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 3, p.wait_cycles)) { ok = false; break; }
           have_q = true;
         }
         // without PV nothing else orders the reuse of an S buffer: wait until the softmax warps have read tile it - 2
-        if (prob_pass && it >= 2 && !wait_bar(BAR(P_FULL + sb), ((it >> 1) - 1) & 1, abort_flag, p.status, 12)) { ok = false; break; }
+        if (prob_pass && it >= 2 && !wait_bar(BAR(P_FULL + sb), ((it >> 1) - 1) & 1, abort_flag, p.status, 12, p.wait_cycles)) { ok = false; break; }
         if (it == 0) TRACE(7);
         tc_fence_after();
         const uint32_t ksm = smem_u32(stage0 + (size_t)s * stage_bytes);
@@ -476,7 +476,7 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
       }
       if (do_attn && ok && prev_it >= 0) ok = issue_pv(prev, prev_it);
       // a CTA whose slice holds no valid key never used Q: its load must still have landed before the CTA retires
-      if (ok && !have_q) ok = wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 3);
+      if (ok && !have_q) ok = wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 3, p.wait_cycles);
       if (*abort_flag) {               // wait for the tensor pipe to finish what was issued before TMEM is freed
         tc_commit(BAR(DRAIN));
         drain_bar(BAR(DRAIN), 0);
@@ -512,7 +512,7 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
         const int sb = it & 1;
         const int c_lo = min(rep * chunk_keys, x.nv), c_hi = min((rep + 1) * chunk_keys, x.nv);
         // a warp that gave up keeps walking the tiles so that the four warps meet at every barrier below
-        if (!dead && !wait_bar_warp(BAR(S_FULL + sb), (it >> 1) & 1, abort_flag, p.status, 9)) dead = true;
+        if (!dead && !wait_bar_warp(BAR(S_FULL + sb), (it >> 1) & 1, abort_flag, p.status, 9, p.wait_cycles)) dead = true;
         tc_fence_after();
         float* cs = colsum + (size_t)sb * 4 * KT + (size_t)(warp - 2) * KT;
 #pragma unroll 1
@@ -568,7 +568,7 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
         // its replica owns nothing
         const bool idle = q4 * 32 - rep * rows_rep >= M_rt;
         const int c_lo = idle ? x.nv : min(rep * chunk_keys, x.nv), c_hi = min((rep + 1) * chunk_keys, x.nv);
-        if (!wait_bar_warp(BAR(S_FULL + sb), (it >> 1) & 1, abort_flag, p.status, 9)) { ok = false; break; }
+        if (!wait_bar_warp(BAR(S_FULL + sb), (it >> 1) & 1, abort_flag, p.status, 9, p.wait_cycles)) { ok = false; break; }
         if (tid == 64 && it == 0) TRACE(10);
         tc_fence_after();
         const uint32_t s_addr = lane_addr + (uint32_t)sb * S_STRIDE;
@@ -610,7 +610,7 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
         }
         if (it > 0 && __any_sync(0xffffffffu, grow)) {
           // every PV issued so far must have landed before the rows are rewritten; PV of this tile waits for our arrive
-          if (!wait_bar_warp(BAR(PV_DONE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag, p.status, 8)) { ok = false; break; }
+          if (!wait_bar_warp(BAR(PV_DONE + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag, p.status, 8, p.wait_cycles)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll 1
           for (int c = 0; c < D / 16; ++c) {
@@ -663,7 +663,7 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
         l_run += psum;
         // ---- V rows past the source's count may hold anything: zero them so that 0 * V stays 0 ----
         if (x.nv < x.n_mma) {
-          if (!wait_bar_warp(BAR(FULL_V + s), (it / NS) & 1, abort_flag, p.status, 10)) { ok = false; break; }
+          if (!wait_bar_warp(BAR(FULL_V + s), (it / NS) & 1, abort_flag, p.status, 10, p.wait_cycles)) { ok = false; break; }
           unsigned char* vs = stage0 + (size_t)s * stage_bytes + kv_bytes;
           const int nz = (x.n_mma - x.nv) * H * 8;     // 16-byte chunks to clear
           for (int i = (warp - 2) * 32 + lane; i < nz; i += 128) {
@@ -709,7 +709,7 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
         const Tile x = tile_of(t, tiles1, KT, KT2, n1, n2);
         if (x.nv == 0) continue;
         const int s = it % NS;
-        if (!wait_bar_warp(BAR(FULL_K + s), (it / NS) & 1, abort_flag, p.status, 11)) break;
+        if (!wait_bar_warp(BAR(FULL_K + s), (it / NS) & 1, abort_flag, p.status, 11, p.wait_cycles)) break;
         if (x.src1) {
           // one key per lane: a_j = scale * <qbar, k_j>; the 128-byte swizzle keeps 32 consecutive rows conflict-free
           const unsigned char* kst = stage0 + (size_t)s * stage_bytes;
@@ -790,7 +790,7 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
     if (rep == 0) lm_s[m_local] = make_float2(mstar, lsum);
     // the finished accumulator row: TMEM -> weight -> shared memory, 32 columns at a time
     const bool have_o = sm_ok && sm_tiles > 0 &&
-                        wait_bar_warp(BAR(PV_DONE + ((sm_tiles - 1) & 1)), ((sm_tiles - 1) >> 1) & 1, abort_flag, p.status, 6);
+                        wait_bar_warp(BAR(PV_DONE + ((sm_tiles - 1) & 1)), ((sm_tiles - 1) >> 1) & 1, abort_flag, p.status, 6, p.wait_cycles);
     tc_fence_after();
 #pragma unroll 1
     for (int c = 0; c < D / 32; ++c) {
@@ -1023,15 +1023,11 @@ size_t umma_smem_bytes(int D, int KT, bool dual) {
 }
 
 template <int D, bool PROB, bool DUAL>
-cudaError_t launch_umma_d(const UmmaMaps& tm, const UmmaParams& up, const AttnPlan& pl, cudaStream_t st) {
+cudaError_t launch_umma_d(const UmmaMaps& tm, const UmmaParams& up, const AttnPlan& pl, bool pdl, cudaStream_t st) {
   auto kern = attn_umma_bf16_kernel<D, PROB, DUAL>;
-  static size_t configured = 0;
-  if (pl.smem_bytes > configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
-    if (e != cudaSuccess) return e;
-    (void)cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    configured = pl.smem_bytes;
-  }
+  static SmemConfig configured;
+  cudaError_t e = configure_smem(reinterpret_cast<const void*>(kern), pl.smem_bytes, configured, true);
+  if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(pl.splits, up.a.Hkv * up.row_tiles, up.a.B);
   cfg.blockDim = dim3(UM_THREADS);
@@ -1039,8 +1035,7 @@ cudaError_t launch_umma_d(const UmmaMaps& tm, const UmmaParams& up, const AttnPl
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
   int na = 0;
-  const char* e = getenv("SDLLM_PDL");       // SDLLM_PDL=0 turns programmatic dependent launch off (tuning and test aid)
-  if (!(e && e[0] == '0')) {
+  if (pdl) {
     attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[na].val.programmaticStreamSerializationAllowed = 1;
     ++na;
@@ -1074,48 +1069,46 @@ bool umma_supported(int dtype, int D, int M, int b) {
 bool umma_tail_is_fused(const AttnPlan& pl, int D, int M, int n1_max, bool pool, bool merge) {
   const size_t merge_bytes = merge && pl.splits > 1 ? (size_t)pl.splits * (M < 128 ? M : 128) * D * 4 : 0;
   bool fused = merge_bytes <= 256 * 1024 && (!pool || n1_max <= 8192);
-  if (const char* e = getenv("SDLLM_FUSED_TAIL")) fused = e[0] == '1' && (!pool || n1_max <= 8192);   // tuning aid
+  const int forced = tuning().fused_tail;
+  if (forced >= 0) fused = forced == 1 && (!pool || n1_max <= 8192);
   return fused;
 }
 
-AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, int n2) {
+AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, int n2, const Tuning& tn) {
   AttnPlan pl{};
   pl.kind = 2; pl.tma = true; pl.cluster = 1; pl.fused_tail = true;
   pl.threads = UM_THREADS; pl.stages = UM_STAGES;
+  const int sms = sm_count();
   const int G = M / b;
   pl.row_tiles = M <= 128 ? 1 : (G + 128 / b - 1) / (128 / b);
   pl.rep = M <= 32 ? 4 : (M <= 64 ? 2 : 1);
   const long long units = (long long)B * Hkv * pl.row_tiles;
   // Several waves of CTAs: the small-footprint variant puts two of them on an SM, so that one's set-up and way out
   // overlap the other's streaming. It works on 64-key tiles, which leaves room for two replicas of the rows at most.
-  pl.dual = units >= 2 * kNumSMs && n2 > 0;          // measured: pays for the reuse step, not for the refresh step
-  if (const char* e = getenv("SDLLM_DUAL")) pl.dual = e[0] == '1';      // tuning and test aid
+  pl.dual = units >= 2 * sms && n2 > 0;              // measured: pays for the reuse step, not for the refresh step
+  if (tn.dual >= 0) pl.dual = tn.dual == 1;
   if (pl.dual && pl.rep > 2) pl.rep = 2;
-  long long want = kNumSMs / units;
+  long long want = sms / units;
   if (want < 1) want = 1;
-  if (const char* e = getenv("SDLLM_SPLITS")) { if (atoi(e) >= 1) want = atoi(e); }   // tuning aid
+  if (tn.splits > 0) want = tn.splits;
   // Reuse step with replicated rows (few query rows per head, so a tile costs a softmax warp little): a CTA works
   // best on about four 128-key tiles. With fewer, the set-up of the CTAs and the merge of their partials weigh more
-  // than the streaming they save (LLaDA-shaped layer, 6 tiles per head: 2 splits 11.5 us, 4 splits 12.5 us, 1 split
-  // 12.4 us; 18 tiles per head: 4 splits 17.6 us, 2 splits 20.0 us).
-  if (n2 > 0 && pl.rep > 1 && !pl.dual && !getenv("SDLLM_SPLITS")) {
+  // than the streaming they save.
+  if (n2 > 0 && pl.rep > 1 && !pl.dual && tn.splits <= 0) {
     const long long cap = ((n1_max + 127) / 128 + 1 + 3) / 4;
     if (want > cap) want = cap;
   }
   const int kt2 = n2 > 0 ? (n2 < 128 ? n2 : 128) : 0;
   pl.key_tile = 128;
   if (pl.rep <= 2 && (n1_max + 127) / 128 + (n2 > 0 ? 1 : 0) < want) pl.key_tile = 64;
-  if (const char* e = getenv("SDLLM_KEY_TILE")) {   // tuning aid
-    if (atoi(e) == 64 && pl.rep <= 2) pl.key_tile = 64;
-    if (atoi(e) == 128) pl.key_tile = 128;
-  }
+  if (tn.key_tile == 64 && pl.rep <= 2) pl.key_tile = 64;
+  if (tn.key_tile == 128) pl.key_tile = 128;
   if (pl.dual) { pl.key_tile = 64; pl.stages = 2; }
   // A reuse step with few heads and a short cache: rather than many one-tile splits whose merge needs a second launch,
   // take at most eight splits of 128-key tiles, which one cluster merges on chip.
   const int tiles128 = (n1_max + 127) / 128 + (n2 > 0 ? 1 : 0);
-  const bool no_cluster = (getenv("SDLLM_CLUSTER") && getenv("SDLLM_CLUSTER")[0] == '0') ||
-                          (getenv("SDLLM_FUSED_TAIL") && getenv("SDLLM_FUSED_TAIL")[0] == '0');
-  if (!pl.dual && !no_cluster && !getenv("SDLLM_SPLITS") && !getenv("SDLLM_KEY_TILE") && n2 > 0 && want > 8 && tiles128 <= 16) {
+  const bool no_cluster = tn.cluster == 0 || tn.fused_tail == 0;
+  if (!pl.dual && !no_cluster && tn.splits <= 0 && tn.key_tile == 0 && n2 > 0 && want > 8 && tiles128 <= 16) {
     pl.key_tile = 128;
     want = tiles128 < 8 ? tiles128 : 8;
   }
@@ -1132,37 +1125,32 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
   pl.smem_bytes = umma_smem_bytes(D, pl.key_tile, pl.dual);
   // Few key splits of a small problem: make them one thread-block cluster, so that they merge through distributed shared
   // memory instead of the workspace. Only where the whole grid is one wave (a cluster needs all its SMs at once).
-  {
-    // SDLLM_CLUSTER=0 (or SDLLM_FUSED_TAIL=0): never (tuning and test aid). Several row tiles only at the reuse step:
-    // the probability pass of the refresh step pools over all row tiles of a head, which one cluster does not span.
-    if (!no_cluster && pl.splits >= 2 && pl.splits <= 8 && (pl.row_tiles == 1 || n2 > 0) && pl.key_tile == 128 &&
-        units * pl.splits <= kNumSMs && n1_max <= 8192)
-      pl.cluster = pl.splits;
-  }
+  // Several row tiles only at the reuse step: the probability pass of the refresh step pools over all row tiles of a
+  // head, which one cluster does not span.
+  if (!no_cluster && pl.splits >= 2 && pl.splits <= 8 && (pl.row_tiles == 1 || n2 > 0) && pl.key_tile == 128 &&
+      units * pl.splits <= sms && n1_max <= 8192)
+    pl.cluster = pl.splits;
   return pl;
 }
 
 cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cudaStream_t st) {
+  const Tuning tn = tuning();
   UmmaMaps tm;
   UmmaParams up{};
   up.a = p;
   up.a.splits = pl.splits;
+  up.a.wait_cycles = tn.wait_cycles;
   up.KT = pl.key_tile; up.KT2 = pl.key_tile2; up.R = pl.rep; up.row_tiles = pl.row_tiles;
   up.heads_rt = pl.row_tiles == 1 ? p.G : 128 / p.b;
   const bool pool = p.want_scores && p.pooled != nullptr;
-  {
-    const char* e = getenv("SDLLM_EARLY_LOADS");   // SDLLM_EARLY_LOADS=0: no loads before the grid dependency (test aid)
-    up.early_src1 = (p.n2 > 0 && p.n1_max > 0 && !(e && e[0] == '0')) ? 1 : 0;
-  }
+  up.early_src1 = (p.n2 > 0 && p.n1_max > 0 && tn.early_loads != 0) ? 1 : 0;
   up.prob_pass = p.prob_pass;
   up.cluster = pl.cluster;
   {
-    const char* e = getenv("SDLLM_LPT");               // SDLLM_LPT=0/1 forces the ordering off/on (tuning and test aid)
     const long long ctas = (long long)pl.splits * p.Hkv * pl.row_tiles * p.B;
-    up.lpt = (p.n1_per_seq != nullptr && p.B >= 4 && p.B <= 64 && ctas > kNumSMs) ? 1 : 0;
-    if (e) up.lpt = (e[0] == '1' && p.n1_per_seq != nullptr && p.B >= 2 && p.B <= 64) ? 1 : 0;
+    up.lpt = (p.n1_per_seq != nullptr && p.B >= 4 && p.B <= 64 && ctas > sm_count()) ? 1 : 0;
+    if (tn.lpt >= 0) up.lpt = (tn.lpt == 1 && p.n1_per_seq != nullptr && p.B >= 2 && p.B <= 64) ? 1 : 0;
   }
-  if (up.cluster > 1) up.fused_tail = 1;     // set again below; the cluster tail never needs the second launch
   up.fused_tail = (pl.cluster > 1 || umma_tail_is_fused(pl, D, p.M, p.n1_max, pool || p.prob_pass, p.out != nullptr && !p.prob_pass)) ? 1 : 0;
   memset(&tm, 0, sizeof(tm));
   bool ok = true;
@@ -1180,12 +1168,13 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
   }
   if (!ok) return cudaErrorInvalidValue;
   cudaError_t err;
+  const bool pdl = tn.pdl != 0;
   if (pl.dual) {
-    if (up.prob_pass) err = D == 128 ? launch_umma_d<128, true, true>(tm, up, pl, st) : launch_umma_d<64, true, true>(tm, up, pl, st);
-    else err = D == 128 ? launch_umma_d<128, false, true>(tm, up, pl, st) : launch_umma_d<64, false, true>(tm, up, pl, st);
+    if (up.prob_pass) err = D == 128 ? launch_umma_d<128, true, true>(tm, up, pl, pdl, st) : launch_umma_d<64, true, true>(tm, up, pl, pdl, st);
+    else err = D == 128 ? launch_umma_d<128, false, true>(tm, up, pl, pdl, st) : launch_umma_d<64, false, true>(tm, up, pl, pdl, st);
   } else {
-    if (up.prob_pass) err = D == 128 ? launch_umma_d<128, true, false>(tm, up, pl, st) : launch_umma_d<64, true, false>(tm, up, pl, st);
-    else err = D == 128 ? launch_umma_d<128, false, false>(tm, up, pl, st) : launch_umma_d<64, false, false>(tm, up, pl, st);
+    if (up.prob_pass) err = D == 128 ? launch_umma_d<128, true, false>(tm, up, pl, pdl, st) : launch_umma_d<64, true, false>(tm, up, pl, pdl, st);
+    else err = D == 128 ? launch_umma_d<128, false, false>(tm, up, pl, pdl, st) : launch_umma_d<64, false, false>(tm, up, pl, pdl, st);
   }
   if (err != cudaSuccess || up.fused_tail) return err;
   const bool merge = p.out != nullptr && !p.prob_pass && pl.splits > 1;
@@ -1200,8 +1189,7 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   int na = 0;
-  const char* e = getenv("SDLLM_PDL");
-  if (!(e && e[0] == '0')) {
+  if (pdl) {
     attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[na].val.programmaticStreamSerializationAllowed = 1;
     ++na;
@@ -1213,15 +1201,21 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
 
 // ---------------------------------------------------------------------------------------------------------
 // Dispatch between the kernel families
-AttnPlan plan_attention_legacy(int dtype, int D, int M, int B, int Hkv, int n_keys_max);
+AttnPlan plan_attention_legacy(int dtype, int D, int M, int B, int Hkv, int n_keys_max, const Tuning& tn);
 cudaError_t launch_attn_legacy(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st);
+bool kt_supported(int dtype, int D, int M, int b);
+AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int n2, const Tuning& tn);
+cudaError_t launch_attn_kt(const AttnParams& p, const AttnPlan& pl, int D, cudaStream_t st);
 
-AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_max, int n2) {
-  // bf16 goes to the tcgen05 kernel wherever it applies; fp32 and the remaining bf16 shapes to the cp.async kernels.
-  // SDLLM_KERNEL=cpasync forces the latter (test aid).
-  const char* kern = getenv("SDLLM_KERNEL");
-  if (!(kern && kern[0] == 'c') && umma_supported(dtype, D, M, b)) return plan_attention_umma(D, M, b, B, Hkv, n1_max, n2);
-  AttnPlan pl = plan_attention_legacy(dtype, D, M, B, Hkv, n1_max + n2);
+AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_max, int n2, bool prob_scores) {
+  // bf16 goes to the tcgen05 kernels wherever they apply: heads with at most 64 query rows to the kernel that puts the
+  // keys on the accumulator rows (it has no softmax-probability saliency pass), the rest to the one that puts the
+  // queries there; fp32 and the remaining bf16 shapes go to the cp.async kernels. Tuning::kernel forces a family.
+  const Tuning tn = tuning();
+  const bool kt_ok = kt_supported(dtype, D, M, b) && !prob_scores;
+  if ((tn.kernel == 0 || tn.kernel == 3) && kt_ok) return plan_attention_kt(D, M, b, B, Hkv, n1_max, n2, tn);
+  if (tn.kernel != 1 && umma_supported(dtype, D, M, b)) return plan_attention_umma(D, M, b, B, Hkv, n1_max, n2, tn);
+  AttnPlan pl = plan_attention_legacy(dtype, D, M, B, Hkv, n1_max + n2, tn);
   pl.tma = false; pl.cluster = 1; pl.warp_keys = 32; pl.kind = 0;
   pl.part_rows = pl.splits > 1 ? (size_t)pl.splits * M : 0;      // partial rows the kernels leave per (sequence, KV head)
   pl.n_counters = 0; pl.fused_tail = false;
@@ -1230,6 +1224,7 @@ AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_m
 }
 
 cudaError_t launch_attn_partial(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st) {
+  if (plan.kind == 3) return launch_attn_kt(p, plan, D, st);
   if (plan.kind == 2) return launch_attn_umma(p, plan, D, st);
   return launch_attn_legacy(p, plan, dtype, D, st);
 }

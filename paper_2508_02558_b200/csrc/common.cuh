@@ -8,7 +8,6 @@
 
 namespace sdllm {
 
-constexpr int kNumSMs = 148;          // B200
 constexpr int kMaxRows = 256;         // b * G rows of one KV head handled by one CTA
 constexpr int kMaxSplits = 64;        // key-axis splits per (sequence, KV head)
 constexpr float kLog2e = 1.4426950408889634f;
@@ -27,7 +26,8 @@ struct AttnPlan {
   int threads;
   bool tma;         // the kernel is fed by TMA (tcgen05 kernel), else by cp.async
   size_t smem_bytes;
-  int kind;         // 0: cp.async kernels (fp32 FMA / bf16 mma.sync), 2: TMA + tcgen05 kernel
+  int kind;         // 0: cp.async kernels (fp32 FMA / bf16 mma.sync), 2: tcgen05 kernel, queries on the accumulator rows,
+                    // 3: tcgen05 kernel, keys on the accumulator rows (its key splits merge inside their cluster)
   int key_tile2;    // tcgen05 kernel: keys per tile of source 2
   int rep;          // tcgen05 kernel: replicas of the query rows along the 128 accumulator rows
   int row_tiles;    // tcgen05 kernel: 128-row tiles of the b*G rows
@@ -58,6 +58,7 @@ struct AttnParams {
   int splits;                  // partials per (sequence, KV head) in the workspace
   int splits_total;            // CTAs along the key axis per (sequence, KV head) = splits * cluster size
   int32_t* status;             // device status word: set non-zero when a bounded wait gave up
+  long long wait_cycles;       // limit of an abortable device-side wait, in clock cycles
   int32_t* counters;           // completion counters (tcgen05 kernel), zero between calls
   float* pooled;               // refresh with a fused tail: pooled scores [B][Hkv][n1_max], else null
   int window, pool_kind, per_region;
@@ -96,7 +97,7 @@ struct CompactParams {
   int64_t kv_stride_bytes[3], c_stride_bytes[3];
 };
 
-AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_max, int n2);
+AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_max, int n2, bool prob_scores);
 
 bool umma_tail_is_fused(const AttnPlan& pl, int D, int M, int n1_max, bool pool, bool merge);
 bool umma_supported(int dtype, int D, int M, int b);

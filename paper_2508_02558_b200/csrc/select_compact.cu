@@ -1,8 +1,7 @@
 // Top-k selection over the pooled importance scores and the K/V gather-compaction
 // (Algorithm 1: "n <- floor(|I| r)", "TopKIndices(I, n)", "Select(K_f, I)", "Select(V_f, I)").
-#include <stdlib.h>
-
 #include "common.cuh"
+#include "tuning.cuh"
 
 namespace sdllm {
 namespace {
@@ -416,10 +415,11 @@ __global__ void __launch_bounds__(256) compact_kv_kernel(const CompactParams p) 
 cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st) {
   // Tens of thousands of candidates per head and few heads (all clusters resident at once): a cluster of CTAs per head;
   // with many heads one CTA per head already fills the GPU and measured several times faster than clusters.
-  // SDLLM_SELECT=cluster / single forces either wherever the cluster kernel applies (tuning and test aid).
+  // Tuning::select forces either wherever the cluster kernel applies.
   const int cand = p.Lmax - p.b;
-  bool clustered = cand > 8192 && (long long)p.B * p.Hkv * SELC_CTAS <= kNumSMs;
-  if (const char* e = getenv("SDLLM_SELECT")) clustered = e[0] == 'c';
+  bool clustered = cand > 8192 && (long long)p.B * p.Hkv * SELC_CTAS <= sm_count();
+  const int forced = tuning().select;
+  if (forced != 0) clustered = forced == 2;
   if (clustered && cand >= 1 && cand <= SELC_CTAS * SELC_SLICE) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(SELC_CTAS, p.Hkv, p.B);
@@ -431,13 +431,10 @@ cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st) {
     cfg.attrs = attr; cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, select_topk_cluster_kernel, p);
   }
-  static size_t configured = 0;
+  static SmemConfig configured;
   const size_t smem = ((size_t)p.smem_keys + p.smem_keys / 32 + 1) * 4;
-  if (smem > configured) {
-    const cudaError_t e = cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = smem;
-  }
+  const cudaError_t e = configure_smem(reinterpret_cast<const void*>(select_topk_kernel), smem, configured, false);
+  if (e != cudaSuccess) return e;
   select_topk_kernel<<<dim3(p.Hkv, p.B), SEL_THREADS, smem, st>>>(p);
   return cudaGetLastError();
 }

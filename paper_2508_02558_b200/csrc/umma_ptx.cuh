@@ -3,7 +3,7 @@
 // Meant to be included inside `namespace sdllm { namespace { ... } }` of a .cu file.
 #pragma once
 
-constexpr long long kWaitCycles = 400000000LL;   // ~0.2 s
+constexpr long long kDrainCycles = 400000000LL;   // ~0.2 s: limit of the waits that let in-flight work land on the way out
 
 // ---------------------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -141,14 +141,16 @@ __device__ __forceinline__ Tile tile_of(int t, int tiles1, int KT, int KT2, int 
   return x;
 }
 
-// Bounded wait on an mbarrier phase. Returns false when the CTA is aborting (this wait or another one expired).
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int code) {
+// Bounded wait on an mbarrier phase (`limit` clock cycles). Returns false when the CTA is aborting (this wait or another
+// one expired).
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int code,
+                                         long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
       atomicExch(status, code);
       return false;
@@ -156,13 +158,14 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
   }
 }
 // The same for a whole warp: every lane takes the same decision, so warp-synchronous instructions stay converged.
-__device__ __forceinline__ bool wait_bar_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int code) {
-  return __all_sync(0xffffffffu, wait_bar(bar, parity, abort_flag, status, code)) != 0;
+__device__ __forceinline__ bool wait_bar_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int code,
+                                              long long limit) {
+  return __all_sync(0xffffffffu, wait_bar(bar, parity, abort_flag, status, code, limit)) != 0;
 }
 // Bounded wait that ignores the abort flag (used while draining in-flight work on the way out).
 __device__ __forceinline__ void drain_bar(uint32_t bar, uint32_t parity) {
   const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kWaitCycles) return;
+    if (clock64() - t0 > kDrainCycles) return;
   }
 }

@@ -20,3 +20,16 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture
+def tuning():
+    """Apply overrides of the library's launch planner for one test: tuning(splits=3, kernel=2). Reset afterwards."""
+    from paper_2508_02558_b200 import binding as B
+    B.tuning_reset()
+
+    def apply(**kw):
+        for name, value in kw.items():
+            B.tuning_set(name, value)
+    yield apply
+    B.tuning_reset()

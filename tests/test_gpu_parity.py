@@ -131,10 +131,12 @@ def test_batch_with_an_empty_cache_and_a_full_one():
 @pytest.mark.parametrize("policy", [
     dict(select=B.SELECT_PER_REGION_CEIL), dict(select=B.SELECT_PREFIX_ONLY), dict(pool=B.POOL_AVG),
 ])
-def test_policies(policy, monkeypatch):
+def test_policies(policy, tuning):
     cfg = _small("pol", "bf16", 4, 2, 128, 190, 96, retention=0.3, salient_frac=0.02)
     _run_sequence_case(cfg, seed=5, block=1, **policy)
-    monkeypatch.setenv("SDLLM_SELECT", "cluster")        # two regions, each split over the CTAs of a cluster
+    tuning(select=2)                                     # two regions, each split over the CTAs of a cluster
+    _run_sequence_case(cfg, seed=5, block=1, **policy)
+    tuning(select=0, kernel=2)                           # the attention kernel with the queries on the accumulator rows
     _run_sequence_case(cfg, seed=5, block=1, **policy)
 
 
@@ -145,24 +147,27 @@ def test_pool_windows(window):
     assert stats["set_mismatch"] == 0
 
 
-@pytest.mark.parametrize("env", [
-    {"SDLLM_KERNEL": "cpasync"},                          # cp.async + mma.sync kernels, separate merge launch
-    {"SDLLM_KERNEL": "cpasync", "SDLLM_SPLITS": "3"},
-    {"SDLLM_PDL": "0"},                                   # no programmatic dependent launch
-    {"SDLLM_SPLITS": "7"}, {"SDLLM_SPLITS": "1"},         # other key-split counts of the tcgen05 kernel
-    {"SDLLM_SPLITS": "5", "SDLLM_FUSED_TAIL": "0"},       # split merge and pooling in the second launch
-    {"SDLLM_EARLY_LOADS": "0"},                           # no loads ahead of the grid dependency
-    {"SDLLM_CLUSTER": "0", "SDLLM_SPLITS": "4"},          # key splits merged by the last CTA instead of a cluster
-    {"SDLLM_SPLITS": "4"},                                # ... and by a cluster of four
-    {"SDLLM_DUAL": "1", "SDLLM_SPLITS": "1"},             # small-footprint variant (two CTAs per SM)
-    {"SDLLM_DUAL": "1", "SDLLM_SPLITS": "3"},
-    {"SDLLM_KEY_TILE": "64", "SDLLM_SPLITS": "2"},        # 64-key tiles
-    {"SDLLM_SELECT": "cluster"},                          # top-k by a cluster of CTAs per head
+@pytest.mark.parametrize("plan", [
+    dict(kernel=1),                                      # cp.async + mma.sync kernels, separate merge launch
+    dict(kernel=1, splits=3),
+    dict(pdl=0),                                         # no programmatic dependent launch
+    dict(splits=7), dict(splits=1), dict(splits=3),      # other key-split counts (cluster sizes) of the key-row kernel
+    dict(splits=2, stages=3), dict(splits=1, stages=2),  # ... and ring depths
+    dict(early_loads=0),                                 # no loads ahead of the grid dependency
+    dict(kernel=2),                                      # the tcgen05 kernel with the queries on the accumulator rows
+    dict(kernel=2, splits=7), dict(kernel=2, splits=1),
+    dict(kernel=2, splits=5, fused_tail=0),              # split merge and pooling in the second launch
+    dict(kernel=2, early_loads=0),
+    dict(kernel=2, cluster=0, splits=4),                 # key splits merged by the last CTA instead of a cluster
+    dict(kernel=2, splits=4),                            # ... and by a cluster of four
+    dict(kernel=2, dual=1, splits=1),                    # small-footprint variant (two CTAs per SM)
+    dict(kernel=2, dual=1, splits=3),
+    dict(kernel=2, key_tile=64, splits=2),               # 64-key tiles
+    dict(select=2),                                      # top-k by a cluster of CTAs per head
 ])
-def test_alternative_launch_plans_agree_with_oracle(env, monkeypatch):
+def test_alternative_launch_plans_agree_with_oracle(plan, tuning):
     """Every kernel family, tail placement, tile size and split count gives the same answers."""
-    for k, v in env.items():
-        monkeypatch.setenv(k, v)
+    tuning(**plan)
     _run_sequence_case(_small("alt_mha", "bf16", 4, 4, 128, 403, 130, salient_frac=0.02), seed=12, block=1)
     _run_sequence_case(_small("alt_gqa", "bf16", 8, 2, 128, 300, 64, retention=0.3, salient_frac=0.02), seed=13, block=0)
     _run_sequence_case(_small("alt_gqa7", "bf16", 14, 2, 128, 260, 96, retention=0.4, salient_frac=0.02), seed=14, block=1)
@@ -174,20 +179,18 @@ def test_alternative_launch_plans_agree_with_oracle(env, monkeypatch):
     (_small("prob_gqa7", "bf16", 14, 2, 128, 300, 96, retention=0.25, salient_frac=0.01, sink_tokens=4), 2),   # two row tiles
     (_small("prob_d64", "bf16", 4, 2, 64, 150, 64, salient_frac=0.02), 1),
 ])
-@pytest.mark.parametrize("env", [{}, {"SDLLM_SPLITS": "3", "SDLLM_FUSED_TAIL": "0"}, {"SDLLM_SPLITS": "1"}, {"SDLLM_DUAL": "1"}])
-def test_softmax_probability_saliency(cfg, block, env, monkeypatch):
+@pytest.mark.parametrize("plan", [{}, dict(splits=3, fused_tail=0), dict(splits=1), dict(dual=1)])
+def test_softmax_probability_saliency(cfg, block, plan, tuning):
     """The second reading of "attention scores": mean softmax probability per key (two passes over K)."""
-    for k, v in env.items():
-        monkeypatch.setenv(k, v)
+    tuning(**plan)
     _run_sequence_case(cfg, seed=15, block=block, n_sparse=1, score=B.SCORE_PROB_MEAN)
 
 
-@pytest.mark.parametrize("env", [{}, {"SDLLM_LPT": "1"}, {"SDLLM_LPT": "1", "SDLLM_DUAL": "1", "SDLLM_SPLITS": "1"},
-                                 {"SDLLM_SELECT": "cluster"}])
-def test_ragged_batch(env, monkeypatch):
+@pytest.mark.parametrize("plan", [{}, dict(splits=3), dict(kernel=2), dict(kernel=2, lpt=1), dict(kernel=2, lpt=1, dual=1, splits=1),
+                                  dict(select=2)])
+def test_ragged_batch(plan, tuning):
     import parity_util as U
-    for k_, v_ in env.items():
-        monkeypatch.setenv(k_, v_)
+    tuning(**plan)
     cfg = _small("rag", "bf16", 4, 4, 128, 64, 64, salient_frac=0.02)
     bw = W.make_batch(cfg, [40, 333, 64, 200], seed=7, block=1)
     q, k, v = bw.refresh_inputs(1, pad_value=np.nan)       # padding must never be read
@@ -201,11 +204,10 @@ def test_ragged_batch(env, monkeypatch):
 
 
 @pytest.mark.parametrize("kernel", ["default", "cluster", "single"])
-def test_select_topk_alone_heavy_ties_bit_exact(kernel, monkeypatch):
+def test_select_topk_alone_heavy_ties_bit_exact(kernel, tuning):
     """Plateaus of exactly equal scores (what max pooling produces) must resolve to the lowest positions. The selection
     by one CTA per head and the one by a cluster of CTAs per head (long sequences) must both be exact."""
-    if kernel != "default":
-        monkeypatch.setenv("SDLLM_SELECT", kernel)
+    tuning(select={"default": 0, "single": 1, "cluster": 2}[kernel])
     rng = np.random.default_rng(8)
     for (Bn, Hkv, L, b, o, r) in [(2, 3, 300, 32, 100, 0.5), (1, 2, 2080, 32, 2048, 0.37), (1, 1, 40000, 32, 7, 0.25), (1, 1, 50000, 32, 49000, 0.6),
                                   (1, 2, 64, 32, 0, 0.5), (1, 2, 64, 32, 32, 0.99)]:
