@@ -46,7 +46,7 @@ namespace {
 
 constexpr int KT_THREADS = 192;
 constexpr int KT_MAX_STAGES = 3;
-constexpr int KT_CTRL = 4096;            // control block: barriers, flags, references, sums, received (reference, sum) pairs
+constexpr int KT_CTRL = 3072;            // control block: barriers, flags, references, sums
 
 struct KtMaps {
   CUtensorMap q, k1, v1, k2, v2;
@@ -58,22 +58,48 @@ struct KtParams {
   int S;             // key splits of a unit = CTAs of its cluster (1..8)
   int NS;            // ring slots (128-key K tile + V tile each)
   int PB;            // P^T buffers (1 or 2)
-  int QL;            // query columns a CTA owns in the merge: ceil(N / S)
+  int DL;            // head dimensions a CTA owns in the merge: ceil(D / S)
+  int cpt;           // merge: columns per thread, a multiple of 4
   int gr2;           // rows of a source-2 box: min(32, n2)
   int early_src1;    // 1: source 1 and its count are older than every kernel that may still run (reuse step)
+  int early_trigger; // 1: release the next kernel in the stream as soon as this CTA is set up
   long long wait_cycles;   // limit of every abortable mbarrier wait
 };
 
 #include "umma_ptx.cuh"
 
-__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed;\n" ::: "memory"); }
 __device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release;\n" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire;\n" ::: "memory"); }
-__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
-  asm volatile("st.shared::cluster.f32 [%0], %1;\n" ::"r"(addr), "f"(v) : "memory");
+// Asynchronous stores into the shared memory of a CTA of the cluster; each one reports its bytes to an mbarrier of that
+// CTA (complete_tx, release at cluster scope), so the receiver waits for exactly the data it is owed and for nothing else.
+__device__ __forceinline__ void st_async_f4(uint32_t addr, uint32_t mbar, float x, float y, float z, float w) {
+  asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];\n"
+               ::"r"(addr), "f"(x), "f"(y), "f"(z), "f"(w), "r"(mbar) : "memory");
 }
-__device__ __forceinline__ void st_cluster_f2(uint32_t addr, float x, float y) {
-  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};\n" ::"r"(addr), "f"(x), "f"(y) : "memory");
+__device__ __forceinline__ void st_async_f2(uint32_t addr, uint32_t mbar, float x, float y) {
+  asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];\n"
+               ::"r"(addr), "f"(x), "f"(y), "r"(mbar) : "memory");
+}
+// Bounded wait on an mbarrier that remote CTAs complete: acquire at cluster scope.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool wait_merge(uint32_t bar, volatile int* abort_flag, int32_t* status, long long limit) {
+  if (mbar_try_wait_cluster(bar, 0)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try_wait_cluster(bar, 0)) return true;
+    const bool aborting = *abort_flag != 0;
+    // an aborting CTA still lets its peers' pushes land before it retires (drain limit)
+    if (clock64() - t0 > (aborting ? kDrainCycles : limit)) {
+      if (!aborting) { *abort_flag = 1; atomicExch(status, 13); }
+      else return false;
+    }
+  }
 }
 __device__ __forceinline__ float warp_max_f32(float v) {
   float r;
@@ -155,6 +181,10 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
   const int bi = blockIdx.z, g = blockIdx.y, split = blockIdx.x;
   const int n2 = p.n2;
   const long long wlim = kp.wait_cycles;
+  // The count of source 1 is read ahead of the grid dependency only at the reuse step (it is older than any kernel that
+  // may still run); the load is issued first so that its latency hides behind the set-up.
+  int n1_early = p.n1_max;
+  if (kp.early_src1 && p.n1_per_seq) n1_early = __ldg(p.n1_per_seq + bi);
 
   // ---- shared memory carve-up (1024-byte aligned for the 128-byte swizzle; identical in every CTA of the cluster) ----
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -162,19 +192,21 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
   const uint32_t bars = smem_u32(smem);
   auto BAR = [&](int i) { return bars + 8u * (uint32_t)i; };
   constexpr int Q_FULL = 0, FULL_K = 1, FULL_V = 1 + KT_MAX_STAGES, EMPTY_K = 1 + 2 * KT_MAX_STAGES, EMPTY_V = 1 + 3 * KT_MAX_STAGES;
-  constexpr int S_FULL = 1 + 4 * KT_MAX_STAGES, P_FULL = S_FULL + 2, PV_DONE = S_FULL + 4, DRAIN = S_FULL + 6;
+  constexpr int S_FULL = 1 + 4 * KT_MAX_STAGES, P_FULL = S_FULL + 2, PV_DONE = S_FULL + 4, DRAIN = S_FULL + 6, MERGE = S_FULL + 7;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 260);
-  uint32_t* m_enc = reinterpret_cast<uint32_t*>(smem + 512);        // [64] references (log2 units), order-preserving codes
-  uint32_t* m_old = reinterpret_cast<uint32_t*>(smem + 768);        // [64] references before a raise
+  float* m_ref = reinterpret_cast<float*>(smem + 512);              // [64] references of the columns (log2 units)
+  uint32_t* enc = reinterpret_cast<uint32_t*>(smem + 768);          // [64] scratch of a raise: column maxima, order-preserving codes
   float* l_tot = reinterpret_cast<float*>(smem + 1024);             // [64] sums of this split
-  float* alpha_s = reinterpret_cast<float*>(smem + 1280);           // [64] rescale factors of a raise
+  float* delta_s = reinterpret_cast<float*>(smem + 1280);           // [64] by how much a raise lifts each reference
   float* l_w = reinterpret_cast<float*>(smem + 1536);               // [4][64] per-warp sums
-  float2* ml_recv = reinterpret_cast<float2*>(smem + 2560);         // [S][QL] (reference, sum) pairs pushed by the splits
   unsigned char* q_s = smem + KT_CTRL;                              // [H][NP rows][128 B]
   unsigned char* p_s = q_s + H * NP * 128;                          // [PB][128 key rows][128 B]
   unsigned char* ring = p_s + kp.PB * PBUF;                         // [NS][K tile | V tile]
-  float* recv = reinterpret_cast<float*>(ring + (size_t)NS * SLOT); // [S][QL][D] un-normalised O^T columns pushed by the splits
+  // cluster merge: what the S splits push into this CTA (it owns DL head dimensions of every column)
+  float* recv = reinterpret_cast<float*>(ring + (size_t)NS * SLOT); // [S][NP/4][DL] float4: un-normalised O^T, four columns of one owned head dimension
+  float2* ml_recv = reinterpret_cast<float2*>(recv + (size_t)S * kp.DL * NP);   // [S][NP] (reference, sum) of every column
+  float* w_s = reinterpret_cast<float*>(ml_recv + (size_t)S * NP);  // [S][NP] merge weights, normalisation folded in
 
   if (tid == 0) {                        // the descriptors live in the kernel parameters: fetch them while the CTA sets up
     prefetch_tmap(&tm.k1); prefetch_tmap(&tm.v1);
@@ -193,10 +225,15 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
       mbar_init(BAR(PV_DONE + i), 1);
     }
     mbar_init(BAR(DRAIN), 1);
+    mbar_init(BAR(MERGE), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    if (S > 1) {
+      // what the S splits will push into this CTA: the O^T rows of the head dimensions it owns, and every column's pair
+      const int rows = min(((split + 1) * D + S - 1) / S, D) - (split * D + S - 1) / S;
+      mbar_expect_tx(BAR(MERGE), (uint32_t)(S * (rows * NP * 4 + N * 8)));
+    }
   }
-  if (tid >= 64 && tid < 128) m_enc[tid - 64] = f2ord(-INFINITY);
   // query rows past N (N not a multiple of 32) take part in the MMAs: they must be finite
   if (N < NP)
     for (int i = tid; i < H * (NP - N) * 8; i += KT_THREADS) {
@@ -213,27 +250,28 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   // The next kernel in the stream may start its own set-up now; before it touches anything this kernel writes it
-  // waits for this grid to complete (griddepcontrol.wait below, in that kernel).
-  grid_launch_dependents();
-  if (S > 1) cluster_arrive_relaxed();   // phase 1 of the cluster barrier: "this CTA runs"; waited for before the pushes
+  // waits for this grid to complete (griddepcontrol.wait, in that kernel).
+  if (kp.early_trigger) grid_launch_dependents();
+  if (S > 1) cluster_arrive_release();   // the one cluster barrier: "this CTA runs, its barriers are set up"; waited for before the pushes
 
   // ---- this CTA's share of the key axis, in groups of 32 rows ----
-  // The count of source 1 is read before the grid dependency only at the reuse step (older than any running kernel).
   int n1 = 0, g1 = 0, gb = 0, ge = 0, T = 0;
-  auto read_counts = [&]() {
-    n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
-    n1 = min(max(n1, 0), p.n1_max);
+  auto set_counts = [&](int n1_raw) {
+    n1 = min(max(n1_raw, 0), p.n1_max);
     g1 = (n1 + 31) >> 5;
     const int gt = g1 + ((n2 + 31) >> 5);
     gb = (int)(((long long)split * gt) / S);
     ge = (int)(((long long)(split + 1) * gt) / S);
     T = (ge - gb + 3) >> 2;
   };
-  if (kp.early_src1) read_counts();
-  // Everything but the first loads of the producer lane comes after the kernels in front of this one: the other
-  // threads read the counts, write global memory, or depend on Q.
-  if (tid != 0) {
+  auto read_counts = [&]() { set_counts(p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max); };
+  if (kp.early_src1) set_counts(n1_early);
+  // Everything but the first loads of the producer comes after the kernels in front of this one: the other threads read
+  // the counts, write global memory, or depend on Q. (The whole producer warp stays out of griddepcontrol.wait until
+  // its lane 0 has issued those loads: a warp blocks in that wait as a whole, divergent lanes included.)
+  if (warp != 0) {
     grid_dependency_wait();
+    if (!kp.early_trigger) grid_launch_dependents();
     if (!kp.early_src1) read_counts();
   }
 
@@ -244,41 +282,39 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
 
   if (warp == 0) {
     // ======================================= TMA producer =======================================
-    if (lane == 0) {
-      bool dep = false, ok = true;
-      int k_issued = 0, v_issued = 0;    // tiles whose K / V loads are on their way
-      auto dependency = [&]() {          // everything loaded from here on may have been written by the previous kernels
-        if (dep) return;
-        grid_dependency_wait();
-        dep = true;
-        if (!kp.early_src1) read_counts();
-        mbar_expect_tx(BAR(Q_FULL), (uint32_t)(H * N * 128));
-        for (int h = 0; h < H; ++h) tma_load_4d(smem_u32(q_s + h * NP * 128), &tm.q, BAR(Q_FULL), h * 64, 0, g * p.G, bi);
-      };
-      if (!kp.early_src1) dependency();
-      for (int t = 0; t < T && ok; ++t) {
-        const int s = t % NS;
-        const uint32_t ph = ((t / NS) - 1) & 1;
-        const int gi0 = gb + 4 * t, ng = min(4, ge - gi0);
-        // a tile that needs the ring to turn, or holds rows of source 2, comes after the dependency (and after Q)
-        if (t >= NS || gi0 + ng > g1) dependency();
-        uint32_t bytes = 0;
-        for (int j = 0; j < ng; ++j) bytes += (uint32_t)(H * 128 * (gi0 + j < g1 ? 32 : kp.gr2));
-        const uint32_t kdst = smem_u32(ring + (size_t)s * SLOT), vdst = kdst + KV_BYTES;
-        for (int kv = 0; kv < 2; ++kv) {
-          const int full = kv == 0 ? FULL_K : FULL_V, empty = kv == 0 ? EMPTY_K : EMPTY_V;
-          if (t >= NS && !wait_bar(BAR(empty + s), ph, abort_flag, p.status, 1 + kv, wlim)) { ok = false; break; }
-          mbar_expect_tx(BAR(full + s), bytes);
-          for (int j = 0; j < ng; ++j) {
-            const Group x = group_of(gi0 + j, g1, n1, n2);
-            const CUtensorMap* m = kv == 0 ? (x.src1 ? &tm.k1 : &tm.k2) : (x.src1 ? &tm.v1 : &tm.v2);
-            for (int h = 0; h < H; ++h)
-              tma_load_4d((kv == 0 ? kdst : vdst) + h * HALF + j * 4096, m, BAR(full + s), h * 64, x.row0, g, bi);
-          }
-          if (kv == 0) k_issued = t + 1; else v_issued = t + 1;
+    int t_next = 0, k_issued = 0, v_issued = 0;      // lane 0: next tile to load; tiles whose K / V loads are on their way
+    auto issue_tile = [&](int t) -> bool {           // lane 0 only
+      const int s = t % NS;
+      const uint32_t ph = ((t / NS) - 1) & 1;
+      const int gi0 = gb + 4 * t, ng = min(4, ge - gi0);
+      uint32_t bytes = 0;
+      for (int j = 0; j < ng; ++j) bytes += (uint32_t)(H * 128 * (gi0 + j < g1 ? 32 : kp.gr2));
+      const uint32_t kdst = smem_u32(ring + (size_t)s * SLOT), vdst = kdst + KV_BYTES;
+      for (int kv = 0; kv < 2; ++kv) {
+        const int full = kv == 0 ? FULL_K : FULL_V, empty = kv == 0 ? EMPTY_K : EMPTY_V;
+        if (t >= NS && !wait_bar(BAR(empty + s), ph, abort_flag, p.status, 1 + kv, wlim)) return false;
+        mbar_expect_tx(BAR(full + s), bytes);
+        for (int j = 0; j < ng; ++j) {
+          const Group x = group_of(gi0 + j, g1, n1, n2);
+          const CUtensorMap* m = kv == 0 ? (x.src1 ? &tm.k1 : &tm.k2) : (x.src1 ? &tm.v1 : &tm.v2);
+          for (int h = 0; h < H; ++h)
+            tma_load_4d((kv == 0 ? kdst : vdst) + h * HALF + j * 4096, m, BAR(full + s), h * 64, x.row0, g, bi);
         }
+        if (kv == 0) k_issued = t + 1; else v_issued = t + 1;
       }
-      dependency();                      // a CTA without tiles still loads Q: the MMA lane waits for it before it leaves
+      return true;
+    };
+    // ahead of the dependency: the tiles that fit the ring without turning it and hold rows of source 1 only
+    if (lane == 0 && kp.early_src1)
+      while (t_next < T && t_next < NS && gb + 4 * t_next + min(4, ge - (gb + 4 * t_next)) <= g1) issue_tile(t_next++);
+    __syncwarp();
+    grid_dependency_wait();              // everything loaded from here on may have been written by the previous kernels
+    if (!kp.early_trigger) grid_launch_dependents();
+    if (!kp.early_src1) read_counts();
+    if (lane == 0) {
+      mbar_expect_tx(BAR(Q_FULL), (uint32_t)(H * N * 128));
+      for (int h = 0; h < H; ++h) tma_load_4d(smem_u32(q_s + h * NP * 128), &tm.q, BAR(Q_FULL), h * 64, 0, g * p.G, bi);
+      while (t_next < T && issue_tile(t_next)) ++t_next;
       if (*abort_flag) {
         // let the copies that were issued land before the CTA retires
         for (int j = max(k_issued - NS, 0); j < k_issued; ++j) drain_bar(BAR(FULL_K + j % NS), (j / NS) & 1);
@@ -353,50 +389,70 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
       if (!dead && !wait_bar_warp(BAR(S_FULL + sb), (t >> 1) & 1, abort_flag, p.status, 9, wlim)) dead = true;
       tc_fence_after();
       const bool work = active && !dead;
-      uint32_t sv[NP];
+      float sv[NP];                                    // this key's logits against the N queries, then their scaled distance to the references
       if (work) {
 #pragma unroll
         for (int c = 0; c < NCH; ++c) tmem_ld32(lane_addr + (uint32_t)sb * NP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
         tc_wait_ld();
       } else {
 #pragma unroll
-        for (int c = 0; c < NP; ++c) sv[c] = 0u;
+        for (int c = 0; c < NP; ++c) sv[c] = 0.f;
       }
-      // ---- the references: set from the first tile's column maxima, afterwards only checked ----
-      bool raise = t == 0;
-      if (t > 0) {
-        bool over = false;
-        if (work && valid) {
+      // ---- saliency of this key (refresh step): scale * mean of its N logits ----
+      if (scores && work && valid && x.src1) {
+        float a4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int c = 0; c < NP; ++c) over |= __uint_as_float(sv[c]) * sl2 > ord2f(m_enc[c]) + 8.f;
-        }
-        raise = softmax_barrier_or(over);
-        if (raise) {
-          // (rare) every PV issued so far must have landed before O^T is rewritten; the PV of this tile waits for our arrive
-          if (!dead && !wait_bar_warp(BAR(PV_DONE + ((t - 1) & 1)), ((t - 1) >> 1) & 1, abort_flag, p.status, 8, wlim)) dead = true;
-          tc_fence_after();
-          if (tid - 64 < NP) m_old[tid - 64] = m_enc[tid - 64];
-          softmax_barrier();
-        }
+        for (int c = 0; c < NP; ++c)
+          if (c < N) a4[c & 3] += sv[c];
+        p.raw_scores[(int64_t)(bi * p.Hkv + g) * p.n1_max + x.row0 + lane] = ((a4[0] + a4[1]) + (a4[2] + a4[3])) * (p.scale / (float)N);
       }
-      if (raise) {
+      // ---- the references. The first key of the CTA's first tile lends its logits: it is part of the softmax, so sums
+      //      never vanish, and exp2 of anything up to 2^64 above it is still an ordinary bf16 / fp32 number. Every tile is
+      //      only checked against the references; one that exceeds them by more than 64 raises them (rare). ----
+      if (t == 0) {
+        if (row == 0 && work) {
+#pragma unroll
+          for (int c = 0; c < NP; c += 4)
+            *reinterpret_cast<float4*>(m_ref + c) = make_float4(sv[c] * sl2, sv[c + 1] * sl2, sv[c + 2] * sl2, sv[c + 3] * sl2);
+        }
+        softmax_barrier();
+      }
+      bool over = false;
+#pragma unroll
+      for (int c = 0; c < NP; c += 4) {
+        const float4 m4 = *reinterpret_cast<const float4*>(m_ref + c);
+        sv[c] = fmaf(sv[c], sl2, -m4.x); sv[c + 1] = fmaf(sv[c + 1], sl2, -m4.y);
+        sv[c + 2] = fmaf(sv[c + 2], sl2, -m4.z); sv[c + 3] = fmaf(sv[c + 3], sl2, -m4.w);
+        over |= (sv[c] > 64.f) | (sv[c + 1] > 64.f) | (sv[c + 2] > 64.f) | (sv[c + 3] > 64.f);
+      }
+      if (softmax_barrier_or(over && work && valid)) {
+        // ---- raise the references by the tile's column maxima (where positive) and rescale what has been accumulated.
+        //      Every PV issued so far must have landed before O^T is rewritten; the PV of this tile waits for our arrive. ----
+        if (t > 0 && !dead && !wait_bar_warp(BAR(PV_DONE + ((t - 1) & 1)), ((t - 1) >> 1) & 1, abort_flag, p.status, 8, wlim)) dead = true;
+        tc_fence_after();
+        if (tid - 64 < NP) enc[tid - 64] = f2ord(0.f);
+        softmax_barrier();
         if (work) {
           float mine[NCH];
 #pragma unroll
           for (int c = 0; c < NP; ++c) {
-            const float r = warp_max_f32(valid ? __uint_as_float(sv[c]) : -INFINITY);
+            const float r = warp_max_f32(valid ? sv[c] : -INFINITY);
             if ((c & 31) == lane) mine[c >> 5] = r;
           }
 #pragma unroll
-          for (int c = 0; c < NCH; ++c) atomicMax(m_enc + c * 32 + lane, f2ord(mine[c] * sl2));
+          for (int c = 0; c < NCH; ++c) atomicMax(enc + c * 32 + lane, f2ord(mine[c]));
         }
         softmax_barrier();
-      }
-      if (raise && t > 0) {
-        if (tid - 64 < NP) alpha_s[tid - 64] = fast_exp2(ord2f(m_old[tid - 64]) - ord2f(m_enc[tid - 64]));
+        if (tid - 64 < NP) {
+          const float dlt = ord2f(enc[tid - 64]);      // >= 0
+          delta_s[tid - 64] = dlt;
+          m_ref[tid - 64] += dlt;
+        }
         softmax_barrier();
-        // this thread's TMEM lane is a head dimension of O^T here, not a key: all four warps rescale their lanes
-        if (!dead) {
+#pragma unroll
+        for (int c = 0; c < NP; ++c) sv[c] -= delta_s[c];
+        if (t > 0 && !dead) {
+          // this thread's TMEM lane is a head dimension of O^T here, not a key: all four warps rescale their lanes
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
             uint32_t o32[32];
@@ -404,7 +460,7 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
             tc_wait_ld();
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-              const float a = alpha_s[c * 32 + i];
+              const float a = fast_exp2(-delta_s[c * 32 + i]);
               o32[i] = __float_as_uint(__uint_as_float(o32[i]) * a);
               l_acc[c * 32 + i] *= a;
             }
@@ -413,16 +469,9 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
           }
           tc_wait_st();
         }
+        softmax_barrier();               // delta_s and m_ref are stable again before the next tile reads them
       }
-      // ---- saliency of this key (refresh step): scale * mean of its N logits ----
-      if (scores && work && valid && x.src1) {
-        float a4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int c = 0; c < NP; ++c)
-          if (c < N) a4[c & 3] += __uint_as_float(sv[c]);
-        p.raw_scores[(int64_t)(bi * p.Hkv + g) * p.n1_max + x.row0 + lane] = ((a4[0] + a4[1]) + (a4[2] + a4[3])) * (p.scale / (float)N);
-      }
-      // ---- P^T = exp2(S^T * scale_log2 - reference) as bf16, one 128-byte row per key (128-byte swizzle) ----
+      // ---- P^T = exp2(distance to the reference) as bf16, one 128-byte row per key (128-byte swizzle) ----
       // the P^T buffer is free once the PV that read it has completed
       if (!dead && t >= kp.PB &&
           !wait_bar_warp(BAR(PV_DONE + ((t - kp.PB) & 1)), ((t - kp.PB) >> 1) & 1, abort_flag, p.status, 6, wlim))
@@ -435,8 +484,8 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int c = c8 * 8 + 2 * i;
-            const float e0 = valid ? fast_exp2(fmaf(__uint_as_float(sv[c]), sl2, -ord2f(m_enc[c]))) : 0.f;
-            const float e1 = valid ? fast_exp2(fmaf(__uint_as_float(sv[c + 1]), sl2, -ord2f(m_enc[c + 1]))) : 0.f;
+            const float e0 = fast_exp2(valid ? sv[c] : -INFINITY);
+            const float e1 = fast_exp2(valid ? sv[c + 1] : -INFINITY);
             l_acc[c] += e0; l_acc[c + 1] += e1;
             pk[i] = pack_bf16(e0, e1);
           }
@@ -462,10 +511,11 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
 
   // ======================================= epilogue =======================================
   const bool do_attn = p.out != nullptr;
-  uint32_t ov[NP];                       // softmax warps: this thread's head dimension of O^T, all columns
+  const int DL = kp.DL;                  // head dimensions a CTA owns in the merge: ceil(D / S)
   if (warp >= 2) {
     const int q4 = warp & 3;
-    const int row = q4 * 32 + lane;
+    const int row = q4 * 32 + lane;      // from here on: a head dimension of O^T
+    const int st = tid - 64;             // 0..127
     // ---- column sums over the 128 key rows: shuffle transpose inside a warp (lane i ends up with column i), then the
     //      four warps' rows in a fixed order ----
 #pragma unroll
@@ -485,10 +535,26 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
       }
       l_w[(warp - 2) * 64 + c * 32 + lane] = v[0];
     }
+    if (S > 1 && p.want_scores) __threadfence();       // this thread's raw saliency, ahead of the pushes that tell the peers
     softmax_barrier();
-    if (tid - 64 < NP) l_tot[tid - 64] = (l_w[tid - 64] + l_w[64 + tid - 64]) + (l_w[128 + tid - 64] + l_w[192 + tid - 64]);
-    softmax_barrier();
+    float l_mine = 0.f, m_mine = -INFINITY;            // thread st < NP: sum and reference of column st
+    if (st < NP) {
+      l_mine = (l_w[st] + l_w[64 + st]) + (l_w[128 + st] + l_w[192 + st]);
+      m_mine = T > 0 ? m_ref[st] : -INFINITY;
+      l_tot[st] = l_mine;
+    }
+    if (S > 1) {
+      // every split's (reference, sum) of every column goes to every CTA of the cluster
+      cluster_wait_acquire();            // every CTA of the cluster runs: its shared memory and barriers may be written
+      if (st < N) {
+        const uint32_t ml_a = smem_u32(ml_recv + split * NP + st);
+        for (int r = 0; r < S; ++r) st_async_f2(map_to_cta(ml_a, (uint32_t)r), map_to_cta(BAR(MERGE), (uint32_t)r), m_mine, l_mine);
+      }
+    } else {
+      softmax_barrier();                 // l_tot
+    }
     // ---- the finished accumulator row of this thread ----
+    uint32_t ov[NP];
     const bool have_o = do_attn && !dead && T > 0 &&
                         wait_bar_warp(BAR(PV_DONE + ((T - 1) & 1)), ((T - 1) >> 1) & 1, abort_flag, p.status, 6, wlim);
     tc_fence_after();
@@ -500,75 +566,99 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
 #pragma unroll
       for (int c = 0; c < NP; ++c) ov[c] = 0u;
     }
-    if (S == 1 && do_attn && !*abort_flag) {
-      // one split: normalise and store; a warp writes 32 consecutive bf16 of one output row per column
-      if (row < D) {
+    if (S == 1) {
+      if (do_attn && !*abort_flag) {
+        // one split: normalise and store; a warp writes 32 consecutive bf16 of one output row per column
+        if (row < D) {
 #pragma unroll
-        for (int c = 0; c < NP; ++c) {
-          if (c >= N) break;
-          const float l = l_tot[c];
-          const float inv = l > 0.f ? 1.f / l : 0.f;
-          const int hg = c / p.b, i = c - hg * p.b;
-          reinterpret_cast<__nv_bfloat16*>(p.out)[(int64_t)bi * p.o_stride[0] + (int64_t)(g * p.G + hg) * p.o_stride[1] +
-                                                   (int64_t)i * p.o_stride[2] + row] = __float2bfloat16_rn(__uint_as_float(ov[c]) * inv);
+          for (int c = 0; c < NP; ++c) {
+            if (c >= N) break;
+            const float l = l_tot[c];
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            const int hg = c / p.b, i = c - hg * p.b;
+            reinterpret_cast<__nv_bfloat16*>(p.out)[(int64_t)bi * p.o_stride[0] + (int64_t)(g * p.G + hg) * p.o_stride[1] +
+                                                     (int64_t)i * p.o_stride[2] + row] = __float2bfloat16_rn(__uint_as_float(ov[c]) * inv);
+          }
+        }
+        if (p.lse && st < N) {
+          const int hg = st / p.b, i = st - hg * p.b;
+          p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (m_mine + log2f(l_mine)) * kLn2;
         }
       }
-      if (p.lse && tid - 64 < N) {
-        const int c = tid - 64;
-        const int hg = c / p.b, i = c - hg * p.b;
-        p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (ord2f(m_enc[c]) + log2f(l_tot[c])) * kLn2;
-      }
+    } else if (row < D) {
+      // ---- this head dimension's row of O^T goes to the CTA that owns the dimension, 16 bytes at a time (always, also
+      //      when this CTA is aborting: the owner counts the bytes) ----
+      const int owner = row * S / D;
+      const int dl = row - (owner * D + S - 1) / S;
+      const uint32_t dst = map_to_cta(smem_u32(recv + ((size_t)split * (NP / 4) * DL + dl) * 4), (uint32_t)owner);
+      const uint32_t mb = map_to_cta(BAR(MERGE), (uint32_t)owner);
+#pragma unroll
+      for (int c4 = 0; c4 < NP / 4; ++c4)          // consecutive lanes (head dimensions) write consecutive 16-byte units
+        st_async_f4(dst + (uint32_t)(c4 * DL * 16), mb, __uint_as_float(ov[4 * c4]), __uint_as_float(ov[4 * c4 + 1]),
+                    __uint_as_float(ov[4 * c4 + 2]), __uint_as_float(ov[4 * c4 + 3]));
     }
   }
 
   if (S > 1) {
-    // ---- cluster merge: every split pushes each column to the CTA that owns it; one barrier; owners merge and store ----
-    cluster_wait_acquire();              // phase 1: every CTA of the cluster runs, so its shared memory may be written
-    const int QL = kp.QL;
-    if (warp >= 2 && do_attn) {
-      const int row = (warp & 3) * 32 + lane;
-      const uint32_t recv_a = smem_u32(recv), ml_a = smem_u32(ml_recv);
-      if (row < D) {
-#pragma unroll
-        for (int c = 0; c < NP; ++c) {
-          if (c >= N) break;
-          const int owner = c / QL, ql = c - owner * QL;
-          st_cluster_f32(map_to_cta(recv_a + (uint32_t)(((split * QL + ql) * D + row) * 4), (uint32_t)owner), __uint_as_float(ov[c]));
-        }
-      }
-      if (tid - 64 < N) {
-        const int c = tid - 64;
-        const int owner = c / QL, ql = c - owner * QL;
-        st_cluster_f2(map_to_cta(ml_a + (uint32_t)((split * QL + ql) * 8), (uint32_t)owner), ord2f(m_enc[c]), l_tot[c]);
-      }
-    }
-    __threadfence();                     // the raw saliency of this split, for the peers that pool it
-    cluster_arrive_release();
-    cluster_wait_acquire();
+    // ---- cluster merge: once everything owed to this CTA has landed, it merges and stores the head dimensions it owns ----
+    if (warp < 2) cluster_wait_acquire();              // (the softmax warps passed the cluster barrier before their pushes)
+    wait_merge(BAR(MERGE), abort_flag, p.status, wlim);
     if (warp >= 2 && do_attn && !*abort_flag) {
-      const int row = (warp & 3) * 32 + lane;
-      const int c_lo = split * QL, c_hi = min(c_lo + QL, N);
-      for (int c = c_lo; c < c_hi; ++c) {
-        const int ql = c - c_lo;
+      const int st = tid - 64;
+      // weights of the S splits for column st, the normalisation folded in
+      if (st < N) {
+        float2 x[8];
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2) x[s2] = ml_recv[min(s2, S - 1) * NP + st];
         float mstar = -INFINITY;
-        for (int s2 = 0; s2 < S; ++s2) {
-          const float2 x = ml_recv[s2 * QL + ql];
-          if (x.y > 0.f) mstar = fmaxf(mstar, x.x);
-        }
-        float acc = 0.f, l = 0.f;
-        for (int s2 = 0; s2 < S; ++s2) {
-          const float2 x = ml_recv[s2 * QL + ql];
-          if (!(x.y > 0.f)) continue;
-          const float w = fast_exp2(x.x - mstar);
-          l = fmaf(x.y, w, l);
-          if (row < D) acc = fmaf(recv[(s2 * QL + ql) * D + row], w, acc);
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2)
+          if (s2 < S && x[s2].y > 0.f) mstar = fmaxf(mstar, x[s2].x);
+        float w[8], l = 0.f;
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2) {
+          w[s2] = (s2 < S && x[s2].y > 0.f) ? fast_exp2(x[s2].x - mstar) : 0.f;
+          l = fmaf(x[s2].y, w[s2], l);
         }
         const float inv = l > 0.f ? 1.f / l : 0.f;
-        const int hg = c / p.b, i = c - hg * p.b;
-        if (row < D)
-          reinterpret_cast<__nv_bfloat16*>(p.out)[(int64_t)bi * p.o_stride[0] + (int64_t)(g * p.G + hg) * p.o_stride[1] +
-                                                   (int64_t)i * p.o_stride[2] + row] = __float2bfloat16_rn(acc * inv);
-        if (row == 0 && p.lse) p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2)
+          if (s2 < S) w_s[s2 * NP + st] = w[s2] * inv;
+        if (split == 0 && p.lse) {
+          const int hg = st / p.b, i = st - hg * p.b;
+          p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
+        }
+      }
+      softmax_barrier();
+      // thread -> (owned head dimension, chunk of columns); all loads of a group of four columns are in flight together
+      const int d_lo = (split * D + S - 1) / S, d_hi = min(((split + 1) * D + S - 1) / S, D);
+      const int dl = st % DL, qc = st / DL;
+      const int cpt = kp.cpt;            // columns per thread, a multiple of 4
+      if (d_lo + dl < d_hi) {
+        for (int c0 = qc * cpt; c0 < min((qc + 1) * cpt, N); c0 += 4) {
+          float4 r4[8], w4[8];
+#pragma unroll
+          for (int s2 = 0; s2 < 8; ++s2) {
+            const int sc = min(s2, S - 1);
+            r4[s2] = *reinterpret_cast<const float4*>(recv + ((size_t)(sc * (NP / 4) + (c0 >> 2)) * DL + dl) * 4);
+            w4[s2] = *reinterpret_cast<const float4*>(w_s + sc * NP + c0);
+          }
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (int s2 = 0; s2 < 8; ++s2)
+            if (s2 < S) {
+              acc.x = fmaf(r4[s2].x, w4[s2].x, acc.x); acc.y = fmaf(r4[s2].y, w4[s2].y, acc.y);
+              acc.z = fmaf(r4[s2].z, w4[s2].z, acc.z); acc.w = fmaf(r4[s2].w, w4[s2].w, acc.w);
+            }
+          const float a[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+          for (int i4 = 0; i4 < 4; ++i4) {
+            const int c = c0 + i4;
+            const int hg = c / p.b, i = c - hg * p.b;
+            reinterpret_cast<__nv_bfloat16*>(p.out)[(int64_t)bi * p.o_stride[0] + (int64_t)(g * p.G + hg) * p.o_stride[1] +
+                                                     (int64_t)i * p.o_stride[2] + d_lo + dl] = __float2bfloat16_rn(a[i4]);
+          }
+        }
       }
     }
   } else {
@@ -596,10 +686,11 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
 
 // ---------------------------------------------------------------------------------------------------------
 // Host side
-size_t kt_smem_bytes(int D, int NP, int NS, int PB, int S, int QL) {
+size_t kt_smem_bytes(int D, int NP, int NS, int PB, int S) {
   const size_t H = D / 64;
+  const size_t DL = (D + S - 1) / S;
   return 1024 /*alignment slack*/ + KT_CTRL + H * NP * 128 + (size_t)PB * 128 * 128 + (size_t)NS * 2 * H * 128 * 128 +
-         (S > 1 ? (size_t)S * QL * D * 4 : 0);
+         (S > 1 ? (size_t)S * DL * NP * 4 /*recv*/ + (size_t)S * NP * 12 /*ml_recv, w_s*/ : 0);
 }
 
 template <int D, int NCH>
@@ -655,26 +746,24 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   if (want > by_tiles) want = by_tiles;
   if (tn.splits > 0) want = tn.splits;
   if (want > 8) want = 8;
-  if (want > M) want = M;
   if (want < 1) want = 1;
   const int S = (int)want;
-  const int QL = (M + S - 1) / S;
   const int tiles_cta = ((groups + S - 1) / S + 3) / 4;
   // Ring depth and P^T buffers. With few query columns, and either more CTAs than SMs or a single tile per CTA, the
   // footprint is kept below half an SM, so that two CTAs are resident and the next call's CTAs can start loading while
   // this call's finish; otherwise the CTA takes what one SM has.
-  const size_t half_sm = 113 * 1024;
+  const size_t half_sm = 113 * 1024;     // two CTAs of this size, each with its 1 KB system share, fit one SM
   int NS = 1, PB = 1;
   const bool small = NP == 32 && (units * S > sms || tiles_cta <= 1);
   if (small) {
-    while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, NP, NS + 1, PB, S, QL) <= half_sm) ++NS;
+    while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, NP, NS + 1, PB, S) <= half_sm) ++NS;
   } else {
     PB = 2;
-    while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, NP, NS + 1, PB, S, QL) <= 226 * 1024) ++NS;
+    while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, NP, NS + 1, PB, S) <= 226 * 1024) ++NS;
   }
   if (tn.stages > 0) {
     NS = tn.stages > KT_MAX_STAGES ? KT_MAX_STAGES : tn.stages;
-    while (NS > 1 && kt_smem_bytes(D, NP, NS, PB, S, QL) > 226 * 1024) --NS;
+    while (NS > 1 && kt_smem_bytes(D, NP, NS, PB, S) > 226 * 1024) --NS;
   }
   pl.splits = 1;                        // nothing is left in the workspace: the splits merge inside their cluster
   pl.parts = 1;
@@ -683,7 +772,7 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   pl.m_warps = PB;                      // (field reused: P^T buffers)
   pl.part_rows = 0;
   pl.n_counters = 0;
-  pl.smem_bytes = kt_smem_bytes(D, NP, NS, PB, S, QL);
+  pl.smem_bytes = kt_smem_bytes(D, NP, NS, PB, S);
   return pl;
 }
 
@@ -694,9 +783,15 @@ cudaError_t launch_attn_kt(const AttnParams& p, const AttnPlan& pl, int D, cudaS
   kp.a = p;
   kp.a.wait_cycles = tn.wait_cycles;
   kp.N = p.M; kp.S = pl.cluster; kp.NS = pl.stages; kp.PB = pl.m_warps;
-  kp.QL = (p.M + kp.S - 1) / kp.S;
+  kp.DL = (D + kp.S - 1) / kp.S;
+  {
+    const int NPc = p.M <= 32 ? 32 : 64;
+    const int chunks = 128 / kp.DL;                      // threads that share one owned head dimension
+    kp.cpt = ((NPc + chunks - 1) / chunks + 3) / 4 * 4;
+  }
   kp.gr2 = p.n2 < 32 ? p.n2 : 32;
   kp.early_src1 = (p.n2 > 0 && p.n1_max > 0 && tn.early_loads != 0) ? 1 : 0;
+  kp.early_trigger = tn.trigger != 0 ? 1 : 0;
   kp.wait_cycles = tn.wait_cycles;
   memset(&tm, 0, sizeof(tm));
   bool ok = umma_make_map(&tm.q, p.q, D, p.b, p.Hq, p.B, p.q_stride, p.b, p.G);
