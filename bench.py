@@ -375,7 +375,7 @@ def run_ours(args):
         refresh_only()                              # every layer's cache exists before any reuse step runs
     stream.synchronize()
     d0 = caches[0].desc
-    refresh_launches = B.launch_count(d0, B.OP_REFRESH_SCORES) + B.launch_count(d0, B.OP_SELECT_TOPK) + B.launch_count(d0, B.OP_COMPACT_KV)
+    refresh_launches = B.launch_count(d0, B.OP_REFRESH_SCORES) + B.launch_count(d0, B.OP_SELECT_COMPACT)
     sparse_launches = reuse_steps * B.launch_count(d0, B.OP_SPARSE_BLOCK_ATTN)
     launches_per_step = n_layers * ((refresh_launches if args.phase in ("all", "refresh") else 0) +
                                     (sparse_launches if args.phase in ("all", "sparse") else 0))

@@ -67,7 +67,8 @@ typedef enum {
   SDLLM_OP_SELECT_TOPK = 1,
   SDLLM_OP_COMPACT_KV = 2,
   SDLLM_OP_SPARSE_BLOCK_ATTN = 3,
-  SDLLM_OP_DENSE_ATTN = 4
+  SDLLM_OP_DENSE_ATTN = 4,
+  SDLLM_OP_SELECT_COMPACT = 5
 } sdllm_op;
 
 /* Problem description, filled by the caller. Plain data; set struct_size = sizeof(sdllm_desc). */
@@ -155,6 +156,18 @@ sdllm_status sdllm_select_topk(const sdllm_desc* desc, const float* pooled_score
  * same for v, bit-exact. Rows j >= kept_cnt[i] are zero-filled. */
 sdllm_status sdllm_compact_kv(const sdllm_desc* desc, const void* k, const void* v, const int32_t* kept_idx,
                               const int32_t* kept_cnt, void* k_c, void* v_c, void* cuda_stream);
+
+/* Refresh step, parts 2 and 3 in one call (Algorithm 1 from "n <- floor(|I| r)" to the cache store): exactly the results of
+ * sdllm_select_topk followed by sdllm_compact_kv - the same kept_idx, kept_cnt, k_c and v_c, bit for bit - but, while the
+ * candidates of a head fit the shared memory of a CTA (seq_len_max - block_len <= 8192), in ONE launch: the CTAs that
+ * select a head's entries copy its rows themselves, so the index list makes no round trip through memory. Longer
+ * sequences run the two kernels one after the other inside this call (sdllm_launch_count tells which). The launch may
+ * start while the kernel in front of it in the stream is finishing and reads pooled_scores only once that kernel has
+ * completed; it holds its own dependents back until it has completed, so the reuse step that follows may read the
+ * compacted cache early (see sdllm_sparse_block_attn). */
+sdllm_status sdllm_select_compact(const sdllm_desc* desc, const float* pooled_scores, const int32_t* seq_len,
+                                  const int32_t* block_off, const void* k, const void* v, int32_t* kept_idx,
+                                  int32_t* kept_cnt, void* k_c, void* v_c, void* cuda_stream);
 
 /* Reuse step (cache_state 2, Algorithm 3): out = softmax(scale * Q_b' [K_c ; K_n]^T) [V_c ; V_n] over the first
  * kept_cnt[i] rows of the compacted cache followed by the block's b fresh rows k_blk, v_blk.

@@ -18,12 +18,12 @@ F32, BF16 = 0, 1
 SCORE_LOGIT_MEAN, SCORE_PROB_MEAN = 0, 1
 POOL_MAX, POOL_AVG = 0, 1
 SELECT_JOINT_FLOOR, SELECT_PER_REGION_CEIL, SELECT_PREFIX_ONLY = 0, 1, 2
-OP_REFRESH_SCORES, OP_SELECT_TOPK, OP_COMPACT_KV, OP_SPARSE_BLOCK_ATTN, OP_DENSE_ATTN = range(5)
+OP_REFRESH_SCORES, OP_SELECT_TOPK, OP_COMPACT_KV, OP_SPARSE_BLOCK_ATTN, OP_DENSE_ATTN, OP_SELECT_COMPACT = range(6)
 
 EXPORTS = ("sdllm_version", "sdllm_status_string", "sdllm_workspace_bytes", "sdllm_keep_count", "sdllm_cache_state", "sdllm_launch_count",
            "sdllm_read_status",
            "sdllm_refresh_scores", "sdllm_select_topk", "sdllm_compact_kv", "sdllm_sparse_block_attn",
-           "sdllm_sparse_block_attn_static", "sdllm_dense_attn", "sdllm_tuning_set", "sdllm_tuning_reset")
+           "sdllm_sparse_block_attn_static", "sdllm_dense_attn", "sdllm_select_compact", "sdllm_tuning_set", "sdllm_tuning_reset")
 
 
 class Desc(ctypes.Structure):
@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.sdllm_select_topk.argtypes = [dp, vp, i32p, i32p, vp, vp, vp, ctypes.c_size_t, vp]
         L.sdllm_compact_kv.restype = ctypes.c_int
         L.sdllm_compact_kv.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp]
+        L.sdllm_select_compact.restype = ctypes.c_int
+        L.sdllm_select_compact.argtypes = [dp, vp, i32p, i32p, vp, vp, vp, vp, vp, vp, vp]
         L.sdllm_sparse_block_attn.restype = ctypes.c_int
         L.sdllm_sparse_block_attn.argtypes = [dp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.sdllm_dense_attn.restype = ctypes.c_int
@@ -199,6 +201,13 @@ def select_topk(desc: Desc, pooled_scores, seq_len, block_off, kept_idx, kept_cn
 def compact_kv(desc: Desc, k, v, kept_idx, kept_cnt, k_c, v_c, stream=None):
     _check(lib().sdllm_compact_kv(ctypes.byref(desc), _ptr(k), _ptr(v), _ptr(kept_idx), _ptr(kept_cnt), _ptr(k_c),
                                   _ptr(v_c), _stream(stream)), "sdllm_compact_kv")
+
+
+def select_compact(desc: Desc, pooled_scores, seq_len, block_off, k, v, kept_idx, kept_cnt, k_c, v_c, stream=None):
+    """sdllm_select_topk and sdllm_compact_kv in one call (one launch while a head's candidates fit a CTA)."""
+    _check(lib().sdllm_select_compact(ctypes.byref(desc), _ptr(pooled_scores), _ptr(seq_len), _ptr(block_off), _ptr(k), _ptr(v),
+                                      _ptr(kept_idx), _ptr(kept_cnt), _ptr(k_c), _ptr(v_c), _stream(stream)),
+           "sdllm_select_compact")
 
 
 def sparse_block_attn(desc: Desc, q_blk, k_c, v_c, kept_cnt, k_blk, v_blk, out, workspace, stream=None):

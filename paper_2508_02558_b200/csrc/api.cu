@@ -198,6 +198,8 @@ int32_t sdllm_launch_count(const sdllm_desc* d, int op) {
   if (check_desc(d) != SDLLM_OK) return -1;
   if (op == SDLLM_OP_SELECT_TOPK) return 1;
   if (op == SDLLM_OP_COMPACT_KV) return d->n_keep_max > 0 ? 1 : 0;
+  if (op == SDLLM_OP_SELECT_COMPACT)
+    return select_compact_is_fused(d->seq_len_max, d->block_len, d->n_keep_max) ? 1 : 1 + (d->n_keep_max > 0 ? 1 : 0);
   if (op == SDLLM_OP_DENSE_ATTN) return dense_supported(d) ? 1 : -1;
   if (op != SDLLM_OP_REFRESH_SCORES && op != SDLLM_OP_SPARSE_BLOCK_ATTN) return -1;
   const bool refresh = op == SDLLM_OP_REFRESH_SCORES;
@@ -317,6 +319,31 @@ sdllm_status sdllm_compact_kv(const sdllm_desc* d, const void* k, const void* v,
   p.B = d->batch; p.Hkv = d->n_kv_heads; p.n_keep_max = d->n_keep_max; p.row_bytes = d->head_dim * es; p.Lmax = d->seq_len_max;
   for (int i = 0; i < 3; ++i) { p.kv_stride_bytes[i] = d->kv_stride[i] * es; p.c_stride_bytes[i] = d->c_stride[i] * es; }
   if (cuda_failed(launch_compact(p, reinterpret_cast<cudaStream_t>(cuda_stream)), "compact launch")) return SDLLM_ERR_CUDA;
+  return SDLLM_OK;
+}
+
+sdllm_status sdllm_select_compact(const sdllm_desc* d, const float* pooled_scores, const int32_t* seq_len, const int32_t* block_off,
+                                  const void* k, const void* v, int32_t* kept_idx, int32_t* kept_cnt, void* k_c, void* v_c,
+                                  void* cuda_stream) {
+  sdllm_status st = check_desc(d);
+  if (st != SDLLM_OK) return st;
+  if (!pooled_scores || !block_off || !kept_idx || !kept_cnt) return SDLLM_ERR_INVALID_ARG;
+  if (d->n_keep_max > 0 && (!k || !v || !k_c || !v_c)) return SDLLM_ERR_INVALID_ARG;
+  if (!aligned16(pooled_scores) || !aligned16(kept_idx) || !aligned16(k) || !aligned16(v) || !aligned16(k_c) || !aligned16(v_c))
+    return SDLLM_ERR_INVALID_ARG;
+  if ((st = check_device()) != SDLLM_OK) return st;
+  const int es = elem_size(d->dtype);
+  SelectParams p{};
+  p.pooled = pooled_scores; p.seq_len = seq_len; p.block_off = block_off; p.kept_idx = kept_idx; p.kept_cnt = kept_cnt;
+  p.B = d->batch; p.Hkv = d->n_kv_heads; p.Lmax = d->seq_len_max; p.b = d->block_len; p.n_keep_max = d->n_keep_max;
+  p.mode = d->select; p.retention = d->retention;
+  const int cand = d->seq_len_max - d->block_len;
+  p.smem_keys = cand <= 45056 ? cand : 0;
+  CompactParams c{};
+  c.k = k; c.v = v; c.kept_idx = kept_idx; c.kept_cnt = kept_cnt; c.k_c = k_c; c.v_c = v_c;
+  c.B = d->batch; c.Hkv = d->n_kv_heads; c.n_keep_max = d->n_keep_max; c.row_bytes = d->head_dim * es; c.Lmax = d->seq_len_max;
+  for (int i = 0; i < 3; ++i) { c.kv_stride_bytes[i] = d->kv_stride[i] * es; c.c_stride_bytes[i] = d->c_stride[i] * es; }
+  if (cuda_failed(launch_select_compact(p, c, reinterpret_cast<cudaStream_t>(cuda_stream)), "select + compact launch")) return SDLLM_ERR_CUDA;
   return SDLLM_OK;
 }
 

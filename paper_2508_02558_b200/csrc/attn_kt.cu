@@ -49,7 +49,8 @@ constexpr int KT_MAX_STAGES = 3;
 constexpr int KT_CTRL = 3072;            // control block: barriers, flags, references, sums
 
 struct KtMaps {
-  CUtensorMap q, k1, v1, k2, v2;
+  CUtensorMap q, k1, v1, k2, v2;   // boxes of 32 rows (source 2: min(32, n2))
+  CUtensorMap k1t, v1t;            // source 1 again, boxes of 128 rows: a whole tile per copy
 };
 
 struct KtParams {
@@ -68,7 +69,7 @@ struct KtParams {
 
 #include "umma_ptx.cuh"
 
-__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release;\n" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed;\n" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire;\n" ::: "memory"); }
 // Asynchronous stores into the shared memory of a CTA of the cluster; each one reports its bytes to an mbarrier of that
 // CTA (complete_tx, release at cluster scope), so the receiver waits for exactly the data it is owed and for nothing else.
@@ -100,6 +101,11 @@ __device__ __forceinline__ bool wait_merge(uint32_t bar, volatile int* abort_fla
       else return false;
     }
   }
+}
+// Pulls one box of a tensor into L2 without waiting for it. L2 is the point of coherence, so this is safe for data a
+// kernel in front of this one may still be writing: the later copy into shared memory reads what L2 holds then.
+__device__ __forceinline__ void tma_prefetch_l2(const CUtensorMap* tm, int x, int y, int z, int w) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];\n" ::"l"(tm), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
 }
 __device__ __forceinline__ float warp_max_f32(float v) {
   float r;
@@ -208,8 +214,53 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
   float2* ml_recv = reinterpret_cast<float2*>(recv + (size_t)S * kp.DL * NP);   // [S][NP] (reference, sum) of every column
   float* w_s = reinterpret_cast<float*>(ml_recv + (size_t)S * NP);  // [S][NP] merge weights, normalisation folded in
 
+  // ---- this CTA's share of the key axis, in groups of 32 rows ----
+  int n1 = 0, g1 = 0, gb = 0, ge = 0, T = 0;
+  auto set_counts = [&](int n1_raw) {
+    n1 = min(max(n1_raw, 0), p.n1_max);
+    g1 = (n1 + 31) >> 5;
+    const int gt = g1 + ((n2 + 31) >> 5);
+    gb = (int)(((long long)split * gt) / S);
+    ge = (int)(((long long)(split + 1) * gt) / S);
+    T = (ge - gb + 3) >> 2;
+  };
+  auto read_counts = [&]() { set_counts(p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max); };
+
+  // ---- the producer lane (thread 0) ----
+  int t_next = 0, k_issued = 0, v_issued = 0;        // next tile to load; tiles whose K / V loads are on their way
+  auto tile_groups = [&](int t, int& gi0) { gi0 = gb + 4 * t; return min(4, ge - gi0); };
+  auto issue_tile = [&](int t) -> bool {
+    const int s = t % NS;
+    const uint32_t ph = ((t / NS) - 1) & 1;
+    int gi0;
+    const int ng = tile_groups(t, gi0);
+    const bool whole = ng >= 3 && gi0 + ng <= g1;    // rows of source 1 only: one 128-row box per 64-column half
+    uint32_t bytes = 0;
+    if (whole) bytes = (uint32_t)KV_BYTES;
+    else for (int j = 0; j < ng; ++j) bytes += (uint32_t)(H * 128 * (gi0 + j < g1 ? 32 : kp.gr2));
+    const uint32_t kdst = smem_u32(ring + (size_t)s * SLOT), vdst = kdst + KV_BYTES;
+    for (int kv = 0; kv < 2; ++kv) {
+      const int full = kv == 0 ? FULL_K : FULL_V, empty = kv == 0 ? EMPTY_K : EMPTY_V;
+      if (t >= NS && !wait_bar(BAR(empty + s), ph, abort_flag, p.status, 1 + kv, wlim)) return false;
+      mbar_expect_tx(BAR(full + s), bytes);
+      if (whole) {
+        for (int h = 0; h < H; ++h)
+          tma_load_4d((kv == 0 ? kdst : vdst) + h * HALF, kv == 0 ? &tm.k1t : &tm.v1t, BAR(full + s), h * 64, gi0 * 32, g, bi);
+      } else {
+        for (int j = 0; j < ng; ++j) {
+          const Group x = group_of(gi0 + j, g1, n1, n2);
+          const CUtensorMap* m = kv == 0 ? (x.src1 ? &tm.k1 : &tm.k2) : (x.src1 ? &tm.v1 : &tm.v2);
+          for (int h = 0; h < H; ++h)
+            tma_load_4d((kv == 0 ? kdst : vdst) + h * HALF + j * 4096, m, BAR(full + s), h * 64, x.row0, g, bi);
+        }
+      }
+      if (kv == 0) k_issued = t + 1; else v_issued = t + 1;
+    }
+    return true;
+  };
+
   if (tid == 0) {                        // the descriptors live in the kernel parameters: fetch them while the CTA sets up
-    prefetch_tmap(&tm.k1); prefetch_tmap(&tm.v1);
+    prefetch_tmap(&tm.k1t); prefetch_tmap(&tm.v1t); prefetch_tmap(&tm.k1); prefetch_tmap(&tm.v1);
     if (n2 > 0) { prefetch_tmap(&tm.k2); prefetch_tmap(&tm.v2); }
     prefetch_tmap(&tm.q);
     mbar_init(BAR(Q_FULL), 1);
@@ -233,6 +284,16 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
       const int rows = min(((split + 1) * D + S - 1) / S, D) - (split * D + S - 1) / S;
       mbar_expect_tx(BAR(MERGE), (uint32_t)(S * (rows * NP * 4 + N * 8)));
     }
+    // Ahead of everything else, and of the kernels in front of this one: Q on its way into L2 and, at the reuse step,
+    // the first tiles of the compacted cache straight into the ring - they need nothing but the barriers above. Tiles that would turn the ring, or hold rows of source 2, wait for the dependency.
+    for (int h = 0; h < H; ++h) tma_prefetch_l2(&tm.q, h * 64, 0, g * p.G, bi);
+    if (kp.early_src1) {
+      set_counts(n1_early);
+      int gi0;
+      while (t_next < T && t_next < NS && tile_groups(t_next, gi0) + gi0 <= g1) issue_tile(t_next++);
+      if (ge > g1)                                   // this split holds the block's fresh rows
+        for (int h = 0; h < H; ++h) { tma_prefetch_l2(&tm.k2, h * 64, 0, g, bi); tma_prefetch_l2(&tm.v2, h * 64, 0, g, bi); }
+    }
   }
   // query rows past N (N not a multiple of 32) take part in the MMAs: they must be finite
   if (N < NP)
@@ -252,28 +313,16 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
   // The next kernel in the stream may start its own set-up now; before it touches anything this kernel writes it
   // waits for this grid to complete (griddepcontrol.wait, in that kernel).
   if (kp.early_trigger) grid_launch_dependents();
-  if (S > 1) cluster_arrive_release();   // the one cluster barrier: "this CTA runs, its barriers are set up"; waited for before the pushes
+  // the one cluster barrier: "this CTA runs, its barriers are set up" (their initialisation was released to the cluster by
+  // the fence above); waited for before the pushes
+  if (S > 1) cluster_arrive_relaxed();
 
-  // ---- this CTA's share of the key axis, in groups of 32 rows ----
-  int n1 = 0, g1 = 0, gb = 0, ge = 0, T = 0;
-  auto set_counts = [&](int n1_raw) {
-    n1 = min(max(n1_raw, 0), p.n1_max);
-    g1 = (n1 + 31) >> 5;
-    const int gt = g1 + ((n2 + 31) >> 5);
-    gb = (int)(((long long)split * gt) / S);
-    ge = (int)(((long long)(split + 1) * gt) / S);
-    T = (ge - gb + 3) >> 2;
-  };
-  auto read_counts = [&]() { set_counts(p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max); };
-  if (kp.early_src1) set_counts(n1_early);
-  // Everything but the first loads of the producer comes after the kernels in front of this one: the other threads read
-  // the counts, write global memory, or depend on Q. (The whole producer warp stays out of griddepcontrol.wait until
-  // its lane 0 has issued those loads: a warp blocks in that wait as a whole, divergent lanes included.)
-  if (warp != 0) {
-    grid_dependency_wait();
-    if (!kp.early_trigger) grid_launch_dependents();
-    if (!kp.early_src1) read_counts();
-  }
+  if (kp.early_src1 && tid != 0) set_counts(n1_early);
+  // Everything else comes after the kernels in front of this one: the threads read the counts, write global memory, or
+  // depend on Q. (All lanes of the producer warp take the wait together: a warp blocks in it as a whole.)
+  grid_dependency_wait();
+  if (!kp.early_trigger) grid_launch_dependents();
+  if (!kp.early_src1) read_counts();
 
   float l_acc[NP];                       // softmax warps: this key row's share of every column's sum
 #pragma unroll
@@ -282,35 +331,6 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
 
   if (warp == 0) {
     // ======================================= TMA producer =======================================
-    int t_next = 0, k_issued = 0, v_issued = 0;      // lane 0: next tile to load; tiles whose K / V loads are on their way
-    auto issue_tile = [&](int t) -> bool {           // lane 0 only
-      const int s = t % NS;
-      const uint32_t ph = ((t / NS) - 1) & 1;
-      const int gi0 = gb + 4 * t, ng = min(4, ge - gi0);
-      uint32_t bytes = 0;
-      for (int j = 0; j < ng; ++j) bytes += (uint32_t)(H * 128 * (gi0 + j < g1 ? 32 : kp.gr2));
-      const uint32_t kdst = smem_u32(ring + (size_t)s * SLOT), vdst = kdst + KV_BYTES;
-      for (int kv = 0; kv < 2; ++kv) {
-        const int full = kv == 0 ? FULL_K : FULL_V, empty = kv == 0 ? EMPTY_K : EMPTY_V;
-        if (t >= NS && !wait_bar(BAR(empty + s), ph, abort_flag, p.status, 1 + kv, wlim)) return false;
-        mbar_expect_tx(BAR(full + s), bytes);
-        for (int j = 0; j < ng; ++j) {
-          const Group x = group_of(gi0 + j, g1, n1, n2);
-          const CUtensorMap* m = kv == 0 ? (x.src1 ? &tm.k1 : &tm.k2) : (x.src1 ? &tm.v1 : &tm.v2);
-          for (int h = 0; h < H; ++h)
-            tma_load_4d((kv == 0 ? kdst : vdst) + h * HALF + j * 4096, m, BAR(full + s), h * 64, x.row0, g, bi);
-        }
-        if (kv == 0) k_issued = t + 1; else v_issued = t + 1;
-      }
-      return true;
-    };
-    // ahead of the dependency: the tiles that fit the ring without turning it and hold rows of source 1 only
-    if (lane == 0 && kp.early_src1)
-      while (t_next < T && t_next < NS && gb + 4 * t_next + min(4, ge - (gb + 4 * t_next)) <= g1) issue_tile(t_next++);
-    __syncwarp();
-    grid_dependency_wait();              // everything loaded from here on may have been written by the previous kernels
-    if (!kp.early_trigger) grid_launch_dependents();
-    if (!kp.early_src1) read_counts();
     if (lane == 0) {
       mbar_expect_tx(BAR(Q_FULL), (uint32_t)(H * N * 128));
       for (int h = 0; h < H; ++h) tma_load_4d(smem_u32(q_s + h * NP * 128), &tm.q, BAR(Q_FULL), h * 64, 0, g * p.G, bi);
@@ -651,13 +671,11 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
               acc.z = fmaf(r4[s2].z, w4[s2].z, acc.z); acc.w = fmaf(r4[s2].w, w4[s2].w, acc.w);
             }
           const float a[4] = {acc.x, acc.y, acc.z, acc.w};
+          const int hg = c0 / p.b, i0 = c0 - hg * p.b;    // b is a multiple of 16: the four columns are rows of one head
+          __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] +
+                             (int64_t)(g * p.G + hg) * p.o_stride[1] + (int64_t)i0 * p.o_stride[2] + d_lo + dl;
 #pragma unroll
-          for (int i4 = 0; i4 < 4; ++i4) {
-            const int c = c0 + i4;
-            const int hg = c / p.b, i = c - hg * p.b;
-            reinterpret_cast<__nv_bfloat16*>(p.out)[(int64_t)bi * p.o_stride[0] + (int64_t)(g * p.G + hg) * p.o_stride[1] +
-                                                     (int64_t)i * p.o_stride[2] + d_lo + dl] = __float2bfloat16_rn(a[i4]);
-          }
+          for (int i4 = 0; i4 < 4; ++i4) o[(int64_t)i4 * p.o_stride[2]] = __float2bfloat16_rn(a[i4]);
         }
       }
     }
@@ -798,11 +816,13 @@ cudaError_t launch_attn_kt(const AttnParams& p, const AttnPlan& pl, int D, cudaS
   if (p.n1_max > 0) {
     ok = ok && umma_make_map(&tm.k1, p.k1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 32, 1);
     ok = ok && umma_make_map(&tm.v1, p.v1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 32, 1);
+    ok = ok && umma_make_map(&tm.k1t, p.k1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 128, 1);
+    ok = ok && umma_make_map(&tm.v1t, p.v1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 128, 1);
   }
   if (p.n2 > 0) {
     ok = ok && umma_make_map(&tm.k2, p.k2, D, p.n2, p.Hkv, p.B, p.k2_stride, kp.gr2, 1);
     ok = ok && umma_make_map(&tm.v2, p.v2, D, p.n2, p.Hkv, p.B, p.k2_stride, kp.gr2, 1);
-    if (p.n1_max <= 0) { tm.k1 = tm.k2; tm.v1 = tm.v2; }
+    if (p.n1_max <= 0) { tm.k1 = tm.k2; tm.v1 = tm.v2; tm.k1t = tm.k2; tm.v1t = tm.v2; }
   } else {
     tm.k2 = tm.k1; tm.v2 = tm.v1;
   }

@@ -109,6 +109,8 @@ cudaError_t launch_attn_partial(const AttnParams& p, const AttnPlan& plan, int d
 cudaError_t launch_merge_pool(const MergeParams& p, cudaStream_t st);
 cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st);
 cudaError_t launch_compact(const CompactParams& p, cudaStream_t st);
+cudaError_t launch_select_compact(const SelectParams& p, const CompactParams& cp, cudaStream_t st);
+bool select_compact_is_fused(int Lmax, int b, int n_keep_max);
 
 __host__ __device__ inline int keep_count_total(int pre, int suf, double r, int mode, int* n_pre, int* n_suf) {
   // Algorithm 1: n = floor(|I| * r) in double; the other policies are described in sdllm.h.

@@ -20,6 +20,7 @@ constexpr int SEL_WARPS = SEL_THREADS / 32;
 constexpr int SEL_HIST = 8;               // histogram copies, one per group of warps, to spread shared-memory atomics
 
 struct Segment { int c_lo, c_hi, n; };   // candidate range and how many to keep
+constexpr int CP_ROWS_PER_THREAD = 4;    // gather: rows of K and of V in flight per thread
 
 // Exclusive prefix sum of one value per thread over the whole CTA (thread order); `total` receives the sum.
 __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* warp_tot, uint32_t* total) {
@@ -370,7 +371,6 @@ __global__ void __launch_bounds__(SEL_THREADS) select_topk_cluster_kernel(const 
 }
 
 // Gather of the kept rows: 16 bytes per thread, four rows of K and of V in flight per thread.
-constexpr int CP_ROWS_PER_THREAD = 4;
 
 __global__ void __launch_bounds__(256) compact_kv_kernel(const CompactParams p) {
   const int chunks = p.row_bytes / 16;                 // threads per row
@@ -410,6 +410,213 @@ __global__ void __launch_bounds__(256) compact_kv_kernel(const CompactParams p) 
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Selection and gather in one launch (Algorithm 1 from "n <- floor(|I| r)" to the cache store). R CTAs share a
+// (sequence, KV head): every one of them runs the whole selection of the head on its own - the candidates of a head
+// are a few kilobytes, so repeating the radix select costs no time and needs no exchange - and leaves the ascending
+// list of kept positions in its shared memory. Then CTA r writes the r-th share of kept_idx and copies the K and V rows
+// of that share into the compacted cache, 16 bytes per thread with several rows in flight (zero rows and -1 past the
+// count). The index list never makes a round trip through global memory and one launch is gone.
+// Same integer arithmetic as select_topk_kernel: the result is that kernel's, bit for bit.
+template <int NT>
+__device__ __forceinline__ uint32_t block_exclusive_scan_t(uint32_t v, uint32_t* warp_tot, uint32_t* total) {
+  constexpr int NW = NT / 32;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t incl = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += y;
+  }
+  __syncthreads();                        // warp_tot may still be read from a previous scan
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const uint32_t t = lane < NW ? warp_tot[lane] : 0u;
+    uint32_t ti = t;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, ti, d);
+      if (lane >= d) ti += y;
+    }
+    if (lane < NW) warp_tot[lane] = ti - t;   // exclusive offset of each warp
+    if (lane == 31) warp_tot[NW] = ti;        // grand total
+  }
+  __syncthreads();
+  *total = warp_tot[NW];
+  return warp_tot[warp] + incl - v;
+}
+
+template <int NT>
+__global__ void __launch_bounds__(NT) select_gather_kernel(const SelectParams p, const CompactParams cp) {
+  constexpr int NW = NT / 32;
+  constexpr int HC = NW < SEL_HIST ? NW : SEL_HIST;    // histogram copies
+  extern __shared__ uint32_t dyn_s[];                  // candidate keys (index c + c / 32), then the kept positions
+  __shared__ uint32_t hist[4][HC][256];                // one set per radix pass, cleared once per segment
+  __shared__ uint32_t warp_tot[NW + 1];
+  __shared__ uint32_t sh_prefix, sh_remaining;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int r = blockIdx.x, R = gridDim.x, g = blockIdx.y, bi = blockIdx.z;
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");  // the pooled scores come from the kernel in front
+  int L = p.seq_len ? p.seq_len[bi] : p.Lmax;
+  L = min(max(L, 0), p.Lmax);
+  const int b = p.b;
+  int o = p.block_off[bi];
+  o = min(max(o, 0), max(L - b, 0));
+  const int C = max(L - b, 0);
+  const float* sc = p.pooled + (int64_t)(bi * p.Hkv + g) * p.Lmax;
+  uint32_t* keys_s = dyn_s;
+  int32_t* kept_s = reinterpret_cast<int32_t*>(dyn_s + (p.Lmax - b) + (p.Lmax - b) / 32 + 1);
+  auto cand_pos = [&](int c) { return c < o ? c : c + b; };
+  for (int c = tid; c < C; c += NT) keys_s[c + (c >> 5)] = score_key(sc[cand_pos(c)]);
+
+  int n_pre, n_suf;
+  const int n_total = keep_count_total(o, C - o, p.retention, p.mode, &n_pre, &n_suf);
+  Segment seg[2];
+  int n_seg;
+  if (p.mode == SDLLM_SELECT_JOINT_FLOOR) {
+    seg[0] = {0, C, min(n_total, p.n_keep_max)};
+    n_seg = 1;
+  } else {
+    const int np = min(n_pre, p.n_keep_max);
+    seg[0] = {0, o, np};
+    seg[1] = {o, C, min(n_suf, p.n_keep_max - np)};
+    n_seg = 2;
+  }
+  uint32_t run_out = 0;                                // entries written so far (same value in every thread)
+  __syncthreads();
+
+  for (int si = 0; si < n_seg; ++si) {
+    const int c_lo = seg[si].c_lo, c_hi = seg[si].c_hi, n = seg[si].n;
+    const int len = c_hi - c_lo;
+    if (n <= 0 || len <= 0) continue;
+    const int kpt = (len + NT - 1) / NT;               // candidates per thread, a contiguous run
+    const int my_lo = min(c_lo + tid * kpt, c_hi), my_hi = min(my_lo + kpt, c_hi);
+    uint32_t thr = 0u, need_eq = 0u;
+    const bool take_all = n >= len;
+    if (!take_all) {
+      // ---- radix select of the n-th largest key: four passes of 8 bits, most significant first ----
+      if (tid == 0) { sh_prefix = 0u; sh_remaining = (uint32_t)n; }
+      for (int i = tid; i < 4 * HC * 256; i += NT) (&hist[0][0][0])[i] = 0u;
+      __syncthreads();
+      for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        const uint32_t prefix = sh_prefix;
+        const uint32_t remaining = sh_remaining;
+        const uint32_t himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+        uint32_t* my_hist = hist[pass][warp % HC];
+        // Pooled scores of one head share their leading bits, so most keys of a warp fall into one bin: the lanes of a
+        // warp that hit the same bin are counted by one of them (one shared-memory atomic per distinct bin and warp).
+        for (int j = 0; j < kpt; ++j) {
+          const int c = my_lo + j;
+          uint32_t k = 0u;
+          bool act = c < my_hi;
+          if (act) { k = keys_s[c + (c >> 5)]; act = (k & himask) == prefix; }
+          const uint32_t bin = (k >> shift) & 0xFFu;
+          const uint32_t same = __match_any_sync(0xffffffffu, act ? bin : 0x100u);
+          if (act && (uint32_t)lane == (uint32_t)(__ffs(same) - 1)) atomicAdd(&my_hist[bin], (uint32_t)__popc(same));
+        }
+        __syncthreads();
+        if (tid < 256) {
+          uint32_t h = 0;
+#pragma unroll
+          for (int w = 0; w < HC; ++w) h += hist[pass][w][tid];
+          hist[pass][0][tid] = h;
+        }
+        __syncthreads();
+        if (warp == 0) {
+          // lane handles bins [255 - 8*lane - 7, 255 - 8*lane], scanning downward
+          uint32_t local[8], sum = 0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { local[i] = hist[pass][0][255 - (8 * lane + i)]; sum += local[i]; }
+          uint32_t incl = sum;
+#pragma unroll
+          for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += y;
+          }
+          uint32_t above = incl - sum;            // candidates in bins above this lane's range
+          if (above < remaining && incl >= remaining) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              if (above + local[i] >= remaining) {
+                sh_prefix = prefix | ((uint32_t)(255 - (8 * lane + i)) << shift);
+                sh_remaining = remaining - above;
+                break;
+              }
+              above += local[i];
+            }
+          }
+        }
+        __syncthreads();
+      }
+      thr = sh_prefix;
+      need_eq = sh_remaining;                     // how many candidates equal to thr are still to be kept (>= 1)
+    }
+    // ---- ordered emission into shared memory: a thread's run is contiguous, so thread order is position order ----
+    uint32_t my_eq = 0, my_gt = 0;
+    for (int c = my_lo; c < my_hi; ++c) {
+      const uint32_t k = keys_s[c + (c >> 5)];
+      my_gt += (take_all || k > thr) ? 1u : 0u;
+      my_eq += (!take_all && k == thr) ? 1u : 0u;
+    }
+    uint32_t total_eq, total_keep;
+    const uint32_t eq_before = block_exclusive_scan_t<NT>(my_eq, warp_tot, &total_eq);
+    const uint32_t eq_quota = need_eq > eq_before ? min(need_eq - eq_before, my_eq) : 0u;   // ties kept from this run: its first ones
+    const uint32_t out_before = block_exclusive_scan_t<NT>(my_gt + eq_quota, warp_tot, &total_keep);
+    uint32_t w = run_out + out_before, eq_seen = 0;
+    for (int c = my_lo; c < my_hi; ++c) {
+      const uint32_t k = keys_s[c + (c >> 5)];
+      bool keep = take_all || k > thr;
+      if (!take_all && k == thr) { keep = eq_seen < eq_quota; ++eq_seen; }
+      if (keep) {
+        if (w < (uint32_t)p.n_keep_max) kept_s[w] = cand_pos(c);
+        ++w;
+      }
+    }
+    run_out += total_keep;
+  }
+  __syncthreads();
+  const int kept = min((int)run_out, p.n_keep_max);
+  if (g == 0 && r == 0 && tid == 0) p.kept_cnt[bi] = kept;
+
+  // ---- this CTA's share of the (padded) list: indices out, rows gathered ----
+  const int i_lo = (int)(((long long)r * p.n_keep_max) / R), i_hi = (int)(((long long)(r + 1) * p.n_keep_max) / R);
+  int32_t* out = p.kept_idx + (int64_t)(bi * p.Hkv + g) * p.n_keep_max;
+  for (int i = i_lo + tid; i < i_hi; i += NT) out[i] = i < kept ? kept_s[i] : -1;
+  const int chunks = cp.row_bytes / 16;                // threads per row
+  const int rows_per_pass = NT / chunks;
+  const int c16 = tid % chunks, rl = tid / chunks;
+  const char* kb = reinterpret_cast<const char*>(cp.k) + bi * cp.kv_stride_bytes[0] + g * cp.kv_stride_bytes[1];
+  const char* vb = reinterpret_cast<const char*>(cp.v) + bi * cp.kv_stride_bytes[0] + g * cp.kv_stride_bytes[1];
+  char* kc = reinterpret_cast<char*>(cp.k_c) + bi * cp.c_stride_bytes[0] + g * cp.c_stride_bytes[1];
+  char* vc = reinterpret_cast<char*>(cp.v_c) + bi * cp.c_stride_bytes[0] + g * cp.c_stride_bytes[1];
+  if (rl < rows_per_pass)
+    for (int i0 = i_lo + rl; i0 < i_hi; i0 += CP_ROWS_PER_THREAD * rows_per_pass) {
+      uint4 kv[CP_ROWS_PER_THREAD], vv[CP_ROWS_PER_THREAD];
+#pragma unroll
+      for (int u = 0; u < CP_ROWS_PER_THREAD; ++u) {
+        const int i = i0 + u * rows_per_pass;
+        kv[u] = make_uint4(0u, 0u, 0u, 0u);
+        vv[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (i < i_hi && i < kept) {
+          const int src = kept_s[i];
+          kv[u] = __ldg(reinterpret_cast<const uint4*>(kb + (int64_t)src * cp.kv_stride_bytes[2]) + c16);
+          vv[u] = __ldg(reinterpret_cast<const uint4*>(vb + (int64_t)src * cp.kv_stride_bytes[2]) + c16);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < CP_ROWS_PER_THREAD; ++u) {
+        const int i = i0 + u * rows_per_pass;
+        if (i < i_hi) {
+          reinterpret_cast<uint4*>(kc + (int64_t)i * cp.c_stride_bytes[2])[c16] = kv[u];
+          reinterpret_cast<uint4*>(vc + (int64_t)i * cp.c_stride_bytes[2])[c16] = vv[u];
+        }
+      }
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st) {
@@ -437,6 +644,47 @@ cudaError_t launch_select_topk(const SelectParams& p, cudaStream_t st) {
   if (e != cudaSuccess) return e;
   select_topk_kernel<<<dim3(p.Hkv, p.B), SEL_THREADS, smem, st>>>(p);
   return cudaGetLastError();
+}
+
+cudaError_t launch_compact(const CompactParams& p, cudaStream_t st);
+
+// Whether selection and gather run as one launch: the candidates and the kept list of a head must fit the shared memory
+// of a CTA; longer sequences take the two kernels above one after the other.
+bool select_compact_is_fused(int Lmax, int b, int n_keep_max) {
+  const int cand = Lmax - b;
+  return cand >= 1 && cand <= 8192 && n_keep_max >= 1 && tuning().select == 0;
+}
+
+cudaError_t launch_select_compact(const SelectParams& p, const CompactParams& cp, cudaStream_t st) {
+  if (!select_compact_is_fused(p.Lmax, p.b, p.n_keep_max)) {
+    const cudaError_t e = launch_select_topk(p, st);
+    return e != cudaSuccess ? e : launch_compact(cp, st);
+  }
+  const int cand = p.Lmax - p.b;
+  const size_t smem = ((size_t)cand + cand / 32 + 1 + p.n_keep_max) * 4;
+  // CTAs per head: fill the SMs, but leave every CTA at least 64 rows to copy
+  long long R = sm_count() / ((long long)p.B * p.Hkv);
+  if (R > p.n_keep_max / 64) R = p.n_keep_max / 64;
+  if (tuning().splits > 0) R = tuning().splits;
+  if (R > 16) R = 16;
+  if (R < 1) R = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)R, p.Hkv, p.B);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  int na = 0;
+  if (tuning().pdl != 0) {      // starts while the kernel in front finishes; never releases its own dependents early
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = attr; cfg.numAttrs = na;
+  static SmemConfig configured;
+  const cudaError_t e = configure_smem(reinterpret_cast<const void*>(select_gather_kernel<SEL_THREADS>), smem, configured, false);
+  if (e != cudaSuccess) return e;
+  cfg.blockDim = dim3(SEL_THREADS);
+  return cudaLaunchKernelEx(&cfg, select_gather_kernel<SEL_THREADS>, p, cp);
 }
 
 cudaError_t launch_compact(const CompactParams& p, cudaStream_t st) {

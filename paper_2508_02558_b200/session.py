@@ -21,12 +21,13 @@ class LayerCache:
                  block_len: int = 32, dtype: int = B.BF16, retention: float = 0.5, pool_window: int = 3,
                  pool: int = B.POOL_MAX, score: int = B.SCORE_LOGIT_MEAN, select: int = B.SELECT_JOINT_FLOOR,
                  softmax_scale: float = 0.0, n_keep_max: Optional[int] = None, device: str = "cuda:0",
-                 share_scratch_with: Optional["LayerCache"] = None):
+                 share_scratch_with: Optional["LayerCache"] = None, fused_select: bool = True):
         if not torch.cuda.is_available():
             raise RuntimeError("libsdllm needs a CUDA device; there is no CPU path")
         B.lib()
         self.device = torch.device(device)
         self.tdtype = _TORCH_DTYPE[dtype]
+        self.fused_select = fused_select    # selection and gather through sdllm_select_compact (else the two separate calls)
         probe = B.make_desc(batch=batch, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, head_dim=head_dim,
                             seq_len_max=seq_len_max, block_len=block_len, dtype=dtype, retention=retention,
                             pool_window=pool_window, pool=pool, score=score, select=select, softmax_scale=softmax_scale)
@@ -56,8 +57,11 @@ class LayerCache:
         """q_blk [B,Hq,b,D], k/v [B,Hkv,Lmax,D], seq_len/block_off int32 [B] (seq_len may be None)."""
         d = self.desc
         B.refresh_scores(d, q_blk, k, v, seq_len, block_off, out, lse, self.pooled, self.workspace, stream)
-        B.select_topk(d, self.pooled, seq_len, block_off, self.kept_idx, self.kept_cnt, None, stream)
-        B.compact_kv(d, k, v, self.kept_idx, self.kept_cnt, self.k_c, self.v_c, stream)
+        if self.fused_select:
+            B.select_compact(d, self.pooled, seq_len, block_off, k, v, self.kept_idx, self.kept_cnt, self.k_c, self.v_c, stream)
+        else:
+            B.select_topk(d, self.pooled, seq_len, block_off, self.kept_idx, self.kept_cnt, None, stream)
+            B.compact_kv(d, k, v, self.kept_idx, self.kept_cnt, self.k_c, self.v_c, stream)
         return out
 
     # cache_state 2: attention over Concat(K_c, K_n)
