@@ -44,9 +44,9 @@ namespace sdllm {
 using namespace dev;
 namespace {
 
-constexpr int KT_THREADS = 192;
+constexpr int KT_THREADS = 192;          // two service warps and one softmax warpgroup; 320 with two warpgroups
 constexpr int KT_MAX_STAGES = 3;
-constexpr int KT_CTRL = 3072;            // control block: barriers, flags, references, sums
+constexpr int KT_CTRL = 5120;            // control block: barriers, flags, and per softmax warpgroup references, sums, scratch
 
 struct KtMaps {
   CUtensorMap q, k1, v1, k2, v2;   // boxes of 32 rows (source 2: min(32, n2))
@@ -57,7 +57,7 @@ struct KtParams {
   AttnParams a;
   int N;             // query columns of a KV head (b * G)
   int S;             // key splits of a unit = CTAs of its cluster (1..8)
-  int NS;            // ring slots (128-key K tile + V tile each)
+  int NS;            // ring slots (one 128-key K tile + V tile each)
   int PB;            // P^T buffers (1 or 2)
   int DL;            // head dimensions a CTA owns in the merge: ceil(D / S)
   int cpt;           // merge: columns per thread, a multiple of 4
@@ -113,14 +113,16 @@ __device__ __forceinline__ float warp_max_f32(float v) {
   return r;
 }
 // barrier of the 128 softmax threads that also ORs a predicate over them
-__device__ __forceinline__ bool softmax_barrier_or(bool pred) {
+__device__ __forceinline__ bool softmax_barrier_or(int id, bool pred) {
   uint32_t r;
   asm volatile(
-      "{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.or.pred p, 1, 128, q;\n selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(r) : "r"((uint32_t)pred) : "memory");
+      "{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.or.pred p, %2, 128, q;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(r) : "r"((uint32_t)pred), "r"(id) : "memory");
   return r != 0;
 }
-__device__ __forceinline__ void softmax_barrier() { asm volatile("bar.sync 1, 128;\n" ::: "memory"); }
+// barrier of one softmax warpgroup (ids 1 and 2), and of both (id 3)
+__device__ __forceinline__ void softmax_barrier(int id) { asm volatile("bar.sync %0, 128;\n" ::"r"(id) : "memory"); }
+__device__ __forceinline__ void softmax_barrier_both() { asm volatile("bar.sync 3, 256;\n" ::: "memory"); }
 
 // order-preserving fp32 <-> u32 (larger float <=> larger code), for the shared-memory max of the references
 __device__ __forceinline__ uint32_t f2ord(float x) {
@@ -129,6 +131,11 @@ __device__ __forceinline__ uint32_t f2ord(float x) {
 }
 __device__ __forceinline__ float ord2f(uint32_t k) { return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k); }
 
+// Shared-memory matrix descriptor with the 64-byte swizzle (mode 4 in bits 61-63): rows of 64 bytes, 8 rows per atom.
+__device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+         (1ull << 46) | (4ull << 61);
+}
 // Instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B, M = 128, N = n; A and B K-major or MN-major.
 __device__ __forceinline__ uint32_t kt_idesc(int n, bool a_mn, bool b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
@@ -169,28 +176,37 @@ __device__ __forceinline__ float kt_pool_at(const AttnParams& p, const float* a,
   return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
 }
 
-template <int D, int NCH>
-__global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(const __grid_constant__ KtMaps tm, const KtParams kp) {
+template <int D, int NCH, int WG>
+__global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) attn_kt_kernel(const __grid_constant__ KtMaps tm, const KtParams kp) {
+  constexpr int NTHREADS = 64 + 128 * WG;    // WG softmax warpgroups take the tiles in turn, each with its own accumulator
   constexpr int H = D / 64;                  // 128-byte column halves of a K/V row
   constexpr int NP = NCH * 32;               // query columns padded to the softmax chunking
-  constexpr int HALF = 128 * 128;            // bytes of one 64-column half of a 128-key tile
-  constexpr int KV_BYTES = H * HALF;         // one K (or V) tile
-  constexpr int SLOT = 2 * KV_BYTES;
-  constexpr int PBUF = 128 * 128;            // one P^T buffer: 128 key rows of 64 bf16
-  constexpr uint32_t O_COL = 2 * NP;         // TMEM columns: two S^T buffers of NP, then O^T (64 columns)
-  constexpr uint32_t TMEM_COLS = (2 * NP + 64 <= 128) ? 128 : 256;
+  constexpr int PROW = NP * 2;               // bytes of a P^T row: one key, NP bf16 (64-byte swizzle for 32 columns, 128-byte for 64)
+  constexpr int PBUF = 128 * PROW;           // one P^T buffer: 128 key rows
+  constexpr uint32_t O_COL = 2 * NP;         // TMEM columns: two S^T buffers of NP, then one O^T (NP columns) per warpgroup
+  constexpr uint32_t TMEM_COLS = (2 * NP + NP * WG <= 128) ? 128 : 256;
   const AttnParams& p = kp.a;
   extern __shared__ unsigned char smem_raw[];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int NS = kp.NS, S = kp.S, N = kp.N;
+  constexpr int GPT = 4;                     // groups of 32 keys per tile (compile-time: the address arithmetic of the hot loops hangs on it)
+  constexpr int HALF = GPT * 32 * 128;       // bytes of one 64-column half of a tile
+  constexpr int KV_BYTES = H * HALF;         // one K (or V) tile
+  constexpr int SLOT = 2 * KV_BYTES;
   const int bi = blockIdx.z, g = blockIdx.y, split = blockIdx.x;
   const int n2 = p.n2;
   const long long wlim = kp.wait_cycles;
   // The count of source 1 is read ahead of the grid dependency only at the reuse step (it is older than any kernel that
   // may still run); the load is issued first so that its latency hides behind the set-up.
+  // The line is asked to stay in L2 (evict-last): every reuse step of the block reads it again, first thing, while the
+  // K/V streams of a whole model pass through L2 in between.
   int n1_early = p.n1_max;
-  if (kp.early_src1 && p.n1_per_seq) n1_early = __ldg(p.n1_per_seq + bi);
+  if (kp.early_src1 && p.n1_per_seq) {
+    uint64_t keep;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;\n" : "=l"(keep));
+    asm volatile("ld.global.L2::cache_hint.s32 %0, [%1], %2;\n" : "=r"(n1_early) : "l"(p.n1_per_seq + bi), "l"(keep) : "memory");
+  }
 
   // ---- shared memory carve-up (1024-byte aligned for the 128-byte swizzle; identical in every CTA of the cluster) ----
   const uint32_t raw_addr = smem_u32(smem_raw);
@@ -201,11 +217,14 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
   constexpr int S_FULL = 1 + 4 * KT_MAX_STAGES, P_FULL = S_FULL + 2, PV_DONE = S_FULL + 4, DRAIN = S_FULL + 6, MERGE = S_FULL + 7;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 260);
-  float* m_ref = reinterpret_cast<float*>(smem + 512);              // [64] references of the columns (log2 units)
-  uint32_t* enc = reinterpret_cast<uint32_t*>(smem + 768);          // [64] scratch of a raise: column maxima, order-preserving codes
-  float* l_tot = reinterpret_cast<float*>(smem + 1024);             // [64] sums of this split
-  float* delta_s = reinterpret_cast<float*>(smem + 1280);           // [64] by how much a raise lifts each reference
-  float* l_w = reinterpret_cast<float*>(smem + 1536);               // [4][64] per-warp sums
+  // per softmax warpgroup (wg = 0, 1):
+  const int wg = (WG == 2 && warp >= 6) ? 1 : 0;
+  float* m_ref = reinterpret_cast<float*>(smem + 512) + wg * 64;    // [64] references of the columns (log2 units)
+  uint32_t* enc = reinterpret_cast<uint32_t*>(smem + 1024) + wg * 64;   // [64] scratch of a raise: column maxima, order-preserving codes
+  float* l_tot = reinterpret_cast<float*>(smem + 1536) + wg * 64;   // [64] sums of this split (warpgroup 0: of both once merged)
+  float* delta_s = reinterpret_cast<float*>(smem + 2048) + wg * 64; // [64] by how much a raise lifts each reference
+  float* l_w = reinterpret_cast<float*>(smem + 2560) + wg * 256;    // [4][64] per-warp sums
+  const int bar_id = 1 + wg;               // (a compile-time constant with one warpgroup)
   unsigned char* q_s = smem + KT_CTRL;                              // [H][NP rows][128 B]
   unsigned char* p_s = q_s + H * NP * 128;                          // [PB][128 key rows][128 B]
   unsigned char* ring = p_s + kp.PB * PBUF;                         // [NS][K tile | V tile]
@@ -222,19 +241,19 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
     const int gt = g1 + ((n2 + 31) >> 5);
     gb = (int)(((long long)split * gt) / S);
     ge = (int)(((long long)(split + 1) * gt) / S);
-    T = (ge - gb + 3) >> 2;
+    T = (ge - gb + GPT - 1) / GPT;
   };
   auto read_counts = [&]() { set_counts(p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max); };
 
   // ---- the producer lane (thread 0) ----
   int t_next = 0, k_issued = 0, v_issued = 0;        // next tile to load; tiles whose K / V loads are on their way
-  auto tile_groups = [&](int t, int& gi0) { gi0 = gb + 4 * t; return min(4, ge - gi0); };
+  auto tile_groups = [&](int t, int& gi0) { gi0 = gb + GPT * t; return min(GPT, ge - gi0); };
   auto issue_tile = [&](int t) -> bool {
     const int s = t % NS;
     const uint32_t ph = ((t / NS) - 1) & 1;
     int gi0;
     const int ng = tile_groups(t, gi0);
-    const bool whole = ng >= 3 && gi0 + ng <= g1;    // rows of source 1 only: one 128-row box per 64-column half
+    const bool whole = 4 * ng >= 3 * GPT && gi0 + ng <= g1;   // (nearly) full tile of source 1: one box per 64-column half
     uint32_t bytes = 0;
     if (whole) bytes = (uint32_t)KV_BYTES;
     else for (int j = 0; j < ng; ++j) bytes += (uint32_t)(H * 128 * (gi0 + j < g1 ? 32 : kp.gr2));
@@ -245,13 +264,13 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
       mbar_expect_tx(BAR(full + s), bytes);
       if (whole) {
         for (int h = 0; h < H; ++h)
-          tma_load_4d((kv == 0 ? kdst : vdst) + h * HALF, kv == 0 ? &tm.k1t : &tm.v1t, BAR(full + s), h * 64, gi0 * 32, g, bi);
+          tma_load_4d((kv == 0 ? kdst : vdst) + (uint32_t)(h * HALF), kv == 0 ? &tm.k1t : &tm.v1t, BAR(full + s), h * 64, gi0 * 32, g, bi);
       } else {
         for (int j = 0; j < ng; ++j) {
           const Group x = group_of(gi0 + j, g1, n1, n2);
           const CUtensorMap* m = kv == 0 ? (x.src1 ? &tm.k1 : &tm.k2) : (x.src1 ? &tm.v1 : &tm.v2);
           for (int h = 0; h < H; ++h)
-            tma_load_4d((kv == 0 ? kdst : vdst) + h * HALF + j * 4096, m, BAR(full + s), h * 64, x.row0, g, bi);
+            tma_load_4d((kv == 0 ? kdst : vdst) + (uint32_t)(h * HALF + j * 4096), m, BAR(full + s), h * 64, x.row0, g, bi);
         }
       }
       if (kv == 0) k_issued = t + 1; else v_issued = t + 1;
@@ -297,7 +316,7 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
   }
   // query rows past N (N not a multiple of 32) take part in the MMAs: they must be finite
   if (N < NP)
-    for (int i = tid; i < H * (NP - N) * 8; i += KT_THREADS) {
+    for (int i = tid; i < H * (NP - N) * 8; i += NTHREADS) {
       const int h = i / ((NP - N) * 8), r = i % ((NP - N) * 8);
       reinterpret_cast<uint4*>(q_s + h * NP * 128 + N * 128)[r] = make_uint4(0u, 0u, 0u, 0u);
     }
@@ -346,32 +365,37 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
     // ======================================= MMA issuer =======================================
     if (lane == 0) {
       const uint32_t idesc_s = kt_idesc(NP, false, false);
-      const uint32_t idesc_pv = kt_idesc(64, true, true);
+      const uint32_t idesc_pv = kt_idesc(NP, true, true);
       const uint32_t qsm = smem_u32(q_s);
       bool ok = wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 3, wlim);
-      auto issue_pv = [&](int j) -> bool {
-        const int s = j % NS, pb = j & 1;
-        const int ng = min(4, ge - (gb + 4 * j));
+      const uint32_t ring_a = smem_u32(ring), p_a = smem_u32(p_s);
+      const bool two_p = kp.PB == 2;
+      auto issue_pv = [&](int j, int s, uint32_t par) -> bool {       // tile j lives in ring slot s, in its use of parity par
+        const int pb = j & 1;
+        const int ng = min(GPT, ge - (gb + GPT * j));
         if (!wait_bar(BAR(P_FULL + pb), (j >> 1) & 1, abort_flag, p.status, 4, wlim)) return false;
-        if (!wait_bar(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 5, wlim)) return false;
+        if (!wait_bar(BAR(FULL_V + s), par, abort_flag, p.status, 5, wlim)) return false;
         tc_fence_after();
-        const uint32_t vsm = smem_u32(ring + (size_t)s * SLOT) + KV_BYTES;
-        const uint32_t psm = smem_u32(p_s + (size_t)(j % kp.PB) * PBUF);
+        const uint32_t vsm = ring_a + (uint32_t)s * SLOT + KV_BYTES;
+        const uint32_t psm = p_a + ((two_p && pb) ? (uint32_t)PBUF : 0u);
         // O^T += V^T P^T, 16 keys per instruction. A: the V tile read MN-major (the head dimension runs along M; its two
         // 64-element halves lie HALF bytes apart; with D = 64 both halves alias the same data and rows 64..127 of O^T
-        // are duplicates nobody reads). B: P^T, MN-major, one 64-element half.
+        // are duplicates nobody reads). B: P^T, MN-major: rows of NP bf16, 8 keys per swizzle atom.
         for (int ks = 0; ks < 2 * ng; ++ks)
-          mma_ss(tmem_base + O_COL, smem_desc(vsm + ks * 2048, H == 2 ? (uint32_t)HALF : 0u, 1024u),
-                 smem_desc(psm + ks * 2048, (uint32_t)PBUF, 1024u), idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+          mma_ss(tmem_base + O_COL + (uint32_t)(j % WG) * NP, smem_desc(vsm + ks * 2048, H == 2 ? (uint32_t)HALF : 0u, 1024u),
+                 NP == 64 ? smem_desc(psm + ks * 2048, (uint32_t)PBUF, 1024u) : smem_desc_sw64(psm + ks * 1024, (uint32_t)PBUF, 512u),
+                 idesc_pv, (j >= WG || ks > 0) ? 1u : 0u);
         tc_commit(BAR(PV_DONE + pb));    // two alternating barriers: a waiter is never a whole phase ahead of either
         tc_commit(BAR(EMPTY_V + s));
         return true;
       };
+      int s = 0, s_prev = 0;               // ring slot of tile t and of tile t - 1, and the parities of their uses
+      uint32_t par = 0, par_prev = 0;
       for (int t = 0; t < T && ok; ++t) {
-        const int s = t % NS, sb = t & 1;
-        if (!wait_bar(BAR(FULL_K + s), (t / NS) & 1, abort_flag, p.status, 7, wlim)) { ok = false; break; }
+        const int sb = t & 1;
+        if (!wait_bar(BAR(FULL_K + s), par, abort_flag, p.status, 7, wlim)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t ksm = smem_u32(ring + (size_t)s * SLOT);
+        const uint32_t ksm = ring_a + (uint32_t)s * SLOT;
         const uint32_t d_t = tmem_base + (uint32_t)sb * NP;
         // S^T = K_tile Q^T: the S^T buffer of tile t - 2 is free, its softmax arrived before PV(t - 2) was issued
 #pragma unroll
@@ -382,9 +406,11 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
         }
         tc_commit(BAR(S_FULL + sb));
         tc_commit(BAR(EMPTY_K + s));
-        if (t > 0 && !issue_pv(t - 1)) { ok = false; break; }
+        if (t > 0 && !issue_pv(t - 1, s_prev, par_prev)) { ok = false; break; }
+        s_prev = s; par_prev = par;
+        if (++s == NS) { s = 0; par ^= 1u; }
       }
-      if (ok && T > 0) ok = issue_pv(T - 1);
+      if (ok && T > 0) ok = issue_pv(T - 1, s_prev, par_prev);
       if (*abort_flag) {                 // wait for the tensor pipe to finish what was issued before TMEM is freed
         tc_commit(BAR(DRAIN));
         drain_bar(BAR(DRAIN), 0);
@@ -399,9 +425,12 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16);
     const float sl2 = p.scale_log2;
     const bool scores = p.want_scores != 0;
-    for (int t = 0; t < T; ++t) {
-      const int s = t % NS, sb = t & 1;
-      const int gi0 = gb + 4 * t, ng = min(4, ge - gi0);
+    const int st = (tid - 64) & 127;                   // index inside the warpgroup
+    const uint32_t o_col = O_COL + (uint32_t)wg * NP;  // this warpgroup's accumulator
+    const bool two_p = kp.PB == 2;
+    for (int t = wg; t < T; t += WG) {
+      const int sb = t & 1;
+      const int gi0 = gb + GPT * t, ng = min(GPT, ge - gi0);
       const bool active = q4 < ng;                     // warp-uniform: this warp's group exists in the tile
       Group x{1, 0, 0};
       if (active) x = group_of(gi0 + q4, g1, n1, n2);
@@ -429,13 +458,13 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
       // ---- the references. The first key of the CTA's first tile lends its logits: it is part of the softmax, so sums
       //      never vanish, and exp2 of anything up to 2^64 above it is still an ordinary bf16 / fp32 number. Every tile is
       //      only checked against the references; one that exceeds them by more than 64 raises them (rare). ----
-      if (t == 0) {
+      if (t < WG) {
         if (row == 0 && work) {
 #pragma unroll
           for (int c = 0; c < NP; c += 4)
             *reinterpret_cast<float4*>(m_ref + c) = make_float4(sv[c] * sl2, sv[c + 1] * sl2, sv[c + 2] * sl2, sv[c + 3] * sl2);
         }
-        softmax_barrier();
+        softmax_barrier(bar_id);
       }
       bool over = false;
 #pragma unroll
@@ -445,13 +474,13 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
         sv[c + 2] = fmaf(sv[c + 2], sl2, -m4.z); sv[c + 3] = fmaf(sv[c + 3], sl2, -m4.w);
         over |= (sv[c] > 64.f) | (sv[c + 1] > 64.f) | (sv[c + 2] > 64.f) | (sv[c + 3] > 64.f);
       }
-      if (softmax_barrier_or(over && work && valid)) {
+      if (softmax_barrier_or(bar_id, over && work && valid)) {
         // ---- raise the references by the tile's column maxima (where positive) and rescale what has been accumulated.
         //      Every PV issued so far must have landed before O^T is rewritten; the PV of this tile waits for our arrive. ----
-        if (t > 0 && !dead && !wait_bar_warp(BAR(PV_DONE + ((t - 1) & 1)), ((t - 1) >> 1) & 1, abort_flag, p.status, 8, wlim)) dead = true;
+        if (t >= WG && !dead && !wait_bar_warp(BAR(PV_DONE + ((t - WG) & 1)), ((t - WG) >> 1) & 1, abort_flag, p.status, 8, wlim)) dead = true;
         tc_fence_after();
-        if (tid - 64 < NP) enc[tid - 64] = f2ord(0.f);
-        softmax_barrier();
+        if (st < NP) enc[st] = f2ord(0.f);
+        softmax_barrier(bar_id);
         if (work) {
           float mine[NCH];
 #pragma unroll
@@ -462,21 +491,21 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
 #pragma unroll
           for (int c = 0; c < NCH; ++c) atomicMax(enc + c * 32 + lane, f2ord(mine[c]));
         }
-        softmax_barrier();
-        if (tid - 64 < NP) {
-          const float dlt = ord2f(enc[tid - 64]);      // >= 0
-          delta_s[tid - 64] = dlt;
-          m_ref[tid - 64] += dlt;
+        softmax_barrier(bar_id);
+        if (st < NP) {
+          const float dlt = ord2f(enc[st]);            // >= 0
+          delta_s[st] = dlt;
+          m_ref[st] += dlt;
         }
-        softmax_barrier();
+        softmax_barrier(bar_id);
 #pragma unroll
         for (int c = 0; c < NP; ++c) sv[c] -= delta_s[c];
-        if (t > 0 && !dead) {
+        if (t >= WG && !dead) {
           // this thread's TMEM lane is a head dimension of O^T here, not a key: all four warps rescale their lanes
 #pragma unroll
           for (int c = 0; c < NCH; ++c) {
             uint32_t o32[32];
-            tmem_ld32(lane_addr + O_COL + c * 32, o32);
+            tmem_ld32(lane_addr + o_col + c * 32, o32);
             tc_wait_ld();
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
@@ -484,20 +513,20 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
               o32[i] = __float_as_uint(__uint_as_float(o32[i]) * a);
               l_acc[c * 32 + i] *= a;
             }
-            tmem_st16(lane_addr + O_COL + c * 32, *reinterpret_cast<uint32_t(*)[16]>(&o32[0]));
-            tmem_st16(lane_addr + O_COL + c * 32 + 16, *reinterpret_cast<uint32_t(*)[16]>(&o32[16]));
+            tmem_st16(lane_addr + o_col + c * 32, *reinterpret_cast<uint32_t(*)[16]>(&o32[0]));
+            tmem_st16(lane_addr + o_col + c * 32 + 16, *reinterpret_cast<uint32_t(*)[16]>(&o32[16]));
           }
           tc_wait_st();
         }
-        softmax_barrier();               // delta_s and m_ref are stable again before the next tile reads them
+        softmax_barrier(bar_id);         // delta_s and m_ref are stable again before the next tile reads them
       }
       // ---- P^T = exp2(distance to the reference) as bf16, one 128-byte row per key (128-byte swizzle) ----
       // the P^T buffer is free once the PV that read it has completed
-      if (!dead && t >= kp.PB &&
-          !wait_bar_warp(BAR(PV_DONE + ((t - kp.PB) & 1)), ((t - kp.PB) >> 1) & 1, abort_flag, p.status, 6, wlim))
-        dead = true;
+      const int tp = two_p ? t - 2 : t - 1;            // the tile whose PV read this buffer last
+      if (!dead && tp >= 0 && !wait_bar_warp(BAR(PV_DONE + (tp & 1)), (tp >> 1) & 1, abort_flag, p.status, 6, wlim)) dead = true;
       if (active && !dead) {
-        unsigned char* prow = p_s + (size_t)(t % kp.PB) * PBUF + row * 128;
+        unsigned char* prow = p_s + ((two_p && sb) ? PBUF : 0) + row * PROW;
+        const int swz = NP == 64 ? (row & 7) : ((row >> 1) & 3);     // the 16-byte chunk index is XORed with address bits 7.. of the row
 #pragma unroll
         for (int c8 = 0; c8 < NP / 8; ++c8) {
           uint32_t pk[4];
@@ -509,10 +538,11 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
             l_acc[c] += e0; l_acc[c + 1] += e1;
             pk[i] = pack_bf16(e0, e1);
           }
-          *reinterpret_cast<uint4*>(prow + ((c8 ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          *reinterpret_cast<uint4*>(prow + ((c8 ^ swz) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
         // ---- V rows of this group past its count may hold anything: zero them so that 0 * V stays 0 ----
         if (x.nv < 32) {
+          const int s = t % NS;
           if (!wait_bar_warp(BAR(FULL_V + s), (t / NS) & 1, abort_flag, p.status, 10, wlim)) dead = true;
           unsigned char* vs = ring + (size_t)s * SLOT + KV_BYTES;
           const int nz = dead ? 0 : (32 - x.nv) * H * 8;          // 16-byte chunks to clear
@@ -532,10 +562,12 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
   // ======================================= epilogue =======================================
   const bool do_attn = p.out != nullptr;
   const int DL = kp.DL;                  // head dimensions a CTA owns in the merge: ceil(D / S)
+  uint32_t ov[NP];                       // softmax threads: this thread's head dimension of O^T, all columns
+  float l_mine = 0.f, m_mine = -INFINITY;// softmax thread st < NP: sum and reference of column st
   if (warp >= 2) {
     const int q4 = warp & 3;
     const int row = q4 * 32 + lane;      // from here on: a head dimension of O^T
-    const int st = tid - 64;             // 0..127
+    const int st = (tid - 64) & 127;     // index inside the warpgroup
     // ---- column sums over the 128 key rows: shuffle transpose inside a warp (lane i ends up with column i), then the
     //      four warps' rows in a fixed order ----
 #pragma unroll
@@ -553,51 +585,110 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
           v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
         }
       }
-      l_w[(warp - 2) * 64 + c * 32 + lane] = v[0];
+      l_w[((warp - 2) & 3) * 64 + c * 32 + lane] = v[0];
     }
     if (S > 1 && p.want_scores) __threadfence();       // this thread's raw saliency, ahead of the pushes that tell the peers
-    softmax_barrier();
-    float l_mine = 0.f, m_mine = -INFINITY;            // thread st < NP: sum and reference of column st
+    softmax_barrier(bar_id);
     if (st < NP) {
       l_mine = (l_w[st] + l_w[64 + st]) + (l_w[128 + st] + l_w[192 + st]);
-      m_mine = T > 0 ? m_ref[st] : -INFINITY;
-      l_tot[st] = l_mine;
+      m_mine = T > wg ? m_ref[st] : -INFINITY;
     }
-    if (S > 1) {
-      // every split's (reference, sum) of every column goes to every CTA of the cluster
+    // ---- two warpgroups: the second one's partial (reference, sum, accumulator rows) is folded into the first one's ----
+    const bool fold = WG == 2 && T >= 2;
+    const float* m_a = m_ref - wg * 64; const float* m_b = m_a + 64;
+    const float* l_a = l_tot - wg * 64; const float* l_b = l_a + 64;
+    if (fold) {
+      if (st < NP) l_tot[st] = l_mine;
+      softmax_barrier_both();            // both warpgroups' references and sums are posted
+      if (wg == 0 && st < NP) {
+        const float mb = m_b[st], lb = l_b[st];
+        const bool ha = l_mine > 0.f, hb = lb > 0.f;
+        const float ms = fmaxf(ha ? m_mine : -INFINITY, hb ? mb : -INFINITY);
+        l_mine = (ha ? l_mine * fast_exp2(m_mine - ms) : 0.f) + (hb ? lb * fast_exp2(mb - ms) : 0.f);
+        m_mine = ms;
+      }
+    }
+    if (wg == 0 && S > 1) {
+      // every split's (reference, sum) of every column goes to every CTA of the cluster, ahead of the accumulator rows
       cluster_wait_acquire();            // every CTA of the cluster runs: its shared memory and barriers may be written
       if (st < N) {
         const uint32_t ml_a = smem_u32(ml_recv + split * NP + st);
         for (int r = 0; r < S; ++r) st_async_f2(map_to_cta(ml_a, (uint32_t)r), map_to_cta(BAR(MERGE), (uint32_t)r), m_mine, l_mine);
       }
-    } else {
-      softmax_barrier();                 // l_tot
     }
-    // ---- the finished accumulator row of this thread ----
-    uint32_t ov[NP];
-    const bool have_o = do_attn && !dead && T > 0 &&
-                        wait_bar_warp(BAR(PV_DONE + ((T - 1) & 1)), ((T - 1) >> 1) & 1, abort_flag, p.status, 6, wlim);
+    // ---- the finished accumulator row of this thread (of its warpgroup's accumulator) ----
+    const int t_last = T > wg ? wg + ((T - 1 - wg) / WG) * WG : 0;      // the warpgroup's last tile
+    const bool have_o = do_attn && !dead && T > wg &&
+                        wait_bar_warp(BAR(PV_DONE + (t_last & 1)), (t_last >> 1) & 1, abort_flag, p.status, 6, wlim);
     tc_fence_after();
     if (have_o) {
 #pragma unroll
-      for (int c = 0; c < NCH; ++c) tmem_ld32(tmem_base + ((uint32_t)(q4 * 32) << 16) + O_COL + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[c * 32]));
+      for (int c = 0; c < NCH; ++c)
+        tmem_ld32(tmem_base + ((uint32_t)(q4 * 32) << 16) + O_COL + (uint32_t)wg * NP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[c * 32]));
       tc_wait_ld();
     } else {
 #pragma unroll
       for (int c = 0; c < NP; ++c) ov[c] = 0u;
     }
+    if (fold) {
+      // The rows cross in the first ring slot, once both warpgroups have seen their last PV complete. Every thread scales
+      // its own row to the common references; the factors are recomputed from the posted references and sums.
+      float4* xch = reinterpret_cast<float4*>(ring);                // [NP / 4][128 rows]
+      softmax_barrier_both();
+#pragma unroll
+      for (int c4 = 0; c4 < NP / 4; ++c4) {
+        const float4 ma = *reinterpret_cast<const float4*>(m_a + 4 * c4), mb = *reinterpret_cast<const float4*>(m_b + 4 * c4);
+        const float4 la = *reinterpret_cast<const float4*>(l_a + 4 * c4), lb = *reinterpret_cast<const float4*>(l_b + 4 * c4);
+        const float mav[4] = {ma.x, ma.y, ma.z, ma.w}, mbv[4] = {mb.x, mb.y, mb.z, mb.w};
+        const float lav[4] = {la.x, la.y, la.z, la.w}, lbv[4] = {lb.x, lb.y, lb.z, lb.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const bool ha = lav[u] > 0.f, hb = lbv[u] > 0.f;
+          const float ms = fmaxf(ha ? mav[u] : -INFINITY, hb ? mbv[u] : -INFINITY);
+          const float f = wg == 0 ? (ha ? fast_exp2(mav[u] - ms) : 0.f) : (hb ? fast_exp2(mbv[u] - ms) : 0.f);
+          ov[4 * c4 + u] = __float_as_uint(__uint_as_float(ov[4 * c4 + u]) * f);
+        }
+        if (wg == 1)
+          xch[c4 * 128 + row] = make_float4(__uint_as_float(ov[4 * c4]), __uint_as_float(ov[4 * c4 + 1]), __uint_as_float(ov[4 * c4 + 2]),
+                                            __uint_as_float(ov[4 * c4 + 3]));
+      }
+      softmax_barrier_both();
+      if (wg == 0) {
+#pragma unroll
+        for (int c4 = 0; c4 < NP / 4; ++c4) {
+          const float4 x = xch[c4 * 128 + row];
+          ov[4 * c4] = __float_as_uint(__uint_as_float(ov[4 * c4]) + x.x); ov[4 * c4 + 1] = __float_as_uint(__uint_as_float(ov[4 * c4 + 1]) + x.y);
+          ov[4 * c4 + 2] = __float_as_uint(__uint_as_float(ov[4 * c4 + 2]) + x.z); ov[4 * c4 + 3] = __float_as_uint(__uint_as_float(ov[4 * c4 + 3]) + x.w);
+        }
+      }
+    }
+  }
+  if (warp >= 2 && warp < 6) {           // the first warpgroup carries the result out
+    const int q4 = warp & 3;
+    const int row = q4 * 32 + lane;
+    const int st = tid - 64;
+    if (S == 1) {
+      if (st < NP) l_tot[st] = l_mine > 0.f ? 1.f / l_mine : 0.f;       // one split: the normaliser itself
+      softmax_barrier(1);
+    }
     if (S == 1) {
       if (do_attn && !*abort_flag) {
         // one split: normalise and store; a warp writes 32 consecutive bf16 of one output row per column
         if (row < D) {
+          // column c is row c % b of head c / b of the group: the pointer walks the rows and hops to the next head
+          __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] + (int64_t)(g * p.G) * p.o_stride[1] + row;
+          const int64_t hop = p.o_stride[1] - (int64_t)(p.b - 1) * p.o_stride[2];
+          int i = 0;
 #pragma unroll
-          for (int c = 0; c < NP; ++c) {
+          for (int c = 0; c < NP; c += 4) {
             if (c >= N) break;
-            const float l = l_tot[c];
-            const float inv = l > 0.f ? 1.f / l : 0.f;
-            const int hg = c / p.b, i = c - hg * p.b;
-            reinterpret_cast<__nv_bfloat16*>(p.out)[(int64_t)bi * p.o_stride[0] + (int64_t)(g * p.G + hg) * p.o_stride[1] +
-                                                     (int64_t)i * p.o_stride[2] + row] = __float2bfloat16_rn(__uint_as_float(ov[c]) * inv);
+            const float4 inv = *reinterpret_cast<const float4*>(l_tot + c);
+            const float iv[4] = {inv.x, inv.y, inv.z, inv.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              *o = __float2bfloat16_rn(__uint_as_float(ov[c + u]) * iv[u]);
+              if (++i == p.b) { i = 0; o += hop; } else o += p.o_stride[2];
+            }
           }
         }
         if (p.lse && st < N) {
@@ -621,9 +712,9 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
 
   if (S > 1) {
     // ---- cluster merge: once everything owed to this CTA has landed, it merges and stores the head dimensions it owns ----
-    if (warp < 2) cluster_wait_acquire();              // (the softmax warps passed the cluster barrier before their pushes)
+    if (warp < 2 || warp >= 6) cluster_wait_acquire(); // (the first softmax warpgroup passed the cluster barrier before its pushes)
     wait_merge(BAR(MERGE), abort_flag, p.status, wlim);
-    if (warp >= 2 && do_attn && !*abort_flag) {
+    if (warp >= 2 && warp < 6 && do_attn && !*abort_flag) {
       const int st = tid - 64;
       // weights of the S splits for column st, the normalisation folded in
       if (st < N) {
@@ -649,7 +740,7 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
           p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
         }
       }
-      softmax_barrier();
+      softmax_barrier(1);
       // thread -> (owned head dimension, chunk of columns); all loads of a group of four columns are in flight together
       const int d_lo = (split * D + S - 1) / S, d_hi = min(((split + 1) * D + S - 1) / S, D);
       const int dl = st % DL, qc = st / DL;
@@ -688,7 +779,7 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
     const float* a = p.raw_scores + (int64_t)(bi * p.Hkv + g) * p.n1_max;
     const int p_lo = (int)(((long long)split * p.n1_max) / S), p_hi = (int)(((long long)(split + 1) * p.n1_max) / S);
     const int o = p.block_off[bi];
-    for (int pos = p_lo + tid; pos < p_hi; pos += KT_THREADS)
+    for (int pos = p_lo + tid; pos < p_hi; pos += NTHREADS)
       p.pooled[(int64_t)(bi * p.Hkv + g) * p.n1_max + pos] = kt_pool_at(p, a, n1, o, pos);
   }
 
@@ -704,22 +795,22 @@ __global__ void __launch_bounds__(KT_THREADS, NCH == 1 ? 2 : 1) attn_kt_kernel(c
 
 // ---------------------------------------------------------------------------------------------------------
 // Host side
-size_t kt_smem_bytes(int D, int NP, int NS, int PB, int S) {
+size_t kt_smem_bytes(int D, int NP, int NS, int PB, int S, int GPT) {
   const size_t H = D / 64;
   const size_t DL = (D + S - 1) / S;
-  return 1024 /*alignment slack*/ + KT_CTRL + H * NP * 128 + (size_t)PB * 128 * 128 + (size_t)NS * 2 * H * 128 * 128 +
+  return 1024 /*alignment slack*/ + KT_CTRL + H * NP * 128 + (size_t)PB * 128 * NP * 2 + (size_t)NS * 2 * H * GPT * 32 * 128 +
          (S > 1 ? (size_t)S * DL * NP * 4 /*recv*/ + (size_t)S * NP * 12 /*ml_recv, w_s*/ : 0);
 }
 
-template <int D, int NCH>
+template <int D, int NCH, int WG>
 cudaError_t launch_kt_d(const KtMaps& tm, const KtParams& kp, const AttnPlan& pl, bool pdl, cudaStream_t st) {
-  auto kern = attn_kt_kernel<D, NCH>;
+  auto kern = attn_kt_kernel<D, NCH, WG>;
   static SmemConfig configured;
   cudaError_t e = configure_smem(reinterpret_cast<const void*>(kern), pl.smem_bytes, configured, true);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(kp.S, kp.a.Hkv, kp.a.B);
-  cfg.blockDim = dim3(KT_THREADS);
+  cfg.blockDim = dim3(64 + 128 * WG);
   cfg.dynamicSmemBytes = pl.smem_bytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
@@ -759,38 +850,49 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   const int sms = sm_count();
   // Key splits: enough CTAs to fill the SMs (two per SM with few query columns), but at least one full 128-key tile
   // per CTA, and at most eight (one cluster).
-  long long want = (NP == 32 ? 2 : 1) * (long long)sms / units;
+  long long want = (NP == 32 && groups <= 64 ? 2 : 1) * (long long)sms / units;
   const long long by_tiles = (groups + 3) / 4;
   if (want > by_tiles) want = by_tiles;
   if (tn.splits > 0) want = tn.splits;
   if (want > 8) want = 8;
   if (want < 1) want = 1;
   const int S = (int)want;
-  const int tiles_cta = ((groups + S - 1) / S + 3) / 4;
-  // Ring depth and P^T buffers. With few query columns, and either more CTAs than SMs or a single tile per CTA, the
-  // footprint is kept below half an SM, so that two CTAs are resident and the next call's CTAs can start loading while
-  // this call's finish; otherwise the CTA takes what one SM has.
+  // Footprint, ring depth, P^T buffers and softmax warpgroups:
+  // (a) few query columns and at most two full tiles per CTA: the footprint is kept below half an SM, so that two CTAs
+  //     are resident and the next call's CTAs can start loading while this call's finish;
+  // (b) few query columns and longer walks: the CTA takes what one SM has, and two softmax warpgroups take the tiles in
+  //     turn (one warp per scheduler cannot hide its own latencies; two tiles in flight can);
+  // (c) up to 64 query columns: one CTA per SM, one warpgroup.
+  const int groups_cta = (groups + S - 1) / S;
   const size_t half_sm = 113 * 1024;     // two CTAs of this size, each with its 1 KB system share, fit one SM
-  int NS = 1, PB = 1;
-  const bool small = NP == 32 && (units * S > sms || tiles_cta <= 1);
+  bool small = NP == 32 && groups_cta <= 8;
+  int WG = (NP == 32 && !small) ? 2 : 1;
+  if (tn.dual == 1) { small = NP == 32; WG = 1; }      // force (a) / (b) where they apply
+  if (tn.dual == 0 && NP == 32) { small = false; WG = 2; }
+  const int GPT = 4;
+  const int tiles_cta = (groups_cta + GPT - 1) / GPT;
+  int NS = 1, PB = WG == 2 ? 2 : 1;
   if (small) {
-    while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, NP, NS + 1, PB, S) <= half_sm) ++NS;
+    while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, NP, NS + 1, PB, S, GPT) <= half_sm) ++NS;
   } else {
     PB = 2;
-    while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, NP, NS + 1, PB, S) <= 226 * 1024) ++NS;
+    while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, NP, NS + 1, PB, S, GPT) <= 226 * 1024) ++NS;
   }
   if (tn.stages > 0) {
     NS = tn.stages > KT_MAX_STAGES ? KT_MAX_STAGES : tn.stages;
-    while (NS > 1 && kt_smem_bytes(D, NP, NS, PB, S) > 226 * 1024) --NS;
+    while (NS > 1 && kt_smem_bytes(D, NP, NS, PB, S, GPT) > 226 * 1024) --NS;
   }
   pl.splits = 1;                        // nothing is left in the workspace: the splits merge inside their cluster
   pl.parts = 1;
   pl.cluster = S;
   pl.stages = NS;
   pl.m_warps = PB;                      // (field reused: P^T buffers)
+  pl.c_warps = WG;                      // (field reused: softmax warpgroups)
+  pl.threads = 64 + 128 * WG;
   pl.part_rows = 0;
   pl.n_counters = 0;
-  pl.smem_bytes = kt_smem_bytes(D, NP, NS, PB, S);
+  pl.key_tile = 32 * GPT;
+  pl.smem_bytes = kt_smem_bytes(D, NP, NS, PB, S, GPT);
   return pl;
 }
 
@@ -816,8 +918,8 @@ cudaError_t launch_attn_kt(const AttnParams& p, const AttnPlan& pl, int D, cudaS
   if (p.n1_max > 0) {
     ok = ok && umma_make_map(&tm.k1, p.k1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 32, 1);
     ok = ok && umma_make_map(&tm.v1, p.v1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 32, 1);
-    ok = ok && umma_make_map(&tm.k1t, p.k1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 128, 1);
-    ok = ok && umma_make_map(&tm.v1t, p.v1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 128, 1);
+    ok = ok && umma_make_map(&tm.k1t, p.k1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, pl.key_tile, 1);
+    ok = ok && umma_make_map(&tm.v1t, p.v1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, pl.key_tile, 1);
   }
   if (p.n2 > 0) {
     ok = ok && umma_make_map(&tm.k2, p.k2, D, p.n2, p.Hkv, p.B, p.k2_stride, kp.gr2, 1);
@@ -829,8 +931,9 @@ cudaError_t launch_attn_kt(const AttnParams& p, const AttnPlan& pl, int D, cudaS
   if (!ok) return cudaErrorInvalidValue;
   const bool pdl = tn.pdl != 0;
   const int NP = p.M <= 32 ? 32 : 64;
-  if (NP == 32) return D == 128 ? launch_kt_d<128, 1>(tm, kp, pl, pdl, st) : launch_kt_d<64, 1>(tm, kp, pl, pdl, st);
-  return D == 128 ? launch_kt_d<128, 2>(tm, kp, pl, pdl, st) : launch_kt_d<64, 2>(tm, kp, pl, pdl, st);
+  if (NP == 32 && pl.c_warps == 2) return D == 128 ? launch_kt_d<128, 1, 2>(tm, kp, pl, pdl, st) : launch_kt_d<64, 1, 2>(tm, kp, pl, pdl, st);
+  if (NP == 32) return D == 128 ? launch_kt_d<128, 1, 1>(tm, kp, pl, pdl, st) : launch_kt_d<64, 1, 1>(tm, kp, pl, pdl, st);
+  return D == 128 ? launch_kt_d<128, 2, 1>(tm, kp, pl, pdl, st) : launch_kt_d<64, 2, 1>(tm, kp, pl, pdl, st);
 }
 
 }  // namespace sdllm

@@ -153,6 +153,7 @@ def test_pool_windows(window):
     dict(pdl=0),                                         # no programmatic dependent launch
     dict(splits=7), dict(splits=1), dict(splits=3),      # other key-split counts (cluster sizes) of the key-row kernel
     dict(splits=2, stages=3), dict(splits=1, stages=2),  # ... and ring depths
+    dict(dual=0), dict(dual=0, splits=1), dict(dual=0, splits=3, stages=1), dict(dual=1, splits=1, stages=1),   # two softmax warpgroups / one
     dict(early_loads=0),                                 # no loads ahead of the grid dependency
     dict(kernel=2),                                      # the tcgen05 kernel with the queries on the accumulator rows
     dict(kernel=2, splits=7), dict(kernel=2, splits=1),
@@ -186,7 +187,7 @@ def test_softmax_probability_saliency(cfg, block, plan, tuning):
     _run_sequence_case(cfg, seed=15, block=block, n_sparse=1, score=B.SCORE_PROB_MEAN)
 
 
-@pytest.mark.parametrize("plan", [{}, dict(splits=3), dict(kernel=2), dict(kernel=2, lpt=1), dict(kernel=2, lpt=1, dual=1, splits=1),
+@pytest.mark.parametrize("plan", [{}, dict(splits=3), dict(dual=0, splits=1), dict(dual=0, splits=2), dict(kernel=2), dict(kernel=2, lpt=1), dict(kernel=2, lpt=1, dual=1, splits=1),
                                   dict(select=2)])
 def test_ragged_batch(plan, tuning):
     import parity_util as U
