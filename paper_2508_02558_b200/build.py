@@ -38,8 +38,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     os.makedirs(OBJ_DIR, exist_ok=True)
     extra = ["-Xptxas", "-v"] if verbose else []
-    if os.environ.get("SDLLM_TRACE") == "1":        # kernel timeline points (see attn_umma.cu)
-        extra.append("-DSDLLM_TRACE")
 
     def compile_one(src: str) -> str:
         obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")

@@ -64,6 +64,7 @@ struct KtParams {
   int gr2;           // rows of a source-2 box: min(32, n2)
   int early_src1;    // 1: source 1 and its count are older than every kernel that may still run (reuse step)
   int early_trigger; // 1: release the next kernel in the stream as soon as this CTA is set up
+  int lpt;           // 1: grid z counts the sequences from the longest to the shortest (several waves of ragged work)
   long long wait_cycles;   // limit of every abortable mbarrier wait
 };
 
@@ -185,16 +186,33 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
   constexpr int PBUF = 128 * PROW;           // one P^T buffer: 128 key rows
   constexpr uint32_t O_COL = 2 * NP;         // TMEM columns: two S^T buffers of NP, then one O^T (NP columns) per warpgroup
   constexpr uint32_t TMEM_COLS = (2 * NP + NP * WG <= 128) ? 128 : 256;
-  const AttnParams& p = kp.a;
   extern __shared__ unsigned char smem_raw[];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int NS = kp.NS, S = kp.S, N = kp.N;
+  const AttnParams& p = kp.a;
   constexpr int GPT = 4;                     // groups of 32 keys per tile (compile-time: the address arithmetic of the hot loops hangs on it)
   constexpr int HALF = GPT * 32 * 128;       // bytes of one 64-column half of a tile
   constexpr int KV_BYTES = H * HALF;         // one K (or V) tile
   constexpr int SLOT = 2 * KV_BYTES;
-  const int bi = blockIdx.z, g = blockIdx.y, split = blockIdx.x;
+  const int g = blockIdx.y, split = blockIdx.x;
+  // Which sequence: grid z itself, or, for ragged batches that take several waves, the sequence of that rank when the
+  // batch is ordered from the longest to the shortest - CTAs are handed out in grid order, so the long ones start first
+  // and the short ones fill the tail. Every warp ranks the (at most 64) lengths on its own: no shared memory, no barrier.
+  int bi = blockIdx.z;
+  if (kp.lpt) {
+    if (!kp.early_src1) grid_dependency_wait();        // the lengths may come from the kernel in front
+    const int l0 = lane < p.B ? p.n1_per_seq[lane] : -1, l1 = lane + 32 < p.B ? p.n1_per_seq[lane + 32] : -1;
+    int r0 = 0, r1 = 0;                                // how many sequences come before mine (longer, or equal and earlier)
+    for (int i = 0; i < p.B; ++i) {
+      const int li = __shfl_sync(0xffffffffu, i < 32 ? l0 : l1, i & 31);
+      r0 += (li > l0 || (li == l0 && i < lane)) ? 1 : 0;
+      r1 += (li > l1 || (li == l1 && i < lane + 32)) ? 1 : 0;
+    }
+    const unsigned hit0 = __ballot_sync(0xffffffffu, lane < p.B && r0 == (int)blockIdx.z);
+    const unsigned hit1 = __ballot_sync(0xffffffffu, lane + 32 < p.B && r1 == (int)blockIdx.z);
+    bi = hit0 ? __ffs(hit0) - 1 : (hit1 ? __ffs(hit1) + 31 : (int)blockIdx.z);
+  }
   const int n2 = p.n2;
   const long long wlim = kp.wait_cycles;
   // The count of source 1 is read ahead of the grid dependency only at the reuse step (it is older than any kernel that
@@ -850,7 +868,7 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   const int sms = sm_count();
   // Key splits: enough CTAs to fill the SMs (two per SM with few query columns), but at least one full 128-key tile
   // per CTA, and at most eight (one cluster).
-  long long want = (NP == 32 && groups <= 64 ? 2 : 1) * (long long)sms / units;
+  long long want = (NP == 32 ? 2 : 1) * (long long)sms / units;
   const long long by_tiles = (groups + 3) / 4;
   if (want > by_tiles) want = by_tiles;
   if (tn.splits > 0) want = tn.splits;
@@ -858,14 +876,15 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   if (want < 1) want = 1;
   const int S = (int)want;
   // Footprint, ring depth, P^T buffers and softmax warpgroups:
-  // (a) few query columns and at most two full tiles per CTA: the footprint is kept below half an SM, so that two CTAs
-  //     are resident and the next call's CTAs can start loading while this call's finish;
+  // (a) few query columns and either at most two full tiles per CTA or a grid that fits the GPU only at two CTAs per
+  //     SM: the footprint is kept below half an SM, so that two CTAs are resident and the next call's CTAs can start
+  //     loading while this call's finish;
   // (b) few query columns and longer walks: the CTA takes what one SM has, and two softmax warpgroups take the tiles in
   //     turn (one warp per scheduler cannot hide its own latencies; two tiles in flight can);
   // (c) up to 64 query columns: one CTA per SM, one warpgroup.
   const int groups_cta = (groups + S - 1) / S;
   const size_t half_sm = 113 * 1024;     // two CTAs of this size, each with its 1 KB system share, fit one SM
-  bool small = NP == 32 && groups_cta <= 8;
+  bool small = NP == 32 && (groups_cta <= 8 || (units * S > sms && units * S <= 2 * sms));
   int WG = (NP == 32 && !small) ? 2 : 1;
   if (tn.dual == 1) { small = NP == 32; WG = 1; }      // force (a) / (b) where they apply
   if (tn.dual == 0 && NP == 32) { small = false; WG = 2; }
@@ -912,6 +931,11 @@ cudaError_t launch_attn_kt(const AttnParams& p, const AttnPlan& pl, int D, cudaS
   kp.gr2 = p.n2 < 32 ? p.n2 : 32;
   kp.early_src1 = (p.n2 > 0 && p.n1_max > 0 && tn.early_loads != 0) ? 1 : 0;
   kp.early_trigger = tn.trigger != 0 ? 1 : 0;
+  {
+    const long long ctas = (long long)kp.S * p.Hkv * p.B;
+    kp.lpt = (p.n1_per_seq != nullptr && p.B >= 4 && p.B <= 64 && ctas > sm_count()) ? 1 : 0;
+    if (tn.lpt >= 0) kp.lpt = (tn.lpt == 1 && p.n1_per_seq != nullptr && p.B >= 2 && p.B <= 64) ? 1 : 0;
+  }
   kp.wait_cycles = tn.wait_cycles;
   memset(&tm, 0, sizeof(tm));
   bool ok = umma_make_map(&tm.q, p.q, D, p.b, p.Hq, p.B, p.q_stride, p.b, p.G);

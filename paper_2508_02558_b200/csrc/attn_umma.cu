@@ -199,32 +199,6 @@ __global__ void __launch_bounds__(256) umma_tail_kernel(const UmmaParams up, con
                           (int64_t)p.B * p.Hkv * p.n1_max);
 }
 
-// Optional timeline of CTA (0,0,0): built with -DSDLLM_TRACE, each point stores the global timer in the 8-byte slot
-// `slot` (1..31) of the workspace's 256-byte status block. Compiled out by default.
-#ifdef SDLLM_TRACE
-__device__ __forceinline__ void trace_point(int32_t* status, int slot) {
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    reinterpret_cast<unsigned long long*>(status)[slot] = t;
-    if (slot == 1 || slot == 15) reinterpret_cast<long long*>(status)[slot == 1 ? 30 : 31] = clock64();
-  }
-}
-#define TRACE(slot) trace_point(p.status, slot)
-__device__ __forceinline__ void trace_all(int32_t* status, int slot, bool is_min) {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  unsigned long long* a = reinterpret_cast<unsigned long long*>(status) + slot;
-  if (is_min) atomicMin(a, t); else atomicMax(a, t);
-}
-#define TRACE_MIN(slot) trace_all(p.status, slot, true)
-#define TRACE_MAX(slot) trace_all(p.status, slot, false)
-#else
-#define TRACE(slot) do { } while (0)
-#define TRACE_MIN(slot) do { } while (0)
-#define TRACE_MAX(slot) do { } while (0)
-#endif
-
 // PROB selects the second pass of the probability saliency; it is a template parameter so that the attention kernel proper
 // does not carry that pass's code.
 // DUAL is the small-footprint variant for grids of several waves: 64-key tiles, a two-slot ring, 256 TMEM columns and at
@@ -264,7 +238,6 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
   }
   const int g = blockIdx.y / up.row_tiles, rt = blockIdx.y - g * up.row_tiles;
   const int split = blockIdx.x;
-  if (tid == 0) { TRACE(1); TRACE_MAX(24); }
   const int tiles1 = (p.n1_max + KT - 1) / KT;
   const int tiles2 = (p.n2 + KT2 - 1) / KT2;
   const int tiles_all = tiles1 + tiles2;
@@ -363,7 +336,6 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
     *abort_flag = 0;
     *last_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
-    TRACE(2);
     if (!zero_q && (do_s || do_scores)) {
       if (up.early_src1) {
         // Reuse step: the compacted cache and its count were written before the previous kernel in the stream even
@@ -377,10 +349,8 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
         prod_n1 = p.n1_per_seq ? p.n1_per_seq[bi] : p.n1_max;
         prod_n1 = min(max(prod_n1, 0), p.n1_max);
       }
-      TRACE(4);
       issue_q();
       produce(NS - prod_it, false);
-      TRACE(5);
     }
   }
   if (zero_q)
@@ -394,7 +364,6 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  if (tid == 0) TRACE(3);
 
   grid_dependency_wait();              // everything below may read what earlier kernels in the stream wrote
   grid_launch_dependents();
@@ -432,9 +401,7 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
       auto issue_pv = [&](const Tile& x, int j) -> bool {
         const int s = j % NS, pb = j & 1;
         if (!wait_bar(BAR(P_FULL + pb), (j >> 1) & 1, abort_flag, p.status, 4, p.wait_cycles)) return false;
-        if (j == 0) TRACE(8);
         if (!wait_bar(BAR(FULL_V + s), (j / NS) & 1, abort_flag, p.status, 5, p.wait_cycles)) return false;
-        if (j == 0) TRACE(9);
         tc_fence_after();
         const uint32_t vsm = smem_u32(stage0 + (size_t)s * stage_bytes) + kv_bytes;
         const uint32_t a_t = tmem_base + (uint32_t)pb * S_STRIDE;
@@ -456,7 +423,6 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
         }
         // without PV nothing else orders the reuse of an S buffer: wait until the softmax warps have read tile it - 2
         if (prob_pass && it >= 2 && !wait_bar(BAR(P_FULL + sb), ((it >> 1) - 1) & 1, abort_flag, p.status, 12, p.wait_cycles)) { ok = false; break; }
-        if (it == 0) TRACE(7);
         tc_fence_after();
         const uint32_t ksm = smem_u32(stage0 + (size_t)s * stage_bytes);
         const uint32_t qsm = smem_u32(q_s);
@@ -569,7 +535,6 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
         const bool idle = q4 * 32 - rep * rows_rep >= M_rt;
         const int c_lo = idle ? x.nv : min(rep * chunk_keys, x.nv), c_hi = min((rep + 1) * chunk_keys, x.nv);
         if (!wait_bar_warp(BAR(S_FULL + sb), (it >> 1) & 1, abort_flag, p.status, 9, p.wait_cycles)) { ok = false; break; }
-        if (tid == 64 && it == 0) TRACE(10);
         tc_fence_after();
         const uint32_t s_addr = lane_addr + (uint32_t)sb * S_STRIDE;
         // ---- the owned part of the S row. Chunks of 32 columns that are owned and valid as a whole go through the
@@ -676,10 +641,8 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(BAR(P_FULL + sb));
-        if (tid == 64 && it == 0) TRACE(11);
         ++it;
       }
-      if (tid == 64) TRACE(12);
       sm_ok = ok; sm_tiles = it;
     }
   } else {
@@ -808,7 +771,6 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
             make_float4(__uint_as_float(ov[4 * j]) * w, __uint_as_float(ov[4 * j + 1]) * w, __uint_as_float(ov[4 * j + 2]) * w,
                         __uint_as_float(ov[4 * j + 3]) * w);
     }
-    if (tid == 64) TRACE(27);
   }
   if (do_attn) {
     // all eight warps share the stores: consecutive threads take consecutive float4 of a row; a thread keeps its column
@@ -817,7 +779,6 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
     const float* o_s = reinterpret_cast<const float*>(stage0);
     const float2* lm_s = reinterpret_cast<const float2*>(DUAL ? smem + 1024 : stage0 + 128 * D * 4) + 128;
     __syncthreads();
-    if (tid == 64) TRACE(29);
     const int st = tid;
     if (!*abort_flag) {
       const int d4 = st % D4, r_first = st / D4, r_step = UM_THREADS / D4;
@@ -863,7 +824,6 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
       }
     }
   }
-  if (tid == 64) { TRACE(13); TRACE_MAX(25); }
 
   // ---- fused tail: the last CTA of the unit merges the key splits and pools the saliency; nobody waits ----
   const bool tail_merge = do_attn && p.splits > 1;
@@ -931,7 +891,6 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
   } else if (up.fused_tail && (tail_merge || tail_pool)) {
     __threadfence();
     __syncthreads();
-    if (tid == 0) TRACE_MAX(20);
     bool last = true;
     if (expected > 1) {
       if (tid == 0) {
@@ -941,7 +900,6 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
       __syncthreads();
       last = *last_flag != 0;
     }
-    if (tid == 0) TRACE_MAX(21);
     if (last && !*abort_flag) {
       __threadfence();
       if (tail_merge)
@@ -965,13 +923,13 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
         for (int pos = tid; pos < p.n1_max; pos += UM_THREADS)
           p.pooled[(int64_t)(bi * p.Hkv + g) * p.n1_max + pos] = pool_at(p, a_s, n1, p.block_off[bi], pos);
       }
-      if (tid == 0) TRACE_MAX(22);
-      if (expected > 1 && tid == 0) *counter = 0;               // ready for the next call
     }
+    // ready for the next call, whether or not this one gave up: a counter left at its final value would keep every
+    // later call on this workspace from ever finding its last CTA
+    if (last && expected > 1 && tid == 0) *counter = 0;
   }
 
   // ---- free the tensor memory ----
-  if (tid == 64) TRACE(14);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -979,7 +937,6 @@ __global__ void __launch_bounds__(UM_THREADS, DUAL ? 2 : 1) attn_umma_bf16_kerne
     tc_fence_after();
     tmem_dealloc(tmem_base, TMEM_COLS);
   }
-  if (tid == 0) { TRACE(15); TRACE_MAX(26); TRACE_MAX(16 + (int)blockIdx.x); }
 }
 
 // ---------------------------------------------------------------------------------------------------------

@@ -187,7 +187,7 @@ def test_softmax_probability_saliency(cfg, block, plan, tuning):
     _run_sequence_case(cfg, seed=15, block=block, n_sparse=1, score=B.SCORE_PROB_MEAN)
 
 
-@pytest.mark.parametrize("plan", [{}, dict(splits=3), dict(dual=0, splits=1), dict(dual=0, splits=2), dict(kernel=2), dict(kernel=2, lpt=1), dict(kernel=2, lpt=1, dual=1, splits=1),
+@pytest.mark.parametrize("plan", [{}, dict(splits=3), dict(lpt=1), dict(lpt=1, dual=0, splits=1), dict(dual=0, splits=1), dict(dual=0, splits=2), dict(kernel=2), dict(kernel=2, lpt=1), dict(kernel=2, lpt=1, dual=1, splits=1),
                                   dict(select=2)])
 def test_ragged_batch(plan, tuning):
     import parity_util as U

@@ -347,6 +347,95 @@ def test_refresh_policies_and_variants():
     assert (rq.scores > 0).all() and (rq.scores < 1).all() and rq.kept_idx.shape == rj.kept_idx.shape
 
 
+def _kept_by_library_routines(a, o, n_pre, n_suf, window, kind, per_region, joint_n=None):
+    """The kept candidate set of one head rebuilt from library pieces only: torch max/avg pooling per region (or over the
+    whole candidate axis) and a stable numpy sort by (score descending, index ascending)."""
+    def pooled_of(x):
+        t = torch.from_numpy(np.asarray(x, np.float64))[None, None]
+        if kind == oracle.POOL_MAX:
+            return F.max_pool1d(t, window, 1, window // 2)[0, 0].numpy()
+        return F.avg_pool1d(t, window, 1, window // 2, count_include_pad=True)[0, 0].numpy()
+
+    def top(x, n):
+        order = np.argsort(-x, kind="stable")          # equal scores keep their index order: the lower index wins
+        return np.sort(order[:n])
+    if not per_region:
+        return top(pooled_of(a), joint_n)
+    pre = top(pooled_of(a[:o]), n_pre) if o > 0 else np.zeros(0, np.int64)
+    if n_suf is None:                                  # prefix-sparse: the whole suffix stays
+        suf = np.arange(len(a) - o)
+    else:
+        suf = top(pooled_of(a[o:]), n_suf) if len(a) > o else np.zeros(0, np.int64)
+    return np.concatenate([pre, suf + o])
+
+
+@pytest.mark.parametrize("kind", [oracle.POOL_MAX, oracle.POOL_AVG])
+@pytest.mark.parametrize("window", [3, 5])
+def test_refresh_variant_branches_against_library_routines(kind, window):
+    """Per-region ceil, prefix-only (Algorithm 5) and the AvgPool ablation through refresh(): the kept sets must equal
+    what torch's pooling and a stable sort give region by region. The inputs put a dominant score on the LAST prefix key
+    and on the FIRST suffix key, so pooling across the seam, or a quota taken jointly, changes the kept sets."""
+    rng = np.random.default_rng(61)
+    Hq, Hkv, b, L, D, o = 4, 2, 8, 77, 16, 30
+    q = rng.standard_normal((Hq, b, D))
+    k, v = rng.standard_normal((Hkv, L, D)), rng.standard_normal((Hkv, L, D))
+    G = Hq // Hkv
+    for g in range(Hkv):
+        u = q[g * G:(g + 1) * G].mean(axis=(0, 1))
+        u /= np.linalg.norm(u)
+        k[g, o - 1] += (9.0 if g == 0 else 0.0) * u      # head 0: the last prefix key dominates
+        k[g, o + b] += (0.0 if g == 0 else 9.0) * u      # head 1: the first suffix key dominates
+    r = 0.3
+    C = L - b
+    pos = oracle.candidate_positions(L, b, o)
+    for select in (oracle.SELECT_JOINT_FLOOR, oracle.SELECT_PER_REGION_CEIL, oracle.SELECT_PREFIX_ONLY):
+        res = oracle.refresh(q, k, v, o, r, window, pool_kind=kind, select=select)
+        a = oracle.scores_logit_mean(q, k, o)            # pinned on its own by the linearity and planted-key tests
+        per_region = select != oracle.SELECT_JOINT_FLOOR
+        if select == oracle.SELECT_JOINT_FLOOR:
+            n_pre = n_suf = None
+            joint_n = int(np.floor(C * r))
+        elif select == oracle.SELECT_PER_REGION_CEIL:
+            n_pre, n_suf, joint_n = int(np.ceil(o * r)), int(np.ceil((C - o) * r)), None
+        else:
+            n_pre, n_suf, joint_n = int(np.floor(o * r)), None, None
+        for g in range(Hkv):
+            want = pos[_kept_by_library_routines(a[g], o, n_pre, n_suf, window, kind, per_region, joint_n)]
+            np.testing.assert_array_equal(res.kept_idx[g], want)
+    # the planted inputs bite: with max pooling the joint reading keeps the neighbour across the seam, the per-region one
+    # does not reach over it
+    joint = oracle.refresh(q, k, v, o, r, window, pool_kind=oracle.POOL_MAX, select=oracle.SELECT_JOINT_FLOOR)
+    region = oracle.refresh(q, k, v, o, r, window, pool_kind=oracle.POOL_MAX, select=oracle.SELECT_PER_REGION_CEIL)
+    assert o + b in joint.kept_idx[0] and o - 1 in joint.kept_idx[1]
+    assert joint.pooled[0][o] == joint.pooled[0][o - 1] and region.pooled[0][o] < region.pooled[0][o - 1]
+    assert not np.array_equal(joint.kept_idx[0], region.kept_idx[0]) or not np.array_equal(joint.kept_idx[1], region.kept_idx[1])
+
+
+def test_refresh_probability_scores_against_library_softmax():
+    """SCORE_PROB_MEAN through refresh(): the scores are the column means of torch.softmax over ALL keys (block included)
+    taken over the group's block queries, and on the tiny config the sink and every planted key are kept."""
+    cfg = W.CONFIGS["c1_tiny"]
+    s = W.make_sequence(cfg, seed=0)
+    q, k, v = s.refresh_inputs(1)
+    o, b, L = s.block_off, cfg.block_len, cfg.seq_len
+    res = oracle.refresh(q, k, v, o, cfg.retention, cfg.pool_window, score=oracle.SCORE_PROB_MEAN)
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    scale = 1.0 / np.sqrt(cfg.head_dim)
+    pos = oracle.candidate_positions(L, b, o)
+    for g in range(cfg.n_kv_heads):
+        logits = torch.from_numpy(q[g * G:(g + 1) * G].astype(np.float64)) @ torch.from_numpy(k[g].astype(np.float64)).T * scale
+        probs = torch.softmax(logits, dim=-1).reshape(-1, L).mean(dim=0).numpy()
+        np.testing.assert_allclose(res.scores[g], probs[pos], rtol=1e-12, atol=1e-15)
+        kept = set(res.kept_idx[g].tolist())
+        assert 0 in kept                                               # the sink
+        assert set(int(x) for x in s.planted_pos[g]) <= kept           # the planted salient keys
+    # and the selection on top of those scores is the library one
+    a = res.scores
+    for g in range(cfg.n_kv_heads):
+        want = pos[_kept_by_library_routines(a[g], o, None, None, cfg.pool_window, oracle.POOL_MAX, False, res.n_keep)]
+        np.testing.assert_array_equal(res.kept_idx[g], want)
+
+
 # ------------------------------------------------------------------ generator sanity (shapes, rounding, determinism)
 def test_workload_generator_is_deterministic_and_rounded():
     cfg = W.CONFIGS["c3_dream"]
