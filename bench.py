@@ -33,9 +33,22 @@ from paper_2508_02558_b200 import workloads as W
 
 METRIC = "cached_kv_tokens_per_s_per_layer"
 UNIT = "tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the sparse-attention kernel pair on this workload,
-# from the ncu capture summarised under profiles/ (None until a capture exists for the workload).
-NCU_TRAFFIC_BYTES = {"c2_llada": 11118080}
+PROFILES = os.path.join(ROOT, "profiles")
+
+
+def ncu_traffic(workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the reuse-step kernel on `workload`, read from the ncu
+    summary under profiles/ (a line "traffic_bytes_per_launch: N"); None when no capture of the current kernel exists."""
+    path = os.path.join(PROFILES, "attn_kt_%s_sparse.txt" % workload)
+    if not os.path.exists(path):
+        return None, None
+    for line in open(path):
+        if line.startswith("traffic_bytes_per_launch:"):
+            try:
+                return int(line.split(":")[1].split()[0]), os.path.relpath(path, ROOT)
+            except ValueError:
+                return None, None
+    return None, None
 
 
 def parse_args():
@@ -56,6 +69,7 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--tune", action="append", default=[], metavar="NAME=VALUE",
                     help="override one decision of the library's launch planner (sdllm_tuning_set), e.g. --tune splits=4")
+    ap.add_argument("--no-legs", action="store_true", help="skip the short legs over the other workloads (key 'workloads')")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -89,8 +103,17 @@ def workload_config(args) -> W.WorkloadConfig:
     return cfg
 
 
+def block_schedule(cfg: W.WorkloadConfig, state_of=None):
+    """(dense, refresh, reuse) step counts of one decoding block: cache states 0, 1, 2 of Algorithm 2 over the block's
+    denoising steps. `state_of` is the library's sdllm_cache_state (the closed form min(i, 2) where the library is not
+    loaded: the CPU arm)."""
+    state_of = state_of or (lambda i: min(i, 2))
+    states = [state_of(i) for i in range(cfg.steps_per_block)]
+    return states.count(0), states.count(1), states.count(2)
+
+
 def tokens_per_step(cfg: W.WorkloadConfig, n_layers: int, seq_lens, n_keeps, phase: str = "all") -> int:
-    reuse_steps = cfg.steps_per_block - 2
+    reuse_steps = block_schedule(cfg)[2]
     refresh = sum(seq_lens) if phase in ("all", "refresh") else 0
     sparse = reuse_steps * sum(n + cfg.block_len for n in n_keeps) if phase in ("all", "sparse") else 0
     return n_layers * (refresh + sparse)
@@ -149,6 +172,124 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+
+# ------------------------------------------------------------------------------------------------ per-call timing
+LEGS = [  # (workload, batch, retention override, pool window override, layers rotated so that the working set exceeds L2)
+    ("c3_dream", 1, None, None, 28),
+    ("c4_long", 1, 0.1, 3, 3), ("c4_long", 1, 0.25, 3, 3), ("c4_long", 1, 0.5, 3, 3), ("c4_long", 1, 0.5, 1, 3), ("c4_long", 1, 0.5, 7, 3),
+    ("c5_serving", 1, None, None, 8), ("c5_serving", 4, None, None, 2), ("c5_serving", 16, None, None, 1),
+]
+
+
+def time_calls(torch, dev, cfg, Bn, n_layers, rank, peak, steps=5, n_step_sets=4, sampler_index=None):
+    """Times every call of the path on its own for one workload: the refresh-step attention, top-k, compaction, the two
+    fused in one call, the whole refresh chain and the reuse step, each replayed from a CUDA graph over `n_layers` sets
+    of buffers (together larger than L2). Returns microseconds per call and the fraction of the HBM roof."""
+    import dataclasses
+    from paper_2508_02558_b200 import binding as B
+    from paper_2508_02558_b200.session import LayerCache
+    Hq, Hkv, D, b = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.block_len
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    bdt = B.BF16 if cfg.dtype == "bf16" else B.F32
+
+    def to_dev(x):
+        if cfg.dtype == "bf16":
+            return torch.from_numpy(W.f32_to_bf16_bits(x).reshape(x.shape).view(np.int16)).view(torch.bfloat16).to(dev)
+        return torch.from_numpy(x).to(dev)
+    prompt_lens = W.serving_prompt_lengths(Bn, seed=5 + rank) if cfg.name == "c5_serving" else [cfg.prompt_len] * Bn
+    seq_lens = [p_ + cfg.gen_len for p_ in prompt_lens]
+    L = max(seq_lens)
+    caches, Ks, Vs, Qr, Qs, Kn, Vn = [], [], [], [], [], [], []
+    gen = torch.Generator(device=dev); gen.manual_seed(99 + rank)
+    drift = cfg.drift_std / np.sqrt(D)
+    for l in range(n_layers):
+        bw = W.make_batch(cfg, prompt_lens, seed=rank, layer=l, block=0)
+        q, k, v = bw.refresh_inputs(1)
+        Ks.append(to_dev(k)); Vs.append(to_dev(v)); Qr.append(to_dev(q))
+        caches.append(LayerCache(batch=Bn, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, seq_len_max=L, block_len=b, dtype=bdt,
+                                 retention=cfg.retention, pool_window=cfg.pool_window, device=str(dev),
+                                 share_scratch_with=caches[0] if caches else None))
+        rows = torch.stack([torch.arange(o_, o_ + b, device=dev) for o_ in prompt_lens])
+        gather = rows[:, None, :, None].expand(Bn, Hkv, b, D)
+        kb, vb = Ks[l].gather(2, gather).float(), Vs[l].gather(2, gather).float()
+        Qs.append([(Qr[l].float() + drift * torch.randn(Qr[l].shape, device=dev, generator=gen)).to(tdt) for _ in range(n_step_sets)])
+        Kn.append([(kb + drift * torch.randn(kb.shape, device=dev, generator=gen)).to(tdt) for _ in range(n_step_sets)])
+        Vn.append([(vb + drift * torch.randn(vb.shape, device=dev, generator=gen)).to(tdt) for _ in range(n_step_sets)])
+    d0 = caches[0].desc
+    n_keeps = [B.keep_count(d0, Li, pi)[0] for Li, pi in zip(seq_lens, prompt_lens)]
+    sl = torch.tensor(seq_lens, dtype=torch.int32, device=dev)
+    bo = torch.tensor(prompt_lens, dtype=torch.int32, device=dev)
+    out_r = [torch.empty((Bn, Hq, b, D), dtype=tdt, device=dev) for _ in range(n_layers)]
+    out_s = [torch.empty((Bn, Hq, b, D), dtype=tdt, device=dev) for _ in range(n_layers)]
+    stream = torch.cuda.Stream(device=dev)
+    torch.cuda.synchronize(dev)
+
+    def graph_time(fn, calls):
+        with torch.cuda.stream(stream):
+            fn()
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            fn()
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                g.replay()
+            stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(steps):
+                g.replay()
+            e1.record(stream)
+            stream.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / steps / calls
+
+    c = caches
+    ops = {
+        "refresh_chain": (lambda: [c[l].refresh(Qr[l], Ks[l], Vs[l], sl, bo, out=out_r[l], stream=stream) for l in range(n_layers)], n_layers),
+        "refresh": (lambda: [B.refresh_scores(c[l].desc, Qr[l], Ks[l], Vs[l], sl, bo, out_r[l], None, c[l].pooled, c[l].workspace, stream)
+                             for l in range(n_layers)], n_layers),
+        "topk": (lambda: [B.select_topk(c[l].desc, c[l].pooled, sl, bo, c[l].kept_idx, c[l].kept_cnt, None, stream) for l in range(n_layers)], n_layers),
+        "compact": (lambda: [B.compact_kv(c[l].desc, Ks[l], Vs[l], c[l].kept_idx, c[l].kept_cnt, c[l].k_c, c[l].v_c, stream)
+                             for l in range(n_layers)], n_layers),
+        "select_compact": (lambda: [B.select_compact(c[l].desc, c[l].pooled, sl, bo, Ks[l], Vs[l], c[l].kept_idx, c[l].kept_cnt, c[l].k_c,
+                                                     c[l].v_c, stream) for l in range(n_layers)], n_layers),
+        "reuse": (lambda: [c[l].sparse_step(Qs[l][t], Kn[l][t], Vn[l][t], out_s[l], stream=stream)
+                           for t in range(n_step_sets) for l in range(n_layers)], n_layers * n_step_sets),
+    }
+    sampler = ClockSampler(sampler_index) if sampler_index is not None else None
+    us = {}
+    for name in ("refresh_chain", "refresh", "topk", "compact", "select_compact", "reuse"):   # the chain first: it fills every cache
+        us[name] = graph_time(*ops[name])
+    clocks = sampler.stop() if sampler else None
+    ab = algorithmic_bytes(cfg, seq_lens, n_keeps)
+    ab["refresh_chain"] = ab["refresh"] + ab["topk"] + ab["compact"]
+    ab["select_compact"] = ab["topk"] + ab["compact"]
+    ab["reuse"] = ab["sparse"]
+    rec = {"workload": cfg.name, "batch": Bn, "retention": cfg.retention, "pool_window": cfg.pool_window, "layers_rotated": n_layers,
+           "seq_len_max": L, "n_keep_max": max(n_keeps), "fused_select_compact": B.launch_count(d0, B.OP_SELECT_COMPACT) == 1}
+    for name in us:
+        rec[name + "_us"] = round(us[name], 3)
+        rec["frac_" + name] = round(ab[name] / (us[name] * 1e-6) / 1e9 / peak, 4)
+    rec["clocks"] = clocks
+    del caches, Ks, Vs, Qr, Qs, Kn, Vn
+    torch.cuda.empty_cache()
+    return rec
+
+
+def run_legs(torch, dev, rank, peak, local):
+    """Short legs over the workloads that are not the headline: one record per (workload, batch, retention, window)."""
+    import dataclasses
+    out = []
+    for name, Bn, r, s_, layers in LEGS:
+        cfg = W.CONFIGS[name]
+        if r is not None:
+            cfg = dataclasses.replace(cfg, retention=r)
+        if s_ is not None:
+            cfg = dataclasses.replace(cfg, pool_window=s_)
+        out.append(time_calls(torch, dev, cfg, Bn, layers, rank, peak, sampler_index=local))
+    return out
+
+
 # ------------------------------------------------------------------------------------------------ CPU oracle arm
 def oracle_block_sample(cfg: W.WorkloadConfig, seed: int):
     """One layer x one decoding block through the CPU oracle: 1 refresh + the block's reuse steps. Returns (tokens, seconds)."""
@@ -163,6 +304,49 @@ def oracle_block_sample(cfg: W.WorkloadConfig, seed: int):
         oracle.sparse_block_attention(q2, k_c, v_c, kn, vn)
     dt = time.perf_counter() - t0
     return cfg.seq_len + len(steps) * (r.n_keep + cfg.block_len), dt
+
+
+def oracle_one_thread(workload: str):
+    """The same bounded oracle sample on ONE host thread (a child process with OMP_NUM_THREADS=1, the oracle untouched)."""
+    env = dict(os.environ, OMP_NUM_THREADS="1")
+    try:
+        res = subprocess.run([sys.executable, os.path.abspath(__file__), "--impl", "reference", "--workload", workload, "--steps", "1",
+                              "--warmup", "1"], env=env, capture_output=True, text=True, timeout=240)
+        line = json.loads(res.stdout.strip().splitlines()[-1])
+        return {"value": line["value"], "unit": UNIT, "cores": 1, "sample": line["config"]["sample"]}
+    except Exception as e:                      # the figure is reported context: never let it take the run down
+        return {"value": None, "error": repr(e)[:200]}
+
+
+def oracle_other_workloads():
+    """Bounded oracle samples of the other configurations: the tiny config whole, one refresh + 2 reuse steps of one
+    long-context point and of the serving batches (cached-KV tokens per second, all host threads)."""
+    import dataclasses
+    import oracle
+    out = []
+    jobs = [("c1_tiny", 1, None, 3), ("c3_dream", 1, None, 2), ("c4_long", 1, 0.5, 2), ("c5_serving", 1, None, 2), ("c5_serving", 4, None, 2),
+            ("c5_serving", 16, None, 1)]
+    for name, Bn, r, n_reuse in jobs:
+        cfg = W.CONFIGS[name]
+        if r is not None:
+            cfg = dataclasses.replace(cfg, retention=r)
+        lens = W.serving_prompt_lengths(Bn, seed=5) if name == "c5_serving" else [cfg.prompt_len] * Bn
+        bw = W.make_batch(cfg, lens, seed=0)
+        steps = [bw.sparse_inputs(i) for i in range(2, 2 + n_reuse)]
+        q, k, v = bw.refresh_inputs(1)
+        tok, t0 = 0, time.perf_counter()
+        for i, sq in enumerate(bw.seqs):
+            Li, o = sq.seq_len, sq.block_off
+            res = oracle.refresh(q[i], k[i, :, :Li], v[i, :, :Li], o, cfg.retention, cfg.pool_window)
+            k_c, v_c = oracle.gather_rows(k[i, :, :Li], res.kept_idx), oracle.gather_rows(v[i, :, :Li], res.kept_idx)
+            tok += Li
+            for q2, kn, vn in steps:
+                oracle.sparse_block_attention(q2[i], k_c, v_c, kn[i], vn[i])
+                tok += res.n_keep + cfg.block_len
+        sec = time.perf_counter() - t0
+        out.append({"workload": name, "batch": Bn, "retention": cfg.retention, "value": tok / sec, "unit": UNIT, "cores": omp_threads(),
+                    "seconds": round(sec, 3), "sample": "1 layer: 1 refresh + %d reuse steps" % n_reuse})
+    return out
 
 
 def omp_threads() -> int:
@@ -237,7 +421,8 @@ def run_ours(args):
     cfg = workload_config(args)
     n_layers = args.layers or cfg.n_layers
     Hq, Hkv, D, b = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.block_len
-    reuse_steps = cfg.steps_per_block - 2
+    n_dense, n_refresh, reuse_steps = block_schedule(cfg, B.cache_state)      # Algorithm 2: 1 dense, 1 refresh, 30 reuse
+    assert n_refresh == 1
     tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
     bdt = B.BF16 if cfg.dtype == "bf16" else B.F32
 
@@ -395,13 +580,25 @@ def run_ours(args):
     rf_sec = timed(rf_runner, max(3, args.steps // 2), 3) / max(3, args.steps // 2) / n_layers
     peak, peak_kind = peaks()
     achieved = ab["sparse"] / sp_sec / 1e9
-    roofline = {"bound": "hbm", "kernel": "sdllm_sparse_block_attn (attn_umma_bf16_kernel<128, false, false>: tcgen05 attention, key splits merged through cluster shared memory)", "achieved": achieved,
+    traffic, traffic_file = ncu_traffic(cfg.name)
+    kinds = {3: "attn_kt_kernel: tcgen05 attention with the keys on the accumulator rows, key splits merged through cluster shared memory",
+             2: "attn_umma_bf16_kernel: tcgen05 attention with the queries on the accumulator rows", 0: "cp.async kernels"}
+    roofline = {"bound": "hbm", "kernel": "sdllm_sparse_block_attn (%s)" % kinds.get(3 if Hq // Hkv * b <= 64 and cfg.dtype == "bf16" else 2, ""),
+                "achieved": achieved,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                 "frac_of_8TBps": achieved / 8000.0, "algorithmic_bytes_per_launch": ab["sparse"], "us_per_launch": sp_sec * 1e6,
-                "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+                "traffic": traffic, "traffic_source": traffic_file,
                 "refresh_chain": {"us_per_layer": rf_sec * 1e6, "algorithmic_bytes": ab["refresh"] + ab["topk"] + ab["compact"],
                                   "achieved": (ab["refresh"] + ab["topk"] + ab["compact"]) / rf_sec / 1e9,
                                   "frac": (ab["refresh"] + ab["topk"] + ab["compact"]) / rf_sec / 1e9 / peak}}
+    # every call of the path on its own, for the headline workload and (default run) for the other configurations
+    per_call = None
+    legs = None
+    if rank == 0 and world == 1 and not args.no_legs:
+        per_call = time_calls(torch, dev, cfg, Bn, min(n_layers, 8 if Bn == 1 else 2), rank, peak, sampler_index=local)
+        roofline["calls"] = {k: per_call[k] for k in per_call if k.endswith("_us") or k.startswith("frac_")}
+        if args.workload == "c2_llada" and args.batch == 1 and args.retention is None and args.pool_window is None:
+            legs = run_legs(torch, dev, rank, peak, local)
 
     # ---- end to end: inputs start in pinned host memory, results are read back, every step
     e2e = None
@@ -435,6 +632,9 @@ def run_ours(args):
         ctok, csec = oracle_block_sample(cfg, seed=0)
         cpu_baseline = {"value": ctok / csec, "unit": UNIT, "cores": omp_threads(), "kind": "oracle", "seconds": csec,
                         "sample": "1 layer x 1 block (1 refresh + %d reuse steps) of %s, fp64" % (reuse_steps, cfg.name)}
+        if legs is not None:
+            cpu_baseline["one_thread"] = oracle_one_thread(cfg.name)
+            cpu_baseline["other_workloads"] = oracle_other_workloads()
 
     if rank == 0:
         print(json.dumps({
@@ -448,7 +648,7 @@ def run_ours(args):
                            n_layers * (ab["refresh"] + ab["compact"] / 2) / 1e6),
                        "launch": "eager" if args.no_graph else "cuda_graph_replay", "parallelism": "replicas" if world > 1 else "1gpu"},
             "block_steps_per_s": world * n_layers * (1 + reuse_steps) * args.steps / sec,
-            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks,
+            "roofline": roofline, "workloads": legs, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks,
             "gpu_launches": launches_per_step * args.steps,
         }))
     if world > 1:
