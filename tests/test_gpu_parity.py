@@ -362,3 +362,40 @@ def test_dense_step_strided_tensors_and_argument_checks():
     with pytest.raises(B.SdllmError) as e:
         B.dense_attn(d, qd, kd.view(-1)[4:].view(-1), vd, None, out, None, ws)
     assert e.value.status == B.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("plan", [
+    {},                                  # key-row kernel: its splits still meet in the cluster merge while they give up
+    dict(splits=1),                      # ... one CTA per head
+    dict(kernel=2, cluster=0, splits=3), # query-row kernel, partials and completion counters in the workspace
+    dict(kernel=2),                      # ... cluster tail
+])
+def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_a_usable_library(plan, tuning):
+    """With the limit of the abortable device-side waits set to zero, the first wait that is not already satisfied gives
+    up. Nothing hangs and nothing faults: the call returns, the status word reports the time-out, and after the workspace
+    has been zeroed again the next call (normal limit) matches the oracle. The waits that let copies and MMAs in flight
+    land before a CTA retires keep their own long limit."""
+    import parity_util as U
+    cfg = _small("timeout", "bf16", 4, 4, 128, 330, 64, salient_frac=0.02)
+    s = W.make_sequence(cfg, seed=19, block=0)
+    q, k, v = s.refresh_inputs(1)
+    tuning(**plan)                       # before the workspace is sized
+    g = U.gpu_refresh(q[None], k[None], v[None], [s.seq_len], [s.block_off], "bf16", cfg.retention, cfg.pool_window)
+    q2, kn, vn = s.sparse_inputs(2)
+    want = U.gpu_sparse_step(g, q2[None], kn[None], vn[None], "bf16")          # the plan itself works
+    U.check_sparse_against_oracle(g, want, q2[None], kn[None], vn[None], "bf16")
+    tuning(wait_cycles=0)
+    qd, knd, vnd = U.to_dev(q2[None], "bf16"), U.to_dev(kn[None], "bf16"), U.to_dev(vn[None], "bf16")
+    out = torch.zeros(q2[None].shape, dtype=torch.bfloat16, device=U.DEV)
+    g.cache.sparse_step(qd, knd, vnd, out)
+    torch.cuda.synchronize()                                                   # the call returns
+    assert B.read_status(g.cache.workspace) != 0                               # ... and says that it gave up
+    with pytest.raises(B.SdllmError) as e:
+        B._check(B.lib().sdllm_read_status(g.cache.workspace.data_ptr(), torch.cuda.current_stream().cuda_stream,
+                                           __import__("ctypes").byref(__import__("ctypes").c_int32(0))), "sdllm_read_status")
+    assert e.value.status == B.ERR_TIMEOUT
+    tuning(wait_cycles=400_000_000)
+    g.cache.workspace.zero_()                                                  # what the header asks for after a time-out
+    again = U.gpu_sparse_step(g, q2[None], kn[None], vn[None], "bf16")
+    U.check_sparse_against_oracle(g, again, q2[None], kn[None], vn[None], "bf16")
+    np.testing.assert_array_equal(again, want)
