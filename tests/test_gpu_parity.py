@@ -399,3 +399,34 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_a_usable_library(pl
     again = U.gpu_sparse_step(g, q2[None], kn[None], vn[None], "bf16")
     U.check_sparse_against_oracle(g, again, q2[None], kn[None], vn[None], "bf16")
     np.testing.assert_array_equal(again, want)
+
+
+@pytest.mark.parametrize("plan", [{}, dict(splits=1), dict(splits=2), dict(dual=0, splits=1), dict(dual=0, splits=2), dict(kernel=2)])
+def test_logits_far_above_the_softmax_references(plan, tuning):
+    """The key-row kernel takes its softmax references from the first key of a CTA's first tile and only checks later keys
+    against them; keys whose logits lie more than 2^64 above a reference make it raise the references and rescale what it
+    has accumulated. Here every query shares a strong component with a few keys planted in the first tile (not its first
+    row), in later tiles and in the block's fresh rows, 50 to 100 nats above everything else: refresh and reuse step must
+    still match the oracle."""
+    import parity_util as U
+    tuning(**plan)
+    rng = np.random.default_rng(23)
+    Hq = Hkv = 2
+    D, b, L, o = 128, 32, 900, 700
+    q = rng.standard_normal((Hq, b, D)).astype(np.float32) * 0.3
+    q[:, :, 0] += 3.0
+    k = rng.standard_normal((Hkv, L, D)).astype(np.float32) * 0.3
+    v = rng.standard_normal((Hkv, L, D)).astype(np.float32)
+    for pos, gain in [(5, 300.0), (300, 250.0), (301, 250.0), (640, 200.0), (o + 40 + b, 400.0), (o + 3, 300.0)]:
+        k[:, pos, :] = 0.0
+        k[:, pos, 0] = gain                      # logit = gain * 3 / sqrt(128): 53 to 106 nats (76 to 153 in log2 units) above the rest
+    q, k, v = (W.round_to_dtype(x, "bf16") for x in (q, k, v))
+    g = U.gpu_refresh(q[None], k[None], v[None], [L], [o], "bf16", 0.5, 3)
+    U.check_refresh_against_oracle(g, q[None], k[None], v[None], [L], [o], "bf16", 0.5, 3)
+    U.check_compaction_bit_exact(g, g.k_dev, g.v_dev)
+    q2 = W.round_to_dtype(q + 0.01 * rng.standard_normal(q.shape).astype(np.float32), "bf16")
+    kn, vn = k[:, o:o + b].copy(), v[:, o:o + b].copy()
+    kn[:, 17, :] = 0.0
+    kn[:, 17, 0] = 500.0                         # the largest logit of all sits in the block's fresh rows (the last tile)
+    out = U.gpu_sparse_step(g, q2[None], kn[None], vn[None], "bf16")
+    U.check_sparse_against_oracle(g, out, q2[None], kn[None], vn[None], "bf16")
