@@ -44,9 +44,9 @@ namespace sdllm {
 using namespace dev;
 namespace {
 
-constexpr int KT_THREADS = 192;          // two service warps and one softmax warpgroup; 320 with two warpgroups
 constexpr int KT_MAX_STAGES = 3;
-constexpr int KT_CTRL = 5120;            // control block: barriers, flags, and per softmax warpgroup references, sums, scratch
+constexpr int KT_GRP = 3072;             // control block, per softmax warpgroup: references, raise scratch, sums, saliency partials
+constexpr int KT_CTRL0 = 1024;           // control block, common part: barriers and flags
 
 struct KtMaps {
   CUtensorMap q, k1, v1, k2, v2;   // boxes of 32 rows (source 2: min(32, n2))
@@ -71,6 +71,7 @@ struct KtParams {
 #include "umma_ptx.cuh"
 
 __device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed;\n" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release;\n" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire;\n" ::: "memory"); }
 // Asynchronous stores into the shared memory of a CTA of the cluster; each one reports its bytes to an mbarrier of that
 // CTA (complete_tx, release at cluster scope), so the receiver waits for exactly the data it is owed and for nothing else.
@@ -121,9 +122,10 @@ __device__ __forceinline__ bool softmax_barrier_or(int id, bool pred) {
       : "=r"(r) : "r"((uint32_t)pred), "r"(id) : "memory");
   return r != 0;
 }
-// barrier of one softmax warpgroup (ids 1 and 2), and of both (id 3)
+// barrier of one softmax warpgroup (ids 1 to 4), and of all of them (id 5)
 __device__ __forceinline__ void softmax_barrier(int id) { asm volatile("bar.sync %0, 128;\n" ::"r"(id) : "memory"); }
-__device__ __forceinline__ void softmax_barrier_both() { asm volatile("bar.sync 3, 256;\n" ::: "memory"); }
+template <int NG>
+__device__ __forceinline__ void softmax_barrier_all() { asm volatile("bar.sync 5, %0;\n" ::"n"(128 * NG) : "memory"); }
 
 // order-preserving fp32 <-> u32 (larger float <=> larger code), for the shared-memory max of the references
 __device__ __forceinline__ uint32_t f2ord(float x) {
@@ -177,15 +179,23 @@ __device__ __forceinline__ float kt_pool_at(const AttnParams& p, const float* a,
   return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
 }
 
-template <int D, int NCH, int WG>
-__global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) attn_kt_kernel(const __grid_constant__ KtMaps tm, const KtParams kp) {
-  constexpr int NTHREADS = 64 + 128 * WG;    // WG softmax warpgroups take the tiles in turn, each with its own accumulator
+// WG = 2: two softmax warpgroups take the tiles in turn, each with its own accumulator and references (32 query columns).
+// CG > 1: CG softmax warpgroups share every tile, each owning 32 of the 32 * CG query columns (one accumulator).
+template <int D, int WG, int CG>
+__global__ void __launch_bounds__(64 + 128 * WG * CG, (WG == 1 && CG == 1) ? 2 : 1) attn_kt_kernel(const __grid_constant__ KtMaps tm, const KtParams kp) {
+  static_assert(WG == 1 || CG == 1, "tile-alternating warpgroups only with one column group");
+  constexpr int NG = WG * CG;                // softmax warpgroups
+  constexpr int NTHREADS = 64 + 128 * NG;
   constexpr int H = D / 64;                  // 128-byte column halves of a K/V row
-  constexpr int NP = NCH * 32;               // query columns padded to the softmax chunking
-  constexpr int PROW = NP * 2;               // bytes of a P^T row: one key, NP bf16 (64-byte swizzle for 32 columns, 128-byte for 64)
-  constexpr int PBUF = 128 * PROW;           // one P^T buffer: 128 key rows
-  constexpr uint32_t O_COL = 2 * NP;         // TMEM columns: two S^T buffers of NP, then one O^T (NP columns) per warpgroup
-  constexpr uint32_t TMEM_COLS = (2 * NP + NP * WG <= 128) ? 128 : 256;
+  constexpr int NP = 32;                     // query columns of one softmax thread
+  constexpr int NPT = 32 * CG;               // query columns of the tile (padded)
+  constexpr int PHALVES = (CG + 1) / 2;      // 64-column halves of a P^T row (CG > 1: 128-byte rows, 128-byte swizzle)
+  constexpr int PBUF = CG == 1 ? 128 * 64 : PHALVES * 128 * 128;   // one P^T buffer: 128 key rows (CG = 1: 64-byte rows, 64-byte swizzle)
+  constexpr uint32_t O_COL = 2 * NPT;        // TMEM columns: two S^T buffers of NPT, then one O^T of NPT per tile-alternating warpgroup
+  constexpr uint32_t TMEM_NEED = 2 * NPT + NPT * WG;
+  constexpr int MS = 8;                      // largest cluster (key splits of one unit)
+  constexpr uint32_t TMEM_COLS = TMEM_NEED <= 128 ? 128 : (TMEM_NEED <= 256 ? 256 : 512);
+  constexpr int KT_CTRL = KT_CTRL0 + NG * KT_GRP;
   extern __shared__ unsigned char smem_raw[];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -235,21 +245,27 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
   constexpr int S_FULL = 1 + 4 * KT_MAX_STAGES, P_FULL = S_FULL + 2, PV_DONE = S_FULL + 4, DRAIN = S_FULL + 6, MERGE = S_FULL + 7;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + 260);
-  // per softmax warpgroup (wg = 0, 1):
-  const int wg = (WG == 2 && warp >= 6) ? 1 : 0;
-  float* m_ref = reinterpret_cast<float*>(smem + 512) + wg * 64;    // [64] references of the columns (log2 units)
-  uint32_t* enc = reinterpret_cast<uint32_t*>(smem + 1024) + wg * 64;   // [64] scratch of a raise: column maxima, order-preserving codes
-  float* l_tot = reinterpret_cast<float*>(smem + 1536) + wg * 64;   // [64] sums of this split (warpgroup 0: of both once merged)
-  float* delta_s = reinterpret_cast<float*>(smem + 2048) + wg * 64; // [64] by how much a raise lifts each reference
-  float* l_w = reinterpret_cast<float*>(smem + 2560) + wg * 256;    // [4][64] per-warp sums
-  const int bar_id = 1 + wg;               // (a compile-time constant with one warpgroup)
-  unsigned char* q_s = smem + KT_CTRL;                              // [H][NP rows][128 B]
-  unsigned char* p_s = q_s + H * NP * 128;                          // [PB][128 key rows][128 B]
+  // per softmax warpgroup: its index, and which tiles / columns it takes
+  const int grp = (NG > 1 && warp >= 2) ? (warp - 2) >> 2 : 0;
+  const int wg = WG == 2 ? grp : 0;        // tile parity it works on
+  const int cg = CG > 1 ? grp : 0;         // column group it owns
+  unsigned char* gblk = smem + KT_CTRL0 + grp * KT_GRP;
+  float* m_ref = reinterpret_cast<float*>(gblk);                    // [32] references of the group's columns (log2 units)
+  uint32_t* enc = reinterpret_cast<uint32_t*>(gblk + 256);          // [32] scratch of a raise: column maxima, order-preserving codes
+  float* l_tot = reinterpret_cast<float*>(gblk + 512);              // [32] sums of this split
+  float* delta_s = reinterpret_cast<float*>(gblk + 768);            // [32] by how much a raise lifts each reference
+  float* l_w = reinterpret_cast<float*>(gblk + 1024);               // [4][32] per-warp sums
+  float* sal_s = reinterpret_cast<float*>(gblk + 1536);             // [2][128] this group's share of the keys' logit sums (CG > 1)
+  const int bar_id = 1 + grp;              // (a compile-time constant with one warpgroup)
+  unsigned char* q_s = smem + KT_CTRL;                              // [H][NPT rows][128 B]
+  unsigned char* p_s = q_s + H * NPT * 128;                         // [PB][P^T buffer]
   unsigned char* ring = p_s + kp.PB * PBUF;                         // [NS][K tile | V tile]
-  // cluster merge: what the S splits push into this CTA (it owns DL head dimensions of every column)
-  float* recv = reinterpret_cast<float*>(ring + (size_t)NS * SLOT); // [S][NP/4][DL] float4: un-normalised O^T, four columns of one owned head dimension
-  float2* ml_recv = reinterpret_cast<float2*>(recv + (size_t)S * kp.DL * NP);   // [S][NP] (reference, sum) of every column
-  float* w_s = reinterpret_cast<float*>(ml_recv + (size_t)S * NP);  // [S][NP] merge weights, normalisation folded in
+  // Cluster merge: what the S splits push into this CTA (it owns DL head dimensions of every column). With one column
+  // group the area is its own; with several it would not fit beside the ring, so it lies over the ring and is written
+  // only after a cluster barrier behind every CTA's last PV.
+  float* recv = reinterpret_cast<float*>(CG == 1 ? ring + (size_t)NS * SLOT : ring);   // [S][NPT/4][DL] float4: un-normalised O^T, four columns of one owned head dimension
+  float2* ml_recv = reinterpret_cast<float2*>(recv + (size_t)S * kp.DL * NPT);  // [S][NPT] (reference, sum) of every column
+  float* w_s = reinterpret_cast<float*>(ml_recv + (size_t)S * NPT); // [S][NPT] merge weights, normalisation folded in
 
   // ---- this CTA's share of the key axis, in groups of 32 rows ----
   int n1 = 0, g1 = 0, gb = 0, ge = 0, T = 0;
@@ -309,7 +325,7 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(BAR(S_FULL + i), 1);
-      mbar_init(BAR(P_FULL + i), 4);
+      mbar_init(BAR(P_FULL + i), 4 * CG);
       mbar_init(BAR(PV_DONE + i), 1);
     }
     mbar_init(BAR(DRAIN), 1);
@@ -319,7 +335,7 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
     if (S > 1) {
       // what the S splits will push into this CTA: the O^T rows of the head dimensions it owns, and every column's pair
       const int rows = min(((split + 1) * D + S - 1) / S, D) - (split * D + S - 1) / S;
-      mbar_expect_tx(BAR(MERGE), (uint32_t)(S * (rows * NP * 4 + N * 8)));
+      mbar_expect_tx(BAR(MERGE), (uint32_t)(S * (rows * NPT * 4 + N * 8)));
     }
     // Ahead of everything else, and of the kernels in front of this one: Q on its way into L2 and, at the reuse step,
     // the first tiles of the compacted cache straight into the ring - they need nothing but the barriers above. Tiles that would turn the ring, or hold rows of source 2, wait for the dependency.
@@ -333,10 +349,10 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
     }
   }
   // query rows past N (N not a multiple of 32) take part in the MMAs: they must be finite
-  if (N < NP)
-    for (int i = tid; i < H * (NP - N) * 8; i += NTHREADS) {
-      const int h = i / ((NP - N) * 8), r = i % ((NP - N) * 8);
-      reinterpret_cast<uint4*>(q_s + h * NP * 128 + N * 128)[r] = make_uint4(0u, 0u, 0u, 0u);
+  if (N < NPT)
+    for (int i = tid; i < H * (NPT - N) * 8; i += NTHREADS) {
+      const int h = i / ((NPT - N) * 8), r = i % ((NPT - N) * 8);
+      reinterpret_cast<uint4*>(q_s + h * NPT * 128 + N * 128)[r] = make_uint4(0u, 0u, 0u, 0u);
     }
   if (warp == 1) {                       // the MMA warp owns the tensor memory
     tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
@@ -361,16 +377,14 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
   if (!kp.early_trigger) grid_launch_dependents();
   if (!kp.early_src1) read_counts();
 
-  float l_acc[NP];                       // softmax warps: this key row's share of every column's sum
-#pragma unroll
-  for (int c = 0; c < NP; ++c) l_acc[c] = 0.f;
+  float l_lane = 0.f;                    // softmax warps: the sum over this warp's 32 key rows of column `lane` of its group
   bool dead = false;                     // softmax warps: a wait gave up; the warp keeps meeting the others at every barrier
 
   if (warp == 0) {
     // ======================================= TMA producer =======================================
     if (lane == 0) {
       mbar_expect_tx(BAR(Q_FULL), (uint32_t)(H * N * 128));
-      for (int h = 0; h < H; ++h) tma_load_4d(smem_u32(q_s + h * NP * 128), &tm.q, BAR(Q_FULL), h * 64, 0, g * p.G, bi);
+      for (int h = 0; h < H; ++h) tma_load_4d(smem_u32(q_s + h * NPT * 128), &tm.q, BAR(Q_FULL), h * 64, 0, g * p.G, bi);
       while (t_next < T && issue_tile(t_next)) ++t_next;
       if (*abort_flag) {
         // let the copies that were issued land before the CTA retires
@@ -382,8 +396,8 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
   } else if (warp == 1) {
     // ======================================= MMA issuer =======================================
     if (lane == 0) {
-      const uint32_t idesc_s = kt_idesc(NP, false, false);
-      const uint32_t idesc_pv = kt_idesc(NP, true, true);
+      const uint32_t idesc_s = kt_idesc(NPT, false, false);
+      const uint32_t idesc_pv = kt_idesc(NPT, true, true);
       const uint32_t qsm = smem_u32(q_s);
       bool ok = wait_bar(BAR(Q_FULL), 0, abort_flag, p.status, 3, wlim);
       const uint32_t ring_a = smem_u32(ring), p_a = smem_u32(p_s);
@@ -398,10 +412,10 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
         const uint32_t psm = p_a + ((two_p && pb) ? (uint32_t)PBUF : 0u);
         // O^T += V^T P^T, 16 keys per instruction. A: the V tile read MN-major (the head dimension runs along M; its two
         // 64-element halves lie HALF bytes apart; with D = 64 both halves alias the same data and rows 64..127 of O^T
-        // are duplicates nobody reads). B: P^T, MN-major: rows of NP bf16, 8 keys per swizzle atom.
+        // are duplicates nobody reads). B: P^T, MN-major, 8 keys per swizzle atom; its 64-column halves lie 16 KB apart.
         for (int ks = 0; ks < 2 * ng; ++ks)
-          mma_ss(tmem_base + O_COL + (uint32_t)(j % WG) * NP, smem_desc(vsm + ks * 2048, H == 2 ? (uint32_t)HALF : 0u, 1024u),
-                 NP == 64 ? smem_desc(psm + ks * 2048, (uint32_t)PBUF, 1024u) : smem_desc_sw64(psm + ks * 1024, (uint32_t)PBUF, 512u),
+          mma_ss(tmem_base + O_COL + (uint32_t)(j % WG) * NPT, smem_desc(vsm + ks * 2048, H == 2 ? (uint32_t)HALF : 0u, 1024u),
+                 CG > 1 ? smem_desc(psm + ks * 2048, 128u * 128u, 1024u) : smem_desc_sw64(psm + ks * 1024, (uint32_t)PBUF, 512u),
                  idesc_pv, (j >= WG || ks > 0) ? 1u : 0u);
         tc_commit(BAR(PV_DONE + pb));    // two alternating barriers: a waiter is never a whole phase ahead of either
         tc_commit(BAR(EMPTY_V + s));
@@ -414,12 +428,12 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
         if (!wait_bar(BAR(FULL_K + s), par, abort_flag, p.status, 7, wlim)) { ok = false; break; }
         tc_fence_after();
         const uint32_t ksm = ring_a + (uint32_t)s * SLOT;
-        const uint32_t d_t = tmem_base + (uint32_t)sb * NP;
+        const uint32_t d_t = tmem_base + (uint32_t)sb * NPT;
         // S^T = K_tile Q^T: the S^T buffer of tile t - 2 is free, its softmax arrived before PV(t - 2) was issued
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const uint32_t hk = (ks >> 2) * HALF + (ks & 3) * 32;
-          const uint32_t hq = (ks >> 2) * (NP * 128) + (ks & 3) * 32;
+          const uint32_t hq = (ks >> 2) * (NPT * 128) + (ks & 3) * 32;
           mma_ss(d_t, smem_desc(ksm + hk, 16u, 1024u), smem_desc(qsm + hq, 16u, 1024u), idesc_s, ks > 0 ? 1u : 0u);
         }
         tc_commit(BAR(S_FULL + sb));
@@ -444,7 +458,8 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
     const float sl2 = p.scale_log2;
     const bool scores = p.want_scores != 0;
     const int st = (tid - 64) & 127;                   // index inside the warpgroup
-    const uint32_t o_col = O_COL + (uint32_t)wg * NP;  // this warpgroup's accumulator
+    const uint32_t o_col = O_COL + (uint32_t)wg * NPT + (uint32_t)cg * 32;   // this warpgroup's accumulator (columns)
+    const int n_mine = min(max(N - 32 * cg, 0), 32);   // real query columns among this group's 32
     const bool two_p = kp.PB == 2;
     for (int t = wg; t < T; t += WG) {
       const int sb = t & 1;
@@ -458,20 +473,31 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
       const bool work = active && !dead;
       float sv[NP];                                    // this key's logits against the N queries, then their scaled distance to the references
       if (work) {
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) tmem_ld32(lane_addr + (uint32_t)sb * NP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
+        tmem_ld32(lane_addr + (uint32_t)sb * NPT + (uint32_t)cg * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
         tc_wait_ld();
       } else {
 #pragma unroll
         for (int c = 0; c < NP; ++c) sv[c] = 0.f;
       }
       // ---- saliency of this key (refresh step): scale * mean of its N logits ----
-      if (scores && work && valid && x.src1) {
+      if (scores) {
         float a4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int c = 0; c < NP; ++c)
-          if (c < N) a4[c & 3] += sv[c];
-        p.raw_scores[(int64_t)(bi * p.Hkv + g) * p.n1_max + x.row0 + lane] = ((a4[0] + a4[1]) + (a4[2] + a4[3])) * (p.scale / (float)N);
+          if (c < n_mine) a4[c & 3] += sv[c];
+        float a = (a4[0] + a4[1]) + (a4[2] + a4[3]);
+        if constexpr (CG > 1) {
+          // the key's logits are spread over the column groups: their sums meet in shared memory (two buffers in turn,
+          // so the next tile never overwrites what the first group is still adding up)
+          sal_s[(t & 1) * 128 + row] = a;
+          softmax_barrier_all<NG>();
+          if (cg == 0) {
+#pragma unroll
+            for (int c2 = 1; c2 < CG; ++c2) a += reinterpret_cast<const float*>(gblk + c2 * KT_GRP + 1536)[(t & 1) * 128 + row];
+          }
+        }
+        if (cg == 0 && work && valid && x.src1)
+          p.raw_scores[(int64_t)(bi * p.Hkv + g) * p.n1_max + x.row0 + lane] = a * (p.scale / (float)N);
       }
       // ---- the references. The first key of the CTA's first tile lends its logits: it is part of the softmax, so sums
       //      never vanish, and exp2 of anything up to 2^64 above it is still an ordinary bf16 / fp32 number. Every tile is
@@ -484,14 +510,15 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
         }
         softmax_barrier(bar_id);
       }
-      bool over = false;
+      float far0 = -INFINITY, far1 = -INFINITY;        // the largest distance above a reference
 #pragma unroll
       for (int c = 0; c < NP; c += 4) {
         const float4 m4 = *reinterpret_cast<const float4*>(m_ref + c);
         sv[c] = fmaf(sv[c], sl2, -m4.x); sv[c + 1] = fmaf(sv[c + 1], sl2, -m4.y);
         sv[c + 2] = fmaf(sv[c + 2], sl2, -m4.z); sv[c + 3] = fmaf(sv[c + 3], sl2, -m4.w);
-        over |= (sv[c] > 64.f) | (sv[c + 1] > 64.f) | (sv[c + 2] > 64.f) | (sv[c + 3] > 64.f);
+        far0 = fmaxf(far0, fmaxf(sv[c], sv[c + 1])); far1 = fmaxf(far1, fmaxf(sv[c + 2], sv[c + 3]));
       }
+      const bool over = fmaxf(far0, far1) > 64.f;
       if (softmax_barrier_or(bar_id, over && work && valid)) {
         // ---- raise the references by the tile's column maxima (where positive) and rescale what has been accumulated.
         //      Every PV issued so far must have landed before O^T is rewritten; the PV of this tile waits for our arrive. ----
@@ -500,14 +527,13 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
         if (st < NP) enc[st] = f2ord(0.f);
         softmax_barrier(bar_id);
         if (work) {
-          float mine[NCH];
+          float mine = 0.f;
 #pragma unroll
           for (int c = 0; c < NP; ++c) {
             const float r = warp_max_f32(valid ? sv[c] : -INFINITY);
-            if ((c & 31) == lane) mine[c >> 5] = r;
+            if (c == lane) mine = r;
           }
-#pragma unroll
-          for (int c = 0; c < NCH; ++c) atomicMax(enc + c * 32 + lane, f2ord(mine[c]));
+          atomicMax(enc + lane, f2ord(mine));
         }
         softmax_barrier(bar_id);
         if (st < NP) {
@@ -518,22 +544,16 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
         softmax_barrier(bar_id);
 #pragma unroll
         for (int c = 0; c < NP; ++c) sv[c] -= delta_s[c];
+        l_lane *= fast_exp2(-delta_s[lane]);
         if (t >= WG && !dead) {
           // this thread's TMEM lane is a head dimension of O^T here, not a key: all four warps rescale their lanes
+          uint32_t o32[32];
+          tmem_ld32(lane_addr + o_col, o32);
+          tc_wait_ld();
 #pragma unroll
-          for (int c = 0; c < NCH; ++c) {
-            uint32_t o32[32];
-            tmem_ld32(lane_addr + o_col + c * 32, o32);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float a = fast_exp2(-delta_s[c * 32 + i]);
-              o32[i] = __float_as_uint(__uint_as_float(o32[i]) * a);
-              l_acc[c * 32 + i] *= a;
-            }
-            tmem_st16(lane_addr + o_col + c * 32, *reinterpret_cast<uint32_t(*)[16]>(&o32[0]));
-            tmem_st16(lane_addr + o_col + c * 32 + 16, *reinterpret_cast<uint32_t(*)[16]>(&o32[16]));
-          }
+          for (int i = 0; i < 32; ++i) o32[i] = __float_as_uint(__uint_as_float(o32[i]) * fast_exp2(-delta_s[i]));
+          tmem_st16(lane_addr + o_col, *reinterpret_cast<uint32_t(*)[16]>(&o32[0]));
+          tmem_st16(lane_addr + o_col + 16, *reinterpret_cast<uint32_t(*)[16]>(&o32[16]));
           tc_wait_st();
         }
         softmax_barrier(bar_id);         // delta_s and m_ref are stable again before the next tile reads them
@@ -543,23 +563,30 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
       const int tp = two_p ? t - 2 : t - 1;            // the tile whose PV read this buffer last
       if (!dead && tp >= 0 && !wait_bar_warp(BAR(PV_DONE + (tp & 1)), (tp >> 1) & 1, abort_flag, p.status, 6, wlim)) dead = true;
       if (active && !dead) {
-        unsigned char* prow = p_s + ((two_p && sb) ? PBUF : 0) + row * PROW;
-        const int swz = NP == 64 ? (row & 7) : ((row >> 1) & 3);     // the 16-byte chunk index is XORed with address bits 7.. of the row
+        // CG = 1: rows of 64 bytes, 64-byte swizzle; CG > 1: 128-byte rows per 64-column half, this group's 32 columns
+        // are chunks 4 * (cg & 1) .. of half cg / 2; the 16-byte chunk index is XORed with address bits 7.. of the row
+        unsigned char* prow = p_s + ((two_p && sb) ? PBUF : 0) + (CG == 1 ? row * 64 : (cg >> 1) * (128 * 128) + row * 128);
+        const int swz = CG == 1 ? ((row >> 1) & 3) : (row & 7);
+        const int cbase = CG == 1 ? 0 : 4 * (cg & 1);
+        if (x.nv < 32) {                               // ragged group (warp-uniform): rows past the count contribute nothing
+#pragma unroll
+          for (int c = 0; c < NP; ++c) sv[c] = valid ? sv[c] : -INFINITY;
+        }
 #pragma unroll
         for (int c8 = 0; c8 < NP / 8; ++c8) {
           uint32_t pk[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int c = c8 * 8 + 2 * i;
-            const float e0 = fast_exp2(valid ? sv[c] : -INFINITY);
-            const float e1 = fast_exp2(valid ? sv[c + 1] : -INFINITY);
-            l_acc[c] += e0; l_acc[c + 1] += e1;
+            const float e0 = fast_exp2(sv[c]);
+            const float e1 = fast_exp2(sv[c + 1]);
+            sv[c] = e0; sv[c + 1] = e1;
             pk[i] = pack_bf16(e0, e1);
           }
-          *reinterpret_cast<uint4*>(prow + ((c8 ^ swz) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          *reinterpret_cast<uint4*>(prow + (((cbase + c8) ^ swz) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
         // ---- V rows of this group past its count may hold anything: zero them so that 0 * V stays 0 ----
-        if (x.nv < 32) {
+        if (x.nv < 32 && cg == 0) {
           const int s = t % NS;
           if (!wait_bar_warp(BAR(FULL_V + s), (t / NS) & 1, abort_flag, p.status, 10, wlim)) dead = true;
           unsigned char* vs = ring + (size_t)s * SLOT + KV_BYTES;
@@ -574,50 +601,49 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
       tc_fence_before();
       __syncwarp();
       if (lane == 0 && !dead) mbar_arrive(BAR(P_FULL + sb));
+      // ---- column sums, off the critical path (the MMA warp already has P^T): shuffle transpose over the warp's 32 key
+      //      rows, lane i ends up with the sum of column i ----
+      if (active && !dead) {
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+          const bool up_half = (lane & off) != 0;
+#pragma unroll
+          for (int k = 0; k < off; ++k) {
+            const float send = up_half ? sv[k] : sv[k + off];
+            const float keep = up_half ? sv[k + off] : sv[k];
+            sv[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+          }
+        }
+        l_lane += sv[0];
+      }
     }
   }
 
   // ======================================= epilogue =======================================
   const bool do_attn = p.out != nullptr;
   const int DL = kp.DL;                  // head dimensions a CTA owns in the merge: ceil(D / S)
-  uint32_t ov[NP];                       // softmax threads: this thread's head dimension of O^T, all columns
-  float l_mine = 0.f, m_mine = -INFINITY;// softmax thread st < NP: sum and reference of column st
+  uint32_t ov[NP];                       // softmax threads: this thread's head dimension of O^T, its group's 32 columns
+  float l_mine = 0.f, m_mine = -INFINITY;// softmax thread st < 32: sum and reference of column 32 * cg + st
+  const bool carry = warp >= 2 && (WG == 1 || grp == 0);      // the threads that carry the result out
   if (warp >= 2) {
     const int q4 = warp & 3;
     const int row = q4 * 32 + lane;      // from here on: a head dimension of O^T
     const int st = (tid - 64) & 127;     // index inside the warpgroup
-    // ---- column sums over the 128 key rows: shuffle transpose inside a warp (lane i ends up with column i), then the
-    //      four warps' rows in a fixed order ----
-#pragma unroll
-    for (int c = 0; c < NCH; ++c) {
-      float v[32];
-#pragma unroll
-      for (int i = 0; i < 32; ++i) v[i] = l_acc[c * 32 + i];
-#pragma unroll
-      for (int off = 16; off >= 1; off >>= 1) {
-        const bool up_half = (lane & off) != 0;
-#pragma unroll
-        for (int k = 0; k < off; ++k) {
-          const float send = up_half ? v[k] : v[k + off];
-          const float keep = up_half ? v[k + off] : v[k];
-          v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-        }
-      }
-      l_w[((warp - 2) & 3) * 64 + c * 32 + lane] = v[0];
-    }
+    // ---- column sums over the 128 key rows: the four warps' sums in a fixed order ----
+    l_w[((warp - 2) & 3) * 32 + lane] = l_lane;
     if (S > 1 && p.want_scores) __threadfence();       // this thread's raw saliency, ahead of the pushes that tell the peers
     softmax_barrier(bar_id);
     if (st < NP) {
-      l_mine = (l_w[st] + l_w[64 + st]) + (l_w[128 + st] + l_w[192 + st]);
+      l_mine = (l_w[st] + l_w[32 + st]) + (l_w[64 + st] + l_w[96 + st]);
       m_mine = T > wg ? m_ref[st] : -INFINITY;
     }
-    // ---- two warpgroups: the second one's partial (reference, sum, accumulator rows) is folded into the first one's ----
+    // ---- two tile-alternating warpgroups: the second one's partial (reference, sum, accumulator rows) is folded into the first one's ----
     const bool fold = WG == 2 && T >= 2;
-    const float* m_a = m_ref - wg * 64; const float* m_b = m_a + 64;
-    const float* l_a = l_tot - wg * 64; const float* l_b = l_a + 64;
+    const float* m_a = reinterpret_cast<const float*>(smem + KT_CTRL0); const float* m_b = m_a + KT_GRP / 4;
+    const float* l_a = m_a + 128; const float* l_b = l_a + KT_GRP / 4;
     if (fold) {
       if (st < NP) l_tot[st] = l_mine;
-      softmax_barrier_both();            // both warpgroups' references and sums are posted
+      softmax_barrier_all<NG>();         // both warpgroups' references and sums are posted
       if (wg == 0 && st < NP) {
         const float mb = m_b[st], lb = l_b[st];
         const bool ha = l_mine > 0.f, hb = lb > 0.f;
@@ -626,23 +652,21 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
         m_mine = ms;
       }
     }
-    if (wg == 0 && S > 1) {
+    if (CG == 1 && carry && S > 1) {
       // every split's (reference, sum) of every column goes to every CTA of the cluster, ahead of the accumulator rows
       cluster_wait_acquire();            // every CTA of the cluster runs: its shared memory and barriers may be written
       if (st < N) {
-        const uint32_t ml_a = smem_u32(ml_recv + split * NP + st);
+        const uint32_t ml_a = smem_u32(ml_recv + split * NPT + st);
         for (int r = 0; r < S; ++r) st_async_f2(map_to_cta(ml_a, (uint32_t)r), map_to_cta(BAR(MERGE), (uint32_t)r), m_mine, l_mine);
       }
     }
-    // ---- the finished accumulator row of this thread (of its warpgroup's accumulator) ----
+    // ---- the finished accumulator row of this thread (its group's columns of its warpgroup's accumulator) ----
     const int t_last = T > wg ? wg + ((T - 1 - wg) / WG) * WG : 0;      // the warpgroup's last tile
-    const bool have_o = do_attn && !dead && T > wg &&
-                        wait_bar_warp(BAR(PV_DONE + (t_last & 1)), (t_last >> 1) & 1, abort_flag, p.status, 6, wlim);
+    const bool pv_ok = !dead && T > wg && wait_bar_warp(BAR(PV_DONE + (t_last & 1)), (t_last >> 1) & 1, abort_flag, p.status, 6, wlim);
+    const bool have_o = do_attn && pv_ok;
     tc_fence_after();
     if (have_o) {
-#pragma unroll
-      for (int c = 0; c < NCH; ++c)
-        tmem_ld32(tmem_base + ((uint32_t)(q4 * 32) << 16) + O_COL + (uint32_t)wg * NP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&ov[c * 32]));
+      tmem_ld32(tmem_base + ((uint32_t)(q4 * 32) << 16) + O_COL + (uint32_t)wg * NPT + (uint32_t)cg * 32, ov);
       tc_wait_ld();
     } else {
 #pragma unroll
@@ -652,7 +676,7 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
       // The rows cross in the first ring slot, once both warpgroups have seen their last PV complete. Every thread scales
       // its own row to the common references; the factors are recomputed from the posted references and sums.
       float4* xch = reinterpret_cast<float4*>(ring);                // [NP / 4][128 rows]
-      softmax_barrier_both();
+      softmax_barrier_all<NG>();
 #pragma unroll
       for (int c4 = 0; c4 < NP / 4; ++c4) {
         const float4 ma = *reinterpret_cast<const float4*>(m_a + 4 * c4), mb = *reinterpret_cast<const float4*>(m_b + 4 * c4);
@@ -670,7 +694,7 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
           xch[c4 * 128 + row] = make_float4(__uint_as_float(ov[4 * c4]), __uint_as_float(ov[4 * c4 + 1]), __uint_as_float(ov[4 * c4 + 2]),
                                             __uint_as_float(ov[4 * c4 + 3]));
       }
-      softmax_barrier_both();
+      softmax_barrier_all<NG>();
       if (wg == 0) {
 #pragma unroll
         for (int c4 = 0; c4 < NP / 4; ++c4) {
@@ -681,25 +705,33 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
       }
     }
   }
-  if (warp >= 2 && warp < 6) {           // the first warpgroup carries the result out
+  if (CG > 1 && S > 1) {
+    // Several column groups: the merge area lies over the ring. Every thread of every CTA of the cluster passes one more
+    // cluster barrier; the softmax threads arrive at it only behind their last PV, so behind it no CTA's ring is in use.
+    cluster_wait_acquire();              // (the barrier taken at the start: every CTA runs, its mbarriers are set up)
+    cluster_arrive_release();
+    cluster_wait_acquire();
+  }
+  if (carry) {
     const int q4 = warp & 3;
     const int row = q4 * 32 + lane;
-    const int st = tid - 64;
+    const int st = (tid - 64) & 127;
+    const int c_first = 32 * cg;         // first query column of this group
     if (S == 1) {
       if (st < NP) l_tot[st] = l_mine > 0.f ? 1.f / l_mine : 0.f;       // one split: the normaliser itself
-      softmax_barrier(1);
-    }
-    if (S == 1) {
+      softmax_barrier(bar_id);
       if (do_attn && !*abort_flag) {
         // one split: normalise and store; a warp writes 32 consecutive bf16 of one output row per column
         if (row < D) {
           // column c is row c % b of head c / b of the group: the pointer walks the rows and hops to the next head
-          __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] + (int64_t)(g * p.G) * p.o_stride[1] + row;
+          const int hg0 = c_first / p.b;
+          int i = c_first - hg0 * p.b;
+          __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + (int64_t)bi * p.o_stride[0] + (int64_t)(g * p.G + hg0) * p.o_stride[1] +
+                             (int64_t)i * p.o_stride[2] + row;
           const int64_t hop = p.o_stride[1] - (int64_t)(p.b - 1) * p.o_stride[2];
-          int i = 0;
 #pragma unroll
           for (int c = 0; c < NP; c += 4) {
-            if (c >= N) break;
+            if (c_first + c >= N) break;
             const float4 inv = *reinterpret_cast<const float4*>(l_tot + c);
             const float iv[4] = {inv.x, inv.y, inv.z, inv.w};
 #pragma unroll
@@ -709,72 +741,82 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
             }
           }
         }
-        if (p.lse && st < N) {
-          const int hg = st / p.b, i = st - hg * p.b;
+        if (p.lse && st < NP && c_first + st < N) {
+          const int c = c_first + st;
+          const int hg = c / p.b, i = c - hg * p.b;
           p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (m_mine + log2f(l_mine)) * kLn2;
         }
       }
-    } else if (row < D) {
-      // ---- this head dimension's row of O^T goes to the CTA that owns the dimension, 16 bytes at a time (always, also
-      //      when this CTA is aborting: the owner counts the bytes) ----
-      const int owner = row * S / D;
-      const int dl = row - (owner * D + S - 1) / S;
-      const uint32_t dst = map_to_cta(smem_u32(recv + ((size_t)split * (NP / 4) * DL + dl) * 4), (uint32_t)owner);
-      const uint32_t mb = map_to_cta(BAR(MERGE), (uint32_t)owner);
+    } else {
+      if (CG > 1 && st < NP && c_first + st < N) {     // (one column group: pushed ahead of the accumulator rows, above)
+        const uint32_t ml_a = smem_u32(ml_recv + split * NPT + c_first + st);
+        for (int r = 0; r < S; ++r) st_async_f2(map_to_cta(ml_a, (uint32_t)r), map_to_cta(BAR(MERGE), (uint32_t)r), m_mine, l_mine);
+      }
+      if (row < D) {
+        // ---- this head dimension's row of O^T goes to the CTA that owns the dimension, 16 bytes at a time (always, also
+        //      when this CTA is aborting: the owner counts the bytes) ----
+        const int owner = row * S / D;
+        const int dl = row - (owner * D + S - 1) / S;
+        const uint32_t dst = map_to_cta(smem_u32(recv + ((size_t)(split * (NPT / 4) + 8 * cg) * DL + dl) * 4), (uint32_t)owner);
+        const uint32_t mb = map_to_cta(BAR(MERGE), (uint32_t)owner);
 #pragma unroll
-      for (int c4 = 0; c4 < NP / 4; ++c4)          // consecutive lanes (head dimensions) write consecutive 16-byte units
-        st_async_f4(dst + (uint32_t)(c4 * DL * 16), mb, __uint_as_float(ov[4 * c4]), __uint_as_float(ov[4 * c4 + 1]),
-                    __uint_as_float(ov[4 * c4 + 2]), __uint_as_float(ov[4 * c4 + 3]));
+        for (int c4 = 0; c4 < NP / 4; ++c4)          // consecutive lanes (head dimensions) write consecutive 16-byte units
+          st_async_f4(dst + (uint32_t)(c4 * DL * 16), mb, __uint_as_float(ov[4 * c4]), __uint_as_float(ov[4 * c4 + 1]),
+                      __uint_as_float(ov[4 * c4 + 2]), __uint_as_float(ov[4 * c4 + 3]));
+      }
     }
   }
 
   if (S > 1) {
     // ---- cluster merge: once everything owed to this CTA has landed, it merges and stores the head dimensions it owns ----
-    if (warp < 2 || warp >= 6) cluster_wait_acquire(); // (the first softmax warpgroup passed the cluster barrier before its pushes)
+    if (CG == 1 && !carry) cluster_wait_acquire();     // (the carrying threads passed the cluster barrier before their pushes)
     wait_merge(BAR(MERGE), abort_flag, p.status, wlim);
-    if (warp >= 2 && warp < 6 && do_attn && !*abort_flag) {
-      const int st = tid - 64;
-      // weights of the S splits for column st, the normalisation folded in
-      if (st < N) {
-        float2 x[8];
+    const bool live = do_attn && !*abort_flag;
+    if (carry) {
+      const int st = (tid - 64) & 127;
+      const int c_mine = 32 * cg + st;   // the column whose weights this thread computes (st < 32)
+      // weights of the S splits for that column, the normalisation folded in
+      if (live && st < NP && c_mine < N) {
+        float2 x[MS];
 #pragma unroll
-        for (int s2 = 0; s2 < 8; ++s2) x[s2] = ml_recv[min(s2, S - 1) * NP + st];
+        for (int s2 = 0; s2 < MS; ++s2) x[s2] = ml_recv[min(s2, S - 1) * NPT + c_mine];
         float mstar = -INFINITY;
 #pragma unroll
-        for (int s2 = 0; s2 < 8; ++s2)
+        for (int s2 = 0; s2 < MS; ++s2)
           if (s2 < S && x[s2].y > 0.f) mstar = fmaxf(mstar, x[s2].x);
-        float w[8], l = 0.f;
+        float w[MS], l = 0.f;
 #pragma unroll
-        for (int s2 = 0; s2 < 8; ++s2) {
+        for (int s2 = 0; s2 < MS; ++s2) {
           w[s2] = (s2 < S && x[s2].y > 0.f) ? fast_exp2(x[s2].x - mstar) : 0.f;
           l = fmaf(x[s2].y, w[s2], l);
         }
         const float inv = l > 0.f ? 1.f / l : 0.f;
 #pragma unroll
-        for (int s2 = 0; s2 < 8; ++s2)
-          if (s2 < S) w_s[s2 * NP + st] = w[s2] * inv;
+        for (int s2 = 0; s2 < MS; ++s2)
+          if (s2 < S) w_s[s2 * NPT + c_mine] = w[s2] * inv;
         if (split == 0 && p.lse) {
-          const int hg = st / p.b, i = st - hg * p.b;
+          const int hg = c_mine / p.b, i = c_mine - hg * p.b;
           p.lse[((int64_t)bi * p.Hq + g * p.G + hg) * p.b + i] = (mstar + log2f(l)) * kLn2;
         }
       }
-      softmax_barrier(1);
+      if constexpr (CG > 1) softmax_barrier_all<NG>(); else softmax_barrier(1);
       // thread -> (owned head dimension, chunk of columns); all loads of a group of four columns are in flight together
       const int d_lo = (split * D + S - 1) / S, d_hi = min(((split + 1) * D + S - 1) / S, D);
-      const int dl = st % DL, qc = st / DL;
+      const int sa = 128 * cg + st;      // index among all carrying threads
+      const int dl = sa % DL, qc = sa / DL;
       const int cpt = kp.cpt;            // columns per thread, a multiple of 4
-      if (d_lo + dl < d_hi) {
+      if (live && d_lo + dl < d_hi) {
         for (int c0 = qc * cpt; c0 < min((qc + 1) * cpt, N); c0 += 4) {
-          float4 r4[8], w4[8];
-#pragma unroll
-          for (int s2 = 0; s2 < 8; ++s2) {
-            const int sc = min(s2, S - 1);
-            r4[s2] = *reinterpret_cast<const float4*>(recv + ((size_t)(sc * (NP / 4) + (c0 >> 2)) * DL + dl) * 4);
-            w4[s2] = *reinterpret_cast<const float4*>(w_s + sc * NP + c0);
-          }
           float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          float4 r4[MS], w4[MS];                         // all splits' loads in flight together
 #pragma unroll
-          for (int s2 = 0; s2 < 8; ++s2)
+          for (int s2 = 0; s2 < MS; ++s2) {
+            const int sc = min(s2, S - 1);
+            r4[s2] = *reinterpret_cast<const float4*>(recv + ((size_t)(sc * (NPT / 4) + (c0 >> 2)) * DL + dl) * 4);
+            w4[s2] = *reinterpret_cast<const float4*>(w_s + sc * NPT + c0);
+          }
+#pragma unroll
+          for (int s2 = 0; s2 < MS; ++s2)
             if (s2 < S) {
               acc.x = fmaf(r4[s2].x, w4[s2].x, acc.x); acc.y = fmaf(r4[s2].y, w4[s2].y, acc.y);
               acc.z = fmaf(r4[s2].z, w4[s2].z, acc.z); acc.w = fmaf(r4[s2].w, w4[s2].w, acc.w);
@@ -813,22 +855,26 @@ __global__ void __launch_bounds__(64 + 128 * WG, (NCH == 1 && WG == 1) ? 2 : 1) 
 
 // ---------------------------------------------------------------------------------------------------------
 // Host side
-size_t kt_smem_bytes(int D, int NP, int NS, int PB, int S, int GPT) {
-  const size_t H = D / 64;
+size_t kt_smem_bytes(int D, int CG, int WG, int NS, int PB, int S) {
+  const size_t H = D / 64, NPT = 32 * CG, NG = (size_t)CG * WG;
   const size_t DL = (D + S - 1) / S;
-  return 1024 /*alignment slack*/ + KT_CTRL + H * NP * 128 + (size_t)PB * 128 * NP * 2 + (size_t)NS * 2 * H * GPT * 32 * 128 +
-         (S > 1 ? (size_t)S * DL * NP * 4 /*recv*/ + (size_t)S * NP * 12 /*ml_recv, w_s*/ : 0);
+  const size_t pbuf = CG == 1 ? 128 * 64 : (size_t)((CG + 1) / 2) * 128 * 128;
+  const size_t ring = (size_t)NS * 2 * H * 128 * 128;
+  const size_t merge = S > 1 ? (size_t)S * DL * NPT * 4 /*recv*/ + (size_t)S * NPT * 12 /*ml_recv, w_s*/ : 0;
+  // one column group: the merge area follows the ring; several: it lies over the ring (which must be large enough)
+  const size_t tail = CG == 1 ? ring + merge : (ring > merge ? ring : merge);
+  return 1024 /*alignment slack*/ + KT_CTRL0 + NG * KT_GRP + H * NPT * 128 + (size_t)PB * pbuf + tail;
 }
 
-template <int D, int NCH, int WG>
+template <int D, int WG, int CG>
 cudaError_t launch_kt_d(const KtMaps& tm, const KtParams& kp, const AttnPlan& pl, bool pdl, cudaStream_t st) {
-  auto kern = attn_kt_kernel<D, NCH, WG>;
+  auto kern = attn_kt_kernel<D, WG, CG>;
   static SmemConfig configured;
   cudaError_t e = configure_smem(reinterpret_cast<const void*>(kern), pl.smem_bytes, configured, true);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(kp.S, kp.a.Hkv, kp.a.B);
-  cfg.blockDim = dim3(64 + 128 * WG);
+  cfg.blockDim = dim3(64 + 128 * WG * CG);
   cfg.dynamicSmemBytes = pl.smem_bytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
@@ -847,28 +893,54 @@ cudaError_t launch_kt_d(const KtMaps& tm, const KtParams& kp, const AttnPlan& pl
   return cudaLaunchKernelEx(&cfg, kern, tm, kp);
 }
 
+template <int D>
+cudaError_t launch_kt_shape(const KtMaps& tm, const KtParams& kp, const AttnPlan& pl, int WG, int CG, bool pdl, cudaStream_t st) {
+  if (WG == 2) return launch_kt_d<D, 2, 1>(tm, kp, pl, pdl, st);
+  switch (CG) {
+    case 1: return launch_kt_d<D, 1, 1>(tm, kp, pl, pdl, st);
+    case 2: return launch_kt_d<D, 1, 2>(tm, kp, pl, pdl, st);
+    case 3: return launch_kt_d<D, 1, 3>(tm, kp, pl, pdl, st);
+    default: return launch_kt_d<D, 1, 4>(tm, kp, pl, pdl, st);
+  }
+}
+
 }  // namespace
 
-// Whether the key-row kernel covers a shape: bf16, D in {64, 128}, at most 64 query rows per KV head, block length a
+// Whether the key-row kernel covers a shape: bf16, D in {64, 128}, at most 128 query rows per KV head, block length a
 // multiple of 16.
 bool kt_supported(int dtype, int D, int M, int b) {
-  return umma_supported(dtype, D, M, b) && M <= 64;
+  return umma_supported(dtype, D, M, b) && M <= 128;
+}
+
+// Whether the planner picks it among the shapes it covers. A unit's key splits are the CTAs of one cluster, eight at
+// most. With up to 32 query rows that is enough everywhere. With more, a CTA takes a whole SM, and a few units with
+// long key ranges (8 KV heads, one sequence, 16k keys: 64 CTAs) would leave most SMs idle; the query-row kernel splits
+// those further through its workspace and measured faster there (25 against 38 us), slower with 64 units and more.
+bool kt_preferred(int M, int B, int Hkv, int n1_max, int n2) {
+  if (M <= 32) return true;
+  const long long units = (long long)B * Hkv;
+  const int sms = sm_count();
+  long long S = sms / units;
+  const long long by_tiles = ((n1_max + 31) / 32 + (n2 + 31) / 32 + 3) / 4;
+  if (S > by_tiles) S = by_tiles;
+  if (S > 8) S = 8;
+  if (S < 1) S = 1;
+  return units * S * 4 >= (long long)sms * 3;
 }
 
 AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int n2, const Tuning& tn) {
   (void)b;
   AttnPlan pl{};
   pl.kind = 3; pl.tma = true; pl.fused_tail = true;
-  pl.threads = KT_THREADS;
   pl.key_tile = 128; pl.key_tile2 = n2 < 32 ? n2 : 32;
   pl.rep = 1; pl.row_tiles = 1; pl.rows_rep = M;
-  const int NP = M <= 32 ? 32 : 64;
+  const int CG = (M + 31) / 32;          // column groups of 32 query columns: one softmax warpgroup each
   const int groups = (n1_max + 31) / 32 + (n2 + 31) / 32;
   const long long units = (long long)B * Hkv;
   const int sms = sm_count();
-  // Key splits: enough CTAs to fill the SMs (two per SM with few query columns), but at least one full 128-key tile
+  // Key splits: enough CTAs to fill the SMs (two per SM with one column group), but at least one full 128-key tile
   // per CTA, and at most eight (one cluster).
-  long long want = (NP == 32 ? 2 : 1) * (long long)sms / units;
+  long long want = (CG == 1 ? 2 : 1) * (long long)sms / units;
   const long long by_tiles = (groups + 3) / 4;
   if (want > by_tiles) want = by_tiles;
   if (tn.splits > 0) want = tn.splits;
@@ -876,42 +948,39 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   if (want < 1) want = 1;
   const int S = (int)want;
   // Footprint, ring depth, P^T buffers and softmax warpgroups:
-  // (a) few query columns and either at most two full tiles per CTA or a grid that fits the GPU only at two CTAs per
+  // (a) one column group and either at most two full tiles per CTA or a grid that fits the GPU only at two CTAs per
   //     SM: the footprint is kept below half an SM, so that two CTAs are resident and the next call's CTAs can start
   //     loading while this call's finish;
-  // (b) few query columns and longer walks: the CTA takes what one SM has, and two softmax warpgroups take the tiles in
+  // (b) one column group and longer walks: the CTA takes what one SM has, and two softmax warpgroups take the tiles in
   //     turn (one warp per scheduler cannot hide its own latencies; two tiles in flight can);
-  // (c) up to 64 query columns: one CTA per SM, one warpgroup.
+  // (c) 33 to 128 query columns: one CTA per SM, one softmax warpgroup per 32 columns, all on the same tile.
   const int groups_cta = (groups + S - 1) / S;
   const size_t half_sm = 113 * 1024;     // two CTAs of this size, each with its 1 KB system share, fit one SM
-  bool small = NP == 32 && (groups_cta <= 8 || (units * S > sms && units * S <= 2 * sms));
-  int WG = (NP == 32 && !small) ? 2 : 1;
-  if (tn.dual == 1) { small = NP == 32; WG = 1; }      // force (a) / (b) where they apply
-  if (tn.dual == 0 && NP == 32) { small = false; WG = 2; }
-  const int GPT = 4;
-  const int tiles_cta = (groups_cta + GPT - 1) / GPT;
+  bool small = CG == 1 && (groups_cta <= 8 || (units * S > sms && units * S <= 2 * sms));
+  int WG = (CG == 1 && !small) ? 2 : 1;
+  if (tn.dual == 1) { small = CG == 1; WG = 1; }       // force (a) / (b) where they apply
+  if (tn.dual == 0 && CG == 1) { small = false; WG = 2; }
+  const int tiles_cta = (groups_cta + 3) / 4;
   int NS = 1, PB = WG == 2 ? 2 : 1;
-  if (small) {
-    while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, NP, NS + 1, PB, S, GPT) <= half_sm) ++NS;
-  } else {
-    PB = 2;
-    while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, NP, NS + 1, PB, S, GPT) <= 226 * 1024) ++NS;
-  }
+  const size_t limit = small ? half_sm : 226 * 1024;
+  if (!small && kt_smem_bytes(D, CG, WG, 1, 2, S) <= limit) PB = 2;
+  while (NS < KT_MAX_STAGES && NS < tiles_cta && kt_smem_bytes(D, CG, WG, NS + 1, PB, S) <= limit) ++NS;
+  if (!small && PB == 2 && WG == 1 && NS < 2 && tiles_cta >= 2 && kt_smem_bytes(D, CG, WG, 2, 1, S) <= limit) { PB = 1; NS = 2; }   // a second ring slot is worth more than a second P^T buffer
   if (tn.stages > 0) {
     NS = tn.stages > KT_MAX_STAGES ? KT_MAX_STAGES : tn.stages;
-    while (NS > 1 && kt_smem_bytes(D, NP, NS, PB, S, GPT) > 226 * 1024) --NS;
+    while (NS > 1 && kt_smem_bytes(D, CG, WG, NS, PB, S) > 226 * 1024) --NS;
   }
   pl.splits = 1;                        // nothing is left in the workspace: the splits merge inside their cluster
   pl.parts = 1;
   pl.cluster = S;
   pl.stages = NS;
   pl.m_warps = PB;                      // (field reused: P^T buffers)
-  pl.c_warps = WG;                      // (field reused: softmax warpgroups)
-  pl.threads = 64 + 128 * WG;
+  pl.c_warps = WG;                      // (field reused: tile-alternating softmax warpgroups)
+  pl.warp_keys = CG;                    // (field reused: column groups)
+  pl.threads = 64 + 128 * WG * CG;
   pl.part_rows = 0;
   pl.n_counters = 0;
-  pl.key_tile = 32 * GPT;
-  pl.smem_bytes = kt_smem_bytes(D, NP, NS, PB, S, GPT);
+  pl.smem_bytes = kt_smem_bytes(D, CG, WG, NS, PB, S);
   return pl;
 }
 
@@ -919,14 +988,14 @@ cudaError_t launch_attn_kt(const AttnParams& p, const AttnPlan& pl, int D, cudaS
   const Tuning tn = tuning();
   KtMaps tm;
   KtParams kp{};
+  const int CG = (p.M + 31) / 32, WG = pl.c_warps;
   kp.a = p;
   kp.a.wait_cycles = tn.wait_cycles;
   kp.N = p.M; kp.S = pl.cluster; kp.NS = pl.stages; kp.PB = pl.m_warps;
   kp.DL = (D + kp.S - 1) / kp.S;
   {
-    const int NPc = p.M <= 32 ? 32 : 64;
-    const int chunks = 128 / kp.DL;                      // threads that share one owned head dimension
-    kp.cpt = ((NPc + chunks - 1) / chunks + 3) / 4 * 4;
+    const int chunks = 128 * CG / kp.DL;                 // carrying threads that share one owned head dimension
+    kp.cpt = ((32 * CG + chunks - 1) / chunks + 3) / 4 * 4;
   }
   kp.gr2 = p.n2 < 32 ? p.n2 : 32;
   kp.early_src1 = (p.n2 > 0 && p.n1_max > 0 && tn.early_loads != 0) ? 1 : 0;
@@ -942,8 +1011,8 @@ cudaError_t launch_attn_kt(const AttnParams& p, const AttnPlan& pl, int D, cudaS
   if (p.n1_max > 0) {
     ok = ok && umma_make_map(&tm.k1, p.k1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 32, 1);
     ok = ok && umma_make_map(&tm.v1, p.v1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 32, 1);
-    ok = ok && umma_make_map(&tm.k1t, p.k1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, pl.key_tile, 1);
-    ok = ok && umma_make_map(&tm.v1t, p.v1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, pl.key_tile, 1);
+    ok = ok && umma_make_map(&tm.k1t, p.k1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 128, 1);
+    ok = ok && umma_make_map(&tm.v1t, p.v1, D, p.n1_max, p.Hkv, p.B, p.k1_stride, 128, 1);
   }
   if (p.n2 > 0) {
     ok = ok && umma_make_map(&tm.k2, p.k2, D, p.n2, p.Hkv, p.B, p.k2_stride, kp.gr2, 1);
@@ -954,10 +1023,7 @@ cudaError_t launch_attn_kt(const AttnParams& p, const AttnPlan& pl, int D, cudaS
   }
   if (!ok) return cudaErrorInvalidValue;
   const bool pdl = tn.pdl != 0;
-  const int NP = p.M <= 32 ? 32 : 64;
-  if (NP == 32 && pl.c_warps == 2) return D == 128 ? launch_kt_d<128, 1, 2>(tm, kp, pl, pdl, st) : launch_kt_d<64, 1, 2>(tm, kp, pl, pdl, st);
-  if (NP == 32) return D == 128 ? launch_kt_d<128, 1, 1>(tm, kp, pl, pdl, st) : launch_kt_d<64, 1, 1>(tm, kp, pl, pdl, st);
-  return D == 128 ? launch_kt_d<128, 2, 1>(tm, kp, pl, pdl, st) : launch_kt_d<64, 2, 1>(tm, kp, pl, pdl, st);
+  return D == 128 ? launch_kt_shape<128>(tm, kp, pl, WG, CG, pdl, st) : launch_kt_shape<64>(tm, kp, pl, WG, CG, pdl, st);
 }
 
 }  // namespace sdllm

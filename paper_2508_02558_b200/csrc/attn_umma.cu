@@ -1161,16 +1161,19 @@ cudaError_t launch_attn_umma(const AttnParams& p, const AttnPlan& pl, int D, cud
 AttnPlan plan_attention_legacy(int dtype, int D, int M, int B, int Hkv, int n_keys_max, const Tuning& tn);
 cudaError_t launch_attn_legacy(const AttnParams& p, const AttnPlan& plan, int dtype, int D, cudaStream_t st);
 bool kt_supported(int dtype, int D, int M, int b);
+bool kt_preferred(int M, int B, int Hkv, int n1_max, int n2);
 AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int n2, const Tuning& tn);
 cudaError_t launch_attn_kt(const AttnParams& p, const AttnPlan& pl, int D, cudaStream_t st);
 
 AttnPlan plan_attention(int dtype, int D, int M, int b, int B, int Hkv, int n1_max, int n2, bool prob_scores) {
-  // bf16 goes to the tcgen05 kernels wherever they apply: heads with at most 64 query rows to the kernel that puts the
-  // keys on the accumulator rows (it has no softmax-probability saliency pass), the rest to the one that puts the
-  // queries there; fp32 and the remaining bf16 shapes go to the cp.async kernels. Tuning::kernel forces a family.
+  // bf16 goes to the tcgen05 kernels wherever they apply: heads with at most 128 query rows to the kernel that puts the
+  // keys on the accumulator rows (it has no softmax-probability saliency pass) unless its cluster limit would leave most
+  // SMs idle, the rest to the one that puts the queries there; fp32 and the remaining bf16 shapes go to the cp.async
+  // kernels. Tuning::kernel forces a family.
   const Tuning tn = tuning();
   const bool kt_ok = kt_supported(dtype, D, M, b) && !prob_scores;
-  if ((tn.kernel == 0 || tn.kernel == 3) && kt_ok) return plan_attention_kt(D, M, b, B, Hkv, n1_max, n2, tn);
+  if (kt_ok && (tn.kernel == 3 || (tn.kernel == 0 && kt_preferred(M, B, Hkv, n1_max, n2))))
+    return plan_attention_kt(D, M, b, B, Hkv, n1_max, n2, tn);
   if (tn.kernel != 1 && umma_supported(dtype, D, M, b)) return plan_attention_umma(D, M, b, B, Hkv, n1_max, n2, tn);
   AttnPlan pl = plan_attention_legacy(dtype, D, M, B, Hkv, n1_max + n2, tn);
   pl.tma = false; pl.cluster = 1; pl.warp_keys = 32; pl.kind = 0;

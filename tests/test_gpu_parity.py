@@ -62,6 +62,21 @@ def test_small_cases_span_tiles_heads_and_dtypes(cfg, block):
     _run_sequence_case(cfg, seed=11, block=block)
 
 
+@pytest.mark.parametrize("cfg,block", [
+    (_small("kt_gqa2", "bf16", 8, 4, 128, 517, 64, retention=0.3, salient_frac=0.01), 0),       # 64 query columns: two softmax warpgroups per tile
+    (_small("kt_gqa3", "bf16", 6, 2, 128, 333, 96, retention=0.5, salient_frac=0.02), 1),       # 96: three
+    (_small("kt_gqa4", "bf16", 8, 2, 128, 700, 64, retention=0.4, salient_frac=0.01), 1),       # 128: four
+    (_small("kt_gqa2_d64", "bf16", 4, 2, 64, 150, 64, salient_frac=0.02), 1),
+    (_small("kt_gqa4_blk16", "bf16", 16, 4, 128, 212, 32, block_len=16, salient_frac=0.02), 1), # 64 columns from four heads of 16 rows
+])
+@pytest.mark.parametrize("plan", [dict(kernel=3), dict(kernel=3, splits=1), dict(kernel=3, splits=8)])
+def test_key_row_kernel_on_grouped_heads(cfg, block, plan, tuning):
+    """Up to 128 query columns per KV head on the kernel with the keys on the accumulator rows (the planner picks it
+    for such heads only when there are enough (sequence, KV head) units; here it is forced)."""
+    tuning(**plan)
+    _run_sequence_case(cfg, seed=21, block=block, n_sparse=2)
+
+
 @pytest.mark.parametrize("p,gen,block", [(0, 96, 0), (160, 32, 0), (64, 64, 1)])
 def test_block_at_sequence_edges(p, gen, block):
     """Empty prefix (block first), empty suffix (block last)."""
@@ -151,10 +166,15 @@ def test_pool_windows(window):
     dict(kernel=1),                                      # cp.async + mma.sync kernels, separate merge launch
     dict(kernel=1, splits=3),
     dict(pdl=0),                                         # no programmatic dependent launch
-    dict(splits=7), dict(splits=1), dict(splits=3),      # other key-split counts (cluster sizes) of the key-row kernel
-    dict(splits=2, stages=3), dict(splits=1, stages=2),  # ... and ring depths
-    dict(dual=0), dict(dual=0, splits=1), dict(dual=0, splits=3, stages=1), dict(dual=1, splits=1, stages=1),   # two softmax warpgroups / one
-    dict(early_loads=0),                                 # no loads ahead of the grid dependency
+    # the tcgen05 kernel with the keys on the accumulator rows, forced also for the grouped heads (few units: the planner
+    # would give those to the query-row kernel), where one softmax warpgroup per 32 query columns shares every tile
+    dict(kernel=3),
+    dict(kernel=3, splits=7), dict(kernel=3, splits=1), dict(kernel=3, splits=3),      # key-split counts (cluster sizes)
+    dict(kernel=3, splits=2, stages=3), dict(kernel=3, splits=1, stages=2),            # ... and ring depths
+    dict(kernel=3, dual=0), dict(kernel=3, dual=0, splits=1), dict(kernel=3, dual=0, splits=3, stages=1),   # two softmax warpgroups / one
+    dict(kernel=3, dual=1, splits=1, stages=1),
+    dict(kernel=3, early_loads=0),                       # no loads ahead of the grid dependency
+    dict(kernel=3, pdl=0),
     dict(kernel=2),                                      # the tcgen05 kernel with the queries on the accumulator rows
     dict(kernel=2, splits=7), dict(kernel=2, splits=1),
     dict(kernel=2, splits=5, fused_tail=0),              # split merge and pooling in the second launch
