@@ -224,7 +224,7 @@ sdllm_status sdllm_sparse_block_attn_static(const sdllm_desc* desc, const void* 
  *   "kernel"      attention kernel family: 0 automatic, 1 cp.async, 2 tcgen05 with the queries on the accumulator rows,
  *                 3 tcgen05 with the keys on the accumulator rows (only where that kernel covers the shape)
  *   "pdl"         0: no programmatic dependent launch     "early_loads" 0: no loads ahead of the grid dependency
- *   "cluster", "fused_tail", "dual", "key_tile", "lpt", "stages"   plan details of the tcgen05 kernels
+ *   "cluster", "fused_tail", "dual", "key_tile", "lpt", "stages", "trigger", "persist"   plan details of the tcgen05 kernels
  *   "select"      top-k kernel: 1 one CTA per head, 2 one cluster per head
  *   "wait_cycles" limit, in SM clock cycles, of every abortable device-side wait (default 400 000 000, ~0.2 s). A limit
  *                 of a few cycles makes the first wait that is not already satisfied give up: the call still returns,

@@ -37,6 +37,7 @@
 #include <string.h>
 
 #include "attn_device.cuh"
+#include "kt_params.cuh"
 #include "tuning.cuh"
 #include "umma_host.cuh"
 
@@ -45,139 +46,8 @@ using namespace dev;
 namespace {
 
 constexpr int KT_MAX_STAGES = 3;
-constexpr int KT_GRP = 3072;             // control block, per softmax warpgroup: references, raise scratch, sums, saliency partials
-constexpr int KT_CTRL0 = 1024;           // control block, common part: barriers and flags
 
-struct KtMaps {
-  CUtensorMap q, k1, v1, k2, v2;   // boxes of 32 rows (source 2: min(32, n2))
-  CUtensorMap k1t, v1t;            // source 1 again, boxes of 128 rows: a whole tile per copy
-};
-
-struct KtParams {
-  AttnParams a;
-  int N;             // query columns of a KV head (b * G)
-  int S;             // key splits of a unit = CTAs of its cluster (1..8)
-  int NS;            // ring slots (one 128-key K tile + V tile each)
-  int PB;            // P^T buffers (1 or 2)
-  int DL;            // head dimensions a CTA owns in the merge: ceil(D / S)
-  int cpt;           // merge: columns per thread, a multiple of 4
-  int gr2;           // rows of a source-2 box: min(32, n2)
-  int early_src1;    // 1: source 1 and its count are older than every kernel that may still run (reuse step)
-  int early_trigger; // 1: release the next kernel in the stream as soon as this CTA is set up
-  int lpt;           // 1: grid z counts the sequences from the longest to the shortest (several waves of ragged work)
-  long long wait_cycles;   // limit of every abortable mbarrier wait
-};
-
-#include "umma_ptx.cuh"
-
-__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed;\n" ::: "memory"); }
-__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release;\n" ::: "memory"); }
-__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire;\n" ::: "memory"); }
-// Asynchronous stores into the shared memory of a CTA of the cluster; each one reports its bytes to an mbarrier of that
-// CTA (complete_tx, release at cluster scope), so the receiver waits for exactly the data it is owed and for nothing else.
-__device__ __forceinline__ void st_async_f4(uint32_t addr, uint32_t mbar, float x, float y, float z, float w) {
-  asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];\n"
-               ::"r"(addr), "f"(x), "f"(y), "f"(z), "f"(w), "r"(mbar) : "memory");
-}
-__device__ __forceinline__ void st_async_f2(uint32_t addr, uint32_t mbar, float x, float y) {
-  asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];\n"
-               ::"r"(addr), "f"(x), "f"(y), "r"(mbar) : "memory");
-}
-// Bounded wait on an mbarrier that remote CTAs complete: acquire at cluster scope.
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool wait_merge(uint32_t bar, volatile int* abort_flag, int32_t* status, long long limit) {
-  if (mbar_try_wait_cluster(bar, 0)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-    if (mbar_try_wait_cluster(bar, 0)) return true;
-    const bool aborting = *abort_flag != 0;
-    // an aborting CTA still lets its peers' pushes land before it retires (drain limit)
-    if (clock64() - t0 > (aborting ? kDrainCycles : limit)) {
-      if (!aborting) { *abort_flag = 1; atomicExch(status, 13); }
-      else return false;
-    }
-  }
-}
-// Pulls one box of a tensor into L2 without waiting for it. L2 is the point of coherence, so this is safe for data a
-// kernel in front of this one may still be writing: the later copy into shared memory reads what L2 holds then.
-__device__ __forceinline__ void tma_prefetch_l2(const CUtensorMap* tm, int x, int y, int z, int w) {
-  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];\n" ::"l"(tm), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
-}
-__device__ __forceinline__ float warp_max_f32(float v) {
-  float r;
-  asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;\n" : "=f"(r) : "f"(v));
-  return r;
-}
-// barrier of the 128 softmax threads that also ORs a predicate over them
-__device__ __forceinline__ bool softmax_barrier_or(int id, bool pred) {
-  uint32_t r;
-  asm volatile(
-      "{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.or.pred p, %2, 128, q;\n selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(r) : "r"((uint32_t)pred), "r"(id) : "memory");
-  return r != 0;
-}
-// barrier of one softmax warpgroup (ids 1 to 4), and of all of them (id 5)
-__device__ __forceinline__ void softmax_barrier(int id) { asm volatile("bar.sync %0, 128;\n" ::"r"(id) : "memory"); }
-template <int NG>
-__device__ __forceinline__ void softmax_barrier_all() { asm volatile("bar.sync 5, %0;\n" ::"n"(128 * NG) : "memory"); }
-
-// order-preserving fp32 <-> u32 (larger float <=> larger code), for the shared-memory max of the references
-__device__ __forceinline__ uint32_t f2ord(float x) {
-  const uint32_t u = __float_as_uint(x);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-__device__ __forceinline__ float ord2f(uint32_t k) { return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k); }
-
-// Shared-memory matrix descriptor with the 64-byte swizzle (mode 4 in bits 61-63): rows of 64 bytes, 8 rows per atom.
-__device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
-         (1ull << 46) | (4ull << 61);
-}
-// Instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B, M = 128, N = n; A and B K-major or MN-major.
-__device__ __forceinline__ uint32_t kt_idesc(int n, bool a_mn, bool b_mn) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
-         ((128u >> 4) << 24);
-}
-
-// One group of 32 key rows: where it comes from and how many of its rows are real keys.
-struct Group {
-  int src1;     // 1: source 1, 0: source 2
-  int row0;     // first row inside its source
-  int nv;       // valid rows, 1..32
-};
-__device__ __forceinline__ Group group_of(int gi, int g1, int n1, int n2) {
-  Group x;
-  if (gi < g1) { x.src1 = 1; x.row0 = gi * 32; x.nv = min(n1 - x.row0, 32); }
-  else { x.src1 = 0; x.row0 = (gi - g1) * 32; x.nv = min(n2 - x.row0, 32); }
-  return x;
-}
-
-// Importance of one absolute position: Algorithm 1, MaxPool1D(A, kernel_size = s, padding = s/2) over the candidate
-// axis Concat(prefix, suffix) (AvgPool for the ablation); block positions and padding get -inf. `a` is the raw
-// saliency by absolute position in global memory, written by other CTAs during this launch (read through L2).
-__device__ __forceinline__ float kt_pool_at(const AttnParams& p, const float* a, int L, int o_in, int pos) {
-  const int b = p.b;
-  const int o = min(max(o_in, 0), max(L - b, 0));
-  if (pos >= L || (pos >= o && pos < o + b)) return -INFINITY;
-  const int C = max(L - b, 0), w = (p.window - 1) / 2;
-  const int c = pos < o ? pos : pos - b;
-  int lo = 0, hi = C;
-  if (p.per_region) { if (c < o) hi = o; else lo = o; }
-  float mx = -INFINITY, sum = 0.f;
-  for (int t = c - w; t <= c + w; ++t) {
-    if (t < lo || t >= hi) continue;
-    const float x = __ldcg(a + (t < o ? t : t + b));
-    mx = fmaxf(mx, x);
-    sum += x;
-  }
-  return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
-}
+#include "kt_common.cuh"
 
 // WG = 2: two softmax warpgroups take the tiles in turn, each with its own accumulator and references (32 query columns).
 // CG > 1: CG softmax warpgroups share every tile, each owning 32 of the 32 * CG query columns (one accumulator).
@@ -839,8 +709,7 @@ __global__ void __launch_bounds__(64 + 128 * WG * CG, (WG == 1 && CG == 1) ? 2 :
     const float* a = p.raw_scores + (int64_t)(bi * p.Hkv + g) * p.n1_max;
     const int p_lo = (int)(((long long)split * p.n1_max) / S), p_hi = (int)(((long long)(split + 1) * p.n1_max) / S);
     const int o = p.block_off[bi];
-    for (int pos = p_lo + tid; pos < p_hi; pos += NTHREADS)
-      p.pooled[(int64_t)(bi * p.Hkv + g) * p.n1_max + pos] = kt_pool_at(p, a, n1, o, pos);
+    kt_pool_positions(p, a, p.pooled + (int64_t)(bi * p.Hkv + g) * p.n1_max, n1, o, p_lo + tid, p_hi, NTHREADS);
   }
 
   // ---- free the tensor memory ----
@@ -981,6 +850,16 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   pl.part_rows = 0;
   pl.n_counters = 0;
   pl.smem_bytes = kt_smem_bytes(D, CG, WG, NS, PB, S);
+  // (d) as (b), but with more units than SMs: the CTAs would run in waves, each paying its set-up and its way out with
+  //     the SM's memory pipe idle; one resident CTA per SM walks the units as one sequence of tiles instead.
+  pl.persistent = CG == 1 && S == 1 && WG == 2 && units > sms;
+  if (tn.persist == 0) pl.persistent = false;
+  if (tn.persist >= 1) pl.persistent = CG == 1 && S == 1;
+  if (pl.persistent) {
+    pl.stages = 3; pl.m_warps = 2; pl.c_warps = 2; pl.threads = 64 + 2 * 128;
+    pl.smem_bytes = kt_stream_smem_bytes(D);
+    pl.n_counters = 2;                  // the next unit to hand out, and the CTAs that have finished
+  }
   return pl;
 }
 
@@ -1023,6 +902,10 @@ cudaError_t launch_attn_kt(const AttnParams& p, const AttnPlan& pl, int D, cudaS
   }
   if (!ok) return cudaErrorInvalidValue;
   const bool pdl = tn.pdl != 0;
+  if (pl.persistent) {
+    kp.lpt = (p.n1_per_seq != nullptr && p.B <= 64 && tn.lpt != 0) ? 1 : 0;      // the walk starts with the longest sequences
+    return launch_kt_stream(tm, kp, D, pl.smem_bytes, pdl, st);
+  }
   return D == 128 ? launch_kt_shape<128>(tm, kp, pl, WG, CG, pdl, st) : launch_kt_shape<64>(tm, kp, pl, WG, CG, pdl, st);
 }
 

@@ -35,6 +35,7 @@ struct AttnPlan {
   int rows_rep;     // rows of one partial
   bool fused_tail;  // the attention kernel merges the partials and pools the scores itself
   bool dual;        // tcgen05 kernel, small-footprint variant: two CTAs per SM
+  bool persistent;  // key-row kernel, streaming variant: one resident CTA per SM walks the units
   size_t part_rows; // partial rows per (sequence, KV head) in the workspace (0: none)
   size_t n_counters;// completion counters in the workspace
 };

@@ -32,6 +32,7 @@ bool tuning_set(const char* name, long long value) {
       {"splits", &Tuning::splits}, {"kernel", &Tuning::kernel}, {"pdl", &Tuning::pdl}, {"early_loads", &Tuning::early_loads},
       {"cluster", &Tuning::cluster}, {"fused_tail", &Tuning::fused_tail}, {"dual", &Tuning::dual}, {"key_tile", &Tuning::key_tile},
       {"lpt", &Tuning::lpt}, {"select", &Tuning::select}, {"stages", &Tuning::stages}, {"debug", &Tuning::debug}, {"trigger", &Tuning::trigger},
+      {"persist", &Tuning::persist},
   };
   for (const Field& f : fields)
     if (strcmp(name, f.name) == 0) {

@@ -25,6 +25,8 @@ struct Tuning {
   int select = 0;            // top-k: 1 one CTA per head, 2 a cluster per head
   int stages = 0;            // key-row kernel: ring slots (1..3)
   int trigger = 1;           // key-row kernel: 1 releases the next kernel in the stream at its start, 0 after its own dependency
+  int persist = -1;          // key-row kernel: 0 / 1 forces the streaming variant (resident CTAs walk the units) off / on;
+                             // n >= 2: on, with at most n CTAs (small test shapes then walk several units per CTA)
   int debug = 0;             // 1: print the CUDA error behind an SDLLM_ERR_CUDA to stderr
   long long wait_cycles = 400000000LL;   // limit of an abortable device-side wait, ~0.2 s
 };

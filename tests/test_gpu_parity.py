@@ -175,6 +175,7 @@ def test_pool_windows(window):
     dict(kernel=3, dual=1, splits=1, stages=1),
     dict(kernel=3, early_loads=0),                       # no loads ahead of the grid dependency
     dict(kernel=3, pdl=0),
+    dict(kernel=3, splits=1, persist=1), dict(kernel=3, splits=1, persist=2),   # streaming variant (where one column group suffices)
     dict(kernel=2),                                      # the tcgen05 kernel with the queries on the accumulator rows
     dict(kernel=2, splits=7), dict(kernel=2, splits=1),
     dict(kernel=2, splits=5, fused_tail=0),              # split merge and pooling in the second launch
@@ -208,7 +209,10 @@ def test_softmax_probability_saliency(cfg, block, plan, tuning):
 
 
 @pytest.mark.parametrize("plan", [{}, dict(splits=3), dict(lpt=1), dict(lpt=1, dual=0, splits=1), dict(dual=0, splits=1), dict(dual=0, splits=2), dict(kernel=2), dict(kernel=2, lpt=1), dict(kernel=2, lpt=1, dual=1, splits=1),
-                                  dict(select=2)])
+                                  dict(select=2),
+                                  # streaming variant of the key-row kernel: 16 units on one CTA each, on 3 CTAs (five or six
+                                  # units per CTA, in the order of the lengths) and on a single one, also in batch order
+                                  dict(splits=1, persist=1), dict(splits=1, persist=3), dict(splits=1, persist=3, lpt=0), dict(splits=1, persist=2)])
 def test_ragged_batch(plan, tuning):
     import parity_util as U
     tuning(**plan)
@@ -387,6 +391,7 @@ def test_dense_step_strided_tensors_and_argument_checks():
 @pytest.mark.parametrize("plan", [
     {},                                  # key-row kernel: its splits still meet in the cluster merge while they give up
     dict(splits=1),                      # ... one CTA per head
+    dict(splits=1, persist=2),           # ... streaming variant: two resident CTAs walk the heads
     dict(kernel=2, cluster=0, splits=3), # query-row kernel, partials and completion counters in the workspace
     dict(kernel=2),                      # ... cluster tail
 ])
@@ -421,7 +426,8 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_a_usable_library(pl
     np.testing.assert_array_equal(again, want)
 
 
-@pytest.mark.parametrize("plan", [{}, dict(splits=1), dict(splits=2), dict(dual=0, splits=1), dict(dual=0, splits=2), dict(kernel=2)])
+@pytest.mark.parametrize("plan", [{}, dict(splits=1), dict(splits=2), dict(dual=0, splits=1), dict(dual=0, splits=2), dict(kernel=2),
+                                  dict(splits=1, persist=1), dict(splits=1, persist=2)])
 def test_logits_far_above_the_softmax_references(plan, tuning):
     """The key-row kernel takes its softmax references from the first key of a CTA's first tile and only checks later keys
     against them; keys whose logits lie more than 2^64 above a reference make it raise the references and rescale what it
