@@ -36,10 +36,12 @@ UNIT = "tokens/s"
 PROFILES = os.path.join(ROOT, "profiles")
 
 
-def ncu_traffic(workload: str):
-    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the reuse-step kernel on `workload`, read from the ncu
-    summary under profiles/ (a line "traffic_bytes_per_launch: N"); None when no capture of the current kernel exists."""
-    path = os.path.join(PROFILES, "attn_kt_%s_sparse.txt" % workload)
+def ncu_traffic(kernel: str, workload: str, batch: int):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the reuse-step kernel `kernel` on `workload`, read from
+    the ncu summary under profiles/ (a line "traffic_bytes_per_launch: N"); None when no capture of that kernel on that
+    workload exists."""
+    stem = kernel.replace("_bf16_kernel", "").replace("_kernel", "")
+    path = os.path.join(PROFILES, "%s_%s%s_sparse.txt" % (stem, workload, "_b%d" % batch if batch > 1 else ""))
     if not os.path.exists(path):
         return None, None
     for line in open(path):
@@ -133,21 +135,73 @@ def algorithmic_bytes(cfg: W.WorkloadConfig, seq_lens, n_keeps):
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples the SM clock and the clock-event (throttle) reasons of one GPU while timed regions run: a thread polls NVML
+    every few milliseconds (read-only queries), and only the samples that fall inside a region marked with begin() /
+    end() count. Falls back to an `nvidia-smi -lms` child process when the NVML binding is missing."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    BITS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+    active = None                 # the sampler that timed regions report to
 
     def __init__(self, index: int):
-        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.samples, self.windows, self._t0 = [], [], None
+        self.proc = self.file = self.thread = None
+        self.max_mhz = None
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=self.file, stderr=subprocess.DEVNULL)
-        except OSError:
-            self.proc = None
+            import pynvml
+            import threading
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            self._stop = threading.Event()
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.thread = None
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            try:
+                self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                              "-lms", "100"], stdout=self.file, stderr=subprocess.DEVNULL)
+            except OSError:
+                self.proc = None
+        ClockSampler.active = self
+
+    def _poll(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = float(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+                try:
+                    why = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+                except Exception:
+                    why = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                self.samples.append((time.perf_counter(), mhz, why))
+            except Exception:
+                pass
+            self._stop.wait(0.002)
+
+    def begin(self):
+        self._t0 = time.perf_counter()
+
+    def end(self):
+        if self._t0 is not None:
+            self.windows.append((self._t0, time.perf_counter()))
+            self._t0 = None
 
     def stop(self):
+        if ClockSampler.active is self:
+            ClockSampler.active = None
+        if self.thread is not None:
+            self._stop.set()
+            self.thread.join(timeout=2)
+            inside = [(m, w) for (t, m, w) in self.samples if any(a <= t <= b for a, b in self.windows)] if self.windows else \
+                     [(m, w) for (_, m, w) in self.samples]
+            reasons = sorted({name for _, w in inside for bit, name in self.BITS.items() if w & bit})
+            return {"sm_mhz": statistics.median([m for m, _ in inside]) if inside else None, "sm_max_mhz": self.max_mhz,
+                    "samples": len(inside), "reasons": reasons, "source": "nvml, polled every 2 ms inside the timed regions"}
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -169,8 +223,7 @@ class ClockSampler:
                     reasons.add(n)
         os.unlink(self.file.name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
-
+                "samples": len(sm), "reasons": sorted(reasons), "source": "nvidia-smi -lms 100"}
 
 
 # ------------------------------------------------------------------------------------------------ per-call timing
@@ -232,16 +285,24 @@ def time_calls(torch, dev, cfg, Bn, n_layers, rank, peak, steps=5, n_step_sets=4
         with torch.cuda.graph(g, stream=stream):
             fn()
         with torch.cuda.stream(stream):
-            for _ in range(3):
-                g.replay()
-            stream.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            for _ in range(steps):
+            for _ in range(3):
                 g.replay()
             e1.record(stream)
             stream.synchronize()
-        return e0.elapsed_time(e1) * 1e3 / steps / calls
+            # at least `steps` replays, and enough of them for about 30 ms: the clock sampler polls every few milliseconds
+            n_rep = max(steps, min(2000, int(0.03 / max(e0.elapsed_time(e1) / 3e3, 1e-6)) + 1))
+            if ClockSampler.active:
+                ClockSampler.active.begin()
+            e0.record(stream)
+            for _ in range(n_rep):
+                g.replay()
+            e1.record(stream)
+            stream.synchronize()
+            if ClockSampler.active:
+                ClockSampler.active.end()
+        return e0.elapsed_time(e1) * 1e3 / n_rep / calls
 
     c = caches
     ops = {
@@ -511,11 +572,15 @@ def run_ours(args):
                 dist.barrier()
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if ClockSampler.active:
+                ClockSampler.active.begin()
             e0.record(stream)
             for _ in range(iters):
                 runner()
             e1.record(stream)
             torch.cuda.synchronize()
+            if ClockSampler.active:
+                ClockSampler.active.end()
             if world > 1:
                 dist.barrier()
         return e0.elapsed_time(e1) / 1e3
@@ -580,10 +645,9 @@ def run_ours(args):
     rf_sec = timed(rf_runner, max(3, args.steps // 2), 3) / max(3, args.steps // 2) / n_layers
     peak, peak_kind = peaks()
     achieved = ab["sparse"] / sp_sec / 1e9
-    traffic, traffic_file = ncu_traffic(cfg.name)
-    kinds = {3: "attn_kt_kernel: tcgen05 attention with the keys on the accumulator rows, key splits merged through cluster shared memory",
-             2: "attn_umma_bf16_kernel: tcgen05 attention with the queries on the accumulator rows", 0: "cp.async kernels"}
-    roofline = {"bound": "hbm", "kernel": "sdllm_sparse_block_attn (%s)" % kinds.get(3 if Hq // Hkv * b <= 64 and cfg.dtype == "bf16" else 2, ""),
+    plan_text = B.plan_describe(caches[0].desc, B.OP_SPARSE_BLOCK_ATTN)      # what the library will launch for this call
+    traffic, traffic_file = ncu_traffic(plan_text.split()[0], cfg.name, Bn)
+    roofline = {"bound": "hbm", "kernel": "sdllm_sparse_block_attn (%s)" % plan_text,
                 "achieved": achieved,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                 "frac_of_8TBps": achieved / 8000.0, "algorithmic_bytes_per_launch": ab["sparse"], "us_per_launch": sp_sec * 1e6,

@@ -126,6 +126,13 @@ int32_t sdllm_cache_state(int32_t step_in_block, int32_t delay);
  * -1 for an invalid description or op. Lets a caller account for its launches without tracing them. */
 int32_t sdllm_launch_count(const sdllm_desc* desc, int op);
 
+/* Host-only; the paper has no counterpart. Writes a short NUL-terminated description of the launch plan of an attention
+ * call (`op` = SDLLM_OP_REFRESH_SCORES or SDLLM_OP_SPARSE_BLOCK_ATTN) into buf[0..buf_bytes): the kernel's name first,
+ * then its grid in words, e.g. "attn_kt_kernel splits=6 cluster=6 stages=1 threads=192". For logs and for naming the
+ * kernel a measurement belongs to; the text is not a stable format. The plan depends on the current device's SM
+ * count and on sdllm_tuning_set. Returns SDLLM_ERR_INVALID_ARG for a bad description, op, or a NULL / empty buffer. */
+sdllm_status sdllm_plan_describe(const sdllm_desc* desc, int op, char* buf, size_t buf_bytes);
+
 /* Reads the device status word kept in the first 4 bytes of an attention workspace. The kernels bound every wait
  * on a shared-memory barrier; if one ever expires they record a non-zero code there and run to the end instead of
  * hanging (the outputs of that call are then invalid). The caller zeroes those 4 bytes once after allocating the

@@ -21,7 +21,7 @@ SELECT_JOINT_FLOOR, SELECT_PER_REGION_CEIL, SELECT_PREFIX_ONLY = 0, 1, 2
 OP_REFRESH_SCORES, OP_SELECT_TOPK, OP_COMPACT_KV, OP_SPARSE_BLOCK_ATTN, OP_DENSE_ATTN, OP_SELECT_COMPACT = range(6)
 
 EXPORTS = ("sdllm_version", "sdllm_status_string", "sdllm_workspace_bytes", "sdllm_keep_count", "sdllm_cache_state", "sdllm_launch_count",
-           "sdllm_read_status",
+           "sdllm_plan_describe", "sdllm_read_status",
            "sdllm_refresh_scores", "sdllm_select_topk", "sdllm_compact_kv", "sdllm_sparse_block_attn",
            "sdllm_sparse_block_attn_static", "sdllm_dense_attn", "sdllm_select_compact", "sdllm_tuning_set", "sdllm_tuning_reset")
 
@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
         L.sdllm_keep_count.argtypes = [dp, ctypes.c_int32, ctypes.c_int32] + [ctypes.POINTER(ctypes.c_int32)] * 3
         L.sdllm_launch_count.restype = ctypes.c_int32
         L.sdllm_launch_count.argtypes = [ctypes.POINTER(Desc), ctypes.c_int]
+        L.sdllm_plan_describe.restype = ctypes.c_int
+        L.sdllm_plan_describe.argtypes = [ctypes.POINTER(Desc), ctypes.c_int, ctypes.c_char_p, ctypes.c_size_t]
         L.sdllm_cache_state.restype = ctypes.c_int32
         L.sdllm_cache_state.argtypes = [ctypes.c_int32, ctypes.c_int32]
         L.sdllm_read_status.restype = ctypes.c_int
@@ -171,6 +173,12 @@ def keep_count(desc: Desc, seq_len: int, block_off: int):
 
 def launch_count(desc: Desc, op: int) -> int:
     return int(lib().sdllm_launch_count(ctypes.byref(desc), int(op)))
+
+
+def plan_describe(desc: Desc, op: int) -> str:
+    buf = ctypes.create_string_buffer(256)
+    _check(lib().sdllm_plan_describe(ctypes.byref(desc), int(op), buf, ctypes.c_size_t(256)), "sdllm_plan_describe")
+    return buf.value.decode()
 
 
 def cache_state(step_in_block: int, delay: int = 1) -> int:

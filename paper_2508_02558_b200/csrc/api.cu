@@ -194,6 +194,22 @@ sdllm_status sdllm_keep_count(const sdllm_desc* d, int32_t seq_len, int32_t bloc
   return SDLLM_OK;
 }
 
+sdllm_status sdllm_plan_describe(const sdllm_desc* d, int op, char* buf, size_t buf_bytes) {
+  if (buf == nullptr || buf_bytes == 0) return SDLLM_ERR_INVALID_ARG;
+  buf[0] = 0;
+  if (check_desc(d) != SDLLM_OK || (op != SDLLM_OP_REFRESH_SCORES && op != SDLLM_OP_SPARSE_BLOCK_ATTN)) return SDLLM_ERR_INVALID_ARG;
+  const AttnPlan pl = plan_for(d, op);
+  const char* name = pl.kind == 3 ? (pl.persistent ? "attn_kt_stream_kernel" : "attn_kt_kernel")
+                                  : (pl.kind == 2 ? "attn_umma_bf16_kernel" : (d->dtype == SDLLM_BF16 ? "attn_bf16_kernel" : "attn_f32_kernel"));
+  if (pl.kind == 3)
+    snprintf(buf, buf_bytes, "%s splits=%d cluster=%d stages=%d softmax_warpgroups=%d threads=%d smem=%zu", name, pl.cluster, pl.cluster,
+             pl.stages, pl.c_warps * pl.warp_keys, pl.threads, pl.smem_bytes);
+  else
+    snprintf(buf, buf_bytes, "%s splits=%d cluster=%d stages=%d key_tile=%d threads=%d smem=%zu", name, pl.splits, pl.cluster, pl.stages,
+             pl.key_tile, pl.threads, pl.smem_bytes);
+  return SDLLM_OK;
+}
+
 int32_t sdllm_launch_count(const sdllm_desc* d, int op) {
   if (check_desc(d) != SDLLM_OK) return -1;
   if (op == SDLLM_OP_SELECT_TOPK) return 1;

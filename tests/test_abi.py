@@ -67,6 +67,20 @@ def test_workspace_sizes():
     assert B.workspace_bytes(big, B.OP_REFRESH_SCORES) >= 16 * 32 * 4352 * 4
 
 
+def test_plan_description_is_host_only_and_checks_its_arguments():
+    """Which kernel a shape gets depends on the device (without a Blackwell GPU the planner falls back to the cp.async
+    kernels); the names on a B200 are checked by the GPU tests. Here: a name comes back, and bad arguments are refused."""
+    assert B.plan_describe(_desc(), B.OP_SPARSE_BLOCK_ATTN).startswith("attn_")
+    assert B.plan_describe(_desc(dtype=B.F32), B.OP_REFRESH_SCORES).startswith("attn_f32_kernel ")
+    with pytest.raises(B.SdllmError) as e:
+        B.plan_describe(_desc(), B.OP_SELECT_TOPK)
+    assert e.value.status == B.ERR_INVALID_ARG
+    with pytest.raises(B.SdllmError) as e:
+        B.plan_describe(_desc(pool_window=2), B.OP_REFRESH_SCORES)
+    assert e.value.status == B.ERR_INVALID_ARG
+    assert B.lib().sdllm_plan_describe(__import__("ctypes").byref(_desc()), B.OP_REFRESH_SCORES, None, 0) == B.ERR_INVALID_ARG
+
+
 @pytest.mark.parametrize("bad,status", [
     (dict(pool_window=2), B.ERR_INVALID_ARG), (dict(retention=1.5), B.ERR_INVALID_ARG),
     (dict(n_q_heads=30), B.ERR_INVALID_ARG), (dict(dtype=7), B.ERR_INVALID_ARG),

@@ -456,3 +456,21 @@ def test_logits_far_above_the_softmax_references(plan, tuning):
     kn[:, 17, 0] = 500.0                         # the largest logit of all sits in the block's fresh rows (the last tile)
     out = U.gpu_sparse_step(g, q2[None], kn[None], vn[None], "bf16")
     U.check_sparse_against_oracle(g, out, q2[None], kn[None], vn[None], "bf16")
+
+
+def test_planner_picks_the_kernel_families_where_they_were_measured_to_win():
+    """Which kernel runs which shape on a B200 (sdllm_plan_describe): the benchmark's headline shape the key-row kernel,
+    a 16-sequence serving batch its streaming variant (more units than SMs), grouped heads with few units the query-row
+    kernel, grouped heads with many units the key-row kernel again."""
+    def name(op=B.OP_SPARSE_BLOCK_ATTN, **kw):
+        kw = dict(dict(batch=1, n_q_heads=32, n_kv_heads=32, head_dim=128, seq_len_max=1280, block_len=32, dtype=B.BF16, retention=0.5,
+                       n_keep_max=496), **kw)
+        return B.plan_describe(B.make_desc(**kw), op).split()[0]
+    assert name() == "attn_kt_kernel" and name(B.OP_REFRESH_SCORES) == "attn_kt_kernel"
+    assert name(batch=16, seq_len_max=4352, n_keep_max=2160) == "attn_kt_stream_kernel"
+    assert name(B.OP_REFRESH_SCORES, batch=16, seq_len_max=4352, n_keep_max=2160) == "attn_kt_stream_kernel"
+    assert name(n_q_heads=28, n_kv_heads=4, seq_len_max=4096, n_keep_max=1024) == "attn_umma_bf16_kernel"       # 224 query rows per KV head
+    assert name(n_kv_heads=8, seq_len_max=32768, n_keep_max=16368) == "attn_umma_bf16_kernel"                   # 8 units of 128 rows
+    assert name(batch=8, n_q_heads=16, n_kv_heads=8, seq_len_max=4352, n_keep_max=2048) == "attn_kt_kernel"     # 64 units of 64 rows
+    assert name(dtype=B.F32) == "attn_f32_kernel"
+
