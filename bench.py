@@ -671,22 +671,66 @@ def run_ours(args):
         hQs, hKn, hVn = Qs.cpu().pin_memory(), Kn.cpu().pin_memory(), Vn.cpu().pin_memory()
         h_out_r, h_out_s = out_r.cpu().pin_memory(), out_s.cpu().pin_memory()
 
+        # Two sets of device buffers: while step i runs from one set, the copy stream fills the other with step i + 1's
+        # inputs and a third stream brings step i - 1's outputs back. Every step's inputs still cross PCIe inside the
+        # timed region, every output is read back; the library is driven exactly as in the device-resident measurement.
+        def fresh_like(t):
+            return torch.empty_like(t)
+        sets = [dict(Q=Q_all, K=K_all, V=V_all, Qs=Qs, Kn=Kn, Vn=Vn, out_r=out_r, out_s=out_s, run=step_runner)]
+        if args.phase == "all":
+            s2 = dict(Q=fresh_like(Q_all), K=fresh_like(K_all), V=fresh_like(V_all), Qs=fresh_like(Qs), Kn=fresh_like(Kn), Vn=fresh_like(Vn),
+                      out_r=fresh_like(out_r), out_s=fresh_like(out_s))
+
+            def step_on_second_set():
+                for l in range(n_layers):
+                    caches[l].refresh(s2["Q"][l], s2["K"][l], s2["V"][l], seq_len_t, block_off, out=s2["out_r"][l], stream=stream)
+                for t in range(reuse_steps):
+                    for l in range(n_layers):
+                        caches[l].sparse_step(s2["Qs"][t, l], s2["Kn"][t, l], s2["Vn"][t, l], s2["out_s"][t, l], stream=stream)
+            s2["run"] = make_runner(step_on_second_set)
+            sets.append(s2)
+        h_outs = [(h_out_r, h_out_s)] + [(h_out_r.clone().pin_memory(), h_out_s.clone().pin_memory()) for _ in sets[1:]]
+        copy_in, copy_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        ev_in = [torch.cuda.Event() for _ in sets]      # the set's inputs have arrived
+        ev_run = [torch.cuda.Event() for _ in sets]     # the step on the set has finished
+        ev_out = [torch.cuda.Event() for _ in sets]     # the set's outputs are on the host
+        torch.cuda.synchronize(dev)
+        step_no = [0]
+
         def e2e_step():
-            """The step's inputs come from pinned host memory (one copy per tensor kind), the step runs through the
-            library exactly as in the device-resident measurement, and all of its outputs go back to the host."""
+            i = step_no[0] % len(sets); step_no[0] += 1
+            x = sets[i]
+            copy_in.wait_event(ev_run[i])                # the set's previous step no longer reads its inputs
+            with torch.cuda.stream(copy_in):
+                x["Q"].copy_(hQ, non_blocking=True); x["K"].copy_(hK, non_blocking=True); x["V"].copy_(hV, non_blocking=True)
+                x["Qs"].copy_(hQs, non_blocking=True); x["Kn"].copy_(hKn, non_blocking=True); x["Vn"].copy_(hVn, non_blocking=True)
+                ev_in[i].record(copy_in)
+            stream.wait_event(ev_in[i])
+            stream.wait_event(ev_out[i])                 # the set's previous outputs have left
             with torch.cuda.stream(stream):
-                Q_all.copy_(hQ, non_blocking=True); K_all.copy_(hK, non_blocking=True); V_all.copy_(hV, non_blocking=True)
-                Qs.copy_(hQs, non_blocking=True); Kn.copy_(hKn, non_blocking=True); Vn.copy_(hVn, non_blocking=True)
-                step_runner()
-                h_out_r.copy_(out_r, non_blocking=True); h_out_s.copy_(out_s, non_blocking=True)
-        e2e_iters = max(2, min(args.steps, 5))
-        e2e_sec = timed(e2e_step, e2e_iters, 1)
+                x["run"]()
+                ev_run[i].record(stream)
+            copy_out.wait_event(ev_run[i])
+            with torch.cuda.stream(copy_out):
+                h_outs[i][0].copy_(x["out_r"], non_blocking=True); h_outs[i][1].copy_(x["out_s"], non_blocking=True)
+                ev_out[i].record(copy_out)
+
+        def e2e_run(iters):
+            copy_in.wait_stream(stream); copy_out.wait_stream(stream)      # nothing starts ahead of the timed region
+            for _ in range(iters):
+                e2e_step()
+            stream.wait_stream(copy_in); stream.wait_stream(copy_out)      # the timed region ends when the last output is back
+        e2e_iters = max(2, min(args.steps, 6))
+        e2e_run(2)                                       # warm-up: both sets, all three streams
+        torch.cuda.synchronize(dev)
+        e2e_sec = timed(lambda: e2e_run(e2e_iters), 1, 0)
         e2e_sec = slowest_rank_seconds(e2e_sec, dev)
         esz = Ks[0].element_size()
         h2d = n_layers * Bn * ((2 * Hkv * L * D + Hq * b * D) * esz + reuse_steps * (2 * Hkv * b * D + Hq * b * D) * esz)
         d2h = n_layers * Bn * (1 + reuse_steps) * Hq * b * D * esz
         e2e = {"value": whole_job_value(tok * e2e_iters, world, e2e_sec), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "ms_per_step": 1e3 * e2e_sec / e2e_iters}
+               "ms_per_step": 1e3 * e2e_sec / e2e_iters, "steps": e2e_iters,
+               "overlap": "double-buffered: copies of step i+1 and i-1 run beside step i" if len(sets) > 1 else "none"}
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

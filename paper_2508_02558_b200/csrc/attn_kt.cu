@@ -815,6 +815,10 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   if (tn.splits > 0) want = tn.splits;
   if (want > 8) want = 8;
   if (want < 1) want = 1;
+  // Clusters of 3, 5 or 7 measured slower than the next even size (7.4 / 7.6 / 7.9 us against 6.8 / 7.2 / 7.8 us per
+  // reuse call of 32 heads at 9, 17 and 25 groups): uneven shares of the head dimensions in the merge, and clusters that
+  // pack the SMs of a GPC badly.
+  if (tn.splits <= 0 && want >= 3 && (want & 1) && want + 1 <= groups) want += 1;
   const int S = (int)want;
   // Footprint, ring depth, P^T buffers and softmax warpgroups:
   // (a) one column group and either at most two full tiles per CTA or a grid that fits the GPU only at two CTAs per

@@ -491,12 +491,12 @@ __global__ void __launch_bounds__(KS_THREADS, 1) attn_kt_stream_kernel(const __g
       // ======================================= end of the unit =======================================
       // ---- refresh step: pooling of the head's saliency, once both warpgroups' raw values are in L2 ----
       if (scores) {
-        __threadfence();
+        __threadfence_block();                         // writers and readers of the unit's raw saliency are this CTA's threads
         asm volatile("bar.sync 5, 256;\n" ::: "memory");
         if (p.pooled != nullptr && !*abort_flag) {
           const float* a = p.raw_scores + (int64_t)(bi * p.Hkv + g) * p.n1_max;
           const int o = p.block_off[bi];
-          kt_pool_positions(p, a, p.pooled + (int64_t)(bi * p.Hkv + g) * p.n1_max, x.n1, o, tid - 64, p.n1_max, 256);
+          kt_pool_positions<18>(p, a, p.pooled + (int64_t)(bi * p.Hkv + g) * p.n1_max, x.n1, o, tid - 64, p.n1_max, 256);   // (one round for 4.5k positions)
         }
       }
       // ---- this warpgroup's sums of the 32 columns ----

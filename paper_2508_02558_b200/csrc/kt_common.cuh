@@ -116,18 +116,19 @@ __device__ __forceinline__ float kt_pool_at(const AttnParams& p, const float* a,
   return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
 }
 // Pools the positions first, first + stride, ... below `end` of one head: `out` and `a` are the head's rows of the pooled
-// and of the raw scores. Eight positions at a time, so that their (L2) loads are in flight together instead of one
+// and of the raw scores. NB positions at a time, so that their (L2) loads are in flight together instead of one
 // position's after the other's.
+template <int NB = 8>
 __device__ __forceinline__ void kt_pool_positions(const AttnParams& p, const float* a, float* out, int L, int o, int first, int end, int stride) {
-  for (int pos0 = first; pos0 < end; pos0 += 8 * stride) {
-    float r[8];
+  for (int pos0 = first; pos0 < end; pos0 += NB * stride) {
+    float r[NB];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < NB; ++j) {
       const int pos = pos0 + j * stride;
       r[j] = pos < end ? kt_pool_at(p, a, L, o, pos) : 0.f;
     }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < NB; ++j) {
       const int pos = pos0 + j * stride;
       if (pos < end) out[pos] = r[j];
     }
