@@ -812,17 +812,24 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   long long want = (CG == 1 ? 2 : 1) * (long long)sms / units;
   const long long by_tiles = (groups + 3) / 4;
   if (want > by_tiles) want = by_tiles;
-  // More than half as many units as SMs, each with a walk of eight tiles or more: one whole-SM CTA per unit (footprint
+  // Six groups of 32 keys at most (two tiles, the second one short): one CTA walks both rather than two CTAs one each -
+  // a short second tile costs less than the cluster merge (124 cached keys, 32 heads: 6.0 against 6.9 us; with eight
+  // groups four splits are ahead again, 6.7 against 7.3 us).
+  if (groups <= 6) want = 1;
+  // More than half as many units as SMs, each with a walk of four tiles or more: one whole-SM CTA per unit (footprint
   // (b) below) beats two splits per unit at two CTAs per SM - the same share of the SMs is busy and nothing is merged
-  // (128 units x 17 tiles: 29.6 against 32.8 us; 96 units: 27.8 us; at 5 tiles per unit the two are equal).
-  if (CG == 1 && units * 2 > sms && units <= sms && groups >= 32) want = 1;
+  // (128 units x 17 tiles: 29.6 against 32.8 us; 96 units x 5 tiles: 12.3 against 19.3 us with clusters of three; at
+  // 128 units x 5 tiles the two are equal).
+  if (CG == 1 && units * 2 > sms && units <= sms && groups >= 16) want = 1;
   if (tn.splits > 0) want = tn.splits;
   if (want > 8) want = 8;
   if (want < 1) want = 1;
   // Clusters of 3, 5 or 7 measured slower than the next even size (7.4 / 7.6 / 7.9 us against 6.8 / 7.2 / 7.8 us per
   // reuse call of 32 heads at 9, 17 and 25 groups): uneven shares of the head dimensions in the merge, and clusters that
   // pack the SMs of a GPC badly.
-  if (tn.splits <= 0 && want >= 3 && (want & 1) && want + 1 <= groups && units * (want + 1) <= (CG == 1 ? 2 : 1) * (long long)sms) want += 1;
+  // Where the next even size would leave the one-wave budget, the one below is taken.
+  if (tn.splits <= 0 && want >= 3 && (want & 1))
+    want += (want + 1 <= groups && units * (want + 1) <= (CG == 1 ? 2 : 1) * (long long)sms) ? 1 : -1;
   const int S = (int)want;
   // Footprint, ring depth, P^T buffers and softmax warpgroups:
   // (a) one column group and either at most two full tiles per CTA or a grid that fits the GPU only at two CTAs per
