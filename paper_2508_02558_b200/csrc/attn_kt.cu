@@ -816,11 +816,11 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   // a short second tile costs less than the cluster merge (124 cached keys, 32 heads: 6.0 against 6.9 us; with eight
   // groups four splits are ahead again, 6.7 against 7.3 us).
   if (groups <= 6) want = 1;
-  // More than half as many units as SMs, each with a walk of four tiles or more: one whole-SM CTA per unit (footprint
+  // More than half as many units as SMs, each with a walk of five tiles or more: one whole-SM CTA per unit (footprint
   // (b) below) beats two splits per unit at two CTAs per SM - the same share of the SMs is busy and nothing is merged
   // (128 units x 17 tiles: 29.6 against 32.8 us; 96 units x 5 tiles: 12.3 against 19.3 us with clusters of three; at
   // 128 units x 5 tiles the two are equal).
-  if (CG == 1 && units * 2 > sms && units <= sms && groups >= 16) want = 1;
+  if (CG == 1 && units * 2 > sms && units <= sms && groups >= 20) want = 1;
   if (tn.splits > 0) want = tn.splits;
   if (want > 8) want = 8;
   if (want < 1) want = 1;
@@ -840,7 +840,10 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   // (c) 33 to 128 query columns: one CTA per SM, one softmax warpgroup per 32 columns, all on the same tile.
   const int groups_cta = (groups + S - 1) / S;
   const size_t half_sm = 113 * 1024;     // two CTAs of this size, each with its 1 KB system share, fit one SM
-  bool small = CG == 1 && (groups_cta <= 8 || (units * S > sms && units * S <= 2 * sms));
+  // (more units than SMs with walks of less than seven tiles: two small CTAs per SM overlap their set-up and way out
+  // better than the resident walk of (d), whose cost per unit is about three tiles' worth: 38 against 45 us for 512
+  // units of four tiles)
+  bool small = CG == 1 && (groups_cta <= 8 || (units * S > sms && units * S <= 2 * sms) || (units > sms && groups < 28));
   int WG = (CG == 1 && !small) ? 2 : 1;
   if (tn.dual == 1) { small = CG == 1; WG = 1; }       // force (a) / (b) where they apply
   if (tn.dual == 0 && CG == 1) { small = false; WG = 2; }
