@@ -785,6 +785,9 @@ bool kt_supported(int dtype, int D, int M, int b) {
 // most. With up to 32 query rows that is enough everywhere. With more, a CTA takes a whole SM, and a few units with
 // long key ranges (8 KV heads, one sequence, 16k keys: 64 CTAs) would leave most SMs idle; the query-row kernel splits
 // those further through its workspace and measured faster there (25 against 38 us), slower with 64 units and more.
+// Short walks are latency chains whatever the number of CTAs, and this kernel's chain is the shorter one: up to six
+// tiles per CTA at 64 query columns (8 KV heads x 1024 keys: 8.1 against 14.5 us; x 4096: 12.2 against 15.2), up to two
+// with more columns (12.1 against 13.0 us at 128 columns x 1024 keys; at 4096 keys the query-row kernel is ahead).
 bool kt_preferred(int M, int B, int Hkv, int n1_max, int n2) {
   if (M <= 32) return true;
   const long long units = (long long)B * Hkv;
@@ -794,7 +797,11 @@ bool kt_preferred(int M, int B, int Hkv, int n1_max, int n2) {
   if (S > by_tiles) S = by_tiles;
   if (S > 8) S = 8;
   if (S < 1) S = 1;
-  return units * S * 4 >= (long long)sms * 3;
+  const long long tiles_cta = (by_tiles + S - 1) / S;
+  // (three or four column groups walk a tile in 2 us, the query-row kernel in 1.5: long walks go there even when the
+  // SMs are filled - 32 units x 128 tiles: 70.7 against 79.6 us)
+  if (units * S * 4 >= (long long)sms * 3) return M <= 64 || tiles_cta <= 16;
+  return tiles_cta <= (M <= 64 ? 6 : 2);
 }
 
 AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int n2, const Tuning& tn) {
