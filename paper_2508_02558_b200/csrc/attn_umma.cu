@@ -1025,7 +1025,9 @@ bool umma_supported(int dtype, int D, int M, int b) {
 // the whole GPU.
 bool umma_tail_is_fused(const AttnPlan& pl, int D, int M, int n1_max, bool pool, bool merge) {
   const size_t merge_bytes = merge && pl.splits > 1 ? (size_t)pl.splits * (M < 128 ? M : 128) * D * 4 : 0;
-  bool fused = merge_bytes <= 256 * 1024 && (!pool || n1_max <= 8192);
+  // (a merge of full 128-row partials by the last CTA alone lost to the second launch at every split count measured,
+  // 16.2 against 22.6 us with four splits: the last CTA does it only for small partials)
+  bool fused = merge_bytes <= 32 * 1024 && (!pool || n1_max <= 8192);
   const int forced = tuning().fused_tail;
   if (forced >= 0) fused = forced == 1 && (!pool || n1_max <= 8192);
   return fused;
@@ -1057,6 +1059,15 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
     const long long cap = ((n1_max + 127) / 128 + 1 + 3) / 4;
     if (want > cap) want = cap;
   }
+  // Full 128-row tiles (nothing replicated), from the same sweep as the cluster note below: with at most 24 tiles per
+  // head eight splits beat sixteen (11.4 against 13.7 us at 1024 keys, 13.1 against 14.2 at 2048); with 32 units or more
+  // and at most five tiles per head no split at all beats four (13.1 against 20.8 us at 256 keys, 32 units).
+  // Nine splits (16 units) lost 6 % to eight wherever measured.
+  if (pl.rep == 1 && !pl.dual && tn.splits <= 0) {
+    const int t128 = (n1_max + 127) / 128 + (n2 > 0 ? 1 : 0);
+    if (want > 8 && (t128 <= 24 || want < 16)) want = 8;
+    if (n2 > 0 && units >= 32 && t128 <= 5) want = 1;
+  }
   const int kt2 = n2 > 0 ? (n2 < 128 ? n2 : 128) : 0;
   pl.key_tile = 128;
   if (pl.rep <= 2 && (n1_max + 127) / 128 + (n2 > 0 ? 1 : 0) < want) pl.key_tile = 64;
@@ -1066,7 +1077,12 @@ AttnPlan plan_attention_umma(int D, int M, int b, int B, int Hkv, int n1_max, in
   // A reuse step with few heads and a short cache: rather than many one-tile splits whose merge needs a second launch,
   // take at most eight splits of 128-key tiles, which one cluster merges on chip.
   const int tiles128 = (n1_max + 127) / 128 + (n2 > 0 ? 1 : 0);
-  const bool no_cluster = tn.cluster == 0 || tn.fused_tail == 0;
+  // The cluster tail of this kernel (every split pulls its share of the rows out of its peers' shared memory between two
+  // cluster barriers) measured slower than partials in the workspace at every shape of a sweep over 1 to 8 sequences x
+  // 256 to 4096 cached keys of 4 KV heads x 7 query heads (10 to 80 %: 11.5 against 12.6 us at 1024 keys, 13.1 against
+  // 23.7 us with two sequences), so it is taken only on request (Tuning::cluster = 2); the key-row kernel's push-style
+  // merge is the cluster path that pays.
+  const bool no_cluster = tn.cluster != 2 || tn.fused_tail == 0;
   if (!pl.dual && !no_cluster && tn.splits <= 0 && tn.key_tile == 0 && n2 > 0 && want > 8 && tiles128 <= 16) {
     pl.key_tile = 128;
     want = tiles128 < 8 ? tiles128 : 8;

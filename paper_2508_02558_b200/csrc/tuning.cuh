@@ -17,7 +17,7 @@ struct Tuning {
                              // rows; 3: tcgen05 kernel with the keys on the accumulator rows
   int pdl = 1;               // 0: no programmatic dependent launch
   int early_loads = 1;       // 0: no loads ahead of the grid dependency
-  int cluster = 1;           // 0: the query-row kernel never merges its splits through a cluster
+  int cluster = 1;           // query-row kernel: 2 merges few key splits through a cluster where the shape allows (off otherwise)
   int fused_tail = -1;       // query-row kernel: 0 / 1 forces the tail into the second launch / into the last CTA
   int dual = -1;             // query-row kernel: 0 / 1 forces the two-CTAs-per-SM variant off / on
   int key_tile = 0;          // query-row kernel: 64 or 128

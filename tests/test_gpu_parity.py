@@ -181,7 +181,8 @@ def test_pool_windows(window):
     dict(kernel=2, splits=5, fused_tail=0),              # split merge and pooling in the second launch
     dict(kernel=2, early_loads=0),
     dict(kernel=2, cluster=0, splits=4),                 # key splits merged by the last CTA instead of a cluster
-    dict(kernel=2, splits=4),                            # ... and by a cluster of four
+    dict(kernel=2, cluster=2, splits=4),                 # ... and by a cluster of four
+    dict(kernel=2, cluster=2), dict(kernel=2, cluster=2, splits=7),
     dict(kernel=2, dual=1, splits=1),                    # small-footprint variant (two CTAs per SM)
     dict(kernel=2, dual=1, splits=3),
     dict(kernel=2, key_tile=64, splits=2),               # 64-key tiles
@@ -393,7 +394,7 @@ def test_dense_step_strided_tensors_and_argument_checks():
     dict(splits=1),                      # ... one CTA per head
     dict(splits=1, persist=2),           # ... streaming variant: two resident CTAs walk the heads
     dict(kernel=2, cluster=0, splits=3), # query-row kernel, partials and completion counters in the workspace
-    dict(kernel=2),                      # ... cluster tail
+    dict(kernel=2, cluster=2),           # ... cluster tail
 ])
 def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_a_usable_library(plan, tuning):
     """With the limit of the abortable device-side waits set to zero, the first wait that is not already satisfied gives
