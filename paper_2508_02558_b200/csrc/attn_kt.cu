@@ -36,6 +36,8 @@
 #include <cuda.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "attn_device.cuh"
 #include "kt_params.cuh"
 #include "tuning.cuh"
@@ -735,11 +737,18 @@ size_t kt_smem_bytes(int D, int CG, int WG, int NS, int PB, int S) {
   return 1024 /*alignment slack*/ + KT_CTRL0 + NG * KT_GRP + H * NPT * 128 + (size_t)PB * pbuf + tail;
 }
 
+// what has been set as the kernel's dynamic shared memory limit, per device (one record per kernel: launch and
+// occupancy query both raise it, neither may lower it behind the other's back)
+template <int D, int WG, int CG>
+SmemConfig& kt_smem_config() {
+  static SmemConfig configured;
+  return configured;
+}
+
 template <int D, int WG, int CG>
 cudaError_t launch_kt_d(const KtMaps& tm, const KtParams& kp, const AttnPlan& pl, bool pdl, cudaStream_t st) {
   auto kern = attn_kt_kernel<D, WG, CG>;
-  static SmemConfig configured;
-  cudaError_t e = configure_smem(reinterpret_cast<const void*>(kern), pl.smem_bytes, configured, true);
+  cudaError_t e = configure_smem(reinterpret_cast<const void*>(kern), pl.smem_bytes, kt_smem_config<D, WG, CG>(), true);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(kp.S, kp.a.Hkv, kp.a.B);
@@ -773,6 +782,42 @@ cudaError_t launch_kt_shape(const KtMaps& tm, const KtParams& kp, const AttnPlan
   }
 }
 
+// How many clusters of S whole-SM CTAs (several column groups: footprint (c)) the current device keeps resident at once:
+// cudaOccupancyMaxActiveClusters, asked once per (head dimension, column groups, cluster size) and device. -1: no answer.
+template <int D, int CG>
+int kt_query_clusters(int S) {
+  auto kern = attn_kt_kernel<D, 1, CG>;
+  const size_t smem = 200 * 1024;        // any footprint above half an SM: one CTA per SM
+  if (configure_smem(reinterpret_cast<const void*>(kern), 226 * 1024, kt_smem_config<D, 1, CG>(), true) != cudaSuccess) return -1;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(S, 1, 1);
+  cfg.blockDim = dim3(64 + 128 * CG);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = S; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { (void)cudaGetLastError(); return -1; }
+  return n;
+}
+int kt_resident_clusters(int D, int CG, int S) {
+  static std::mutex mu;
+  static int cache[kMaxDevices][2][5][9];          // [device][D == 128][CG][S]: 0 = not asked yet, else answer + 2
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { (void)cudaGetLastError(); return -1; }
+  if (CG < 2 || CG > 4 || S < 2 || S > 8) return -1;
+  std::lock_guard<std::mutex> lock(mu);
+  int& c = cache[dev][D == 128 ? 1 : 0][CG][S];
+  if (c == 0) {
+    int n = -1;
+    if (D == 128) n = CG == 2 ? kt_query_clusters<128, 2>(S) : (CG == 3 ? kt_query_clusters<128, 3>(S) : kt_query_clusters<128, 4>(S));
+    else n = CG == 2 ? kt_query_clusters<64, 2>(S) : (CG == 3 ? kt_query_clusters<64, 3>(S) : kt_query_clusters<64, 4>(S));
+    c = n + 2;
+  }
+  return c - 2;
+}
+
 }  // namespace
 
 // Whether the key-row kernel covers a shape: bf16, D in {64, 128}, at most 128 query rows per KV head, block length a
@@ -800,7 +845,9 @@ bool kt_preferred(int M, int B, int Hkv, int n1_max, int n2) {
   const long long tiles_cta = (by_tiles + S - 1) / S;
   // (three or four column groups walk a tile in 2 us, the query-row kernel in 1.5: long walks go there even when the
   // SMs are filled - 32 units x 128 tiles: 70.7 against 79.6 us)
-  if (units * S * 4 >= (long long)sms * 3) return M <= 64 || tiles_cta <= 16;
+  // (with 16 to 24 units the query-row kernel, which can use more CTAs, is ahead from five tiles per CTA on: 19.7 against
+  // 22.3 us at 16 units x 33 tiles)
+  if (units * S * 4 >= (long long)sms * 3) return M <= 64 || tiles_cta <= (units >= 32 ? 16 : 4);
   return tiles_cta <= (M <= 64 ? 6 : 2);
 }
 
@@ -837,6 +884,19 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   // Where the next even size would leave the one-wave budget, the one below is taken.
   if (tn.splits <= 0 && want >= 3 && (want & 1))
     want += (want + 1 <= groups && units * (want + 1) <= (CG == 1 ? 2 : 1) * (long long)sms) ? 1 : -1;
+  if (CG > 1 && tn.splits <= 0) {
+    // Whole-SM CTAs: a cluster needs its SMs inside one GPC, so fewer clusters are resident than SMs / S suggests (16
+    // clusters of eight do not fit a B200, 16 of six do, 24 of six do not, 32 of four do). A grid whose clusters do not
+    // all fit runs in two waves: 15.9 against 9.3 us for 16 units x 1024 keys. The device is asked; without an answer
+    // the numbers above stand in.
+    if (by_tiles <= 3 && units >= 24) want = 1;          // (short walks of many units: no split, 7.7 against 9.6 us)
+    while (want > 1) {
+      const int fit = kt_resident_clusters(D, CG, (int)want);
+      const long long room = fit >= 0 ? fit : (want >= 7 ? 12 : (want >= 5 ? 20 : (want >= 3 ? 36 : 74)));
+      if (units <= room) break;
+      want = want > 2 ? ((want - 1) & ~1LL) : 1;
+    }
+  }
   const int S = (int)want;
   // Footprint, ring depth, P^T buffers and softmax warpgroups:
   // (a) one column group and either at most two full tiles per CTA or a grid that fits the GPU only at two CTAs per
