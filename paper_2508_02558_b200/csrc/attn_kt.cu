@@ -784,14 +784,14 @@ cudaError_t launch_kt_shape(const KtMaps& tm, const KtParams& kp, const AttnPlan
 
 // How many clusters of S whole-SM CTAs (several column groups: footprint (c)) the current device keeps resident at once:
 // cudaOccupancyMaxActiveClusters, asked once per (head dimension, column groups, cluster size) and device. -1: no answer.
-template <int D, int CG>
+template <int D, int WG, int CG>
 int kt_query_clusters(int S) {
-  auto kern = attn_kt_kernel<D, 1, CG>;
+  auto kern = attn_kt_kernel<D, WG, CG>;
   const size_t smem = 200 * 1024;        // any footprint above half an SM: one CTA per SM
-  if (configure_smem(reinterpret_cast<const void*>(kern), 226 * 1024, kt_smem_config<D, 1, CG>(), true) != cudaSuccess) return -1;
+  if (configure_smem(reinterpret_cast<const void*>(kern), 226 * 1024, kt_smem_config<D, WG, CG>(), true) != cudaSuccess) return -1;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(S, 1, 1);
-  cfg.blockDim = dim3(64 + 128 * CG);
+  cfg.blockDim = dim3(64 + 128 * WG * CG);
   cfg.dynamicSmemBytes = smem;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -801,18 +801,19 @@ int kt_query_clusters(int S) {
   if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { (void)cudaGetLastError(); return -1; }
   return n;
 }
+// (CG = 1 stands for footprint (b): two tile-alternating softmax warpgroups on one column group)
 int kt_resident_clusters(int D, int CG, int S) {
   static std::mutex mu;
   static int cache[kMaxDevices][2][5][9];          // [device][D == 128][CG][S]: 0 = not asked yet, else answer + 2
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { (void)cudaGetLastError(); return -1; }
-  if (CG < 2 || CG > 4 || S < 2 || S > 8) return -1;
+  if (CG < 1 || CG > 4 || S < 2 || S > 8) return -1;
   std::lock_guard<std::mutex> lock(mu);
   int& c = cache[dev][D == 128 ? 1 : 0][CG][S];
   if (c == 0) {
     int n = -1;
-    if (D == 128) n = CG == 2 ? kt_query_clusters<128, 2>(S) : (CG == 3 ? kt_query_clusters<128, 3>(S) : kt_query_clusters<128, 4>(S));
-    else n = CG == 2 ? kt_query_clusters<64, 2>(S) : (CG == 3 ? kt_query_clusters<64, 3>(S) : kt_query_clusters<64, 4>(S));
+    if (D == 128) n = CG == 1 ? kt_query_clusters<128, 2, 1>(S) : (CG == 2 ? kt_query_clusters<128, 1, 2>(S) : (CG == 3 ? kt_query_clusters<128, 1, 3>(S) : kt_query_clusters<128, 1, 4>(S)));
+    else n = CG == 1 ? kt_query_clusters<64, 2, 1>(S) : (CG == 2 ? kt_query_clusters<64, 1, 2>(S) : (CG == 3 ? kt_query_clusters<64, 1, 3>(S) : kt_query_clusters<64, 1, 4>(S)));
     c = n + 2;
   }
   return c - 2;
@@ -897,6 +898,25 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
       want = want > 2 ? ((want - 1) & ~1LL) : 1;
     }
   }
+  // ... and the same for footprints (a) and (b) below: where the clusters would not all be resident the cluster size goes
+  // down until they are (48 units: clusters of six at two CTAs per SM ran in two waves, 17.8 against 11.4 us with four).
+  auto is_small = [&](long long s_) {
+    const long long gc = (groups + s_ - 1) / s_;
+    return CG == 1 && (gc <= 8 || (units * s_ > sms && units * s_ <= 2 * sms) || (units > sms && groups < (n2 > 0 ? 20 : 28)));
+  };
+  while (CG == 1 && tn.splits <= 0 && tn.dual < 0 && want > 1) {
+    long long room;
+    if (is_small(want)) {
+      // (two CTAs per SM: the occupancy query is too careful here - it would turn away 32 clusters of six, which do run
+      // together - so the rule is the measured one: clusters of three or more fill at most nine tenths of the slots)
+      room = want >= 3 ? (2LL * sms * 9 / 10) / want : units;
+    } else {
+      const int fit = kt_resident_clusters(D, 1, (int)want);
+      room = fit >= 0 ? fit : (want >= 7 ? 12 : (want >= 5 ? 20 : (want >= 3 ? 36 : 74)));
+    }
+    if (units <= room) break;
+    want = want > 2 ? ((want - 1) & ~1LL) : 1;
+  }
   const int S = (int)want;
   // Footprint, ring depth, P^T buffers and softmax warpgroups:
   // (a) one column group and either at most two full tiles per CTA or a grid that fits the GPU only at two CTAs per
@@ -907,10 +927,10 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   // (c) 33 to 128 query columns: one CTA per SM, one softmax warpgroup per 32 columns, all on the same tile.
   const int groups_cta = (groups + S - 1) / S;
   const size_t half_sm = 113 * 1024;     // two CTAs of this size, each with its 1 KB system share, fit one SM
-  // (more units than SMs with walks of less than seven tiles: two small CTAs per SM overlap their set-up and way out
+  // (more units than SMs with walks of less than seven tiles at the refresh step, five at the reuse step: two small CTAs per SM overlap their set-up and way out
   // better than the resident walk of (d), whose cost per unit is about three tiles' worth: 38 against 45 us for 512
   // units of four tiles)
-  bool small = CG == 1 && (groups_cta <= 8 || (units * S > sms && units * S <= 2 * sms) || (units > sms && groups < 28));
+  bool small = CG == 1 && (groups_cta <= 8 || (units * S > sms && units * S <= 2 * sms) || (units > sms && groups < (n2 > 0 ? 20 : 28)));
   int WG = (CG == 1 && !small) ? 2 : 1;
   if (tn.dual == 1) { small = CG == 1; WG = 1; }       // force (a) / (b) where they apply
   if (tn.dual == 0 && CG == 1) { small = false; WG = 2; }
