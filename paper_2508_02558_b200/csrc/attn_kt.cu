@@ -875,7 +875,7 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   // (b) below) beats two splits per unit at two CTAs per SM - the same share of the SMs is busy and nothing is merged
   // (128 units x 17 tiles: 29.6 against 32.8 us; 96 units x 5 tiles: 12.3 against 19.3 us with clusters of three; at
   // 128 units x 5 tiles the two are equal).
-  if (CG == 1 && units * 2 > sms && units <= sms && groups >= 20) want = 1;
+  if (CG == 1 && D == 128 && units * 2 > sms && units <= sms && groups >= 20) want = 1;
   if (tn.splits > 0) want = tn.splits;
   if (want > 8) want = 8;
   if (want < 1) want = 1;
@@ -902,7 +902,7 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   // down until they are (48 units: clusters of six at two CTAs per SM ran in two waves, 17.8 against 11.4 us with four).
   auto is_small = [&](long long s_) {
     const long long gc = (groups + s_ - 1) / s_;
-    return CG == 1 && (gc <= 8 || (units * s_ > sms && units * s_ <= 2 * sms) || (units > sms && groups < (n2 > 0 ? 20 : 28)));
+    return CG == 1 && (D == 64 || gc <= 8 || (units * s_ > sms && units * s_ <= 2 * sms) || (units > sms && groups < (n2 > 0 ? 20 : 28)));
   };
   while (CG == 1 && tn.splits <= 0 && tn.dual < 0 && want > 1) {
     long long room;
@@ -930,7 +930,9 @@ AttnPlan plan_attention_kt(int D, int M, int b, int B, int Hkv, int n1_max, int 
   // (more units than SMs with walks of less than seven tiles at the refresh step, five at the reuse step: two small CTAs per SM overlap their set-up and way out
   // better than the resident walk of (d), whose cost per unit is about three tiles' worth: 38 against 45 us for 512
   // units of four tiles)
-  bool small = CG == 1 && (groups_cta <= 8 || (units * S > sms && units * S <= 2 * sms) || (units > sms && groups < (n2 > 0 ? 20 : 28)));
+  // (head dimension 64: a tile is half the bytes for the same softmax, so the softmax warps are what is short: always two
+  // CTAs per SM - 97.5 against 140 us for 512 units x 4352 keys, 30.2 against 41.1 us for 128 units)
+  bool small = CG == 1 && (D == 64 || groups_cta <= 8 || (units * S > sms && units * S <= 2 * sms) || (units > sms && groups < (n2 > 0 ? 20 : 28)));
   int WG = (CG == 1 && !small) ? 2 : 1;
   if (tn.dual == 1) { small = CG == 1; WG = 1; }       // force (a) / (b) where they apply
   if (tn.dual == 0 && CG == 1) { small = false; WG = 2; }
