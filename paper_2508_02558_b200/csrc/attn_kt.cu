@@ -711,7 +711,7 @@ __global__ void __launch_bounds__(64 + 128 * WG * CG, (WG == 1 && CG == 1) ? 2 :
     const float* a = p.raw_scores + (int64_t)(bi * p.Hkv + g) * p.n1_max;
     const int p_lo = (int)(((long long)split * p.n1_max) / S), p_hi = (int)(((long long)(split + 1) * p.n1_max) / S);
     const int o = p.block_off[bi];
-    kt_pool_positions(p, a, p.pooled + (int64_t)(bi * p.Hkv + g) * p.n1_max, n1, o, p_lo + tid, p_hi, NTHREADS);
+    kt_pool_span(p, a, p.pooled + (int64_t)(bi * p.Hkv + g) * p.n1_max, n1, o, p_lo, p_hi, tid, NTHREADS);
   }
 
   // ---- free the tensor memory ----

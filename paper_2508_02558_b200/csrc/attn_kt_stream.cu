@@ -496,7 +496,7 @@ __global__ void __launch_bounds__(KS_THREADS, 1) attn_kt_stream_kernel(const __g
         if (p.pooled != nullptr && !*abort_flag) {
           const float* a = p.raw_scores + (int64_t)(bi * p.Hkv + g) * p.n1_max;
           const int o = p.block_off[bi];
-          kt_pool_positions<18>(p, a, p.pooled + (int64_t)(bi * p.Hkv + g) * p.n1_max, x.n1, o, tid - 64, p.n1_max, 256);   // (one round for 4.5k positions)
+          kt_pool_span(p, a, p.pooled + (int64_t)(bi * p.Hkv + g) * p.n1_max, x.n1, o, 0, p.n1_max, tid - 64, 256);
         }
       }
       // ---- this warpgroup's sums of the 32 columns ----

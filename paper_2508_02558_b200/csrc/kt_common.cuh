@@ -115,22 +115,56 @@ __device__ __forceinline__ float kt_pool_at(const AttnParams& p, const float* a,
   }
   return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
 }
-// Pools the positions first, first + stride, ... below `end` of one head: `out` and `a` are the head's rows of the pooled
-// and of the raw scores. NB positions at a time, so that their (L2) loads are in flight together instead of one
-// position's after the other's.
-template <int NB = 8>
-__device__ __forceinline__ void kt_pool_positions(const AttnParams& p, const float* a, float* out, int L, int o, int first, int end, int stride) {
-  for (int pos0 = first; pos0 < end; pos0 += NB * stride) {
-    float r[NB];
+// Pools the absolute positions [p_lo, p_hi) of one head with `nthreads` threads (this one is `tid`): `out` and `a` are the
+// head's rows of the pooled and of the raw scores. A thread takes sixteen consecutive candidates at a time: their windows
+// overlap, so 24 loads (all of them issued together: fixed count, clamped addresses) serve sixteen outputs, and the window
+// logic runs on registers. Same values and the same order of the sums as kt_pool_at, which the wider windows still use.
+// (One position at a time, each with its own loop of dependent L2 round trips, cost 16 us per 4352 positions.)
+__device__ __forceinline__ void kt_pool_span(const AttnParams& p, const float* a, float* out, int L, int o_in, int p_lo, int p_hi,
+                                             int tid, int nthreads) {
+  const int b = p.b;
+  const int o = min(max(o_in, 0), max(L - b, 0));
+  const int C = max(L - b, 0), w = (p.window - 1) / 2;
+  for (int pos = p_lo + tid; pos < p_hi; pos += nthreads)       // the block's own positions and the padding
+    if (pos >= L || (pos >= o && pos < o + b)) out[pos] = -INFINITY;
+  auto below = [&](int x) {                                     // candidates whose position lies below x
+    const int c = x <= o ? x : (x <= o + b ? o : x - b);
+    return min(max(c, 0), C);
+  };
+  const int cl = below(p_lo), ch = below(p_hi);
+  if (w > 4 || ch - cl <= 4 * nthreads) {                     // (a few positions per thread: batching does not pay yet)
+    for (int c = cl + tid; c < ch; c += nthreads) {
+      const int pos = c < o ? c : c + b;
+      out[pos] = kt_pool_at(p, a, L, o_in, pos);
+    }
+    return;
+  }
+  constexpr int K = 16;
+  const bool is_max = p.pool_kind == SDLLM_POOL_MAX;
+  for (int c0 = cl + tid * K; c0 < ch; c0 += nthreads * K) {
+    float v[K + 8];
 #pragma unroll
-    for (int j = 0; j < NB; ++j) {
-      const int pos = pos0 + j * stride;
-      r[j] = pos < end ? kt_pool_at(p, a, L, o, pos) : 0.f;
+    for (int i = 0; i < K + 8; ++i) {
+      const int c = min(max(c0 - 4 + i, 0), C - 1);             // (C >= 1 here: the range is not empty)
+      v[i] = __ldcg(a + (c < o ? c : c + b));
     }
 #pragma unroll
-    for (int j = 0; j < NB; ++j) {
-      const int pos = pos0 + j * stride;
-      if (pos < end) out[pos] = r[j];
+    for (int u = 0; u < K; ++u) {
+      const int c = c0 + u;
+      if (c < ch) {
+        int lo = 0, hi = C;
+        if (p.per_region) { if (c < o) hi = o; else lo = o; }
+        float mx = -INFINITY, sum = 0.f;
+#pragma unroll
+        for (int k = -4; k <= 4; ++k) {
+          const int t = c + k;
+          const bool ok = k >= -w && k <= w && t >= lo && t < hi;
+          const float x = v[u + 4 + k];
+          mx = ok ? fmaxf(mx, x) : mx;
+          sum += ok ? x : 0.f;
+        }
+        out[c < o ? c : c + b] = is_max ? mx : sum / (float)p.window;
+      }
     }
   }
 }
