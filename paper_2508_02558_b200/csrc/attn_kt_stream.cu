@@ -186,6 +186,9 @@ __global__ void __launch_bounds__(KS_THREADS, 1) attn_kt_stream_kernel(const __g
       bool ok = true;
       int n_listed = 0;                  // entries of the unit list written so far
       bool ended = false;                // ... the last of them being the end mark
+      // The counter is asked one unit ahead: the answer for unit k + 1 travels (an L2 round trip under full load) while
+      // unit k's loads are issued, instead of holding up the first loads of unit k + 1.
+      int u_ahead = atomicAdd(p.counters, 1);
       for (int k = 0; ok; ++k) {
         // The next unit: whoever asks first gets the longest one left. The list in shared memory has 16 places; the
         // producer never runs more than eight units ahead of the stores (it could, through units without keys).
@@ -196,8 +199,9 @@ __global__ void __launch_bounds__(KS_THREADS, 1) attn_kt_stream_kernel(const __g
             else if (clock64() - t0 > wlim) { *abort_flag = 1; atomicExch(p.status, 15); ok = false; }
           }
         }
-        int u = ok ? atomicAdd(p.counters, 1) : -1;
+        int u = ok ? u_ahead : -1;
         if (u >= n_units) u = -1;
+        if (u >= 0) u_ahead = atomicAdd(p.counters, 1);
         unit_list[k & 15] = u;
         __threadfence_block();
         *n_pub = k + 1;
