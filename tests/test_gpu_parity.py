@@ -474,4 +474,8 @@ def test_planner_picks_the_kernel_families_where_they_were_measured_to_win():
     assert name(n_kv_heads=8, seq_len_max=32768, n_keep_max=16368) == "attn_umma_bf16_kernel"                   # 8 units of 128 rows
     assert name(batch=8, n_q_heads=16, n_kv_heads=8, seq_len_max=4352, n_keep_max=2048) == "attn_kt_kernel"     # 64 units of 64 rows
     assert name(dtype=B.F32) == "attn_f32_kernel"
+    # cluster sizes follow what the device keeps resident at once: 16 units of whole-SM CTAs get clusters of six, not eight
+    plan = B.plan_describe(B.make_desc(batch=2, n_q_heads=16, n_kv_heads=8, head_dim=128, seq_len_max=2080, block_len=32, dtype=B.BF16,
+                                       retention=0.5, n_keep_max=1024), B.OP_SPARSE_BLOCK_ATTN)
+    assert plan.startswith("attn_kt_kernel ") and " cluster=6 " in plan, plan
 
