@@ -115,6 +115,36 @@ __device__ __forceinline__ float kt_pool_at(const AttnParams& p, const float* a,
   }
   return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
 }
+// kt_pool_at for windows of at most 2 W + 1 with a fixed trip count: the window's loads are independent of one another and
+// go out together (the loop of kt_pool_at waits for each before it issues the next: three L2 round trips for a window
+// of three, on the critical path of a call that lasts 12 us). Same values, same order of the sum.
+template <int W>
+__device__ __forceinline__ float kt_pool_at_w(const AttnParams& p, const float* a, int L, int o_in, int pos) {
+  const int b = p.b;
+  const int o = min(max(o_in, 0), max(L - b, 0));
+  if (pos >= L || (pos >= o && pos < o + b)) return -INFINITY;
+  const int C = max(L - b, 0), w = (p.window - 1) / 2;
+  const int c = pos < o ? pos : pos - b;
+  int lo = 0, hi = C;
+  if (p.per_region) { if (c < o) hi = o; else lo = o; }
+  float x[2 * W + 1];
+  bool ok[2 * W + 1];
+#pragma unroll
+  for (int k = -W; k <= W; ++k) {
+    const int t = c + k;
+    ok[k + W] = k >= -w && k <= w && t >= lo && t < hi;
+    const int tt = ok[k + W] ? t : c;                  // (c itself is always a valid candidate)
+    x[k + W] = __ldcg(a + (tt < o ? tt : tt + b));
+  }
+  float mx = -INFINITY, sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < 2 * W + 1; ++i) {
+    mx = ok[i] ? fmaxf(mx, x[i]) : mx;
+    sum += ok[i] ? x[i] : 0.f;
+  }
+  return p.pool_kind == SDLLM_POOL_MAX ? mx : sum / (float)p.window;
+}
+
 // Pools the absolute positions [p_lo, p_hi) of one head with `nthreads` threads (this one is `tid`): `out` and `a` are the
 // head's rows of the pooled and of the raw scores. A thread takes sixteen consecutive candidates at a time: their windows
 // overlap, so 24 loads (all of them issued together: fixed count, clamped addresses) serve sixteen outputs, and the window
@@ -135,7 +165,7 @@ __device__ __forceinline__ void kt_pool_span(const AttnParams& p, const float* a
   if (w > 4 || ch - cl <= 4 * nthreads) {                     // (a few positions per thread: batching does not pay yet)
     for (int c = cl + tid; c < ch; c += nthreads) {
       const int pos = c < o ? c : c + b;
-      out[pos] = kt_pool_at(p, a, L, o_in, pos);
+      out[pos] = w <= 1 ? kt_pool_at_w<1>(p, a, L, o_in, pos) : (w <= 2 ? kt_pool_at_w<2>(p, a, L, o_in, pos) : kt_pool_at(p, a, L, o_in, pos));
     }
     return;
   }
