@@ -171,7 +171,9 @@ sdllm_status sdllm_compact_kv(const sdllm_desc* desc, const void* k, const void*
  * sequences run the two kernels one after the other inside this call (sdllm_launch_count tells which). The launch may
  * start while the kernel in front of it in the stream is finishing and reads pooled_scores only once that kernel has
  * completed; it holds its own dependents back until it has completed, so the reuse step that follows may read the
- * compacted cache early (see sdllm_sparse_block_attn). */
+ * compacted cache early (see sdllm_sparse_block_attn). seq_len and block_off are older than the scores (the refresh
+ * attention in front has read them too) and are read early, under the rule stated at sdllm_sparse_block_attn: only a
+ * caller's own kernel that releases its dependents early must not be the one that writes them directly in front. */
 sdllm_status sdllm_select_compact(const sdllm_desc* desc, const float* pooled_scores, const int32_t* seq_len,
                                   const int32_t* block_off, const void* k, const void* v, int32_t* kept_idx,
                                   int32_t* kept_cnt, void* k_c, void* v_c, void* cuda_stream);

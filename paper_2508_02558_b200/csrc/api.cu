@@ -355,6 +355,7 @@ sdllm_status sdllm_select_compact(const sdllm_desc* d, const float* pooled_score
   p.mode = d->select; p.retention = d->retention;
   const int cand = d->seq_len_max - d->block_len;
   p.smem_keys = cand <= 45056 ? cand : 0;
+  p.early_inputs = (tuning().pdl != 0 && tuning().early_loads != 0) ? 1 : 0;
   CompactParams c{};
   c.k = k; c.v = v; c.kept_idx = kept_idx; c.kept_cnt = kept_cnt; c.k_c = k_c; c.v_c = v_c;
   c.B = d->batch; c.Hkv = d->n_kv_heads; c.n_keep_max = d->n_keep_max; c.row_bytes = d->head_dim * es; c.Lmax = d->seq_len_max;

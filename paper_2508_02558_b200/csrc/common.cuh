@@ -89,6 +89,7 @@ struct SelectParams {
   int B, Hkv, Lmax, b, n_keep_max, mode;
   double retention;
   int smem_keys;               // candidates cached in shared memory (0 = read global every pass)
+  int early_inputs;            // fused kernel: seq_len and block_off are read ahead of the grid dependency
 };
 
 struct CompactParams {

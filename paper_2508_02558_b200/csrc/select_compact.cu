@@ -458,11 +458,21 @@ __global__ void __launch_bounds__(NT) select_gather_kernel(const SelectParams p,
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int r = blockIdx.x, R = gridDim.x, g = blockIdx.y, bi = blockIdx.z;
+  // Ahead of the grid dependency: what does not depend on the kernel in front - the first segment's histograms and (the
+  // caller's lengths and block offsets are older than the scores) the two words that place the block.
+  int L = p.Lmax, o = 0;
+  if (p.early_inputs) {
+    if (p.seq_len) L = __ldcg(p.seq_len + bi);
+    o = __ldcg(p.block_off + bi);
+  }
+  for (int i = tid; i < 4 * HC * 256; i += NT) (&hist[0][0][0])[i] = 0u;
   asm volatile("griddepcontrol.wait;\n" ::: "memory");  // the pooled scores come from the kernel in front
-  int L = p.seq_len ? p.seq_len[bi] : p.Lmax;
+  if (!p.early_inputs) {
+    if (p.seq_len) L = p.seq_len[bi];
+    o = p.block_off[bi];
+  }
   L = min(max(L, 0), p.Lmax);
   const int b = p.b;
-  int o = p.block_off[bi];
   o = min(max(o, 0), max(L - b, 0));
   const int C = max(L - b, 0);
   const float* sc = p.pooled + (int64_t)(bi * p.Hkv + g) * p.Lmax;
@@ -485,6 +495,7 @@ __global__ void __launch_bounds__(NT) select_gather_kernel(const SelectParams p,
     n_seg = 2;
   }
   uint32_t run_out = 0;                                // entries written so far (same value in every thread)
+  bool hist_used = false;
   __syncthreads();
 
   for (int si = 0; si < n_seg; ++si) {
@@ -498,7 +509,9 @@ __global__ void __launch_bounds__(NT) select_gather_kernel(const SelectParams p,
     if (!take_all) {
       // ---- radix select of the n-th largest key: four passes of 8 bits, most significant first ----
       if (tid == 0) { sh_prefix = 0u; sh_remaining = (uint32_t)n; }
-      for (int i = tid; i < 4 * HC * 256; i += NT) (&hist[0][0][0])[i] = 0u;
+      if (hist_used)                               // (the first select finds the histograms cleared at the kernel's start)
+        for (int i = tid; i < 4 * HC * 256; i += NT) (&hist[0][0][0])[i] = 0u;
+      hist_used = true;
       __syncthreads();
       for (int pass = 0; pass < 4; ++pass) {
         const int shift = 24 - 8 * pass;
