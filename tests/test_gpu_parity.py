@@ -229,6 +229,20 @@ def test_ragged_batch(plan, tuning):
     U.check_sparse_against_oracle(g, out, q2, kn, vn, "bf16")
 
 
+@pytest.mark.parametrize("plan", [dict(lpt=1), dict(lpt=1, early_loads=0), dict(lpt=0)])
+def test_ragged_batch_with_equal_lengths_in_length_order(plan, tuning):
+    """Sequences taken from the longest to the shortest: equal lengths must still map grid slots to sequences one to one."""
+    import parity_util as U
+    tuning(**plan)
+    cfg = _small("rag", "bf16", 4, 4, 128, 64, 64, salient_frac=0.02)
+    bw = W.make_batch(cfg, [200, 64, 200, 64, 333], seed=9, block=1)
+    q, k, v = bw.refresh_inputs(1, pad_value=np.nan)
+    g = U.gpu_refresh(q, k, v, bw.seq_len, bw.block_off, "bf16", 0.5, 3)
+    k0, v0 = np.nan_to_num(k), np.nan_to_num(v)
+    U.check_refresh_against_oracle(g, q, k0, v0, bw.seq_len, bw.block_off, "bf16", 0.5, 3)
+    U.check_compaction_bit_exact(g, g.k_dev, g.v_dev)
+
+
 @pytest.mark.parametrize("kernel", ["default", "cluster", "single"])
 def test_select_topk_alone_heavy_ties_bit_exact(kernel, tuning):
     """Plateaus of exactly equal scores (what max pooling produces) must resolve to the lowest positions. The selection
