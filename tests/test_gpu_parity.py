@@ -492,4 +492,13 @@ def test_planner_picks_the_kernel_families_where_they_were_measured_to_win():
     plan = B.plan_describe(B.make_desc(batch=2, n_q_heads=16, n_kv_heads=8, head_dim=128, seq_len_max=2080, block_len=32, dtype=B.BF16,
                                        retention=0.5, n_keep_max=1024), B.OP_SPARSE_BLOCK_ATTN)
     assert plan.startswith("attn_kt_kernel ") and " cluster=6 " in plan, plan
+    # 192 units of long walks (a six-sequence serving batch): one CTA per SM with a ring of three slots, not two small CTAs
+    # per SM with one slot each; short walks keep the small footprint
+    for op in (B.OP_SPARSE_BLOCK_ATTN, B.OP_REFRESH_SCORES):
+        plan = B.plan_describe(B.make_desc(batch=6, n_q_heads=32, n_kv_heads=32, head_dim=128, seq_len_max=4128, block_len=32,
+                                           dtype=B.BF16, retention=0.5, n_keep_max=2048), op)
+        assert plan.startswith("attn_kt_kernel ") and " stages=3 " in plan and " cluster=1 " in plan, plan
+    plan = B.plan_describe(B.make_desc(batch=6, n_q_heads=32, n_kv_heads=32, head_dim=128, seq_len_max=1056, block_len=32,
+                                       dtype=B.BF16, retention=0.5, n_keep_max=512), B.OP_SPARSE_BLOCK_ATTN)
+    assert plan.startswith("attn_kt_kernel ") and " stages=1 " in plan, plan
 
